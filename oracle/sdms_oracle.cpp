@@ -1,0 +1,349 @@
+// CPU oracle for per-step draft construction (arXiv 2503.05330, Method section
+// and Algorithm 1).  TEST INFRASTRUCTURE ONLY: a plain, slow, brute-force
+// restatement of the method, used to check the CUDA library and timed as the
+// CPU baseline.  It shares no code with the CUDA path and is never called by it.
+//
+// What each step follows:
+//   state      - paths y_1..y_N that grow token by token ("Dynamic Draft Pool
+//                Construction"), with the model probability of every generated
+//                token (the p_theta of Eq. 5).
+//   match      - Eq. 3: every position of every OTHER path of the same prompt
+//                whose prefix ends with the query path's k-token suffix.
+//   candidates - the tokens following each match (at most D of them).
+//   DAG        - "Consensus-Driven Draft Extraction": layer d holds the distinct
+//                d-th follower tokens; edge (u,v) between layers d-1 and d
+//                carries Eq. 5: alpha * sum_i p_i + (1-alpha) * Freq(u->v).
+//   search     - greedy walk: at each layer take the token whose summed
+//                in-edge weight is highest; stop at length D or at a leaf.
+//   accept     - "Draft acceptance": longest prefix of the draft equal to the
+//                sampled tokens.
+//
+// Readings where the paper is silent (all restated in the design notes):
+//   * followers start one position after the matched suffix;
+//   * a match needs at least one follower; a path never searches itself;
+//   * probabilities are held as integers pq = round_half_even(exp(logprob)*2^30),
+//     sums S are exact 64-bit integers, so results do not depend on the order
+//     of accumulation;  Freq(u->v) is the raw instance count;
+//   * weight = alpha*(S/2^30) + (1-alpha)*cnt evaluated in double, each
+//     operation rounded separately (build with -ffp-contract=off);
+//   * the walk only moves to successors of the node it stands on (mode 0);
+//     mode 1 takes the best node of each layer regardless of the previous one;
+//   * ties go to the smallest token id.
+//
+// Pins (tests/, CPU only): hand-worked example from Eq. 3 / Eq. 5 with dyadic
+// probabilities; match set against regex/numpy searches and closed-form counts;
+// alpha = 0 against collections.Counter; conservation invariants; enumeration
+// of every root-to-node DAG path; pq against 50-digit decimal arithmetic;
+// acceptance against os.path.commonprefix.  Behaviour on real model traces
+// (the paper's Table 1) is "parity unpinned": it needs the models and datasets.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <map>
+#include <thread>
+#include <utility>
+#include <vector>
+#include <algorithm>
+
+namespace {
+
+constexpr int64_t ONE_Q30 = int64_t(1) << 30;
+
+enum : uint32_t {
+  ST_BAD_COUNT = 1u, ST_CAPACITY = 2u, ST_BAD_TOKEN = 4u, ST_BAD_LOGPROB = 8u,
+};
+
+struct Acc { int64_t S = 0; int64_t cnt = 0; };
+
+struct PathResult {
+  bool valid = false;                       // query existed (len >= k, path not full)
+  int root = -1;
+  std::vector<std::pair<int, int>> matches; // (path j, index e of last matched token)
+  // layers[d-1] for d = 1..D
+  std::vector<std::map<int, Acc>> nodes;
+  std::vector<std::map<std::pair<int, int>, Acc>> edges;  // key (u, v)
+  std::vector<int> draft;
+  std::vector<double> score, edge_w;
+};
+
+struct Ctx {
+  int G, N, L, V, D, mode;
+  double alpha;
+  std::vector<std::vector<int32_t>> tok, pq;
+  std::vector<PathResult> res;
+};
+
+// Eq. 5 with S in units of 2^-30 (probability sum) and cnt = Freq.
+double weight(double alpha, int64_t S, int64_t cnt) {
+  double t1 = alpha * (double)S;
+  t1 = t1 * (1.0 / (double)ONE_Q30);
+  double t2 = (1.0 - alpha) * (double)cnt;
+  return t1 + t2;
+}
+
+// pq = round_half_even(exp(logprob) * 2^30), clamped to [0, 2^30]; NaN -> 0.
+int32_t prob_to_fixed(float lp, uint32_t* status) {
+  if (std::isnan(lp)) { if (status) *status |= ST_BAD_LOGPROB; return 0; }
+  if (lp >= 0.0f) return (int32_t)ONE_Q30;
+  long double y = expl((long double)lp) * (long double)ONE_Q30;
+  long double r = rintl(y);   // default rounding mode: to nearest, ties to even
+  if (r < 0) r = 0;
+  if (r > (long double)ONE_Q30) r = (long double)ONE_Q30;
+  return (int32_t)r;
+}
+
+uint32_t append_impl(Ctx* c, const int32_t* tokens, const float* logprobs, const int32_t* pqs,
+                     const int32_t* counts, int a_max) {
+  uint32_t st = 0;
+  int P = c->G * c->N;
+  for (int p = 0; p < P; ++p) {
+    int n = counts[p];
+    if (n < 0) { st |= ST_BAD_COUNT; n = 0; }
+    if (n > a_max) { st |= ST_BAD_COUNT; n = a_max; }
+    int room = c->L - (int)c->tok[p].size();
+    if (n > room) { st |= ST_CAPACITY; n = room; }
+    for (int a = 0; a < n; ++a) {
+      int32_t t = tokens[(size_t)p * a_max + a];
+      if (t < 0 || t >= c->V) { st |= ST_BAD_TOKEN; break; }   // path keeps what came before
+      int32_t q = pqs ? pqs[(size_t)p * a_max + a]
+                      : prob_to_fixed(logprobs[(size_t)p * a_max + a], &st);
+      c->tok[p].push_back(t);
+      c->pq[p].push_back(q);
+    }
+  }
+  return st;
+}
+
+void build_path(Ctx* c, int k, int i) {
+  PathResult& r = c->res[i];
+  r = PathResult();
+  r.nodes.resize(c->D);
+  r.edges.resize(c->D);
+  const std::vector<int32_t>& yi = c->tok[i];
+  int len_i = (int)yi.size();
+  if (k < 1 || len_i < k || len_i >= c->L) return;    // no query: too short, or path is full
+  r.valid = true;
+  r.root = yi[len_i - 1];
+  int g = i / c->N;
+  // Eq. 3: every other path j of the prompt, every end position e with a follower.
+  for (int j = g * c->N; j < (g + 1) * c->N; ++j) {
+    if (j == i) continue;
+    const std::vector<int32_t>& yj = c->tok[j];
+    int len_j = (int)yj.size();
+    for (int e = k - 1; e <= len_j - 2; ++e) {
+      bool same = true;
+      for (int t = 0; t < k; ++t)
+        if (yj[e - k + 1 + t] != yi[len_i - k + t]) { same = false; break; }
+      if (same) r.matches.push_back({j, e});
+    }
+  }
+  // Layered DAG: one instance per (candidate, layer).
+  for (const auto& m : r.matches) {
+    int j = m.first, e = m.second;
+    int len_j = (int)c->tok[j].size();
+    int n_m = std::min(c->D, len_j - 1 - e);
+    for (int d = 1; d <= n_m; ++d) {
+      int u = c->tok[j][e + d - 1];
+      int v = c->tok[j][e + d];
+      int64_t p = c->pq[j][e + d];
+      Acc& ed = r.edges[d - 1][{u, v}];
+      ed.S += p; ed.cnt += 1;
+      Acc& nd = r.nodes[d - 1][v];
+      nd.S += p; nd.cnt += 1;
+    }
+  }
+  // Greedy extraction.
+  int cur = r.root;
+  for (int d = 1; d <= c->D; ++d) {
+    bool found = false; int best_v = -1; double best_w = 0.0; double best_e = 0.0;
+    for (const auto& kv : r.nodes[d - 1]) {       // ascending token id
+      int v = kv.first;
+      auto it = r.edges[d - 1].find({cur, v});
+      bool succ = it != r.edges[d - 1].end();
+      if (c->mode == 0 && !succ) continue;
+      double w = weight(c->alpha, kv.second.S, kv.second.cnt);
+      if (!found || w > best_w) {                 // strict: ties keep the smaller token
+        found = true; best_v = v; best_w = w;
+        best_e = succ ? weight(c->alpha, it->second.S, it->second.cnt) : 0.0;
+      }
+    }
+    if (!found) break;
+    r.draft.push_back(best_v);
+    r.score.push_back(best_w);
+    r.edge_w.push_back(best_e);
+    cur = best_v;
+  }
+}
+
+struct NodeRow { int tok; int64_t S, cnt; double w; };
+
+}  // namespace
+
+extern "C" {
+
+void* orc_create(int G, int N, int L, int V, int D, float alpha, int mode) {
+  Ctx* c = new Ctx();
+  c->G = G; c->N = N; c->L = L; c->V = V; c->D = D; c->mode = mode;
+  c->alpha = (double)alpha;
+  c->tok.resize((size_t)G * N); c->pq.resize((size_t)G * N); c->res.resize((size_t)G * N);
+  return c;
+}
+
+void orc_destroy(void* h) { delete (Ctx*)h; }
+
+int32_t orc_prob_to_fixed(float lp) { return prob_to_fixed(lp, nullptr); }
+
+double orc_weight(float alpha, int64_t S, int64_t cnt) { return weight((double)alpha, S, cnt); }
+
+uint32_t orc_append(void* h, const int32_t* tokens, const float* logprobs, const int32_t* counts, int a_max) {
+  return append_impl((Ctx*)h, tokens, logprobs, nullptr, counts, a_max);
+}
+
+// Same as orc_append but with the fixed-point probabilities given directly
+// (used by the hand-worked examples, whose probabilities are dyadic).
+uint32_t orc_append_fixed(void* h, const int32_t* tokens, const int32_t* pq, const int32_t* counts, int a_max) {
+  return append_impl((Ctx*)h, tokens, nullptr, pq, counts, a_max);
+}
+
+void orc_get_lengths(void* h, int32_t* out) {
+  Ctx* c = (Ctx*)h;
+  for (size_t p = 0; p < c->tok.size(); ++p) out[p] = (int32_t)c->tok[p].size();
+}
+
+void orc_get_history(void* h, int p, int32_t* tok, int32_t* pq) {
+  Ctx* c = (Ctx*)h;
+  std::memcpy(tok, c->tok[p].data(), c->tok[p].size() * 4);
+  std::memcpy(pq, c->pq[p].data(), c->pq[p].size() * 4);
+}
+
+void orc_build_path(void* h, int k, int i) { build_path((Ctx*)h, k, i); }
+
+// All paths; nthreads > 1 fans the (independent) query paths out over threads.
+void orc_build_all(void* h, int k, int nthreads) {
+  Ctx* c = (Ctx*)h;
+  int P = c->G * c->N;
+  if (nthreads <= 1) { for (int i = 0; i < P; ++i) build_path(c, k, i); return; }
+  std::vector<std::thread> th;
+  for (int t = 0; t < nthreads; ++t)
+    th.emplace_back([=]() { for (int i = t; i < P; i += nthreads) build_path(c, k, i); });
+  for (auto& x : th) x.join();
+}
+
+int orc_num_matches(void* h, int i) { return (int)((Ctx*)h)->res[i].matches.size(); }
+
+// Global positions j*L + e, ascending.
+void orc_get_matches(void* h, int i, int32_t* gpos) {
+  Ctx* c = (Ctx*)h;
+  size_t n = 0;
+  for (const auto& m : c->res[i].matches) gpos[n++] = m.first * c->L + m.second;
+}
+
+void orc_layer_counts(void* h, int i, int d, int32_t* n_nodes, int32_t* n_edges) {
+  const PathResult& r = ((Ctx*)h)->res[i];
+  *n_nodes = (int32_t)r.nodes[d - 1].size();
+  *n_edges = (int32_t)r.edges[d - 1].size();
+}
+
+void orc_get_nodes(void* h, int i, int d, int32_t* tok, int64_t* S, int64_t* cnt) {
+  size_t n = 0;
+  for (const auto& kv : ((Ctx*)h)->res[i].nodes[d - 1]) { tok[n] = kv.first; S[n] = kv.second.S; cnt[n] = kv.second.cnt; ++n; }
+}
+
+void orc_get_edges(void* h, int i, int d, int32_t* u, int32_t* v, int64_t* S, int64_t* cnt) {
+  size_t n = 0;
+  for (const auto& kv : ((Ctx*)h)->res[i].edges[d - 1]) {
+    u[n] = kv.first.first; v[n] = kv.first.second; S[n] = kv.second.S; cnt[n] = kv.second.cnt; ++n;
+  }
+}
+
+int orc_get_draft(void* h, int i, int32_t* tok, double* score, double* edge_w) {
+  const PathResult& r = ((Ctx*)h)->res[i];
+  for (size_t d = 0; d < r.draft.size(); ++d) { tok[d] = r.draft[d]; score[d] = r.score[d]; edge_w[d] = r.edge_w[d]; }
+  return (int)r.draft.size();
+}
+
+// Drafts of all paths in the library's output layout: tok [P][D] (unused = -1),
+// len [P], score / edge_w [P][D] as float (unused = 0).
+void orc_get_drafts(void* h, int32_t* tok, int32_t* len, float* score, float* edge_w) {
+  Ctx* c = (Ctx*)h;
+  int P = c->G * c->N;
+  for (int i = 0; i < P; ++i) {
+    const PathResult& r = c->res[i];
+    len[i] = (int32_t)r.draft.size();
+    for (int d = 0; d < c->D; ++d) {
+      bool on = d < (int)r.draft.size();
+      tok[(size_t)i * c->D + d] = on ? r.draft[d] : -1;
+      score[(size_t)i * c->D + d] = on ? (float)r.score[d] : 0.0f;
+      edge_w[(size_t)i * c->D + d] = on ? (float)r.edge_w[d] : 0.0f;
+    }
+  }
+}
+
+// Truncated view of the DAG of path i: per layer the B best nodes by
+// (weight desc, token asc); per kept node of layer d its Ke best out-edges to
+// layer d+1 by (weight desc, destination token asc).  Unused slots: token -1.
+// node_* are [D][B], node_count [D], edge_* are [D][B][Ke], out_degree [D][B].
+void orc_get_export(void* h, int i, int B, int Ke,
+                    int32_t* node_tok, int64_t* node_S, int32_t* node_cnt, int32_t* node_count,
+                    int32_t* edge_dst, int64_t* edge_S, int32_t* edge_cnt, int32_t* out_degree) {
+  Ctx* c = (Ctx*)h;
+  const PathResult& r = c->res[i];
+  int D = c->D;
+  for (int x = 0; x < D * B; ++x) { node_tok[x] = -1; node_S[x] = 0; node_cnt[x] = 0; out_degree[x] = 0; }
+  for (int x = 0; x < D * B * Ke; ++x) { edge_dst[x] = -1; edge_S[x] = 0; edge_cnt[x] = 0; }
+  for (int d = 1; d <= D; ++d) {
+    node_count[d - 1] = (int32_t)r.nodes[d - 1].size();
+    std::vector<NodeRow> rows;
+    for (const auto& kv : r.nodes[d - 1])
+      rows.push_back({kv.first, kv.second.S, kv.second.cnt, weight(c->alpha, kv.second.S, kv.second.cnt)});
+    std::stable_sort(rows.begin(), rows.end(), [](const NodeRow& a, const NodeRow& b) {
+      return a.w > b.w || (a.w == b.w && a.tok < b.tok); });
+    for (int b = 0; b < B && b < (int)rows.size(); ++b) {
+      size_t nx = (size_t)(d - 1) * B + b;
+      node_tok[nx] = rows[b].tok; node_S[nx] = rows[b].S; node_cnt[nx] = (int32_t)rows[b].cnt;
+      if (d == D) continue;
+      std::vector<NodeRow> out;
+      for (const auto& kv : r.edges[d])              // edges between layers d and d+1
+        if (kv.first.first == rows[b].tok)
+          out.push_back({kv.first.second, kv.second.S, kv.second.cnt, weight(c->alpha, kv.second.S, kv.second.cnt)});
+      out_degree[nx] = (int32_t)out.size();
+      std::stable_sort(out.begin(), out.end(), [](const NodeRow& a, const NodeRow& b) {
+        return a.w > b.w || (a.w == b.w && a.tok < b.tok); });
+      for (int e = 0; e < Ke && e < (int)out.size(); ++e) {
+        size_t ex = nx * Ke + e;
+        edge_dst[ex] = out[e].tok; edge_S[ex] = out[e].S; edge_cnt[ex] = (int32_t)out[e].cnt;
+      }
+    }
+  }
+}
+
+// "Draft acceptance": tau_p = longest t <= draft_len[p] with draft[0..t) == sampled[0..t).
+void orc_accept(void* h, const int32_t* draft_tok, const int32_t* draft_len, const int32_t* sampled,
+                int32_t* accept_len) {
+  Ctx* c = (Ctx*)h;
+  int P = c->G * c->N, D = c->D;
+  for (int p = 0; p < P; ++p) {
+    int t = 0;
+    while (t < draft_len[p] && t < D && draft_tok[(size_t)p * D + t] == sampled[(size_t)p * (D + 1) + t]) ++t;
+    accept_len[p] = t;
+  }
+}
+
+// Acceptance followed by the state update: path p appends sampled[p][0 .. tau_p]
+// (the accepted tokens plus the model's own next token), at most max_append
+// tokens, cut at capacity (no status for that cut) and before a token outside [0, V).
+uint32_t orc_accept_commit(void* h, const int32_t* draft_tok, const int32_t* draft_len, const int32_t* sampled,
+                           const float* sampled_logprobs, int max_append, int32_t* accept_len) {
+  Ctx* c = (Ctx*)h;
+  int P = c->G * c->N, D = c->D;
+  orc_accept(h, draft_tok, draft_len, sampled, accept_len);
+  std::vector<int32_t> counts(P);
+  for (int p = 0; p < P; ++p) {
+    int n = std::min(accept_len[p] + 1, max_append);
+    n = std::min(n, c->L - (int)c->tok[p].size());
+    counts[p] = n;
+  }
+  return append_impl(c, sampled, sampled_logprobs, nullptr, counts.data(), D + 1);
+}
+
+}  // extern "C"

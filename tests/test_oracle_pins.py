@@ -1,0 +1,457 @@
+"""Pins of the CPU oracle against what the paper and plain mathematics fix.
+
+Nothing here touches the CUDA library.  Each check is chosen so that a
+plausible mistake in the oracle (dropped term, off-by-one position, self match,
+wrong tie rule, transposed edge) fails at least one of them.
+"""
+import collections
+import decimal
+import itertools
+import json
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import Oracle
+from paper_2503_05330_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+Q30 = 1 << 30
+
+
+def load_paths(o, paths, probs=None, logprobs=None):
+    """Append whole paths (ragged) in one call."""
+    a_max = max(len(p) for p in paths)
+    tok = np.zeros((o.P, a_max), np.int32)
+    cnt = np.array([len(p) for p in paths], np.int32)
+    for i, p in enumerate(paths):
+        tok[i, :len(p)] = p
+    if probs is not None:
+        pq = np.zeros((o.P, a_max), np.int32)
+        for i, p in enumerate(probs):
+            pq[i, :len(p)] = [int(round(x * Q30)) for x in p]
+        return o.append_fixed(tok, pq, cnt)
+    lp = np.zeros((o.P, a_max), np.float32)
+    for i, p in enumerate(logprobs):
+        lp[i, :len(p)] = p
+    return o.append(tok, lp, cnt)
+
+
+# ----------------------------------------------------------------------------
+# fixed-point probability
+# ----------------------------------------------------------------------------
+def test_prob_to_fixed_against_50_digit_decimal():
+    decimal.getcontext().prec = 60
+    rng = synth.Stream(99)
+    lps = np.concatenate([(-8.0 * rng.uniform(1500)).astype(np.float32),
+                          (-1e-3 * rng.uniform(300)).astype(np.float32),
+                          np.array([-20.0, -30.0, -50.0, -1e-7, -0.6931472], np.float32)])
+    for lp in lps:
+        exact = (decimal.Decimal(float(lp)).exp() * Q30).to_integral_value(rounding=decimal.ROUND_HALF_EVEN)
+        assert oracle.prob_to_fixed(float(lp)) == int(exact), lp
+
+
+def test_prob_to_fixed_special_values():
+    assert oracle.prob_to_fixed(0.0) == Q30
+    assert oracle.prob_to_fixed(1.5) == Q30          # a probability cannot exceed one
+    assert oracle.prob_to_fixed(float("-inf")) == 0
+    assert oracle.prob_to_fixed(-100.0) == 0
+    assert oracle.prob_to_fixed(float("nan")) == 0
+    # monotone in the logprob
+    xs = np.linspace(-12, 0, 400).astype(np.float32)
+    v = [oracle.prob_to_fixed(float(x)) for x in xs]
+    assert all(a <= b for a, b in zip(v, v[1:]))
+
+
+def test_weight_is_eq5_in_exact_cases():
+    # alpha = 1: pure probability sum; alpha = 0: pure count; alpha = 1/2: dyadic mix.
+    assert oracle.weight(1.0, 3 * Q30 // 4, 2) == 0.75
+    assert oracle.weight(0.0, 3 * Q30 // 4, 2) == 2.0
+    assert oracle.weight(0.5, 3 * Q30 // 4, 2) == 1.375
+    assert oracle.weight(0.25, Q30 // 2, 3) == 0.25 * 0.5 + 0.75 * 3
+
+
+# ----------------------------------------------------------------------------
+# the hand-worked example
+# ----------------------------------------------------------------------------
+@pytest.fixture()
+def worked():
+    with open(os.path.join(GOLDEN, "worked_example.json")) as f:
+        return json.load(f)
+
+
+def make_worked(w, alpha=None, mode=0, probs=None):
+    o = Oracle(1, 3, w["capacity"], 16, w["D"], alpha=w["alpha"] if alpha is None else alpha, mode=mode)
+    assert load_paths(o, w["paths"], probs=probs or w["prob"]) == 0
+    return o
+
+
+def test_worked_example_matches_dag_and_draft(worked):
+    w = worked
+    o = make_worked(w)
+    o.build_path(w["k"], 0)
+    L = w["capacity"]
+    assert o.matches(0).tolist() == [j * L + e for j, e in w["matches"]]
+    for d in (1, 2, 3):
+        nodes, edges = o.layer(0, d)
+        assert edges == {(u, v): (int(s * Q30), c) for u, v, s, c in w["edges"][str(d)]}
+        assert nodes == {v: (int(s * Q30), c) for v, s, c in w["nodes"][str(d)]}
+    tok, score, edge_w = o.draft(0)
+    assert tok.tolist() == w["draft"]
+    assert score.tolist() == w["draft_score"]
+    assert edge_w.tolist() == w["draft_edge_w"]
+    assert int(score[0] * Q30) == w["draft_S_fixed"]
+    # following the heaviest out-edge instead of the heaviest node would give another draft
+    assert w["heaviest_out_edge_walk"] != w["draft"]
+    for i, want in w["other_queries"].items():
+        o.build_path(w["k"], int(i))
+        assert o.draft(int(i))[0].tolist() == want
+
+
+def test_worked_example_layer_argmax_mode(worked):
+    o = make_worked(worked, mode=1)
+    o.build_path(worked["k"], 0)
+    assert o.draft(0)[0].tolist() == worked["layer_argmax_walk"]
+
+
+def test_worked_example_tie_goes_to_smaller_token(worked):
+    w = worked
+    probs = [list(p) for p in w["prob"]]
+    pj, idx, val = w["tie_variant"]["set"]
+    probs[pj][idx] = val
+    o = make_worked(w, probs=probs)
+    o.build_path(w["k"], 0)
+    nodes, _ = o.layer(0, 1)
+    assert nodes[3][0] == nodes[4][0]
+    assert o.draft(0)[0][0] == w["tie_variant"]["first_token"]
+
+
+def test_worked_example_alpha_half(worked):
+    w = worked
+    o = make_worked(w, alpha=w["alpha_half_variant"]["alpha"])
+    o.build_path(w["k"], 0)
+    nodes, _ = o.layer(0, 1)
+    assert oracle.weight(0.5, *nodes[3]) == w["alpha_half_variant"]["W_1_3"]
+    assert oracle.weight(0.5, *nodes[4]) == w["alpha_half_variant"]["W_1_4"]
+    assert o.draft(0)[1][0] == w["alpha_half_variant"]["W_1_3"]
+
+
+def test_worked_example_accept_and_commit(worked):
+    w = worked
+    o = make_worked(w)
+    o.build_all(w["k"])
+    tok, ln, _, _ = o.drafts()
+    D = w["D"]
+    sampled = np.full((3, D + 1), 15, np.int32)
+    sampled[0] = w["accept"]["sampled"]
+    lens0 = o.lengths().copy()
+    tau, st = o.accept_commit(tok, ln, sampled, np.full((3, D + 1), -0.5, np.float32), D + 1)
+    assert st == 0
+    assert tau[0] == w["accept"]["tau"]
+    h, _ = o.history(0)
+    assert h[lens0[0]:].tolist() == w["accept"]["committed"]
+    # a path whose draft is rejected outright still receives the model's own token
+    assert tau[2] == 0 and o.lengths()[2] == lens0[2] + 1
+
+
+def test_reconverging_branches_merge_into_one_node():
+    # two candidates diverge at layer 1 and meet again at layer 2 in the same
+    # token: one node there, two in-edges, its score the sum over both.
+    paths = [[9, 1], [1, 2, 7, 5], [1, 3, 7, 5], [8, 8]]
+    probs = [[0.5, 0.5], [0.5, 0.5, 0.25, 0.5], [0.5, 0.25, 0.5, 0.5], [0.5, 0.5]]
+    o = Oracle(1, 4, 8, 16, 3)
+    load_paths(o, paths, probs=probs)
+    o.build_path(1, 0)
+    nodes, edges = o.layer(0, 2)
+    assert nodes == {7: (int(0.75 * Q30), 2)}
+    assert edges == {(2, 7): (Q30 // 4, 1), (3, 7): (Q30 // 2, 1)}
+    nodes3, edges3 = o.layer(0, 3)
+    assert edges3 == {(7, 5): (Q30, 2)}
+    assert o.draft(0)[0].tolist() == [2, 7, 5]
+
+
+# ----------------------------------------------------------------------------
+# the match set (Eq. 3)
+# ----------------------------------------------------------------------------
+def regex_matches(tokens, lens, N, L, i, k):
+    """Eq. 3 by overlapping regex search on byte strings (tokens < 256)."""
+    q = bytes(tokens[i, lens[i] - k:lens[i]].tolist())
+    g = i // N
+    out = []
+    for j in range(g * N, (g + 1) * N):
+        if j == i:
+            continue
+        hay = bytes(tokens[j, :lens[j]].tolist())
+        for m in re.finditer(b"(?=" + re.escape(q) + b")", hay):
+            e = m.start() + k - 1
+            if e <= lens[j] - 2:
+                out.append(j * L + e)
+    return sorted(out)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_match_set_equals_regex_search(seed):
+    G, N, L, V = 2, 4, 24, 3 + seed % 2
+    tokens, lps = synth.small_random(G * N, L, V, seed)
+    rng = synth.Stream(1000 + seed)
+    lens = (3 + rng.uniform(G * N) * (L - 4)).astype(np.int32)     # ragged, none full
+    o = Oracle(G, N, L, V, 4)
+    o.append(tokens, lps, lens)
+    for k in (1, 2, 3):
+        o.build_all(k)
+        for i in range(G * N):
+            assert o.matches(i).tolist() == regex_matches(tokens, lens, N, L, i, k), (seed, k, i)
+
+
+def test_k1_is_numpy_where():
+    tokens, lps = synth.small_random(4, 40, 5, 7)
+    lens = np.array([40 - 1, 33, 17, 25], np.int32)
+    o = Oracle(1, 4, 40, 5, 3)
+    o.append(tokens, lps, lens)
+    o.build_all(1)
+    for i in range(4):
+        want = []
+        for j in range(4):
+            if j != i:
+                e = np.where(tokens[j, :lens[j] - 1] == tokens[i, lens[i] - 1])[0]
+                want += (j * 40 + e).tolist()
+        assert o.matches(i).tolist() == want
+
+
+def test_all_equal_tokens_closed_form_and_disjoint_alphabets():
+    # every window of a constant path matches: len_j - k positions per other path
+    L, N = 32, 3
+    lens = np.array([10, 20, 31], np.int32)
+    o = Oracle(1, N, L, 4, 4)
+    o.append(np.full((N, L), 2, np.int32), np.full((N, L), -0.1, np.float32), lens)
+    for k in (1, 2, 5):
+        o.build_all(k)
+        for i in range(N):
+            assert len(o.matches(i)) == sum(lens[j] - k for j in range(N) if j != i)
+    # paths over disjoint alphabets never match
+    tok = np.stack([np.arange(L) % 3, 3 + np.arange(L) % 3, 6 + np.arange(L) % 3]).astype(np.int32)
+    o = Oracle(1, N, L, 9, 4)
+    o.append(tok, np.full((N, L), -0.1, np.float32), lens)
+    o.build_all(1)
+    assert all(len(o.matches(i)) == 0 for i in range(N))
+
+
+def test_matching_never_crosses_prompts_and_needs_k_tokens():
+    tok = np.tile(np.array([1, 2, 3, 1, 2, 3, 1, 2], np.int32), (4, 1))
+    o = Oracle(2, 2, 16, 4, 2)
+    o.append(tok, np.full(tok.shape, -0.2, np.float32), np.array([8, 8, 8, 1], np.int32))
+    o.build_all(2)
+    assert all(m // 16 == 1 for m in o.matches(0))       # path 0 only sees path 1
+    assert all(m // 16 == 3 for m in o.matches(2))
+    assert len(o.matches(3)) == 0 and o.draft(3)[0].size == 0   # one token cannot form a 2-token query
+
+
+def test_full_path_builds_no_draft_but_is_still_a_source():
+    tok = np.tile(np.array([1, 2, 1, 2, 1, 2, 1, 2], np.int32), (2, 1))
+    o = Oracle(1, 2, 8, 4, 2)
+    o.append(tok, np.full(tok.shape, -0.2, np.float32), np.array([8, 4], np.int32))
+    o.build_all(1)
+    assert o.draft(0)[0].size == 0              # path 0 is at capacity
+    assert len(o.matches(1)) == 3               # token 2 inside the full path, last one has no follower
+    assert o.draft(1)[0].tolist() == [1, 2]
+
+
+# ----------------------------------------------------------------------------
+# DAG aggregation (Eq. 5) - invariants and the alpha = 0 special case
+# ----------------------------------------------------------------------------
+def follower_slices(tokens, pqs, lens, L, D, gpos):
+    j, e = divmod(int(gpos), L)
+    n = min(D, lens[j] - 1 - e)
+    return tokens[j, e:e + n + 1], pqs[j][e + 1:e + n + 1]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_dag_invariants_and_counter(seed):
+    G, N, L, V, D = 1, 5, 40, 3, 5
+    tokens, lps = synth.small_random(G * N, L, V, 50 + seed)
+    rng = synth.Stream(2000 + seed)
+    lens = (6 + rng.uniform(N) * (L - 7)).astype(np.int32)
+    for alpha in (1.0, 0.0):
+        o = Oracle(G, N, L, V, D, alpha=alpha)
+        o.append(tokens, lps, lens)
+        pqs = [o.history(p)[1] for p in range(N)]
+        k = 1 + seed % 2
+        o.build_all(k)
+        for i in range(N):
+            m = o.matches(i)
+            cands = [follower_slices(tokens, pqs, lens, L, D, g) for g in m]
+            for d in range(1, D + 1):
+                nodes, edges = o.layer(i, d)
+                live = [(t, p) for t, p in cands if len(p) >= d]
+                # counts are a Counter over follower pairs / follower tokens
+                assert {key: c for key, (_, c) in edges.items()} == dict(
+                    collections.Counter((int(t[d - 1]), int(t[d])) for t, _ in live))
+                assert {key: c for key, (_, c) in nodes.items()} == dict(
+                    collections.Counter(int(t[d]) for t, _ in live))
+                # probability mass is conserved from instances to edges to nodes
+                assert sum(s for s, _ in nodes.values()) == sum(int(p[d - 1]) for _, p in live)
+                for v, (s, c) in nodes.items():
+                    assert s == sum(es for (u2, v2), (es, _) in edges.items() if v2 == v)
+                    assert c == sum(ec for (u2, v2), (_, ec) in edges.items() if v2 == v)
+                # every edge starts in a node of the previous layer
+                if d > 1:
+                    prev_nodes, _ = o.layer(i, d - 1)
+                    assert {u for u, _ in edges} <= set(prev_nodes)
+                    for u, (_, c) in prev_nodes.items():
+                        ended = sum(1 for t, p in cands if len(p) == d - 1 and int(t[d - 1]) == u)
+                        assert sum(ec for (u2, _), (_, ec) in edges.items() if u2 == u) == c - ended
+                else:
+                    assert {u for u, _ in edges} <= {int(tokens[i, lens[i] - 1])}
+            if alpha == 0.0:
+                _, score, edge_w = o.draft(i)
+                assert all(float(x).is_integer() for x in score) and all(float(x).is_integer() for x in edge_w)
+
+
+def test_alpha_one_scores_agree_with_real_valued_sum():
+    G, N, L, V, D = 1, 6, 64, 4, 4
+    tokens, lps = synth.small_random(N, L, V, 77)
+    lens = np.full(N, L - 1, np.int32)
+    o = Oracle(G, N, L, V, D)
+    o.append(tokens, lps, lens)
+    o.build_all(1)
+    for i in range(N):
+        m = o.matches(i)
+        for d in range(1, D + 1):
+            nodes, _ = o.layer(i, d)
+            real = collections.defaultdict(float)
+            for g in m:
+                j, e = divmod(int(g), L)
+                if e + d <= lens[j] - 1:
+                    real[int(tokens[j, e + d])] += float(np.exp(np.float64(lps[j, e + d])))
+            for v, (s, c) in nodes.items():
+                assert abs(s / Q30 - real[v]) <= c * 2.0 ** -31 + 1e-12
+
+
+# ----------------------------------------------------------------------------
+# greedy search against enumeration of every DAG path
+# ----------------------------------------------------------------------------
+def all_dag_paths(o, i, root, D):
+    """Every root-to-node path of the layered DAG, by exhaustive extension."""
+    layers = [o.layer(i, d) for d in range(1, D + 1)]
+    paths = {()}
+    frontier = [((), root)]
+    for d in range(D):
+        nxt = []
+        for pref, u in frontier:
+            for (eu, ev) in layers[d][1]:
+                if eu == u:
+                    nxt.append((pref + (ev,), ev))
+        paths.update(p for p, _ in nxt)
+        frontier = list(set(nxt))
+    return paths, layers
+
+
+@pytest.mark.parametrize("seed,alpha", list(itertools.product(range(5), (1.0, 0.5))))
+def test_draft_is_greedy_path_of_the_dag(seed, alpha):
+    G, N, L, V, D = 1, 4, 24, 3, 4
+    tokens, lps = synth.small_random(N, L, V, 300 + seed)
+    rng = synth.Stream(3000 + seed)
+    lens = (4 + rng.uniform(N) * (L - 5)).astype(np.int32)
+    o = Oracle(G, N, L, V, D, alpha=alpha)
+    o.append(tokens, lps, lens)
+    o.build_all(1)
+    for i in range(N):
+        root = int(tokens[i, lens[i] - 1])
+        paths, layers = all_dag_paths(o, i, root, D)
+        draft, score, edge_w = o.draft(i)
+        draft = tuple(int(x) for x in draft)
+        assert draft in paths                                         # a path of the DAG
+        for d in range(len(draft) + 1):
+            ext = sorted({p[d] for p in paths if len(p) > d and p[:d] == draft[:d]})
+            if d == len(draft):
+                assert d == D or not ext                              # stops at D or at a leaf
+                break
+            w = {v: oracle.weight(alpha, *layers[d][0][v]) for v in ext}
+            best = max(w.values())
+            assert draft[d] == min(v for v in ext if w[v] == best)    # argmax, ties to the smaller id
+            assert score[d] == w[draft[d]]
+            u = root if d == 0 else draft[d - 1]
+            assert edge_w[d] == oracle.weight(alpha, *layers[d][1][(u, draft[d])])
+
+
+def test_layer_argmax_mode_is_per_layer_max():
+    N, L, V, D = 4, 24, 3, 4
+    tokens, lps = synth.small_random(N, L, V, 411)
+    o = Oracle(1, N, L, V, D, mode=1)
+    o.append(tokens, lps, np.full(N, L - 2, np.int32))
+    o.build_all(1)
+    for i in range(N):
+        draft, score, _ = o.draft(i)
+        for d in range(1, D + 1):
+            nodes, _ = o.layer(i, d)
+            if not nodes:
+                assert len(draft) == d - 1
+                break
+            w = {v: oracle.weight(1.0, *sc) for v, sc in nodes.items()}
+            assert draft[d - 1] == min(v for v in w if w[v] == max(w.values()))
+
+
+# ----------------------------------------------------------------------------
+# export view, acceptance, append rules
+# ----------------------------------------------------------------------------
+def test_export_view_is_sorted_truncation_of_the_full_dag():
+    N, L, V, D, B, Ke = 5, 48, 4, 4, 3, 2
+    tokens, lps = synth.small_random(N, L, V, 512)
+    o = Oracle(1, N, L, V, D, alpha=0.5)
+    o.append(tokens, lps, np.full(N, L - 3, np.int32))
+    o.build_all(1)
+    for i in range(N):
+        ex = o.export(i, B, Ke)
+        for d in range(1, D + 1):
+            nodes, _ = o.layer(i, d)
+            order = sorted(nodes, key=lambda v: (-oracle.weight(0.5, *nodes[v]), v))
+            assert ex["node_count"][d - 1] == len(nodes)
+            kept = [int(x) for x in ex["node_tok"][d - 1] if x >= 0]
+            assert kept == order[:B]
+            if d < D:
+                _, nxt = o.layer(i, d + 1)
+                for b, u in enumerate(kept):
+                    out = {v: sc for (uu, v), sc in nxt.items() if uu == u}
+                    eorder = sorted(out, key=lambda v: (-oracle.weight(0.5, *out[v]), v))
+                    assert ex["out_degree"][d - 1, b] == len(out)
+                    assert [int(x) for x in ex["edge_dst"][d - 1, b] if x >= 0] == eorder[:Ke]
+                    for e, v in enumerate(eorder[:Ke]):
+                        assert (int(ex["edge_S"][d - 1, b, e]), int(ex["edge_cnt"][d - 1, b, e])) == out[v]
+
+
+def test_accept_is_longest_common_prefix_exhaustive():
+    D = 4
+    cases = []
+    for dl in range(D + 1):
+        for draft in itertools.product((0, 1), repeat=dl):
+            for samp in itertools.product((0, 1), repeat=D + 1):
+                cases.append((draft, samp))
+    P = len(cases)
+    o = Oracle(1, P, 8, 2, D)
+    dt = np.full((P, D), -1, np.int32); dlens = np.zeros(P, np.int32); sm = np.zeros((P, D + 1), np.int32)
+    for p, (draft, samp) in enumerate(cases):
+        dt[p, :len(draft)] = draft; dlens[p] = len(draft); sm[p] = samp
+    tau = o.accept(dt, dlens, sm)
+    for p, (draft, samp) in enumerate(cases):
+        assert tau[p] == len(os.path.commonprefix([list(draft), list(samp[:len(draft)])]))
+
+
+def test_append_rules_and_status():
+    o = Oracle(1, 4, 6, 10, 2)
+    tok = np.array([[1, 2, 3, 4], [1, 2, 3, 4], [1, 99, 3, 4], [1, 2, 3, 4]], np.int32)
+    lp = np.full((4, 4), -0.3, np.float32)
+    st = o.append(tok, lp, np.array([4, 0, 4, 7], np.int32))
+    assert st == oracle.ST_BAD_TOKEN | oracle.ST_BAD_COUNT
+    assert o.lengths().tolist() == [4, 0, 1, 4]          # cut before the bad token; count clamped
+    st = o.append(tok, lp, np.array([4, 2, 0, 0], np.int32))
+    assert st == oracle.ST_CAPACITY
+    assert o.lengths().tolist() == [6, 2, 1, 4]
+    assert o.history(0)[0].tolist() == [1, 2, 3, 4, 1, 2]
+    lp[0, 0] = np.nan
+    st = o.append(tok, lp, np.array([0, 1, 1, 1], np.int32))
+    assert st == 0                                        # the NaN entry was not among the appended
+    st = o.append(tok, np.full((4, 4), np.nan, np.float32), np.array([0, 1, 0, 0], np.int32))
+    assert st == oracle.ST_BAD_LOGPROB and o.history(1)[1][-1] == 0

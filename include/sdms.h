@@ -1,0 +1,190 @@
+/*
+ * sdms - draft-token construction for multi-sample speculative decoding on one
+ * NVIDIA B200 (sm_100a).  Method: arXiv 2503.05330, section "Method" and
+ * Algorithm 1 ("Self-Consistency Draft Token Generation").
+ *
+ * A context holds G independent prompts with N reasoning paths each.  Every
+ * decode step the caller
+ *   1. asks for one draft per path            (sdms_build_drafts),
+ *   2. lets its model verify the drafts       (not part of this library),
+ *   3. reports the sampled tokens             (sdms_accept, which can also
+ *      append them; or sdms_append directly).
+ *
+ * Conventions that hold for every entry point
+ *   - "d_" pointers are DEVICE pointers owned by the caller; everything else is
+ *     host memory.  The library allocates no device memory: all of its device
+ *     state lives in the caller's workspace (sdms_workspace_bytes bytes, 256-byte
+ *     aligned).  The context is a small host object.
+ *   - Path index p = g * paths_per_group + n.  Rows of per-path arrays are
+ *     contiguous ([P][x], row-major, int32/float32).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     only enqueue work; none waits for the device except sdms_create,
+ *     sdms_get_status and sdms_profile_read.
+ *   - Return value: 0 on success, a negative SDMS_ERR_* otherwise.  Nothing
+ *     throws, aborts or traps.  Conditions only visible on the device set bits
+ *     in a device status word (SDMS_STATUS_*); the offending item is clamped or
+ *     skipped as described per call and the rest of the batch proceeds.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ */
+#ifndef SDMS_H_
+#define SDMS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SDMS_OK                      0
+#define SDMS_ERR_INVALID_ARG        -1
+#define SDMS_ERR_WORKSPACE_TOO_SMALL -2
+#define SDMS_ERR_CUDA               -3
+#define SDMS_ERR_BAD_STATE          -4
+
+/* Device status bits (sticky until sdms_get_status clears them). */
+#define SDMS_STATUS_BAD_COUNT      0x01u /* append count outside [0, row width]: clamped          */
+#define SDMS_STATUS_CAPACITY       0x02u /* sdms_append beyond the path capacity: truncated       */
+#define SDMS_STATUS_BAD_TOKEN      0x04u /* token outside [0, vocab): path keeps what came before */
+#define SDMS_STATUS_BAD_LOGPROB    0x08u /* NaN logprob: stored as probability 0                  */
+#define SDMS_STATUS_INDEX_FULL     0x10u /* n-gram table had no free bucket (cannot happen with the sized workspace) */
+#define SDMS_STATUS_MATCH_OVERFLOW 0x20u /* match workspace exhausted: the affected paths get draft_len 0 */
+
+#define SDMS_MAX_K      16   /* largest supported k_max           */
+#define SDMS_MAX_DRAFT  32   /* largest supported max_draft_len   */
+#define SDMS_MAX_PATHS_PER_GROUP 1024
+#define SDMS_MAX_DAG_NODES 32  /* largest dag_nodes_per_layer      */
+#define SDMS_MAX_DAG_EDGES 16  /* largest dag_edges_per_node       */
+
+typedef struct sdms_ctx sdms_ctx;
+
+typedef struct {
+  uint32_t struct_size;          /* sizeof(sdms_config), for ABI checks                       */
+  int32_t  num_groups;           /* G: independent prompts; matching never crosses prompts    */
+  int32_t  paths_per_group;      /* N: parallel samples of one prompt (the paper's N)         */
+  int32_t  capacity;             /* L: tokens kept per path; a path at L builds no more drafts
+                                    but is still searched by the others                      */
+  int32_t  vocab;                /* V: tokens must lie in [0, V)                              */
+  int32_t  k_max;                /* largest query suffix length that will be asked for        */
+  int32_t  max_draft_len;        /* D: the paper's maximum draft token length                 */
+  int32_t  max_append;           /* most tokens a path may gain per sdms_accept commit        */
+  int32_t  dag_nodes_per_layer;  /* B: nodes kept per layer in the DAG export, 0 = no export  */
+  int32_t  dag_edges_per_node;   /* Ke: out-edges kept per exported node                      */
+  int32_t  search_mode;          /* 0: walk to the best successor of the current node;
+                                    1: best node of each layer regardless of the previous one */
+  float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
+  int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
+} sdms_config;
+
+/* Bytes of device workspace a context with this configuration needs (host only,
+ * no CUDA call). */
+int sdms_workspace_bytes(const sdms_config* cfg, size_t* bytes);
+
+/* Create a context over caller-owned device memory.  Zero-fills the workspace on
+ * the default stream and waits for it.  Starts with all paths empty. */
+int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ctx** out);
+
+/* Forget every token (same effect as destroying and re-creating the context). */
+int sdms_reset(sdms_ctx* ctx, void* stream);
+
+/* Frees the host object only. */
+int sdms_destroy(sdms_ctx* ctx);
+
+/*
+ * State update ("Dynamic Draft Pool Construction": the partial sequences
+ * y_i^{1:t} grow every step).  Path p gains d_tokens[p][0 .. d_counts[p]) with
+ * the model's log-probability of each of those tokens (the p_theta of Eq. 5 is
+ * exp(logprob), stored as round_half_even(exp(logprob) * 2^30) in [0, 2^30]).
+ * Rows are `row_width` wide (1 <= row_width; any width, e.g. a prefill chunk).
+ * The new positions' n-grams (n = 1..k_max) enter the prompt's hash tables.
+ * Clamping: count outside [0, row_width] -> BAD_COUNT; beyond capacity ->
+ * CAPACITY, truncated; token outside [0, V) -> BAD_TOKEN, the path keeps the
+ * tokens before it.
+ */
+int sdms_append(sdms_ctx* ctx, const int32_t* d_tokens, const float* d_logprobs,
+                const int32_t* d_counts, int32_t row_width, void* stream);
+
+/*
+ * One draft per path (Algorithm 1 with exact matching, epsilon = 0):
+ *   query      the last k tokens of path i                       (1 <= k <= k_max)
+ *   match      Eq. 3: every end position e in every other path j of the same
+ *              prompt with y_j[e-k+1..e] equal to the query and e <= len_j - 2
+ *   candidates the up to D tokens that follow each match
+ *   DAG        layer d = distinct d-th followers; edge (u,v) between layers d-1
+ *              and d accumulates S = sum of fixed-point probabilities of v and
+ *              cnt = number of instances; Eq. 5 weight = alpha*S/2^30 + (1-alpha)*cnt
+ *              evaluated in binary64; a node's score is Eq. 5 on its summed in-edges
+ *   search     greedy walk from the query's last token, ties to the smaller token
+ *              id, until D tokens or a node without successor.
+ * Outputs: d_draft_tok [P][D] (unused entries -1), d_draft_len [P],
+ * d_draft_score [P][D] = score of each chosen node, d_draft_edge_w [P][D] =
+ * weight of the edge taken (unused 0; either float array may be NULL).
+ * Paths shorter than k, full paths and paths without a match get draft_len 0.
+ * Read-only with respect to the path histories.
+ */
+int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d_draft_len,
+                      float* d_draft_score, float* d_draft_edge_w, void* stream);
+
+/*
+ * "Draft acceptance": d_accept_len[p] = longest t <= d_draft_len[p] with
+ * d_draft_tok[p][0..t) == d_sampled[p][0..t), d_sampled being [P][D+1] tokens
+ * sampled by the model at the draft positions plus one more.
+ * If d_sampled_logprobs ([P][D+1]) is not NULL the call also commits: path p
+ * appends d_sampled[p][0 .. min(tau_p + 1, max_append)) exactly as sdms_append
+ * would, except that reaching capacity silently truncates.
+ */
+int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draft_len,
+                const int32_t* d_sampled, const float* d_sampled_logprobs,
+                int32_t* d_accept_len, void* stream);
+
+/* ---- inspection (used by the parity tests; not part of a decode step) ------- */
+
+/* Matches of the last sdms_build_drafts: d_offsets [P+1] (exclusive prefix sums)
+ * and d_gpos = global positions j*L + e of every match, grouped per query path,
+ * in no particular order inside a group.  At most `cap` positions are written;
+ * d_offsets always holds the true counts. */
+int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t cap, void* stream);
+
+/* DAG export of the last sdms_build_drafts (needs dag_nodes_per_layer > 0).
+ * Layer index d-1 for d = 1..D.  Per layer the B best nodes by (score desc,
+ * token asc): node_tok/node_S/node_cnt [P][D][B] (unused token -1), the true
+ * number of nodes node_count [P][D].  Per kept node of layer d its Ke best
+ * out-edges to layer d+1 by (weight desc, destination asc): edge_dst/edge_S/
+ * edge_cnt [P][D][B][Ke] and the true out-degree out_degree [P][D][B].
+ * S values are int64 sums of fixed-point probabilities. */
+int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t* d_node_cnt,
+                 int32_t* d_node_count, int32_t* d_edge_dst, int64_t* d_edge_S,
+                 int32_t* d_edge_cnt, int32_t* d_out_degree, void* stream);
+
+/* Copies the stores: d_tok / d_pq [P][L], d_len [P] (any may be NULL). */
+int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_t* d_len, void* stream);
+
+/* Waits for `stream`, returns the status bits in *host_flags and clears them. */
+int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream);
+
+/* ---- measurement hooks (no counterpart in the paper) ----------------------- */
+
+#define SDMS_KERNEL_APPEND 0
+#define SDMS_KERNEL_PROBE  1
+#define SDMS_KERNEL_SCAN   2
+#define SDMS_KERNEL_DAG    3
+#define SDMS_KERNEL_ACCEPT 4
+#define SDMS_NUM_KERNELS   5
+
+/* Number of kernels this context has launched since creation. */
+int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches);
+
+/* When enabled every kernel launch is bracketed by CUDA events on its stream. */
+int sdms_profile_enable(sdms_ctx* ctx, int32_t on);
+
+/* Waits for the recorded events; adds up per kernel the elapsed milliseconds and
+ * the launches since the last read (arrays of SDMS_NUM_KERNELS). */
+int sdms_profile_read(sdms_ctx* ctx, float* ms, uint64_t* launches);
+
+const char* sdms_strerror(int code);
+const char* sdms_kernel_name(int kernel);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SDMS_H_ */

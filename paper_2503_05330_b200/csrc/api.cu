@@ -1,0 +1,307 @@
+// C entry points: argument checks, workspace carving, launches, measurement hooks.
+#include <new>
+#include <vector>
+#include <cstring>
+#include "sdms_internal.h"
+
+using namespace sdms;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t tok, pq, len, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, matches;
+  size_t x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
+  size_t total;
+  uint32_t table_cap;
+  int64_t match_cap;
+};
+
+int check_config(const sdms_config* c) {
+  if (!c || c->struct_size != sizeof(sdms_config)) return SDMS_ERR_INVALID_ARG;
+  if (c->num_groups < 1 || c->paths_per_group < 1 || c->paths_per_group > SDMS_MAX_PATHS_PER_GROUP)
+    return SDMS_ERR_INVALID_ARG;
+  if (c->capacity < 2 || c->vocab < 1 || c->vocab > (1 << 26)) return SDMS_ERR_INVALID_ARG;
+  if (c->k_max < 1 || c->k_max > SDMS_MAX_K) return SDMS_ERR_INVALID_ARG;
+  if (c->max_draft_len < 1 || c->max_draft_len > SDMS_MAX_DRAFT) return SDMS_ERR_INVALID_ARG;
+  if (c->max_append < 1 || c->max_append > c->max_draft_len + 1) return SDMS_ERR_INVALID_ARG;
+  if (c->dag_nodes_per_layer < 0 || c->dag_nodes_per_layer > SDMS_MAX_DAG_NODES) return SDMS_ERR_INVALID_ARG;
+  if (c->dag_nodes_per_layer > 0 && (c->dag_edges_per_node < 1 || c->dag_edges_per_node > SDMS_MAX_DAG_EDGES))
+    return SDMS_ERR_INVALID_ARG;
+  if (c->search_mode != 0 && c->search_mode != 1) return SDMS_ERR_INVALID_ARG;
+  if (!(c->alpha >= 0.0f && c->alpha <= 1.0f)) return SDMS_ERR_INVALID_ARG;
+  if (c->match_capacity < 0 || c->match_capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;
+  const int64_t P = (int64_t)c->num_groups * c->paths_per_group;
+  if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
+  return SDMS_OK;
+}
+
+Layout make_layout(const sdms_config* c) {
+  Layout l;
+  const size_t P = (size_t)c->num_groups * c->paths_per_group;
+  const size_t L = c->capacity, D = c->max_draft_len, B = c->dag_nodes_per_layer, Ke = c->dag_edges_per_node;
+  // twice as many buckets as positions a prompt can hold: load factor <= 1/2
+  uint32_t cap = 64;
+  while ((size_t)cap < 2 * (size_t)c->paths_per_group * L) cap <<= 1;
+  l.table_cap = cap;
+  int64_t mc = c->match_capacity;
+  if (mc == 0) {
+    const int64_t worst = (int64_t)P * c->paths_per_group * (int64_t)L;   // every position matches every query
+    mc = worst < (1LL << 26) ? worst : (1LL << 26);
+  }
+  l.match_cap = mc;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  l.tok = take((P * L + SDMS_MAX_DRAFT + 8) * 4);
+  l.pq = take((P * L + SDMS_MAX_DRAFT + 8) * 4);
+  l.len = take(P * 4);
+  l.status = take(4);
+  l.index = take((size_t)c->num_groups * c->k_max * cap * kBucketWords * 4);
+  l.q_fp = take(P * 4); l.q_mode = take(P * 4); l.q_reserved = take(P * 4);
+  l.q_off = take(P * 4); l.q_cursor = take(P * 4);
+  l.g_nscan = take((size_t)c->num_groups * 4);
+  l.matches = take((size_t)mc * 4);
+  l.x_node_tok = take(P * D * B * 4); l.x_node_S = take(P * D * B * 8); l.x_node_cnt = take(P * D * B * 4);
+  l.x_node_count = take(P * D * 4);
+  l.x_edge_dst = take(P * D * B * Ke * 4); l.x_edge_S = take(P * D * B * Ke * 8);
+  l.x_edge_cnt = take(P * D * B * Ke * 4); l.x_out_degree = take(P * D * B * 4);
+  l.total = o;
+  return l;
+}
+
+struct EventPair { cudaEvent_t a, b; int kernel; };
+
+}  // namespace
+
+struct sdms_ctx {
+  sdms_config cfg;
+  Layout lay;
+  Dev dev;
+  unsigned char* ws;
+  uint64_t launches;
+  bool profiling;
+  bool built;
+  std::vector<EventPair> pending;
+  std::vector<EventPair> pool;
+  float prof_ms[SDMS_NUM_KERNELS];
+  uint64_t prof_n[SDMS_NUM_KERNELS];
+};
+
+namespace {
+
+template <class F>
+int timed(sdms_ctx* ctx, int kernel, cudaStream_t stream, F launch) {
+  EventPair ev{};
+  if (ctx->profiling) {
+    if (!ctx->pool.empty()) { ev = ctx->pool.back(); ctx->pool.pop_back(); }
+    else if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) return SDMS_ERR_CUDA;
+    ev.kernel = kernel;
+    cudaEventRecord(ev.a, stream);
+  }
+  const cudaError_t e = launch();
+  ++ctx->launches;
+  if (ctx->profiling) { cudaEventRecord(ev.b, stream); ctx->pending.push_back(ev); }
+  return e == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sdms_workspace_bytes(const sdms_config* cfg, size_t* bytes) {
+  if (!bytes) return SDMS_ERR_INVALID_ARG;
+  const int rc = check_config(cfg);
+  if (rc != SDMS_OK) return rc;
+  *bytes = make_layout(cfg).total;
+  return SDMS_OK;
+}
+
+int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ctx** out) {
+  if (!out) return SDMS_ERR_INVALID_ARG;
+  *out = nullptr;
+  const int rc = check_config(cfg);
+  if (rc != SDMS_OK) return rc;
+  if (!d_workspace || ((uintptr_t)d_workspace & (kAlign - 1))) return SDMS_ERR_INVALID_ARG;
+  const Layout lay = make_layout(cfg);
+  if (bytes < lay.total) return SDMS_ERR_WORKSPACE_TOO_SMALL;
+  if (dag_kernel_setup() != cudaSuccess) return SDMS_ERR_CUDA;
+  if (cudaMemsetAsync(d_workspace, 0, lay.total, 0) != cudaSuccess) return SDMS_ERR_CUDA;
+  if (cudaStreamSynchronize(0) != cudaSuccess) return SDMS_ERR_CUDA;
+  sdms_ctx* ctx = new (std::nothrow) sdms_ctx();
+  if (!ctx) return SDMS_ERR_BAD_STATE;
+  ctx->cfg = *cfg;
+  ctx->lay = lay;
+  ctx->ws = static_cast<unsigned char*>(d_workspace);
+  ctx->launches = 0;
+  ctx->profiling = false;
+  ctx->built = false;
+  std::memset(ctx->prof_ms, 0, sizeof(ctx->prof_ms));
+  std::memset(ctx->prof_n, 0, sizeof(ctx->prof_n));
+  Dev& d = ctx->dev;
+  d.G = cfg->num_groups; d.N = cfg->paths_per_group; d.L = cfg->capacity; d.V = cfg->vocab;
+  d.k_max = cfg->k_max; d.D = cfg->max_draft_len; d.max_append = cfg->max_append;
+  d.B = cfg->dag_nodes_per_layer; d.Ke = cfg->dag_nodes_per_layer ? cfg->dag_edges_per_node : 0;
+  d.mode = cfg->search_mode; d.P = d.G * d.N;
+  d.alpha = (double)cfg->alpha;
+  d.table_cap = lay.table_cap; d.match_cap = lay.match_cap;
+  unsigned char* w = ctx->ws;
+  d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len);
+  d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);
+  d.q_fp = (uint32_t*)(w + lay.q_fp); d.q_mode = (int32_t*)(w + lay.q_mode);
+  d.q_reserved = (int32_t*)(w + lay.q_reserved); d.q_off = (int32_t*)(w + lay.q_off);
+  d.q_cursor = (int32_t*)(w + lay.q_cursor); d.g_nscan = (int32_t*)(w + lay.g_nscan);
+  d.matches = (int32_t*)(w + lay.matches);
+  d.x_node_tok = (int32_t*)(w + lay.x_node_tok); d.x_node_S = (int64_t*)(w + lay.x_node_S);
+  d.x_node_cnt = (int32_t*)(w + lay.x_node_cnt); d.x_node_count = (int32_t*)(w + lay.x_node_count);
+  d.x_edge_dst = (int32_t*)(w + lay.x_edge_dst); d.x_edge_S = (int64_t*)(w + lay.x_edge_S);
+  d.x_edge_cnt = (int32_t*)(w + lay.x_edge_cnt); d.x_out_degree = (int32_t*)(w + lay.x_out_degree);
+  *out = ctx;
+  return SDMS_OK;
+}
+
+int sdms_reset(sdms_ctx* ctx, void* stream) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the path store need not be cleared: lengths say what is valid
+  const Layout& l = ctx->lay;
+  if (cudaMemsetAsync(ctx->ws + l.len, 0, l.matches - l.len, st) != cudaSuccess) return SDMS_ERR_CUDA;
+  ctx->built = false;
+  return SDMS_OK;
+}
+
+int sdms_destroy(sdms_ctx* ctx) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  for (auto& e : ctx->pending) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  for (auto& e : ctx->pool) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  delete ctx;
+  return SDMS_OK;
+}
+
+int sdms_append(sdms_ctx* ctx, const int32_t* d_tokens, const float* d_logprobs, const int32_t* d_counts,
+                int32_t row_width, void* stream) {
+  if (!ctx || !d_tokens || !d_logprobs || !d_counts || row_width < 1) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  return timed(ctx, SDMS_KERNEL_APPEND, st,
+               [&] { return launch_append(ctx->dev, d_tokens, d_logprobs, d_counts, row_width, st); });
+}
+
+int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d_draft_len,
+                      float* d_draft_score, float* d_draft_edge_w, void* stream) {
+  if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
+  if (k < 1 || k > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, st); });
+  if (rc != SDMS_OK) return rc;
+  rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+  if (rc != SDMS_OK) return rc;
+  rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
+    return launch_dag(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+  if (rc == SDMS_OK) ctx->built = true;
+  return rc;
+}
+
+int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draft_len, const int32_t* d_sampled,
+                const float* d_sampled_logprobs, int32_t* d_accept_len, void* stream) {
+  if (!ctx || !d_draft_tok || !d_draft_len || !d_sampled || !d_accept_len) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  return timed(ctx, SDMS_KERNEL_ACCEPT, st, [&] {
+    return launch_accept(ctx->dev, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, st); });
+}
+
+int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t cap, void* stream) {
+  if (!ctx || !d_offsets || (!d_gpos && cap)) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->built) return SDMS_ERR_BAD_STATE;
+  const cudaError_t e = launch_compact_matches(ctx->dev, d_offsets, d_gpos, cap, (cudaStream_t)stream);
+  ++ctx->launches;
+  return e == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
+int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t* d_node_cnt,
+                 int32_t* d_node_count, int32_t* d_edge_dst, int64_t* d_edge_S, int32_t* d_edge_cnt,
+                 int32_t* d_out_degree, void* stream) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->built || ctx->dev.B == 0) return SDMS_ERR_BAD_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dev& d = ctx->dev;
+  const size_t nb = (size_t)d.P * d.D * d.B, ne = nb * d.Ke;
+  bool ok = true;
+  auto copy = [&](void* dst, const void* src, size_t bytes) {
+    if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  };
+  copy(d_node_tok, d.x_node_tok, nb * 4); copy(d_node_S, d.x_node_S, nb * 8); copy(d_node_cnt, d.x_node_cnt, nb * 4);
+  copy(d_node_count, d.x_node_count, (size_t)d.P * d.D * 4);
+  copy(d_edge_dst, d.x_edge_dst, ne * 4); copy(d_edge_S, d.x_edge_S, ne * 8); copy(d_edge_cnt, d.x_edge_cnt, ne * 4);
+  copy(d_out_degree, d.x_out_degree, nb * 4);
+  return ok ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
+int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_t* d_len, void* stream) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dev& d = ctx->dev;
+  const size_t n = (size_t)d.P * d.L * 4;
+  bool ok = true;
+  if (d_tok) ok = ok && cudaMemcpyAsync(d_tok, d.tok, n, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (d_pq) ok = ok && cudaMemcpyAsync(d_pq, d.pq, n, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (d_len) ok = ok && cudaMemcpyAsync(d_len, d.len, (size_t)d.P * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  return ok ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
+int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream) {
+  if (!ctx || !host_flags) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(host_flags, ctx->dev.status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SDMS_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->dev.status, 0, 4, st) != cudaSuccess) return SDMS_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SDMS_ERR_CUDA;
+  return SDMS_OK;
+}
+
+int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches) {
+  if (!ctx || !launches) return SDMS_ERR_INVALID_ARG;
+  *launches = ctx->launches;
+  return SDMS_OK;
+}
+
+int sdms_profile_enable(sdms_ctx* ctx, int32_t on) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  ctx->profiling = on != 0;
+  return SDMS_OK;
+}
+
+int sdms_profile_read(sdms_ctx* ctx, float* ms, uint64_t* launches) {
+  if (!ctx || !ms || !launches) return SDMS_ERR_INVALID_ARG;
+  for (auto& e : ctx->pending) {
+    float t = 0.f;
+    if (cudaEventSynchronize(e.b) != cudaSuccess || cudaEventElapsedTime(&t, e.a, e.b) != cudaSuccess)
+      return SDMS_ERR_CUDA;
+    ctx->prof_ms[e.kernel] += t;
+    ctx->prof_n[e.kernel] += 1;
+    ctx->pool.push_back(e);
+  }
+  ctx->pending.clear();
+  for (int k = 0; k < SDMS_NUM_KERNELS; ++k) {
+    ms[k] = ctx->prof_ms[k]; launches[k] = ctx->prof_n[k];
+    ctx->prof_ms[k] = 0.f; ctx->prof_n[k] = 0;
+  }
+  return SDMS_OK;
+}
+
+const char* sdms_strerror(int code) {
+  switch (code) {
+    case SDMS_OK: return "ok";
+    case SDMS_ERR_INVALID_ARG: return "invalid argument";
+    case SDMS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SDMS_ERR_CUDA: return "CUDA call failed";
+    case SDMS_ERR_BAD_STATE: return "call not valid in this state";
+    default: return "unknown error";
+  }
+}
+
+const char* sdms_kernel_name(int kernel) {
+  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept"};
+  return kernel >= 0 && kernel < SDMS_NUM_KERNELS ? names[kernel] : "?";
+}
+
+}  // extern "C"

@@ -1,0 +1,218 @@
+// State update and acceptance kernels.
+//
+// append_kernel : one CTA per path; writes tokens and fixed-point probabilities
+//                 into the path store and inserts the n-grams (n = 1..k_max) that
+//                 end at each new position into the prompt's hash tables.
+// accept_kernel : one CTA per path; longest accepted prefix of the draft
+//                 ("Draft acceptance"), optionally followed by the same append.
+#include "sdms_internal.h"
+
+namespace sdms {
+
+namespace {
+
+struct dd { double hi, lo; };
+
+__device__ __forceinline__ dd two_sum(double a, double b) {
+  double s = __dadd_rn(a, b);
+  double bb = __dsub_rn(s, a);
+  double e = __dadd_rn(__dsub_rn(a, __dsub_rn(s, bb)), __dsub_rn(b, bb));
+  return {s, e};
+}
+__device__ __forceinline__ dd quick_two_sum(double a, double b) {   // |a| >= |b|
+  double s = __dadd_rn(a, b);
+  return {s, __dsub_rn(b, __dsub_rn(s, a))};
+}
+__device__ __forceinline__ dd two_prod(double a, double b) {
+  double p = __dmul_rn(a, b);
+  return {p, __fma_rn(a, b, -p)};
+}
+__device__ __forceinline__ dd dd_add(dd a, dd b) {
+  dd s = two_sum(a.hi, b.hi);
+  dd t = two_sum(a.lo, b.lo);
+  s.lo = __dadd_rn(s.lo, t.hi);
+  s = quick_two_sum(s.hi, s.lo);
+  s.lo = __dadd_rn(s.lo, t.lo);
+  return quick_two_sum(s.hi, s.lo);
+}
+__device__ __forceinline__ dd dd_mul(dd a, dd b) {
+  dd p = two_prod(a.hi, b.hi);
+  p.lo = __dadd_rn(p.lo, __dadd_rn(__dmul_rn(a.hi, b.lo), __dmul_rn(a.lo, b.hi)));
+  return quick_two_sum(p.hi, p.lo);
+}
+__device__ __forceinline__ dd dd_div_small(dd a, double n) {        // n a small positive integer
+  double q = __ddiv_rn(a.hi, n);
+  double rem = __fma_rn(-q, n, a.hi);                                // exact remainder
+  double ql = __ddiv_rn(__dadd_rn(rem, a.lo), n);
+  return quick_two_sum(q, ql);
+}
+
+// round_half_even(exp(lp) * 2^30) clamped to [0, 2^30].  exp is evaluated in
+// double-double arithmetic (about 100 bits) so that the rounding decision is
+// that of the exact real number: argument reduction by a split ln 2, Taylor
+// series of exp on |r| <= ln2/2, scaling by a power of two.
+__device__ int32_t prob_to_fixed(float lp, uint32_t* st) {
+  const int32_t one = 1 << 30;
+  if (lp != lp) { *st |= SDMS_STATUS_BAD_LOGPROB; return 0; }
+  if (lp >= 0.0f) return one;
+  if (lp < -40.0f) return 0;                       // exp(-40) * 2^30 < 1e-8
+  const double x = (double)lp;
+  const double ln2_hi = 6.93147180369123816490e-01;  // 32 significant bits: m * ln2_hi is exact
+  const double ln2_lo = 1.90821492927058770002e-10;  // ln 2 - ln2_hi
+  const double m = rint(__dmul_rn(x, 1.44269504088896338700e+00));
+  dd r = {__fma_rn(-m, ln2_hi, x), 0.0};             // exact: the difference fits in 53 bits
+  dd ml = two_prod(m, ln2_lo);
+  r = dd_add(r, dd{-ml.hi, -ml.lo});
+  dd sum = {1.0, 0.0};
+  dd term = {1.0, 0.0};
+  for (int n = 1; n <= 24; ++n) {
+    term = dd_div_small(dd_mul(term, r), (double)n);
+    sum = dd_add(sum, term);
+  }
+  const int sh = (int)m + 30;
+  const double yh = ldexp(sum.hi, sh), yl = ldexp(sum.lo, sh);
+  long long n = __double2ll_rn(yh);
+  const double d = __dadd_rn(__dsub_rn(yh, (double)n), yl);
+  if (d > 0.5 || (d == 0.5 && (n & 1))) ++n;
+  else if (d < -0.5 || (d == -0.5 && (n & 1))) --n;
+  if (n < 0) n = 0;
+  if (n > one) n = one;
+  return (int32_t)n;
+}
+
+// Adds one occurrence of an n-gram (hash h) ending at prompt-local position lpos.
+__device__ void index_insert(const Dev& s, int g, int n, uint64_t h, uint32_t lpos, uint32_t* st) {
+  uint32_t* table = index_table(s, g, n);
+  const uint32_t fp = gram_fp(h);
+  uint32_t b = gram_bucket(h, s.table_cap);
+  for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
+    uint32_t* bucket = table + (size_t)b * kBucketWords;
+    const uint32_t old = atomicCAS(&bucket[0], 0u, fp);
+    if (old == 0u || old == fp) {
+      const uint32_t slot = atomicAdd(&bucket[1], 1u);
+      if (slot < (uint32_t)kInlineSlots) bucket[2 + slot] = lpos;
+      return;
+    }
+    b = (b + 1) & (s.table_cap - 1);
+  }
+  *st |= SDMS_STATUS_INDEX_FULL;
+}
+
+// Block-cooperative append of n validated tokens to path p whose length is len0.
+__device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_t* in_tok,
+                              const float* in_lp, uint32_t* st) {
+  int32_t* tok = s.tok + (size_t)p * s.L;
+  int32_t* pq = s.pq + (size_t)p * s.L;
+  for (int a = threadIdx.x; a < n; a += blockDim.x) {
+    tok[len0 + a] = in_tok[a];
+    pq[len0 + a] = prob_to_fixed(in_lp[a], st);
+  }
+  const int g = p / s.N;
+  const uint32_t lbase = (uint32_t)(p - g * s.N) * (uint32_t)s.L;
+  for (int w = threadIdx.x; w < n * s.k_max; w += blockDim.x) {
+    const int a = w / s.k_max, nn = w % s.k_max + 1;
+    const int pos = len0 + a;
+    if (pos + 1 < nn) continue;
+    uint64_t h = gram_init(nn);
+    for (int t = pos - nn + 1; t <= pos; ++t)
+      h = gram_step(h, t < len0 ? tok[t] : in_tok[t - len0]);   // old tokens from the store, new from the input
+    index_insert(s, g, nn, gram_final(h), lbase + (uint32_t)pos, st);
+  }
+}
+
+__global__ void __launch_bounds__(128) append_kernel(Dev s, const int32_t* __restrict__ tokens,
+                                                     const float* __restrict__ logprobs,
+                                                     const int32_t* __restrict__ counts, int row_width) {
+  const int p = blockIdx.x;
+  __shared__ int sh_len0, sh_n, sh_bad;
+  __shared__ uint32_t sh_st;
+  if (threadIdx.x == 0) {
+    uint32_t st = 0;
+    int n = counts[p];
+    if (n < 0) { st |= SDMS_STATUS_BAD_COUNT; n = 0; }
+    if (n > row_width) { st |= SDMS_STATUS_BAD_COUNT; n = row_width; }
+    const int len0 = s.len[p];
+    if (n > s.L - len0) { st |= SDMS_STATUS_CAPACITY; n = s.L - len0; }
+    sh_len0 = len0; sh_n = n; sh_bad = n; sh_st = st;
+  }
+  __syncthreads();
+  const int32_t* in_tok = tokens + (size_t)p * row_width;
+  const float* in_lp = logprobs + (size_t)p * row_width;
+  for (int a = threadIdx.x; a < sh_n; a += blockDim.x) {
+    const int32_t t = in_tok[a];
+    if (t < 0 || t >= s.V) atomicMin(&sh_bad, a);
+  }
+  __syncthreads();
+  uint32_t st = 0;
+  const int n = sh_bad;
+  if (threadIdx.x == 0 && n < sh_n) st |= SDMS_STATUS_BAD_TOKEN;
+  append_tokens(s, p, sh_len0, n, in_tok, in_lp, &st);
+  if (st) atomicOr(&sh_st, st);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s.len[p] = sh_len0 + n;
+    if (sh_st) atomicOr(s.status, sh_st);
+  }
+}
+
+__global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __restrict__ draft_tok,
+                                                     const int32_t* __restrict__ draft_len,
+                                                     const int32_t* __restrict__ sampled,
+                                                     const float* __restrict__ sampled_lp,
+                                                     int32_t* __restrict__ accept_len) {
+  const int p = blockIdx.x;
+  __shared__ int sh_len0, sh_n, sh_bad;
+  __shared__ uint32_t sh_st;
+  const int32_t* smp = sampled + (size_t)p * (s.D + 1);
+  if (threadIdx.x < 32) {
+    int dl = draft_len[p];
+    dl = dl < 0 ? 0 : (dl > s.D ? s.D : dl);
+    const int d = threadIdx.x;
+    const bool differs = d >= dl || draft_tok[(size_t)p * s.D + d] != smp[d];
+    const unsigned first = __ffs(__ballot_sync(0xffffffffu, differs));   // 0 only if all 32 lanes agree
+    const int tau = first ? (int)first - 1 : 32;
+    if (d == 0) {
+      accept_len[p] = tau;
+      int n = 0, len0 = 0;
+      if (sampled_lp) {
+        len0 = s.len[p];
+        n = min(min(tau + 1, s.max_append), s.L - len0);
+      }
+      sh_len0 = len0; sh_n = n; sh_bad = n; sh_st = 0;
+    }
+  }
+  if (!sampled_lp) return;
+  __syncthreads();
+  for (int a = threadIdx.x; a < sh_n; a += blockDim.x) {
+    const int32_t t = smp[a];
+    if (t < 0 || t >= s.V) atomicMin(&sh_bad, a);
+  }
+  __syncthreads();
+  uint32_t st = 0;
+  const int n = sh_bad;
+  if (threadIdx.x == 0 && n < sh_n) st |= SDMS_STATUS_BAD_TOKEN;
+  append_tokens(s, p, sh_len0, n, smp, sampled_lp + (size_t)p * (s.D + 1), &st);
+  if (st) atomicOr(&sh_st, st);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s.len[p] = sh_len0 + n;
+    if (sh_st) atomicOr(s.status, sh_st);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_append(const Dev& s, const int32_t* tokens, const float* logprobs, const int32_t* counts,
+                          int row_width, cudaStream_t stream) {
+  append_kernel<<<s.P, 128, 0, stream>>>(s, tokens, logprobs, counts, row_width);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t* draft_len,
+                          const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
+                          cudaStream_t stream) {
+  accept_kernel<<<s.P, 128, 0, stream>>>(s, draft_tok, draft_len, sampled, sampled_lp, accept_len);
+  return cudaGetLastError();
+}
+
+}  // namespace sdms

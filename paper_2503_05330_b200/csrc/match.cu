@@ -1,0 +1,271 @@
+// Cross-path suffix match (Eq. 3).
+//
+// probe_kernel : one thread per query path.  Hashes the path's last k tokens,
+//                finds the bucket of that k-gram in the prompt's table and reads
+//                its occurrence count.  The count is an upper bound on the number
+//                of matches, so it sizes the query's slice of the match list.
+//                Up to kInlineSlots occurrences are stored in the bucket itself:
+//                such queries are answered here, from one 32-byte sector.  The
+//                others are handed to the scan.
+// scan_kernel  : one CTA per 1024-token tile of one path.  The tile is staged in
+//                shared memory with 128-bit loads; the fingerprints of the
+//                prompt's scan queries sit in a small shared hash set; every
+//                position hashes its k-gram, probes the set and verifies hits
+//                token by token.  Matches are counted per query in shared
+//                memory, one global atomic per (CTA, query) reserves the output
+//                range, and a second pass writes the positions.
+#include "sdms_internal.h"
+
+namespace sdms {
+
+namespace {
+
+constexpr int kProbeThreads = 1024;
+
+__device__ __forceinline__ long long block_exclusive_scan(long long v, long long* warp_tot, long long* total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  long long x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) warp_tot[wid] = x;
+  __syncthreads();
+  if (wid == 0) {
+    long long w = lane < (int)(blockDim.x >> 5) ? warp_tot[lane] : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long y = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += y;
+    }
+    warp_tot[lane] = w;                       // inclusive over warps
+  }
+  __syncthreads();
+  const long long before = wid ? warp_tot[wid - 1] : 0;
+  *total = warp_tot[(blockDim.x >> 5) - 1];
+  return before + x - v;
+}
+
+__global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
+  __shared__ long long warp_tot[32];
+  __shared__ long long sh_carry;
+  for (int g = threadIdx.x; g < s.G; g += blockDim.x) s.g_nscan[g] = 0;
+  if (threadIdx.x == 0) sh_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < s.P; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    int mode = Q_NONE;
+    uint32_t fp = 0, count = 0;
+    const uint32_t* bucket = nullptr;
+    int len_i = 0, g = 0;
+    if (i < s.P) {
+      len_i = s.len[i];
+      g = i / s.N;
+      if (len_i >= k && len_i < s.L) {
+        const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
+        uint64_t h = gram_init(k);
+        for (int t = 0; t < k; ++t) h = gram_step(h, q[t]);
+        h = gram_final(h);
+        fp = gram_fp(h);
+        const uint32_t* table = index_table(s, g, k);
+        uint32_t b = gram_bucket(h, s.table_cap);
+        for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
+          const uint32_t* cand = table + (size_t)b * kBucketWords;
+          const uint32_t w0 = cand[0];
+          if (w0 == fp) { bucket = cand; break; }
+          if (w0 == 0u) break;
+          b = (b + 1) & (s.table_cap - 1);
+        }
+        if (bucket) {
+          count = bucket[1];
+          mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
+        }
+      }
+    }
+    long long total;
+    const long long off = sh_carry + block_exclusive_scan((long long)count, warp_tot, &total);
+    if (mode != Q_NONE && off + (long long)count > s.match_cap) {
+      mode = Q_NONE;
+      atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+    }
+    if (i < s.P) {
+      int written = 0;
+      if (mode == Q_INLINE) {
+        const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
+        for (uint32_t sl = 0; sl < count; ++sl) {
+          const uint32_t lpos = bucket[2 + sl];
+          const int j = g * s.N + (int)(lpos / (uint32_t)s.L);
+          const int e = (int)(lpos % (uint32_t)s.L);
+          if (j == i || e > s.len[j] - 2) continue;
+          const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
+          bool same = true;
+          for (int t = 0; t < k; ++t) same = same && (c[t] == q[t]);
+          if (same) s.matches[off + written++] = j * s.L + e;
+        }
+      } else if (mode == Q_SCAN) {
+        atomicAdd(&s.g_nscan[g], 1);
+      }
+      s.q_fp[i] = fp;
+      s.q_mode[i] = mode;
+      s.q_reserved[i] = mode == Q_NONE ? 0 : (int32_t)count;
+      s.q_off[i] = (int32_t)(off < s.match_cap ? off : s.match_cap);
+      s.q_cursor[i] = written;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) sh_carry += total;
+    __syncthreads();
+  }
+}
+
+constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
+
+__global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
+  const int j = blockIdx.y;                    // path whose history is scanned
+  const int g = j / s.N;
+  if (s.g_nscan[g] == 0) return;
+  const int len_j = s.len[j];
+  const int t0 = blockIdx.x * kScanTile;
+  const int e_lo = max(t0, k - 1);
+  const int e_hi = min(t0 + kScanTile - 1, len_j - 2);     // inclusive; needs one follower
+  if (e_lo > e_hi) return;
+
+  __shared__ __align__(16) int32_t sh_tok[kHalo + kScanTile];
+  __shared__ int32_t sh_qid[SDMS_MAX_PATHS_PER_GROUP];
+  __shared__ uint32_t sh_qfp[SDMS_MAX_PATHS_PER_GROUP];
+  __shared__ int32_t sh_cnt[SDMS_MAX_PATHS_PER_GROUP];
+  __shared__ int32_t sh_base[SDMS_MAX_PATHS_PER_GROUP];
+  __shared__ int32_t sh_set[kSetSlots];
+  __shared__ int sh_nq;
+
+  if (threadIdx.x == 0) sh_nq = 0;
+  for (int x = threadIdx.x; x < kSetSlots; x += blockDim.x) sh_set[x] = -1;
+  // stage the tile (and the tokens just before it)
+  const int32_t* row = s.tok + (size_t)j * s.L;
+  const int hi = min(t0 + kScanTile, s.L);
+  if ((s.L & 3) == 0) {
+    const int4* src = reinterpret_cast<const int4*>(row + t0);
+    int4* dst = reinterpret_cast<int4*>(sh_tok + kHalo);
+    for (int x = threadIdx.x; x < (hi - t0) / 4; x += blockDim.x) dst[x] = __ldg(src + x);
+  } else {
+    for (int x = threadIdx.x; x < hi - t0; x += blockDim.x) sh_tok[kHalo + x] = __ldg(row + t0 + x);
+  }
+  for (int x = threadIdx.x; x < kHalo; x += blockDim.x) {
+    const int idx = t0 - kHalo + x;
+    sh_tok[x] = idx >= 0 ? __ldg(row + idx) : -1;
+  }
+  __syncthreads();
+  // the prompt's scan queries (a path never searches itself)
+  for (int n = threadIdx.x; n < s.N; n += blockDim.x) {
+    const int i = g * s.N + n;
+    if (i != j && s.q_mode[i] == Q_SCAN) {
+      const int sl = atomicAdd(&sh_nq, 1);
+      const uint32_t fp = s.q_fp[i];
+      sh_qid[sl] = i;
+      sh_qfp[sl] = fp;
+      sh_cnt[sl] = 0;
+      uint32_t hs = (fp >> 1) & (kSetSlots - 1);
+      while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (kSetSlots - 1);
+    }
+  }
+  __syncthreads();
+  const int nq = sh_nq;
+  if (nq == 0) return;
+
+  constexpr int kPer = kScanTile / kScanThreads;
+  uint32_t fps[kPer];
+  bool any = false;
+#pragma unroll
+  for (int r = 0; r < kPer; ++r) {
+    const int e = t0 + r * kScanThreads + threadIdx.x;
+    fps[r] = 0;
+    if (e < e_lo || e > e_hi) continue;
+    const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
+    uint64_t h = gram_init(k);
+    for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
+    const uint32_t fp = gram_fp(gram_final(h));
+    fps[r] = fp;
+    uint32_t hs = (fp >> 1) & (kSetSlots - 1);
+    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
+      if (sh_qfp[sl] != fp) continue;
+      const int i = sh_qid[sl];
+      const int32_t* q = s.tok + (size_t)i * s.L + (s.len[i] - k);
+      bool same = true;
+      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(q + t));
+      if (same) { atomicAdd(&sh_cnt[sl], 1); any = true; }
+    }
+  }
+  if (!__syncthreads_or(any)) return;
+  for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
+    const int c = sh_cnt[sl];
+    sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
+    sh_cnt[sl] = 0;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < kPer; ++r) {
+    const uint32_t fp = fps[r];
+    if (fp == 0) continue;
+    const int e = t0 + r * kScanThreads + threadIdx.x;
+    const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
+    uint32_t hs = (fp >> 1) & (kSetSlots - 1);
+    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
+      if (sh_qfp[sl] != fp) continue;
+      const int i = sh_qid[sl];
+      const int32_t* q = s.tok + (size_t)i * s.L + (s.len[i] - k);
+      bool same = true;
+      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(q + t));
+      if (!same) continue;
+      const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
+      if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = j * s.L + e;
+      else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+    }
+  }
+}
+
+// Inspection only: packs the per-query slices of the match list.
+__global__ void __launch_bounds__(kProbeThreads) compact_matches_kernel(Dev s, int32_t* offsets, int32_t* gpos,
+                                                                        size_t cap) {
+  __shared__ long long warp_tot[32];
+  __shared__ long long sh_carry;
+  if (threadIdx.x == 0) sh_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < s.P; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    long long m = 0;
+    if (i < s.P && s.q_mode[i] != Q_NONE) m = min(s.q_cursor[i], s.q_reserved[i]);
+    long long total;
+    const long long off = sh_carry + block_exclusive_scan(m, warp_tot, &total);
+    if (i < s.P) offsets[i] = (int32_t)off;
+    __syncthreads();
+    if (threadIdx.x == 0) sh_carry += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) offsets[s.P] = (int32_t)sh_carry;
+  __syncthreads();
+  for (int i = 0; i < s.P; ++i) {
+    const int m = offsets[i + 1] - offsets[i];
+    for (int x = threadIdx.x; x < m; x += blockDim.x)
+      if ((size_t)(offsets[i] + x) < cap) gpos[offsets[i] + x] = s.matches[(size_t)s.q_off[i] + x];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
+  probe_kernel<<<1, kProbeThreads, 0, stream>>>(s, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
+  dim3 grid((s.L + kScanTile - 1) / kScanTile, s.P);
+  scan_kernel<<<grid, kScanThreads, 0, stream>>>(s, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream) {
+  compact_matches_kernel<<<1, kProbeThreads, 0, stream>>>(s, offsets, gpos, cap);
+  return cudaGetLastError();
+}
+
+}  // namespace sdms

@@ -1,0 +1,79 @@
+// Device-side view of a context and helpers shared by the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "sdms.h"
+
+namespace sdms {
+
+constexpr int kBucketWords = 8;        // one 32-byte sector: fingerprint, count, 6 positions
+constexpr int kInlineSlots = kBucketWords - 2;
+constexpr int kHalo = SDMS_MAX_K;      // tokens staged in front of a scan tile
+constexpr int kScanTile = 1024;        // history tokens per scan CTA
+constexpr int kScanThreads = 256;
+constexpr int kDagThreads = 256;
+constexpr int kDagCap = 1024;          // entries of the shared-memory node / edge tables
+
+enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
+
+// Everything a kernel needs, passed by value.
+struct Dev {
+  int32_t G, N, L, V, k_max, D, max_append, B, Ke, mode, P;
+  double alpha;
+  uint32_t table_cap;                  // buckets per (prompt, n) table, power of two
+  int64_t match_cap;
+  // path store
+  int32_t* tok;                        // [P][L]
+  int32_t* pq;                         // [P][L] fixed-point probabilities
+  int32_t* len;                        // [P]
+  uint32_t* status;
+  uint32_t* index;                     // [G][k_max][table_cap][kBucketWords]
+  // per-query scratch of the last build
+  uint32_t* q_fp;                      // [P]
+  int32_t* q_mode;                     // [P]
+  int32_t* q_reserved;                 // [P] match slots reserved (index count)
+  int32_t* q_off;                      // [P] start in `matches`
+  int32_t* q_cursor;                   // [P] matches written
+  int32_t* g_nscan;                    // [G] queries of the prompt that need the scan
+  int32_t* matches;                    // [match_cap] global positions j*L+e
+  // DAG export of the last build
+  int32_t* x_node_tok; int64_t* x_node_S; int32_t* x_node_cnt; int32_t* x_node_count;
+  int32_t* x_edge_dst; int64_t* x_edge_S; int32_t* x_edge_cnt; int32_t* x_out_degree;
+};
+
+// 64-bit hash of an n-gram, fed token by token (oldest first).
+__device__ __forceinline__ uint64_t gram_init(int n) {
+  return 0x9E3779B97F4A7C15ull * (uint64_t)(n + 1);
+}
+__device__ __forceinline__ uint64_t gram_step(uint64_t h, int32_t tok) {
+  h = (h ^ (uint64_t)(uint32_t)tok) * 0xFF51AFD7ED558CCDull;
+  return h ^ (h >> 29);
+}
+__device__ __forceinline__ uint64_t gram_final(uint64_t h) {
+  h *= 0xC4CEB9FE1A85EC53ull;
+  return h ^ (h >> 32);
+}
+// Non-zero 32-bit fingerprint (0 marks an empty bucket) and bucket number.
+__device__ __forceinline__ uint32_t gram_fp(uint64_t h) { return (uint32_t)(h >> 32) | 1u; }
+__device__ __forceinline__ uint32_t gram_bucket(uint64_t h, uint32_t cap) { return (uint32_t)h & (cap - 1); }
+
+__device__ __forceinline__ uint32_t* index_table(const Dev& s, int g, int n) {
+  return s.index + ((size_t)(g * s.k_max + (n - 1)) * s.table_cap) * kBucketWords;
+}
+
+// Eq. 5 on integer sums: alpha * S / 2^30 + (1 - alpha) * cnt, every operation
+// rounded on its own (no fused multiply-add), so that any two evaluations of
+// the same (S, cnt) agree bit for bit.
+__device__ __forceinline__ double eq5_weight(double alpha, unsigned long long S, unsigned int cnt) {
+  double t1 = __dmul_rn(alpha, (double)S);
+  t1 = __dmul_rn(t1, 1.0 / 1073741824.0);
+  double t2 = __dmul_rn(__dsub_rn(1.0, alpha), (double)cnt);
+  return __dadd_rn(t1, t2);
+}
+
+// Total order of the export and of the search: larger weight first, then smaller token.
+__device__ __forceinline__ bool ranks_before(double wa, int ta, double wb, int tb) {
+  return wa > wb || (wa == wb && ta < tb);
+}
+
+}  // namespace sdms

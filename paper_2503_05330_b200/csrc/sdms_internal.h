@@ -1,0 +1,19 @@
+// Host-side launchers, one per translation unit of kernels.
+#pragma once
+#include "sdms_dev.cuh"
+
+namespace sdms {
+
+cudaError_t launch_append(const Dev& s, const int32_t* tokens, const float* logprobs, const int32_t* counts,
+                          int row_width, cudaStream_t stream);
+cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t* draft_len,
+                          const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
+                          cudaStream_t stream);
+cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream);
+cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream);
+cudaError_t launch_dag(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                       float* draft_edge_w, cudaStream_t stream);
+cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream);
+cudaError_t dag_kernel_setup();
+
+}  // namespace sdms

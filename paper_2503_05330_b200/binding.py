@@ -1,0 +1,264 @@
+"""ctypes binding of ``libsdms.so``.
+
+Module-level functions carry the names of the C entry points and only marshal
+arguments (torch tensors -> device pointers, torch stream -> cudaStream_t).
+``Sdms`` bundles a context with the buffers a decode loop needs.  Every step of
+the path runs inside the CUDA library; nothing here computes, and there is no
+CPU fallback: loading fails loudly when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdms.so")
+
+SDMS_OK = 0
+ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE = -1, -2, -3, -4
+STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
+STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
+NUM_KERNELS = 5
+KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept")
+
+EXPORTS = (
+    "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
+    "sdms_build_drafts", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
+    "sdms_debug_read_history", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
+    "sdms_profile_read", "sdms_strerror", "sdms_kernel_name",
+)
+
+
+class SdmsConfig(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("num_groups", C.c_int32), ("paths_per_group", C.c_int32),
+        ("capacity", C.c_int32), ("vocab", C.c_int32), ("k_max", C.c_int32),
+        ("max_draft_len", C.c_int32), ("max_append", C.c_int32), ("dag_nodes_per_layer", C.c_int32),
+        ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
+        ("match_capacity", C.c_int64),
+    ]
+
+
+def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
+                match_capacity=0) -> SdmsConfig:
+    return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
+                      B, Ke, search_mode, alpha, match_capacity)
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2503_05330_b200.build` (there is no CPU fallback)")
+        l = C.CDLL(LIB_PATH)
+        vp, i32 = C.c_void_p, C.c_int32
+        l.sdms_workspace_bytes.argtypes = [C.POINTER(SdmsConfig), C.POINTER(C.c_size_t)]
+        l.sdms_create.argtypes = [C.POINTER(SdmsConfig), vp, C.c_size_t, C.POINTER(vp)]
+        l.sdms_reset.argtypes = [vp, vp]
+        l.sdms_destroy.argtypes = [vp]
+        l.sdms_append.argtypes = [vp, vp, vp, vp, i32, vp]
+        l.sdms_build_drafts.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+        l.sdms_accept.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
+        l.sdms_get_dag.argtypes = [vp] * 10
+        l.sdms_debug_read_history.argtypes = [vp] * 5
+        l.sdms_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        l.sdms_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        l.sdms_profile_enable.argtypes = [vp, i32]
+        l.sdms_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_uint64)]
+        l.sdms_strerror.argtypes = [C.c_int]
+        l.sdms_strerror.restype = C.c_char_p
+        l.sdms_kernel_name.argtypes = [C.c_int]
+        l.sdms_kernel_name.restype = C.c_char_p
+        _lib = l
+    return _lib
+
+
+class SdmsError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {lib().sdms_strerror(code).decode()} ({code})")
+
+
+def _check(code, where):
+    if code != SDMS_OK:
+        raise SdmsError(code, where)
+
+
+def _dp(t):
+    """Device pointer of a CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def _sp(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+# ---- the C entry points, one to one ------------------------------------------
+def sdms_workspace_bytes(cfg: SdmsConfig) -> int:
+    n = C.c_size_t(0)
+    _check(lib().sdms_workspace_bytes(C.byref(cfg), C.byref(n)), "sdms_workspace_bytes")
+    return n.value
+
+
+def sdms_create(cfg: SdmsConfig, workspace: torch.Tensor):
+    h = C.c_void_p()
+    _check(lib().sdms_create(C.byref(cfg), _dp(workspace), workspace.numel() * workspace.element_size(),
+                             C.byref(h)), "sdms_create")
+    return h
+
+
+def sdms_reset(ctx, stream=None):
+    _check(lib().sdms_reset(ctx, _sp(stream)), "sdms_reset")
+
+
+def sdms_destroy(ctx):
+    _check(lib().sdms_destroy(ctx), "sdms_destroy")
+
+
+def sdms_append(ctx, tokens, logprobs, counts, stream=None):
+    assert tokens.dtype == torch.int32 and logprobs.dtype == torch.float32 and counts.dtype == torch.int32
+    _check(lib().sdms_append(ctx, _dp(tokens), _dp(logprobs), _dp(counts), tokens.shape[1], _sp(stream)),
+           "sdms_append")
+
+
+def sdms_build_drafts(ctx, k, draft_tok, draft_len, draft_score=None, draft_edge_w=None, stream=None):
+    _check(lib().sdms_build_drafts(ctx, k, _dp(draft_tok), _dp(draft_len), _dp(draft_score), _dp(draft_edge_w),
+                                   _sp(stream)), "sdms_build_drafts")
+
+
+def sdms_accept(ctx, draft_tok, draft_len, sampled, sampled_logprobs, accept_len, stream=None):
+    _check(lib().sdms_accept(ctx, _dp(draft_tok), _dp(draft_len), _dp(sampled), _dp(sampled_logprobs),
+                             _dp(accept_len), _sp(stream)), "sdms_accept")
+
+
+def sdms_get_matches(ctx, offsets, gpos, stream=None):
+    _check(lib().sdms_get_matches(ctx, _dp(offsets), _dp(gpos), gpos.numel(), _sp(stream)), "sdms_get_matches")
+
+
+def sdms_get_dag(ctx, node_tok, node_S, node_cnt, node_count, edge_dst, edge_S, edge_cnt, out_degree, stream=None):
+    _check(lib().sdms_get_dag(ctx, _dp(node_tok), _dp(node_S), _dp(node_cnt), _dp(node_count), _dp(edge_dst),
+                              _dp(edge_S), _dp(edge_cnt), _dp(out_degree), _sp(stream)), "sdms_get_dag")
+
+
+def sdms_debug_read_history(ctx, tok, pq, lens, stream=None):
+    _check(lib().sdms_debug_read_history(ctx, _dp(tok), _dp(pq), _dp(lens), _sp(stream)), "sdms_debug_read_history")
+
+
+def sdms_get_status(ctx, stream=None) -> int:
+    f = C.c_uint32(0)
+    _check(lib().sdms_get_status(ctx, C.byref(f), _sp(stream)), "sdms_get_status")
+    return f.value
+
+
+def sdms_launch_count(ctx) -> int:
+    n = C.c_uint64(0)
+    _check(lib().sdms_launch_count(ctx, C.byref(n)), "sdms_launch_count")
+    return n.value
+
+
+def sdms_profile_enable(ctx, on: bool):
+    _check(lib().sdms_profile_enable(ctx, int(on)), "sdms_profile_enable")
+
+
+def sdms_profile_read(ctx):
+    ms = (C.c_float * NUM_KERNELS)()
+    n = (C.c_uint64 * NUM_KERNELS)()
+    _check(lib().sdms_profile_read(ctx, ms, n), "sdms_profile_read")
+    return {KERNEL_NAMES[k]: (float(ms[k]), int(n[k])) for k in range(NUM_KERNELS)}
+
+
+# ---- convenience wrapper ------------------------------------------------------
+class Sdms:
+    """A context plus the device buffers of one decode loop (allocation and
+    marshalling only)."""
+
+    def __init__(self, G, N, L, V, k_max, D, device="cuda:0", **kw):
+        self.cfg = make_config(G, N, L, V, k_max, D, **kw)
+        self.G, self.N, self.L, self.V, self.k_max, self.D = G, N, L, V, k_max, D
+        self.P = G * N
+        self.B, self.Ke = self.cfg.dag_nodes_per_layer, self.cfg.dag_edges_per_node
+        self.device = torch.device(device)
+        nbytes = sdms_workspace_bytes(self.cfg)
+        self.workspace_bytes = nbytes
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            self.ctx = sdms_create(self.cfg, self.workspace)
+        P, D_ = self.P, D
+        dev = self.device
+        self.draft_tok = torch.empty((P, D_), dtype=torch.int32, device=dev)
+        self.draft_len = torch.empty(P, dtype=torch.int32, device=dev)
+        self.draft_score = torch.empty((P, D_), dtype=torch.float32, device=dev)
+        self.draft_edge_w = torch.empty((P, D_), dtype=torch.float32, device=dev)
+        self.accept_len = torch.empty(P, dtype=torch.int32, device=dev)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            sdms_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self, stream=None):
+        sdms_reset(self.ctx, stream)
+
+    def append(self, tokens, logprobs, counts, stream=None):
+        sdms_append(self.ctx, tokens, logprobs, counts, stream)
+
+    def build_drafts(self, k, stream=None):
+        sdms_build_drafts(self.ctx, k, self.draft_tok, self.draft_len, self.draft_score, self.draft_edge_w, stream)
+        return self.draft_tok, self.draft_len
+
+    def accept(self, sampled, sampled_logprobs=None, stream=None):
+        sdms_accept(self.ctx, self.draft_tok, self.draft_len, sampled, sampled_logprobs, self.accept_len, stream)
+        return self.accept_len
+
+    def status(self, stream=None) -> int:
+        return sdms_get_status(self.ctx, stream)
+
+    def matches(self, cap=None):
+        """(offsets [P+1], positions) of the last build, as CPU tensors."""
+        offsets = torch.empty(self.P + 1, dtype=torch.int32, device=self.device)
+        probe = torch.empty(1, dtype=torch.int32, device=self.device)
+        lib().sdms_get_matches(self.ctx, _dp(offsets), _dp(probe), 0, _sp(None))
+        total = int(offsets[-1].item())
+        gpos = torch.empty(max(total, 1), dtype=torch.int32, device=self.device)
+        sdms_get_matches(self.ctx, offsets, gpos)
+        return offsets.cpu(), gpos[:total].cpu()
+
+    def dag(self):
+        P, D, B, Ke, dev = self.P, self.D, self.B, self.Ke, self.device
+        r = dict(node_tok=torch.empty((P, D, B), dtype=torch.int32, device=dev),
+                 node_S=torch.empty((P, D, B), dtype=torch.int64, device=dev),
+                 node_cnt=torch.empty((P, D, B), dtype=torch.int32, device=dev),
+                 node_count=torch.empty((P, D), dtype=torch.int32, device=dev),
+                 edge_dst=torch.empty((P, D, B, Ke), dtype=torch.int32, device=dev),
+                 edge_S=torch.empty((P, D, B, Ke), dtype=torch.int64, device=dev),
+                 edge_cnt=torch.empty((P, D, B, Ke), dtype=torch.int32, device=dev),
+                 out_degree=torch.empty((P, D, B), dtype=torch.int32, device=dev))
+        sdms_get_dag(self.ctx, r["node_tok"], r["node_S"], r["node_cnt"], r["node_count"], r["edge_dst"],
+                     r["edge_S"], r["edge_cnt"], r["out_degree"])
+        return {k: v.cpu().numpy() for k, v in r.items()}
+
+    def history(self):
+        tok = torch.empty((self.P, self.L), dtype=torch.int32, device=self.device)
+        pq = torch.empty((self.P, self.L), dtype=torch.int32, device=self.device)
+        lens = torch.empty(self.P, dtype=torch.int32, device=self.device)
+        sdms_debug_read_history(self.ctx, tok, pq, lens)
+        return tok.cpu().numpy(), pq.cpu().numpy(), lens.cpu().numpy()

@@ -1,0 +1,175 @@
+"""CUDA library against the CPU oracle, element by element, on the same seeded
+inputs.  Integer results (tokens, positions, sums, counts) must be identical;
+float weights agree within 1e-5 relative (harness.RTOL)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2503_05330_b200 import synth  # noqa: E402
+import harness  # noqa: E402
+from harness import Pair, run_protocol  # noqa: E402
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_worked_example_on_device():
+    w = json.load(open(os.path.join(GOLDEN, "worked_example.json")))
+    # logprobs whose probabilities are the example's dyadic values up to fp32 rounding
+    pair = Pair(1, 3, w["capacity"], 16, 2, w["D"], B=4, Ke=4)
+    a_max = max(len(p) for p in w["paths"])
+    tok = np.zeros((3, a_max), np.int32); lp = np.zeros((3, a_max), np.float32)
+    for i, p in enumerate(w["paths"]):
+        tok[i, :len(p)] = p
+        lp[i, :len(p)] = np.log(np.array(w["prob"][i]))
+    pair.append(tok, lp, np.array([len(p) for p in w["paths"]], np.int32), expect_status=0)
+    pair.check_history()
+    t, ln = pair.build_and_compare(w["k"])
+    assert t[0, :ln[0]].tolist() == w["draft"]
+    assert t[2, :ln[2]].tolist() == w["other_queries"]["2"] and ln[1] == 0
+    sampled = np.full((3, w["D"] + 1), 15, np.int32)
+    sampled[0] = w["accept"]["sampled"]
+    tau = pair.accept_and_compare(sampled, np.full(sampled.shape, -0.5, np.float32))
+    assert tau[0] == w["accept"]["tau"]
+    pair.check_history()
+
+
+def test_fixed_point_probabilities_match_on_many_logprobs():
+    P, L = 8, 4096
+    rng = synth.Stream(4242)
+    lp = np.concatenate([-12.0 * rng.uniform(P * L - 64), np.array([0.0, -0.0, -1e-8, -40.0, -41.0, -25.0, -21.4, -21.5]),
+                         -30.0 * rng.uniform(56)]).astype(np.float32).reshape(P, L)
+    tok = np.zeros((P, L), np.int32)
+    pair = Pair(1, P, L, 4, 1, 2)
+    pair.append(tok, lp, np.full(P, L, np.int32), expect_status=0)
+    pair.check_history()
+
+
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("alpha,mode", [(1.0, 0), (0.5, 0), (0.0, 0), (1.0, 1)])
+def test_dense_tiny_vocab_every_step(seed, alpha, mode):
+    # tiny vocabulary: matches, merges and ties everywhere; ragged lengths
+    G, N, L, V, D, k_max = 2, 4, 48, 3 + seed % 2, 4, 3
+    tokens, lps = synth.small_random(G * N, L, V, 900 + seed)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, B=4, Ke=3)
+        start = 3 + (np.arange(G * N) * 5 + seed) % 9
+        st = run_protocol(pair, tokens, lps, k, steps=40, warm=0, start_lens=start,
+                          commit_in_accept=bool(seed % 2))
+        assert st["steps"] > 0
+
+
+def test_append_clamping_and_status_bits():
+    pair = Pair(1, 4, 6, 10, 2, 2)
+    tok = np.array([[1, 2, 3, 4], [1, 2, 3, 4], [1, 99, 3, 4], [1, 2, 3, 4]], np.int32)
+    lp = np.full((4, 4), -0.3, np.float32)
+    pair.append(tok, lp, np.array([4, 0, 4, 7], np.int32), expect_status=0x04 | 0x01)
+    pair.append(tok, lp, np.array([4, 2, 0, 0], np.int32), expect_status=0x02)
+    pair.append(tok, np.full((4, 4), np.nan, np.float32), np.array([0, 1, 0, 0], np.int32), expect_status=0x08)
+    pair.check_history()
+    pair.build_and_compare(1)
+    pair.build_and_compare(2)
+
+
+def test_empty_and_degenerate_states():
+    # nothing appended yet, then a single token per path, then k larger than some paths
+    pair = Pair(2, 3, 16, 5, 3, 3, B=2, Ke=2)
+    _, ln = pair.build_and_compare(1)
+    assert ln.sum() == 0
+    tok = np.ones((6, 4), np.int32); lp = np.full((6, 4), -1.0, np.float32)
+    pair.append(tok, lp, np.array([1, 1, 1, 0, 1, 0], np.int32), expect_status=0)
+    pair.build_and_compare(1)
+    pair.append(tok, lp, np.array([4, 0, 2, 4, 0, 1], np.int32), expect_status=0)
+    for k in (1, 2, 3):
+        pair.build_and_compare(k)
+    # all paths identical and constant: every window matches
+    pair = Pair(1, 4, 64, 2, 4, 8, B=3, Ke=2, alpha=0.5)
+    pair.append(np.ones((4, 60), np.int32), np.full((4, 60), -0.7, np.float32), np.array([60, 33, 5, 1], np.int32),
+                expect_status=0)
+    for k in (1, 2, 4):
+        pair.build_and_compare(k)
+
+
+def test_full_paths_are_sources_only():
+    N, L = 3, 32
+    tokens, lps = synth.small_random(N, L, 3, 5)
+    pair = Pair(1, N, L, 3, 2, 4)
+    pair.append(tokens, lps, np.array([L, L - 1, 10], np.int32), expect_status=0)
+    _, ln = pair.build_and_compare(1)
+    assert ln[0] == 0
+
+
+def test_match_workspace_overflow_is_reported_not_fatal():
+    N, L = 4, 64
+    pair = Pair(1, N, L, 2, 1, 2, match_capacity=100)
+    pair.g.append(harness.t32(np.zeros((N, L - 1), np.int32), pair.dev),
+                  harness.t32(np.full((N, L - 1), -0.5, np.float32), pair.dev),
+                  harness.t32(np.full(N, L - 1, np.int32), pair.dev))
+    assert pair.g.status() == 0
+    pair.g.build_drafts(1)
+    assert pair.g.status() == 0x20
+    assert (pair.g.draft_len.cpu().numpy() == 0).all()      # every query needs more than 100 slots
+
+
+@pytest.mark.parametrize("k", [1, 2, 3])
+def test_config1_full_protocol(k):
+    w = synth.WORKLOADS[1]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D)
+    st = run_protocol(pair, tokens, lps, k, steps=w.steps, warm=w.k_max)
+    assert st["steps"] == w.steps
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_config2_full_protocol(k):
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D)
+    st = run_protocol(pair, tokens, lps, k, steps=w.steps, warm=w.k_max, commit_in_accept=(k % 2 == 0))
+    assert st["steps"] > 100
+
+
+@pytest.mark.parametrize("k", [1, 4])
+def test_config3_protocol(k):
+    w = synth.WORKLOADS[3]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D)
+    # start from partly filled, ragged histories so the 200 steps end near capacity
+    start = 1200 + (np.arange(w.P) * 37) % 500
+    st = run_protocol(pair, tokens, lps, k, steps=200, warm=0, start_lens=start, check_every=10)
+    assert st["steps"] == 200
+
+
+@pytest.mark.parametrize("fill", [0.3, 0.97])
+def test_config4_sampled_steps(fill):
+    w = synth.WORKLOADS[4]
+    tokens, lps = synth.make_streams(w)
+    for k in (1, 3, 5):
+        pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=4, Ke=2, max_append=w.D)
+        start = (int(w.L * fill) - (np.arange(w.P) * 13) % 97).astype(np.int32)
+        run_protocol(pair, tokens, lps, k, steps=3, warm=0, start_lens=start, commit_in_accept=True)
+        del pair
+
+
+@pytest.mark.parametrize("k", [1, 2, 8])
+def test_config5_sampled_steps(k):
+    # heavy fan-out: k = 1 queries on frequent tokens match tens of thousands of positions
+    w = synth.WORKLOADS[5]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D)
+    start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+    sample = list(range(0, w.P, 16))
+    # the oracle's brute-force scan of 2M positions per query is slow: two steps, full compare on a sample of paths
+    P, L, D = pair.P, pair.L, pair.D
+    pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+    for step in range(2):
+        lens = pair.o.lengths()
+        pair.build_and_compare(k, paths=sample)
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
+        pair.accept_and_compare(sampled, sampled_lp)
+    pair.check_history()
+    torch.cuda.synchronize()

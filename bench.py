@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Throughput of per-step draft construction on synthetic multi-path streams.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole path for all paths of the workload:
+sdms_build_drafts (query, match, gather, DAG, search) followed by sdms_accept
+with commit (acceptance check and state update with index insertion).  The
+suffix length cycles k = 1..k_max over the steps.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_05330_b200 import synth  # noqa: E402
+
+METRIC = "draft-construction paths*steps/sec at N=16 (and us/step)"
+UNIT = "paths*steps/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def k_of(step, k_max):
+    return 1 + step % k_max
+
+
+# ----------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ----------------------------------------------------------------------------
+def oracle_run(w, tokens, logprobs, max_steps, budget_s, threads=1):
+    """Decode protocol on the oracle; returns (paths*steps, seconds, steps, restarts)."""
+    from oracle import Oracle
+    done = 0
+    units = 0
+    secs = 0.0
+    runs = 0
+    while done < max_steps and secs < budget_s:
+        o = Oracle(w.G, w.N, w.L, w.V, w.D)
+        lens = np.full(w.P, w.k_max, np.int32)
+        o.append(tokens[:, :w.k_max], logprobs[:, :w.k_max], lens)
+        runs += 1
+        step = 0
+        while done < max_steps and secs < budget_s:
+            lens = o.lengths()
+            active = int((lens < w.L).sum())
+            if active == 0 or step >= w.steps:
+                break
+            sampled, sampled_lp = synth.sampled_window(tokens, logprobs, lens, w.D + 1)
+            t0 = time.perf_counter()
+            o.build_all(k_of(step, w.k_max), nthreads=threads)
+            tok, ln, _, _ = o.drafts()
+            o.accept_commit(tok, ln, sampled, sampled_lp, w.D)
+            secs += time.perf_counter() - t0
+            units += active
+            done += 1
+            step += 1
+    return units, secs, done, runs
+
+
+def reference_main(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    tokens, logprobs = synth.make_streams(w)
+    oracle_run(w, tokens, logprobs, args.warmup, 30.0)
+    units, secs, steps, runs = oracle_run(w, tokens, logprobs, args.steps, 120.0)
+    value = units / secs
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32/int64 (f64 weights)",
+        "data": "synthetic", "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{steps} decode steps of {w.name} ({runs} run(s) from the warm start)"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {"workload": w.name, "groups": w.G, "paths_per_group": w.N, "capacity": w.L, "vocab": w.V,
+            "k": f"cycles 1..{w.k_max} over the steps", "max_draft_len": w.D,
+            "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)"}
+
+
+# ----------------------------------------------------------------------------
+# clocks during the timed region (NVML, in-process)
+# ----------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.sm, self.reasons, self.max_sm = [], set(), None
+        self._halt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._halt.is_set():
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join()
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_sm,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+class Runner:
+    """Device-resident replay of the decode protocol of one workload."""
+
+    def __init__(self, w, seed, device, B, Ke):
+        import torch
+        from paper_2503_05330_b200 import binding
+        self.torch, self.binding, self.w, self.device = torch, binding, w, device
+        self.tokens, self.logprobs = synth.make_streams(w, seed)
+        self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke)
+        dev = self.s.device
+        self.warm_tok = torch.from_numpy(np.ascontiguousarray(self.tokens[:, :w.k_max])).to(dev)
+        self.warm_lp = torch.from_numpy(np.ascontiguousarray(self.logprobs[:, :w.k_max])).to(dev)
+        self.warm_cnt = torch.full((w.P,), w.k_max, dtype=torch.int32, device=dev)
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        self.plan = None
+
+    def start_run(self):
+        self.s.reset()
+        self.s.append(self.warm_tok, self.warm_lp, self.warm_cnt)
+
+    def dry_run(self):
+        """Plays one run to record, per step, the sampled windows (what the model
+        would return), the live path count and the algorithmic bytes."""
+        torch, w, s = self.torch, self.w, self.s
+        dev = s.device
+        self.start_run()
+        sampled_all, lp_all, active, bytes_scan, bytes_dag, bytes_io = [], [], [], [], [], []
+        matches = []
+        for step in range(w.steps):
+            _, _, lens = s.history()
+            live = int((lens < w.L).sum())
+            if live == 0:
+                break
+            sm, lp = synth.sampled_window(self.tokens, self.logprobs, lens, w.D + 1)
+            s.build_drafts(k_of(step, w.k_max))
+            off, gpos = s.matches()
+            gpos = gpos.numpy().astype(np.int64)
+            j, e = gpos // w.L, gpos % w.L
+            n_m = np.minimum(w.D, lens[j] - 1 - e)
+            matches.append(len(gpos))
+            bytes_scan.append(4 * int(lens.sum()))
+            bytes_dag.append(int(8 * n_m.sum() + 4 * len(gpos) + w.P * (12 * w.D + 4)))
+            s.accept(torch.from_numpy(sm).to(dev), torch.from_numpy(lp).to(dev))
+            tau = s.accept_len.cpu().numpy()
+            gained = np.minimum(np.minimum(tau + 1, w.D), w.L - lens)
+            bytes_io.append(int(gained.sum()) * (8 + 8 + w.k_max * 32) + w.P * (w.D + 1) * 8)
+            sampled_all.append(sm); lp_all.append(lp); active.append(live)
+        assert s.status() == 0
+        self.plan = dict(
+            sampled=torch.from_numpy(np.stack(sampled_all)).to(dev), lp=torch.from_numpy(np.stack(lp_all)).to(dev),
+            sampled_host=torch.from_numpy(np.stack(sampled_all)).pin_memory(),
+            lp_host=torch.from_numpy(np.stack(lp_all)).pin_memory(),
+            active=active, steps=len(active),
+            bytes={"scan": float(np.mean(bytes_scan)), "dag": float(np.mean(bytes_dag)),
+                   "accept": float(np.mean(bytes_io))},
+            mean_matches_per_step=float(np.mean(matches)))
+        return self.plan
+
+    def timed_steps(self, K, flush=True, e2e=False):
+        """Times exactly K steps (CUDA events around each step on the launch
+        stream), restarting the run when it ends.  Returns (ms, paths*steps)."""
+        torch, w, s, plan = self.torch, self.w, self.s, self.plan
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        units = 0
+        done = 0
+        if e2e:
+            h_acc = torch.empty(w.P, dtype=torch.int32).pin_memory()
+            h_tok = torch.empty((w.P, w.D), dtype=torch.int32).pin_memory()
+            h_len = torch.empty(w.P, dtype=torch.int32).pin_memory()
+            d_sm = torch.empty((w.P, w.D + 1), dtype=torch.int32, device=s.device)
+            d_lp = torch.empty((w.P, w.D + 1), dtype=torch.float32, device=s.device)
+        while done < K:
+            self.start_run()
+            for step in range(plan["steps"]):
+                if done == K:
+                    break
+                if flush:
+                    self.flush.zero_()
+                a, b = ev[done]
+                a.record()
+                if e2e:
+                    d_sm.copy_(plan["sampled_host"][step], non_blocking=True)
+                    d_lp.copy_(plan["lp_host"][step], non_blocking=True)
+                    s.build_drafts(k_of(step, w.k_max))
+                    s.accept(d_sm, d_lp)
+                    h_acc.copy_(s.accept_len, non_blocking=True)
+                    h_tok.copy_(s.draft_tok, non_blocking=True)
+                    h_len.copy_(s.draft_len, non_blocking=True)
+                    b.record()
+                    b.synchronize()                 # the caller reads the result before its next step
+                else:
+                    s.build_drafts(k_of(step, w.k_max))
+                    s.accept(plan["sampled"][step], plan["lp"][step])
+                    b.record()
+                units += plan["active"][step]
+                done += 1
+        torch.cuda.synchronize()
+        ms = sum(a.elapsed_time(b) for a, b in ev)
+        return ms, units
+
+
+def ours_main(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_05330_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    device = f"cuda:{local}"
+    # every rank owns its own prompts (different seed): no data-path collective
+    run = Runner(w, synth.BASE_SEED + w.index + 7919 * rank, device, args.dag_nodes, args.dag_edges)
+    plan = run.dry_run()
+
+    run.timed_steps(max(args.warmup, 3))
+    sampler = ClockSampler(local)
+    sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = binding.sdms_launch_count(run.s.ctx)
+    t0 = time.perf_counter()
+    ms, units = run.timed_steps(args.steps)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    wall = time.perf_counter() - t0
+    launches = binding.sdms_launch_count(run.s.ctx) - launches0
+    clocks = sampler.stop()
+
+    # end to end through host buffers
+    run.timed_steps(3, e2e=True)
+    ms_e2e, units_e2e = run.timed_steps(args.steps, e2e=True)
+
+    # per-kernel times over a further pass of the same steps
+    binding.sdms_profile_enable(run.s.ctx, True)
+    run.timed_steps(args.steps)
+    prof = binding.sdms_profile_read(run.s.ctx)
+    binding.sdms_profile_enable(run.s.ctx, False)
+    # warm-L2 figure for context (no flush between steps)
+    ms_warm, units_warm = run.timed_steps(args.steps, flush=False)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        u = torch.tensor([units, units_e2e], dtype=torch.float64, device=device)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+        ms, ms_e2e = t.tolist()
+        units, units_e2e = u.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_file):
+        peak, peak_src = float(json.load(open(peaks_file))["hbm_gbs"]), "measured copy bandwidth (burst)"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    per_kernel = {}
+    for name, (kms, n) in prof.items():
+        if n:
+            us = 1e3 * kms / n
+            b = plan["bytes"].get(name)
+            per_kernel[name] = {"launches": n, "us_per_launch": us, "share": kms / sum(v[0] for v in prof.values()),
+                                "algorithmic_bytes_per_launch": b,
+                                "gbs": (b / (us * 1e-6) / 1e9) if b else None}
+    dom = max((n for n in per_kernel if per_kernel[n]["gbs"] is not None), key=lambda n: per_kernel[n]["share"])
+    achieved = per_kernel[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                "note": "the whole store of this workload is 128 KiB: a step is bound by launch and "
+                        "dependent-access latency, not by bandwidth"}
+
+    line = {
+        "metric": METRIC, "value": units / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "us_per_step": 1e3 * ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32/int64 (f64 weights)", "data": "synthetic", "config": workload_config(w),
+        "e2e": {"value": units_e2e / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": 1e3 * ms_e2e / args.steps,
+                "h2d_bytes_per_step": w.P * (w.D + 1) * 8, "d2h_bytes_per_step": w.P * (w.D + 2) * 4},
+        "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
+        "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
+        "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
+        "run_steps": plan["steps"], "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 4 * w.steps, 20.0)
+        line["cpu_baseline"] = {"value": units_c / secs_c, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "us_per_step": 1e6 * secs_c / steps_c,
+                                "sample": f"{steps_c} decode steps of {w.name} ({runs_c} run(s) from the warm start)"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2)
+    ap.add_argument("--dag-nodes", type=int, default=8, help="nodes per layer in the DAG export (0 = off)")
+    ap.add_argument("--dag-edges", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        reference_main(args, w)
+    else:
+        ours_main(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -41,6 +41,7 @@ extern "C" {
 #define SDMS_ERR_WORKSPACE_TOO_SMALL -2
 #define SDMS_ERR_CUDA               -3
 #define SDMS_ERR_BAD_STATE          -4
+#define SDMS_ERR_TOO_LARGE          -5
 
 /* Device status bits (sticky until sdms_get_status clears them). */
 #define SDMS_STATUS_BAD_COUNT      0x01u /* append count outside [0, row width]: clamped          */
@@ -161,6 +162,38 @@ int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_
 
 /* Waits for `stream`, returns the status bits in *host_flags and clears them. */
 int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream);
+
+/* ---- for callers that cannot allocate device memory ------------------------- */
+
+/*
+ * The paper has no counterpart of this call; it exists for one kind of caller.
+ * A sampler plug-in that runs inside a serving engine usually finds the GPU's
+ * memory already handed out: the engine reserves almost all free HBM for its
+ * KV-cache pool at start-up, a later cudaMalloc may fail or stall every stream of
+ * the device, and the plug-in has no access to the engine's own allocator.  Such
+ * a caller cannot provide the workspace a context needs.  This call finds the
+ * Eq. 3 matches straight from path histories the caller already holds, and the
+ * only extra device memory it uses - two int32 counters per path - is a fixed
+ * 128 KiB array inside the library image (present on every GPU that loads the
+ * library, until the process exits).  It calls no cudaMalloc / cudaFree and no
+ * allocating routine of any library.
+ *
+ *   d_tok [P][capacity], d_len [P] : the histories (inputs, P = groups * paths)
+ *   d_offsets [P+1], d_gpos [cap]  : same meaning as in sdms_get_matches; a path
+ *       shorter than k, or full, has no query and therefore no matches
+ *
+ * Limits and sharing: P <= SDMS_NOALLOC_MAX_PATHS, otherwise SDMS_ERR_TOO_LARGE
+ * and nothing is launched.  All calls on a device share the one array; each call
+ * zeroes the counters it uses before counting, so calls in sequence on a stream
+ * are independent of each other, but two calls whose kernels overlap on the GPU
+ * (different streams, different threads) race and give wrong results.  The first
+ * call on each device looks up the array's device address; make that first call
+ * outside any stream capture.
+ */
+#define SDMS_NOALLOC_MAX_PATHS 16384
+int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, int32_t num_groups,
+                       int32_t paths_per_group, int32_t capacity, int32_t k, int32_t* d_offsets,
+                       int32_t* d_gpos, size_t cap, void* stream);
 
 /* ---- measurement hooks (no counterpart in the paper) ----------------------- */
 

@@ -17,7 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdms.so")
 
 SDMS_OK = 0
-ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE = -1, -2, -3, -4
+ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE, ERR_TOO_LARGE = -1, -2, -3, -4, -5
+NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
 NUM_KERNELS = 5
@@ -27,7 +28,7 @@ EXPORTS = (
     "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
     "sdms_build_drafts", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
-    "sdms_profile_read", "sdms_strerror", "sdms_kernel_name",
+    "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc",
 )
 
 
@@ -73,6 +74,7 @@ def lib():
         l.sdms_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         l.sdms_profile_enable.argtypes = [vp, i32]
         l.sdms_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_uint64)]
+        l.sdms_match_noalloc.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, C.c_size_t, vp]
         l.sdms_strerror.argtypes = [C.c_int]
         l.sdms_strerror.restype = C.c_char_p
         l.sdms_kernel_name.argtypes = [C.c_int]
@@ -178,6 +180,18 @@ def sdms_profile_read(ctx):
     n = (C.c_uint64 * NUM_KERNELS)()
     _check(lib().sdms_profile_read(ctx, ms, n), "sdms_profile_read")
     return {KERNEL_NAMES[k]: (float(ms[k]), int(n[k])) for k in range(NUM_KERNELS)}
+
+
+def sdms_match_noalloc(tok, lens, num_groups, paths_per_group, k, offsets, gpos, stream=None):
+    """Eq. 3 matches straight from caller-held histories ``tok [P][L]`` / ``lens [P]``.
+
+    For callers that cannot allocate device memory (for example a sampler plug-in
+    inside a serving engine whose KV-cache pool already owns the free HBM): needs
+    no context and no workspace; its only scratch is a fixed array inside the
+    library.  ``offsets [P+1]`` and ``gpos`` are the caller's output tensors."""
+    assert tok.dtype == torch.int32 and lens.dtype == torch.int32
+    _check(lib().sdms_match_noalloc(_dp(tok), _dp(lens), num_groups, paths_per_group, tok.shape[1], k,
+                                    _dp(offsets), _dp(gpos), gpos.numel(), _sp(stream)), "sdms_match_noalloc")
 
 
 # ---- convenience wrapper ------------------------------------------------------

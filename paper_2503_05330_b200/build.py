@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdms.so")
-SOURCES = ["api.cu", "append.cu", "match.cu", "dag.cu"]
+SOURCES = ["api.cu", "append.cu", "match.cu", "dag.cu", "match_static.cu"]
 HEADERS = ["sdms_dev.cuh", "sdms_internal.h"]
 
 

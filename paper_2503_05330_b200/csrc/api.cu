@@ -295,6 +295,7 @@ const char* sdms_strerror(int code) {
     case SDMS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SDMS_ERR_CUDA: return "CUDA call failed";
     case SDMS_ERR_BAD_STATE: return "call not valid in this state";
+    case SDMS_ERR_TOO_LARGE: return "size beyond the fixed maximum of this entry point";
     default: return "unknown error";
   }
 }

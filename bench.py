@@ -168,6 +168,7 @@ class Runner:
         dev = s.device
         self.start_run()
         sampled_all, lp_all, active, bytes_scan, bytes_dag, bytes_io = [], [], [], [], [], []
+        bytes_fused, bytes_useful, scan_queries = [], [], []
         matches = []
         for step in range(w.steps):
             _, _, lens = s.history()
@@ -183,6 +184,14 @@ class Runner:
             matches.append(len(gpos))
             bytes_scan.append(4 * int(lens.sum()))
             bytes_dag.append(int(8 * n_m.sum() + 4 * len(gpos) + w.P * (12 * w.D + 4)))
+            # the fused kernel: a query answered by scanning streams the other paths of its prompt
+            k = k_of(step, w.k_max)
+            modes = s.query_modes()
+            glen = lens.reshape(w.G, w.N).sum(1).repeat(w.N)
+            probe_b = int((modes > 0).sum()) * (32 + 4 * k) + 4 * w.P
+            bytes_fused.append(int(4 * (glen - lens)[modes == 2].sum()) + probe_b + bytes_dag[-1])
+            bytes_useful.append(probe_b + 4 * k * len(gpos) + bytes_dag[-1])      # index model: verify each match
+            scan_queries.append(int((modes == 2).sum()))
             s.accept(torch.from_numpy(sm).to(dev), torch.from_numpy(lp).to(dev))
             tau = s.accept_len.cpu().numpy()
             gained = np.minimum(np.minimum(tau + 1, w.D), w.L - lens)
@@ -195,7 +204,8 @@ class Runner:
             lp_host=torch.from_numpy(np.stack(lp_all)).pin_memory(),
             active=active, steps=len(active),
             bytes={"scan": float(np.mean(bytes_scan)), "dag": float(np.mean(bytes_dag)),
-                   "accept": float(np.mean(bytes_io))},
+                   "accept": float(np.mean(bytes_io)), "build_fused": float(np.mean(bytes_fused))},
+            useful_bytes_build=float(np.mean(bytes_useful)), scan_queries_per_step=float(np.mean(scan_queries)),
             mean_matches_per_step=float(np.mean(matches)))
         return self.plan
 
@@ -315,6 +325,9 @@ def ours_main(args, w):
     achieved = per_kernel[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                "bytes_model": "what this kernel's method must read: index bucket per query, the other paths of the "
+                               "prompt for each scanned query, followers of every match, outputs",
+                "useful_bytes_per_launch_index_model": plan["useful_bytes_build"],
                 "note": "the whole store of this workload is 128 KiB: a step is bound by launch and "
                         "dependent-access latency, not by bandwidth"}
 
@@ -328,7 +341,7 @@ def ours_main(args, w):
         "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
         "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
-        "run_steps": plan["steps"], "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges},
+        "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges},
     }
     if world == 1 and not args.no_cpu_baseline:
         units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 4 * w.steps, 20.0)

@@ -160,6 +160,10 @@ int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t*
 /* Copies the stores: d_tok / d_pq [P][L], d_len [P] (any may be NULL). */
 int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_t* d_len, void* stream);
 
+/* How each path's query of the last sdms_build_drafts was answered: d_modes [P],
+ * 0 = no query or no index entry, 1 = from the index bucket, 2 = by scanning. */
+int sdms_debug_read_query_modes(sdms_ctx* ctx, int32_t* d_modes, void* stream);
+
 /* Waits for `stream`, returns the status bits in *host_flags and clears them. */
 int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream);
 
@@ -202,7 +206,8 @@ int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, int32_t num_g
 #define SDMS_KERNEL_SCAN   2
 #define SDMS_KERNEL_DAG    3
 #define SDMS_KERNEL_ACCEPT 4
-#define SDMS_NUM_KERNELS   5
+#define SDMS_KERNEL_BUILD_FUSED 5   /* probe + scan + dag in one launch (small prompts) */
+#define SDMS_NUM_KERNELS   6
 
 /* Number of kernels this context has launched since creation. */
 int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches);

@@ -21,13 +21,13 @@ ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE, ERR_TOO_LARGE
 NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
-NUM_KERNELS = 5
-KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept")
+NUM_KERNELS = 6
+KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused")
 
 EXPORTS = (
     "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
     "sdms_build_drafts", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
-    "sdms_debug_read_history", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
+    "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc",
 )
 
@@ -70,6 +70,7 @@ def lib():
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
         l.sdms_get_dag.argtypes = [vp] * 10
         l.sdms_debug_read_history.argtypes = [vp] * 5
+        l.sdms_debug_read_query_modes.argtypes = [vp, vp, vp]
         l.sdms_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         l.sdms_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         l.sdms_profile_enable.argtypes = [vp, i32]
@@ -157,6 +158,10 @@ def sdms_get_dag(ctx, node_tok, node_S, node_cnt, node_count, edge_dst, edge_S, 
 
 def sdms_debug_read_history(ctx, tok, pq, lens, stream=None):
     _check(lib().sdms_debug_read_history(ctx, _dp(tok), _dp(pq), _dp(lens), _sp(stream)), "sdms_debug_read_history")
+
+
+def sdms_debug_read_query_modes(ctx, modes, stream=None):
+    _check(lib().sdms_debug_read_query_modes(ctx, _dp(modes), _sp(stream)), "sdms_debug_read_query_modes")
 
 
 def sdms_get_status(ctx, stream=None) -> int:
@@ -269,6 +274,11 @@ class Sdms:
         sdms_get_dag(self.ctx, r["node_tok"], r["node_S"], r["node_cnt"], r["node_count"], r["edge_dst"],
                      r["edge_S"], r["edge_cnt"], r["out_degree"])
         return {k: v.cpu().numpy() for k, v in r.items()}
+
+    def query_modes(self):
+        modes = torch.empty(self.P, dtype=torch.int32, device=self.device)
+        sdms_debug_read_query_modes(self.ctx, modes)
+        return modes.cpu().numpy()
 
     def history(self):
         tok = torch.empty((self.P, self.L), dtype=torch.int32, device=self.device)

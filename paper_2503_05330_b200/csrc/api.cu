@@ -146,6 +146,8 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.mode = cfg->search_mode; d.P = d.G * d.N;
   d.alpha = (double)cfg->alpha;
   d.table_cap = lay.table_cap; d.match_cap = lay.match_cap;
+  // small prompts: every query path gets a private slice of N*L match slots and one CTA does the whole build
+  d.fused = (int64_t)d.N * d.L <= kFusedMaxTokens && (int64_t)d.P * d.N * d.L <= lay.match_cap;
   unsigned char* w = ctx->ws;
   d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len);
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);
@@ -192,6 +194,12 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
   if (k < 1 || k > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  if (ctx->dev.fused) {
+    const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
+      return launch_build_fused(ctx->dev, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+    if (rc == SDMS_OK) ctx->built = true;
+    return rc;
+  }
   int rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, st); });
   if (rc != SDMS_OK) return rc;
   rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
@@ -249,6 +257,13 @@ int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_
   return ok ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
+int sdms_debug_read_query_modes(sdms_ctx* ctx, int32_t* d_modes, void* stream) {
+  if (!ctx || !d_modes) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->built) return SDMS_ERR_BAD_STATE;
+  return cudaMemcpyAsync(d_modes, ctx->dev.q_mode, (size_t)ctx->dev.P * 4, cudaMemcpyDeviceToDevice,
+                         (cudaStream_t)stream) == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
 int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream) {
   if (!ctx || !host_flags) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
@@ -301,7 +316,7 @@ const char* sdms_strerror(int code) {
 }
 
 const char* sdms_kernel_name(int kernel) {
-  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept"};
+  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept", "build_fused"};
   return kernel >= 0 && kernel < SDMS_NUM_KERNELS ? names[kernel] : "?";
 }
 

@@ -57,6 +57,14 @@ __device__ int32_t prob_to_fixed(float lp, uint32_t* st) {
   if (lp >= 0.0f) return one;
   if (lp < -40.0f) return 0;                       // exp(-40) * 2^30 < 1e-8
   const double x = (double)lp;
+  {
+    // plain double first: exp() is within 1 ulp, so y is within 2e-7 of the true value;
+    // only a fraction that close to one half needs the exact evaluation below
+    const double y = __dmul_rn(exp(x), 1073741824.0);
+    const double fl = floor(y);
+    const double frac = __dsub_rn(y, fl);
+    if (fabs(__dsub_rn(frac, 0.5)) > 1e-5) return (int32_t)fl + (frac > 0.5 ? 1 : 0);
+  }
   const double ln2_hi = 6.93147180369123816490e-01;  // 32 significant bits: m * ln2_hi is exact
   const double ln2_lo = 1.90821492927058770002e-10;  // ln 2 - ln2_hi
   const double m = rint(__dmul_rn(x, 1.44269504088896338700e+00));

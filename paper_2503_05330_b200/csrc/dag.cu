@@ -1,20 +1,27 @@
-// Follower gather, layered DAG aggregation (Eq. 5) and greedy extraction.
+// Follower gather, layered DAG aggregation (Eq. 5) and greedy extraction, plus
+// the single-launch build for small prompts.
 //
-// dag_kernel : one CTA per query path.  Layer by layer (d = 1..D) every match m
-//              contributes its d-th follower v = tok[e+d] with the fixed-point
-//              probability pq[e+d]; contributions to the same token merge in a
-//              shared-memory hash table (node = distinct token of the layer):
-//                S_all / c_all : sum over every candidate      -> node score
-//                S_cur / c_cur : candidates coming from the node the walk stands
-//                                on                             -> successor test
-//                                                                  and edge weight
-//              All sums are integers, so the order of the atomics cannot change
-//              a result.  After the pass one warp picks the best successor; with
-//              the export enabled other warps select the B best nodes of the
-//              layer and the Ke best out-edges of the nodes kept one layer up.
-//              A layer with more distinct tokens than the table holds is
-//              processed in several passes, each over the tokens of one residue
-//              class, so that any fan-out fits a fixed amount of shared memory.
+// Every match m of query path i contributes, at layer d = 1..D, its d-th
+// follower v = tok[e+d] with the fixed-point probability pq[e+d].  A node is a
+// distinct token of a layer, an edge a distinct (previous token, token) pair; S
+// and cnt of nodes and edges are integer sums, so the order of accumulation
+// (atomics, warp shuffles) cannot change a result.
+//
+// Two ways through, both per query path in one CTA:
+//   dag_small (M <= 32 matches, the common case): lane m owns candidate m and
+//     each WARP owns a layer, so all layers aggregate at the same time.  Lanes
+//     with the same follower token (__match_any_sync) form a node, lanes that
+//     also share the previous token form an edge; sums run over the lanes of a
+//     group, ranks over the group leaders.  One barrier, then one warp walks the
+//     layers (a warp-wide arg-max per layer).
+//   dag_block (any M): layers in sequence; every warp takes 32 candidates at a
+//     time, pre-aggregates equal tokens with the same warp primitives and lets
+//     the group leaders add into shared-memory hash tables (32-bit atomics with
+//     explicit carry).  After the pass one warp picks the best successor; with
+//     the export enabled other warps select the B best nodes of the layer and the
+//     Ke best out-edges of the nodes kept one layer up.  A layer with more
+//     distinct tokens than the table holds is processed in several passes, each
+//     over the tokens of one residue class, so any fan-out fits the same tables.
 #include "sdms_internal.h"
 
 namespace sdms {
@@ -22,10 +29,13 @@ namespace sdms {
 namespace {
 
 typedef unsigned long long u64;
+constexpr unsigned FULL = 0xffffffffu;
 constexpr int CAP = kDagCap;
-constexpr int kWarps = kDagThreads / 32;
 constexpr int MAXB = SDMS_MAX_DAG_NODES;
 constexpr int MAXKE = SDMS_MAX_DAG_EDGES;
+constexpr int kStageWords = 8192;      // followers (token, pq) of all matches staged in shared memory when M*D fits
+constexpr int kListCap = 2048;         // matches a fused CTA keeps in shared memory besides its global slice
+static_assert(kStageWords >= 4 * 32 * SDMS_MAX_DRAFT, "dag_small keeps its per-layer lanes in the staging area");
 
 struct Cand {            // a node or an edge competing in a selection
   double w; u64 S; unsigned cnt; int tok; int valid;
@@ -35,11 +45,11 @@ __device__ __forceinline__ Cand warp_best(Cand c) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     Cand x;
-    x.w = __shfl_xor_sync(0xffffffffu, c.w, o);
-    x.S = __shfl_xor_sync(0xffffffffu, c.S, o);
-    x.cnt = __shfl_xor_sync(0xffffffffu, c.cnt, o);
-    x.tok = __shfl_xor_sync(0xffffffffu, c.tok, o);
-    x.valid = __shfl_xor_sync(0xffffffffu, c.valid, o);
+    x.w = __shfl_xor_sync(FULL, c.w, o);
+    x.S = __shfl_xor_sync(FULL, c.S, o);
+    x.cnt = __shfl_xor_sync(FULL, c.cnt, o);
+    x.tok = __shfl_xor_sync(FULL, c.tok, o);
+    x.valid = __shfl_xor_sync(FULL, c.valid, o);
     if (x.valid && (!c.valid || ranks_before(x.w, x.tok, c.w, c.tok))) c = x;
   }
   return c;
@@ -70,23 +80,55 @@ __device__ int warp_topk(int ncand, Get get, int K, int* out_tok, u64* out_S, un
   return r;
 }
 
+// Sums of val over the lanes of group a and of group b; `live` (warp-uniform)
+// lists the lanes worth visiting.
+__device__ __forceinline__ void group_sums(unsigned live, unsigned a, unsigned b, unsigned val, u64* sa, u64* sb) {
+  u64 x = 0, y = 0;
+  for (unsigned rem = live; rem; rem &= rem - 1) {
+    const int src = __ffs(rem) - 1;
+    const unsigned t = __shfl_sync(FULL, val, src);
+    if (a >> src & 1) x += t;
+    if (b >> src & 1) y += t;
+  }
+  *sa = x; *sb = y;
+}
+
+// 64-bit add on a (lo, hi) pair of shared words with 32-bit atomics: whoever
+// makes the low word wrap carries into the high word.
+__device__ __forceinline__ void add64(unsigned* lo, unsigned* hi, u64 v) {
+  const unsigned l = (unsigned)v;
+  unsigned h = (unsigned)(v >> 32);
+  const unsigned old = atomicAdd(lo, l);
+  if (old + l < old) ++h;
+  if (h) atomicAdd(hi, h);
+}
+__device__ __forceinline__ u64 get64(const unsigned* lo, const unsigned* hi, int x) {
+  return ((u64)hi[x] << 32) | lo[x];
+}
+
 struct Smem {
-  u64* n_Sall; u64* n_Scur; u64* e_S;
-  int* n_key; unsigned* n_call; unsigned* n_ccur; int* n_touch;
-  int* e_key; unsigned* e_c; int* e_touch;
+  // node table: key = token; sums over all candidates and over those coming from the current node
+  int* n_key; unsigned* n_Slo; unsigned* n_Shi; unsigned* n_Clo; unsigned* n_Chi; unsigned* n_call; unsigned* n_ccur;
+  int* n_touch;
+  // edge table (export): key = token * MAXB + slot of the kept source node
+  int* e_key; unsigned* e_Slo; unsigned* e_Shi; unsigned* e_c; int* e_touch;
   // export lists
   u64* r_node_S; int* r_node_tok; unsigned* r_node_cnt;
   u64* r_edge_S; int* r_edge_dst; unsigned* r_edge_cnt;
   u64* t_S; int* t_tok; unsigned* t_cnt;        // per-warp scratch for merging
   int* kept; int* r_nedge; int* r_outdeg;
+  int* st_tok; int* st_pq;                      // staged followers [m*D + d-1], token -1 = past the path's end
+  int* list;                                    // fused kernel: first kListCap matches
 };
+
+constexpr int kMaxWarps = 32;
 
 template <bool EXPORT>
 __host__ __device__ constexpr size_t dag_smem_bytes() {
-  size_t b = (size_t)CAP * (8 + 8 + 4 + 4 + 4 + 4);
+  size_t b = (size_t)CAP * 8 * 4 + (size_t)kStageWords * 8 + (size_t)kListCap * 4;
   if (EXPORT) {
-    b += (size_t)CAP * (8 + 4 + 4 + 4);
-    b += (size_t)MAXB * 16 + (size_t)MAXB * MAXKE * 16 + (size_t)kWarps * 32 * 16 + (size_t)MAXB * 12;
+    b += (size_t)CAP * 5 * 4;
+    b += (size_t)MAXB * 16 + (size_t)MAXB * MAXKE * 16 + (size_t)kMaxWarps * 32 * 16 + (size_t)MAXB * 12;
   }
   return b;
 }
@@ -95,29 +137,35 @@ template <bool EXPORT>
 __device__ Smem carve(unsigned char* base) {
   Smem m;
   u64* p8 = reinterpret_cast<u64*>(base);
-  m.n_Sall = p8; p8 += CAP;
-  m.n_Scur = p8; p8 += CAP;
   if (EXPORT) {
-    m.e_S = p8; p8 += CAP;
     m.r_node_S = p8; p8 += MAXB;
     m.r_edge_S = p8; p8 += MAXB * MAXKE;
-    m.t_S = p8; p8 += kWarps * 32;
+    m.t_S = p8; p8 += kMaxWarps * 32;
   }
   int* p4 = reinterpret_cast<int*>(p8);
+  m.st_tok = p4; p4 += kStageWords;
+  m.st_pq = p4; p4 += kStageWords;
   m.n_key = p4; p4 += CAP;
+  m.n_Slo = reinterpret_cast<unsigned*>(p4); p4 += CAP;
+  m.n_Shi = reinterpret_cast<unsigned*>(p4); p4 += CAP;
+  m.n_Clo = reinterpret_cast<unsigned*>(p4); p4 += CAP;
+  m.n_Chi = reinterpret_cast<unsigned*>(p4); p4 += CAP;
   m.n_call = reinterpret_cast<unsigned*>(p4); p4 += CAP;
   m.n_ccur = reinterpret_cast<unsigned*>(p4); p4 += CAP;
   m.n_touch = p4; p4 += CAP;
+  m.list = p4; p4 += kListCap;
   if (EXPORT) {
     m.e_key = p4; p4 += CAP;
+    m.e_Slo = reinterpret_cast<unsigned*>(p4); p4 += CAP;
+    m.e_Shi = reinterpret_cast<unsigned*>(p4); p4 += CAP;
     m.e_c = reinterpret_cast<unsigned*>(p4); p4 += CAP;
     m.e_touch = p4; p4 += CAP;
     m.r_node_tok = p4; p4 += MAXB;
     m.r_node_cnt = reinterpret_cast<unsigned*>(p4); p4 += MAXB;
     m.r_edge_dst = p4; p4 += MAXB * MAXKE;
     m.r_edge_cnt = reinterpret_cast<unsigned*>(p4); p4 += MAXB * MAXKE;
-    m.t_tok = p4; p4 += kWarps * 32;
-    m.t_cnt = reinterpret_cast<unsigned*>(p4); p4 += kWarps * 32;
+    m.t_tok = p4; p4 += kMaxWarps * 32;
+    m.t_cnt = reinterpret_cast<unsigned*>(p4); p4 += kMaxWarps * 32;
     m.kept = p4; p4 += MAXB;
     m.r_nedge = p4; p4 += MAXB;
     m.r_outdeg = p4; p4 += MAXB;
@@ -128,22 +176,10 @@ __device__ Smem carve(unsigned char* base) {
 __device__ __forceinline__ unsigned slot_hash(unsigned x) { return (x * 2654435761u) >> 22; }   // 10 bits = CAP
 static_assert(CAP == 1024, "slot_hash yields 10 bits");
 
+// Defaults of one query path: no draft, empty export.
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
-                                                          int32_t* __restrict__ draft_len,
-                                                          float* __restrict__ draft_score,
-                                                          float* __restrict__ draft_edge_w) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  Smem sm = carve<EXPORT>(smem_raw);
-  __shared__ int sh_nn, sh_ne, sh_overflow, sh_found, sh_cur, sh_nkept, sh_nnode_run, sh_node_total;
-  __shared__ double sh_best_w, sh_best_ew;
-  __shared__ int sh_best_tok, sh_best_valid;
-
-  const int i = blockIdx.x;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int D = s.D, B = s.B, Ke = s.Ke;
-
-  // defaults: no draft, empty export
+__device__ void write_defaults(const Dev& s, int i, int32_t* draft_tok, float* draft_score, float* draft_edge_w) {
+  const int tid = threadIdx.x, D = s.D, B = s.B, Ke = s.Ke;
   for (int d = tid; d < D; d += blockDim.x) {
     draft_tok[(size_t)i * D + d] = -1;
     if (draft_score) draft_score[(size_t)i * D + d] = 0.0f;
@@ -160,17 +196,159 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
     }
     for (int d = tid; d < D; d += blockDim.x) s.x_node_count[(size_t)i * D + d] = 0;
   }
-  const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
-  if (M == 0) {
-    if (tid == 0) draft_len[i] = 0;
-    return;
+}
+
+// ---------------------------------------------------------------------------
+// M <= 32: one warp per layer, then one warp walks.  The export rows must hold
+// their defaults already (write_defaults followed by a barrier).
+// ---------------------------------------------------------------------------
+template <bool EXPORT>
+__device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
+                          int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int D = s.D, B = s.B, Ke = s.Ke;
+  const int root = s.tok[(size_t)i * s.L + s.len[i] - 1];
+  // per layer and lane: follower token, previous token, node score, edge weight; per layer: leader masks
+  int* L_v = sm.st_tok;
+  int* L_u = sm.st_tok + 32 * SDMS_MAX_DRAFT;
+  unsigned* L_lead = reinterpret_cast<unsigned*>(sm.st_tok + 2 * 32 * SDMS_MAX_DRAFT);
+  unsigned* L_elead = L_lead + SDMS_MAX_DRAFT;
+  double* L_W = reinterpret_cast<double*>(sm.st_pq);
+  double* L_we = L_W + 32 * SDMS_MAX_DRAFT;
+
+  int gpos = 0, n_m = 0;
+  if (lane < M) {
+    gpos = mlist[lane];
+    const int j = gpos / s.L;
+    n_m = min(D, s.len[j] - 1 - (gpos - j * s.L));
   }
-  const int32_t* mlist = s.matches + s.q_off[i];
+  for (int d = warp + 1; d <= D; d += nwarps) {
+    const bool alive = d <= n_m;                        // candidate reaches layer d
+    const bool alive_prev = lane < M && d - 1 <= n_m;   // ... reached layer d-1 (layer 0 is the root)
+    const int v = alive ? __ldg(s.tok + gpos + d) : -1;
+    const unsigned p = alive ? (unsigned)__ldg(s.pq + gpos + d) : 0u;
+    const int u = !alive_prev ? -1 : (d == 1 ? root : __ldg(s.tok + gpos + d - 1));
+    const unsigned live = __ballot_sync(FULL, alive);
+    const unsigned gv = __match_any_sync(FULL, v);                     // lanes on the same node
+    const unsigned gu = __match_any_sync(FULL, u);                     // lanes with the same previous node
+    const unsigned ge = gv & gu;                                       // lanes on the same edge
+    u64 S_all, S_uv;
+    group_sums(live, gv, ge, p, &S_all, &S_uv);
+    const unsigned c_all = __popc(gv), c_uv = __popc(ge);
+    const bool leader = alive && lane == __ffs(gv) - 1;
+    const bool eleader = alive && lane == __ffs(ge) - 1;
+    const double W = eq5_weight(s.alpha, S_all, c_all);
+    const double w_uv = eq5_weight(s.alpha, S_uv, c_uv);
+    const unsigned leaders = __ballot_sync(FULL, leader), eleaders = __ballot_sync(FULL, eleader);
+    L_v[(d - 1) * 32 + lane] = v; L_u[(d - 1) * 32 + lane] = u;
+    L_W[(d - 1) * 32 + lane] = W; L_we[(d - 1) * 32 + lane] = w_uv;
+    if (lane == 0) { L_lead[d - 1] = leaders; L_elead[d - 1] = eleaders; }
+    if (EXPORT && live) {
+      int rank = 0;
+      for (unsigned rem = leaders; rem; rem &= rem - 1) {
+        const int src = __ffs(rem) - 1;
+        const double ow = __shfl_sync(FULL, W, src);
+        const int ot = __shfl_sync(FULL, v, src);
+        if (ranks_before(ow, ot, W, v)) ++rank;
+      }
+      if (leader && rank < B) {
+        const size_t nx = ((size_t)i * D + (d - 1)) * B + rank;
+        s.x_node_tok[nx] = v; s.x_node_S[nx] = (int64_t)S_all; s.x_node_cnt[nx] = (int32_t)c_all;
+      }
+      if (lane == 0) s.x_node_count[(size_t)i * D + (d - 1)] = __popc(leaders);
+      if (d > 1) {
+        // rank of each previous-layer node, recomputed here so that layers stay independent
+        const unsigned pu = alive_prev ? (unsigned)__ldg(s.pq + gpos + d - 1) : 0u;
+        const unsigned live_prev = __ballot_sync(FULL, alive_prev);
+        u64 S_u, unused;
+        group_sums(live_prev, gu, 0u, pu, &S_u, &unused);
+        const double W_u = eq5_weight(s.alpha, S_u, __popc(gu));
+        const bool uleader = alive_prev && lane == __ffs(gu) - 1;
+        const unsigned uleaders = __ballot_sync(FULL, uleader);
+        int urank = 0;
+        for (unsigned rem = uleaders; rem; rem &= rem - 1) {
+          const int src = __ffs(rem) - 1;
+          const double ow = __shfl_sync(FULL, W_u, src);
+          const int ot = __shfl_sync(FULL, u, src);
+          if (ranks_before(ow, ot, W_u, u)) ++urank;
+        }
+        const int slot_u = __shfl_sync(FULL, urank, __ffs(gu) - 1);     // export slot of this lane's source node
+        int erank = 0, deg = 0;
+        for (unsigned rem = eleaders; rem; rem &= rem - 1) {
+          const int src = __ffs(rem) - 1;
+          const double ow = __shfl_sync(FULL, w_uv, src);
+          const int ot = __shfl_sync(FULL, v, src);
+          const int ou = __shfl_sync(FULL, u, src);
+          if (ou == u) { ++deg; if (ranks_before(ow, ot, w_uv, v)) ++erank; }
+        }
+        if (eleader && slot_u < B) {
+          const size_t nb = ((size_t)i * D + (d - 2)) * B + slot_u;
+          if (erank < Ke) {
+            s.x_edge_dst[nb * Ke + erank] = v; s.x_edge_S[nb * Ke + erank] = (int64_t)S_uv;
+            s.x_edge_cnt[nb * Ke + erank] = (int32_t)c_uv;
+          }
+          if (erank == 0) s.x_out_degree[nb] = deg;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  int cur = root, emitted = 0;
+  for (int d = 1; d <= D; ++d) {
+    const int v = L_v[(d - 1) * 32 + lane], u = L_u[(d - 1) * 32 + lane];
+    const bool el = L_elead[d - 1] >> lane & 1, ld = L_lead[d - 1] >> lane & 1;
+    Cand c;
+    c.valid = s.mode == 1 ? ld : (el && u == cur);
+    c.w = L_W[(d - 1) * 32 + lane]; c.tok = v; c.S = 0; c.cnt = 0;
+    c = warp_best(c);
+    if (!c.valid) break;
+    const unsigned emask = __ballot_sync(FULL, el && u == cur && v == c.tok);   // the edge taken, if it exists
+    const double we = __shfl_sync(FULL, L_we[(d - 1) * 32 + lane], emask ? __ffs(emask) - 1 : 0);
+    if (lane == 0) {
+      draft_tok[(size_t)i * D + (d - 1)] = c.tok;
+      if (draft_score) draft_score[(size_t)i * D + (d - 1)] = (float)c.w;
+      if (draft_edge_w) draft_edge_w[(size_t)i * D + (d - 1)] = emask ? (float)we : 0.0f;
+    }
+    cur = c.tok;
+    ++emitted;
+  }
+  if (lane == 0) draft_len[i] = emitted;
+}
+
+// ---------------------------------------------------------------------------
+// any M: layers in sequence, shared-memory hash tables
+// ---------------------------------------------------------------------------
+template <bool EXPORT>
+__device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
+                          int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
+  __shared__ int sh_nn, sh_ne, sh_overflow, sh_found, sh_cur, sh_nkept, sh_nnode_run, sh_node_total;
+  __shared__ double sh_best_w, sh_best_ew;
+  __shared__ int sh_best_tok, sh_best_valid;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int D = s.D, B = s.B, Ke = s.Ke;
   const int root = s.tok[(size_t)i * s.L + s.len[i] - 1];
 
+  // stage every follower once: one round trip to memory instead of one per layer
+  const bool staged = M * D <= kStageWords;
+  if (staged) {
+    for (int x = tid; x < M * D; x += blockDim.x) {
+      const int m = x / D, dd = x - m * D + 1;
+      const int gpos = mlist[m];
+      const int j = gpos / s.L;
+      const int e = gpos - j * s.L;
+      const bool on = e + dd <= s.len[j] - 1;
+      sm.st_tok[x] = on ? __ldg(s.tok + gpos + dd) : -1;
+      sm.st_pq[x] = on ? __ldg(s.pq + gpos + dd) : 0;
+    }
+  }
   for (int x = tid; x < CAP; x += blockDim.x) {
-    sm.n_key[x] = -1; sm.n_Sall[x] = 0; sm.n_Scur[x] = 0; sm.n_call[x] = 0; sm.n_ccur[x] = 0;
-    if (EXPORT) { sm.e_key[x] = -1; sm.e_S[x] = 0; sm.e_c[x] = 0; }
+    sm.n_key[x] = -1; sm.n_Slo[x] = 0; sm.n_Shi[x] = 0; sm.n_Clo[x] = 0; sm.n_Chi[x] = 0;
+    sm.n_call[x] = 0; sm.n_ccur[x] = 0;
+    if (EXPORT) { sm.e_key[x] = -1; sm.e_Slo[x] = 0; sm.e_Shi[x] = 0; sm.e_c[x] = 0; }
   }
   if (tid == 0) { sh_nn = 0; sh_ne = 0; sh_overflow = 0; sh_cur = root; sh_nkept = 0; }
   __syncthreads();
@@ -191,44 +369,77 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
       __syncthreads();
       bool overflowed = false;
       for (int part = 0; part < npart && !overflowed; ++part) {
-        // ---- accumulate this residue class of follower tokens ----
-        for (int m = tid; m < M; m += blockDim.x) {
-          const int gpos = mlist[m];
-          const int j = gpos / s.L;
-          const int e = gpos - j * s.L;
-          if (e + d > s.len[j] - 1) continue;
-          const int v = __ldg(s.tok + gpos + d);
-          if (npart > 1 && v % npart != part) continue;
-          const int u = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
-          const u64 p = (u64)(unsigned)__ldg(s.pq + gpos + d);
-          unsigned h = slot_hash((unsigned)(v / npart));
-          int slot = -1;
-          for (int probe = 0; probe < CAP; ++probe) {
-            const int old = atomicCAS(&sm.n_key[h], -1, v);
-            if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
-            if (old == -1 || old == v) { slot = (int)h; break; }
-            h = (h + 1) & (CAP - 1);
+        // ---- accumulate this residue class of follower tokens, 32 candidates per warp at a time ----
+        for (int base = warp * 32; base < M; base += nwarps * 32) {
+          const int m = base + lane;
+          int v = -1, u = -1;
+          unsigned p = 0;
+          if (m < M) {
+            if (staged) {
+              v = sm.st_tok[m * D + d - 1];
+              if (v >= 0) { u = d == 1 ? root : sm.st_tok[m * D + d - 2]; p = (unsigned)sm.st_pq[m * D + d - 1]; }
+            } else {
+              const int gpos = mlist[m];
+              const int j = gpos / s.L;
+              if (gpos - j * s.L + d <= s.len[j] - 1) {
+                v = __ldg(s.tok + gpos + d);
+                u = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
+                p = (unsigned)__ldg(s.pq + gpos + d);
+              }
+            }
+            if (v >= 0 && npart > 1 && v % npart != part) v = -1;
           }
-          if (slot < 0) { sh_overflow = 1; continue; }
-          atomicAdd(&sm.n_Sall[slot], p);
-          atomicAdd(&sm.n_call[slot], 1u);
-          if (u == cur) { atomicAdd(&sm.n_Scur[slot], p); atomicAdd(&sm.n_ccur[slot], 1u); }
+          const bool on = v >= 0;
+          const unsigned live = __ballot_sync(FULL, on);
+          if (live == 0) continue;
+          const unsigned gv = __match_any_sync(FULL, v);
+          const unsigned fc = __ballot_sync(FULL, on && u == cur);
+          u64 S_all, S_cur;
+          group_sums(live, gv, gv & fc, p, &S_all, &S_cur);
+          if (on && lane == __ffs(gv) - 1) {                             // one insert per distinct token of the warp
+            unsigned h = slot_hash((unsigned)(v / npart));
+            int slot = -1;
+            for (int probe = 0; probe < CAP; ++probe) {
+              const int old = atomicCAS(&sm.n_key[h], -1, v);
+              if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
+              if (old == -1 || old == v) { slot = (int)h; break; }
+              h = (h + 1) & (CAP - 1);
+            }
+            if (slot < 0) {
+              sh_overflow = 1;
+            } else {
+              add64(&sm.n_Slo[slot], &sm.n_Shi[slot], S_all);
+              atomicAdd(&sm.n_call[slot], (unsigned)__popc(gv));
+              const unsigned cc = __popc(gv & fc);
+              if (cc) { add64(&sm.n_Clo[slot], &sm.n_Chi[slot], S_cur); atomicAdd(&sm.n_ccur[slot], cc); }
+            }
+          }
           if (EXPORT && d > 1) {
             int b = -1;
-            for (int x = 0; x < nkept; ++x) if (sm.kept[x] == u) { b = x; break; }
-            if (b >= 0) {
-              const int ekey = v * MAXB + b;                 // (destination, kept source) in one word
-              unsigned he = slot_hash((unsigned)(v / npart) * 37u + (unsigned)b);
-              int es = -1;
-              for (int probe = 0; probe < CAP; ++probe) {
-                const int old = atomicCAS(&sm.e_key[he], -1, ekey);
-                if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
-                if (old == -1 || old == ekey) { es = (int)he; break; }
-                he = (he + 1) & (CAP - 1);
+            if (on) for (int x = 0; x < nkept; ++x) if (sm.kept[x] == u) { b = x; break; }
+            const bool has_src = b >= 0;
+            const unsigned srcs = __ballot_sync(FULL, has_src);
+            if (srcs) {
+              const unsigned ge = gv & __match_any_sync(FULL, has_src ? u : -1);
+              u64 S_uv, unused;
+              group_sums(srcs, ge, 0u, p, &S_uv, &unused);
+              if (has_src && lane == __ffs(ge) - 1) {
+                const int ekey = v * MAXB + b;                 // (destination, kept source) in one word
+                unsigned he = slot_hash((unsigned)(v / npart) * 37u + (unsigned)b);
+                int es = -1;
+                for (int probe = 0; probe < CAP; ++probe) {
+                  const int old = atomicCAS(&sm.e_key[he], -1, ekey);
+                  if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
+                  if (old == -1 || old == ekey) { es = (int)he; break; }
+                  he = (he + 1) & (CAP - 1);
+                }
+                if (es < 0) {
+                  sh_overflow = 1;
+                } else {
+                  add64(&sm.e_Slo[es], &sm.e_Shi[es], S_uv);
+                  atomicAdd(&sm.e_c[es], (unsigned)__popc(ge));
+                }
               }
-              if (es < 0) { sh_overflow = 1; continue; }
-              atomicAdd(&sm.e_S[es], p);
-              atomicAdd(&sm.e_c[es], 1u);
             }
           }
         }
@@ -238,19 +449,14 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
         if (!overflowed) {
           // ---- selections, one warp each ----
           if (warp == 0 && walking) {
-            auto get = [&](int x) {
-              const int sl = sm.n_touch[x];
-              Cand c;
-              c.tok = sm.n_key[sl]; c.S = sm.n_Sall[sl]; c.cnt = sm.n_call[sl];
-              c.valid = s.mode == 1 || sm.n_ccur[sl] > 0;
-              c.w = eq5_weight(s.alpha, c.S, c.cnt);
-              // carry the slot in place of the count: the edge weight is read from it below
-              c.cnt = (unsigned)sl;
-              return c;
-            };
             Cand best; best.valid = 0; best.w = 0; best.tok = 0; best.S = 0; best.cnt = 0;
             for (int x = lane; x < nn; x += 32) {
-              const Cand c = get(x);
+              const int sl = sm.n_touch[x];
+              Cand c;
+              c.tok = sm.n_key[sl]; c.S = 0;
+              c.valid = s.mode == 1 || sm.n_ccur[sl] > 0;
+              c.w = eq5_weight(s.alpha, get64(sm.n_Slo, sm.n_Shi, sl), sm.n_call[sl]);
+              c.cnt = (unsigned)sl;                  // carry the slot: the edge weight is read from it below
               if (c.valid && (!best.valid || ranks_before(c.w, c.tok, best.w, best.tok))) best = c;
             }
             best = warp_best(best);
@@ -258,14 +464,14 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
                 (!sh_best_valid || ranks_before(best.w, best.tok, sh_best_w, sh_best_tok))) {
               const int sl = (int)best.cnt;
               sh_best_valid = 1; sh_best_w = best.w; sh_best_tok = best.tok;
-              sh_best_ew = sm.n_ccur[sl] ? eq5_weight(s.alpha, sm.n_Scur[sl], sm.n_ccur[sl]) : 0.0;
+              sh_best_ew = sm.n_ccur[sl] ? eq5_weight(s.alpha, get64(sm.n_Clo, sm.n_Chi, sl), sm.n_ccur[sl]) : 0.0;
             }
           }
           if (EXPORT && warp == 1) {
             const int nrun = sh_nnode_run;
             auto get = [&](int x) {
               Cand c; c.valid = 1;
-              if (x < nn) { const int sl = sm.n_touch[x]; c.tok = sm.n_key[sl]; c.S = sm.n_Sall[sl]; c.cnt = sm.n_call[sl]; }
+              if (x < nn) { const int sl = sm.n_touch[x]; c.tok = sm.n_key[sl]; c.S = get64(sm.n_Slo, sm.n_Shi, sl); c.cnt = sm.n_call[sl]; }
               else { c.tok = sm.r_node_tok[x - nn]; c.S = sm.r_node_S[x - nn]; c.cnt = sm.r_node_cnt[x - nn]; }
               c.w = eq5_weight(s.alpha, c.S, c.cnt);
               return c;
@@ -276,17 +482,18 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
             if (lane == 0) { sh_nnode_run = got; sh_node_total += nn; }
           }
           if (EXPORT && warp >= 2 && d > 1) {
-            for (int b = warp - 2; b < nkept; b += kWarps - 2) {
+            for (int b = warp - 2; b < nkept; b += nwarps - 2) {
               const int nrun = sm.r_nedge[b];
               int deg = 0;
               for (int x = lane; x < ne; x += 32) deg += sm.e_key[sm.e_touch[x]] % MAXB == b;
 #pragma unroll
-              for (int o = 16; o > 0; o >>= 1) deg += __shfl_xor_sync(0xffffffffu, deg, o);
+              for (int o = 16; o > 0; o >>= 1) deg += __shfl_xor_sync(FULL, deg, o);
               auto get = [&](int x) {
                 Cand c;
                 if (x < ne) {
                   const int sl = sm.e_touch[x];
-                  c.valid = sm.e_key[sl] % MAXB == b; c.tok = sm.e_key[sl] / MAXB; c.S = sm.e_S[sl]; c.cnt = sm.e_c[sl];
+                  c.valid = sm.e_key[sl] % MAXB == b; c.tok = sm.e_key[sl] / MAXB;
+                  c.S = get64(sm.e_Slo, sm.e_Shi, sl); c.cnt = sm.e_c[sl];
                 } else {
                   const int y = b * MAXKE + (x - ne);
                   c.valid = 1; c.tok = sm.r_edge_dst[y]; c.S = sm.r_edge_S[y]; c.cnt = sm.r_edge_cnt[y];
@@ -309,12 +516,13 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
         // ---- wipe the touched slots for the next pass ----
         for (int x = tid; x < nn; x += blockDim.x) {
           const int sl = sm.n_touch[x];
-          sm.n_key[sl] = -1; sm.n_Sall[sl] = 0; sm.n_Scur[sl] = 0; sm.n_call[sl] = 0; sm.n_ccur[sl] = 0;
+          sm.n_key[sl] = -1; sm.n_Slo[sl] = 0; sm.n_Shi[sl] = 0; sm.n_Clo[sl] = 0; sm.n_Chi[sl] = 0;
+          sm.n_call[sl] = 0; sm.n_ccur[sl] = 0;
         }
         if (EXPORT)
           for (int x = tid; x < ne; x += blockDim.x) {
             const int sl = sm.e_touch[x];
-            sm.e_key[sl] = -1; sm.e_S[sl] = 0; sm.e_c[sl] = 0;
+            sm.e_key[sl] = -1; sm.e_Slo[sl] = 0; sm.e_Shi[sl] = 0; sm.e_c[sl] = 0;
           }
         __syncthreads();
         if (tid == 0) { sh_nn = 0; sh_ne = 0; sh_overflow = 0; }
@@ -376,14 +584,182 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
   if (tid == 0) draft_len[i] = emitted;
 }
 
+// Gather + DAG + search for query path i over its M (> 0) matches in mlist
+// (shared or global memory).  Called by all threads of the CTA, after a barrier
+// that follows write_defaults.
+template <bool EXPORT>
+__device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
+                                          int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                                          float* draft_edge_w) {
+  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, draft_tok, draft_len, draft_score, draft_edge_w);
+  else dag_block<EXPORT>(s, sm, i, M, mlist, draft_tok, draft_len, draft_score, draft_edge_w);
+}
+
+template <bool EXPORT>
+__global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
+                                                          int32_t* __restrict__ draft_len,
+                                                          float* __restrict__ draft_score,
+                                                          float* __restrict__ draft_edge_w) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Smem sm = carve<EXPORT>(smem_raw);
+  const int i = blockIdx.x;
+  write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
+  const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
+  if (M == 0) {
+    if (threadIdx.x == 0) draft_len[i] = 0;
+    return;
+  }
+  __syncthreads();
+  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], draft_tok, draft_len, draft_score, draft_edge_w);
+}
+
+// Whole draft construction of one query path in one CTA, for prompts whose
+// histories are small enough that every CTA can afford to read them itself:
+// probe the index; a k-gram with at most kInlineSlots occurrences is answered
+// from its bucket, any other by streaming the other paths of the prompt with
+// 128-bit loads (last token first, the rest of the window on a hit); then the
+// gather / DAG / search phase runs on the matches just found.  The matches also
+// go to the path's private slice of the match list for inspection.
+template <bool EXPORT>
+__global__ void __launch_bounds__(kDagThreads) build_fused_kernel(Dev s, int k, int32_t* __restrict__ draft_tok,
+                                                                  int32_t* __restrict__ draft_len,
+                                                                  float* __restrict__ draft_score,
+                                                                  float* __restrict__ draft_edge_w) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Smem sm = carve<EXPORT>(smem_raw);
+  __shared__ int sh_mode, sh_M;
+  __shared__ uint32_t sh_count, sh_pos[kInlineSlots];
+  __shared__ int32_t sh_q[SDMS_MAX_K];
+  __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
+  const int i = blockIdx.x, tid = threadIdx.x;
+  const int g = i / s.N;
+  for (int n = tid; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
+  const int slice = s.N * s.L;
+  int32_t* my_matches = s.matches + (size_t)i * slice;
+
+  if (tid == 0) {
+    const int len_i = s.len[i];
+    int mode = Q_NONE;
+    uint32_t fp = 0, count = 0;
+    if (len_i >= k && len_i < s.L) {
+      const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
+      uint64_t h = gram_init(k);
+      for (int t = 0; t < k; ++t) { const int32_t x = q[t]; sh_q[t] = x; h = gram_step(h, x); }
+      h = gram_final(h);
+      fp = gram_fp(h);
+      const uint32_t* table = index_table(s, g, k);
+      uint32_t b = gram_bucket(h, s.table_cap);
+      for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
+        const uint4* cand = reinterpret_cast<const uint4*>(table + (size_t)b * kBucketWords);
+        const uint4 lo = cand[0];
+        if (lo.x == fp) {
+          const uint4 hi = cand[1];
+          count = lo.y;
+          sh_pos[0] = lo.z; sh_pos[1] = lo.w; sh_pos[2] = hi.x; sh_pos[3] = hi.y; sh_pos[4] = hi.z; sh_pos[5] = hi.w;
+          mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
+          break;
+        }
+        if (lo.x == 0u) break;
+        b = (b + 1) & (s.table_cap - 1);
+      }
+    }
+    sh_mode = mode; sh_count = count; sh_M = 0;
+    s.q_fp[i] = fp; s.q_mode[i] = mode; s.q_reserved[i] = mode == Q_NONE ? 0 : slice; s.q_off[i] = i * slice;
+  }
+  write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
+  __syncthreads();
+  const int mode = sh_mode;
+  if (mode == Q_INLINE) {
+    if (tid < (int)sh_count) {
+      const uint32_t lpos = sh_pos[tid];
+      const int jn = (int)(lpos / (uint32_t)s.L);
+      const int j = g * s.N + jn;
+      const int e = (int)(lpos % (uint32_t)s.L);
+      if (j != i && e <= sh_len[jn] - 2) {
+        const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
+        bool same = true;
+        for (int t = 0; t < k; ++t) same = same && (c[t] == sh_q[t]);
+        if (same) {
+          const int at = atomicAdd(&sh_M, 1);
+          sm.list[at] = j * s.L + e;
+          my_matches[at] = j * s.L + e;
+        }
+      }
+    }
+  } else if (mode == Q_SCAN) {
+    // every other path of the prompt, all loads independent of each other:
+    // compare the last token of the query first, the rest of the window on a hit
+    const int last = sh_q[k - 1];
+    const int32_t* gtok = s.tok + (size_t)g * s.N * s.L;
+    auto hit = [&](int jn, int e) {
+      const int32_t* row = gtok + (size_t)jn * s.L;
+      for (int t = 0; t < k - 1; ++t) if (__ldg(row + e - (k - 1) + t) != sh_q[t]) return;
+      const int at = atomicAdd(&sh_M, 1);
+      const int pos = (g * s.N + jn) * s.L + e;
+      if (at < kListCap) sm.list[at] = pos;
+      my_matches[at] = pos;
+    };
+    if ((s.L & 3) == 0) {
+      const int per = s.L >> 2, total = s.N * per;
+      const int4* g4 = reinterpret_cast<const int4*>(gtok);
+      constexpr int kBatch = 8;
+      for (int x0 = tid; x0 < total; x0 += kBatch * blockDim.x) {
+        int4 w[kBatch];
+        int jn[kBatch], e0[kBatch], e_hi[kBatch];
+#pragma unroll
+        for (int r = 0; r < kBatch; ++r) {
+          const int x = x0 + r * blockDim.x;
+          e_hi[r] = -1; e0[r] = 0; jn[r] = 0;
+          if (x < total) {
+            jn[r] = x / per; e0[r] = 4 * (x - jn[r] * per);
+            e_hi[r] = g * s.N + jn[r] == i ? -1 : sh_len[jn[r]] - 2;     // last position with a follower
+            if (e0[r] <= e_hi[r]) w[r] = __ldg(g4 + x);
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < kBatch; ++r) {
+          if (e0[r] > e_hi[r]) continue;
+          if (w[r].x == last && e0[r] >= k - 1) hit(jn[r], e0[r]);
+          if (w[r].y == last && e0[r] + 1 >= k - 1 && e0[r] + 1 <= e_hi[r]) hit(jn[r], e0[r] + 1);
+          if (w[r].z == last && e0[r] + 2 >= k - 1 && e0[r] + 2 <= e_hi[r]) hit(jn[r], e0[r] + 2);
+          if (w[r].w == last && e0[r] + 3 >= k - 1 && e0[r] + 3 <= e_hi[r]) hit(jn[r], e0[r] + 3);
+        }
+      }
+    } else {
+      const int total = s.N * s.L;
+      for (int x = tid; x < total; x += blockDim.x) {
+        const int jn = x / s.L, e = x - jn * s.L;
+        if (g * s.N + jn == i || e < k - 1 || e > sh_len[jn] - 2) continue;
+        if (__ldg(gtok + x) == last) hit(jn, e);
+      }
+    }
+  }
+  __syncthreads();
+  const int M = sh_M;
+  if (tid == 0) s.q_cursor[i] = M;
+  if (M == 0) {
+    if (tid == 0) draft_len[i] = 0;
+    return;
+  }
+  dag_phase<EXPORT>(s, sm, i, M, M <= kListCap ? sm.list : my_matches, draft_tok, draft_len, draft_score,
+                    draft_edge_w);
+}
+
 }  // namespace
 
 cudaError_t dag_kernel_setup() {
   cudaError_t e = cudaFuncSetAttribute(dag_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)dag_smem_bytes<false>());
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(dag_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)dag_smem_bytes<true>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(dag_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dag_smem_bytes<true>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(build_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dag_smem_bytes<true>());
+  return e;
 }
 
 cudaError_t launch_dag(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
@@ -394,6 +770,17 @@ cudaError_t launch_dag(const Dev& s, int32_t* draft_tok, int32_t* draft_len, flo
   else
     dag_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, draft_tok, draft_len, draft_score,
                                                                             draft_edge_w);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_build_fused(const Dev& s, int k, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                               float* draft_edge_w, cudaStream_t stream) {
+  if (s.B > 0)
+    build_fused_kernel<true><<<s.P, kDagThreads, dag_smem_bytes<true>(), stream>>>(s, k, draft_tok, draft_len,
+                                                                                   draft_score, draft_edge_w);
+  else
+    build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, k, draft_tok, draft_len,
+                                                                                    draft_score, draft_edge_w);
   return cudaGetLastError();
 }
 

@@ -13,12 +13,14 @@ constexpr int kScanTile = 1024;        // history tokens per scan CTA
 constexpr int kScanThreads = 256;
 constexpr int kDagThreads = 256;
 constexpr int kDagCap = 1024;          // entries of the shared-memory node / edge tables
+constexpr int kFusedMaxTokens = 131072; // largest N*L a CTA scans on its own
 
 enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
 
 // Everything a kernel needs, passed by value.
 struct Dev {
   int32_t G, N, L, V, k_max, D, max_append, B, Ke, mode, P;
+  int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
   double alpha;
   uint32_t table_cap;                  // buckets per (prompt, n) table, power of two
   int64_t match_cap;

@@ -204,7 +204,7 @@ __device__ void write_defaults(const Dev& s, int i, int32_t* draft_tok, float* d
 // ---------------------------------------------------------------------------
 template <bool EXPORT>
 __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                          int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          const int32_t* plen, int poff, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                           float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int D = s.D, B = s.B, Ke = s.Ke;
@@ -221,7 +221,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   if (lane < M) {
     gpos = mlist[lane];
     const int j = gpos / s.L;
-    n_m = min(D, s.len[j] - 1 - (gpos - j * s.L));
+    n_m = min(D, plen[j - poff] - 1 - (gpos - j * s.L));
   }
   for (int d = warp + 1; d <= D; d += nwarps) {
     const bool alive = d <= n_m;                        // candidate reaches layer d
@@ -322,7 +322,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
 // ---------------------------------------------------------------------------
 template <bool EXPORT>
 __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                          int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          const int32_t* plen, int poff, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                           float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   __shared__ int sh_nn, sh_ne, sh_overflow, sh_found, sh_cur, sh_nkept, sh_nnode_run, sh_node_total;
   __shared__ double sh_best_w, sh_best_ew;
@@ -340,7 +340,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       const int gpos = mlist[m];
       const int j = gpos / s.L;
       const int e = gpos - j * s.L;
-      const bool on = e + dd <= s.len[j] - 1;
+      const bool on = e + dd <= plen[j - poff] - 1;
       sm.st_tok[x] = on ? __ldg(s.tok + gpos + dd) : -1;
       sm.st_pq[x] = on ? __ldg(s.pq + gpos + dd) : 0;
     }
@@ -369,77 +369,52 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       __syncthreads();
       bool overflowed = false;
       for (int part = 0; part < npart && !overflowed; ++part) {
-        // ---- accumulate this residue class of follower tokens, 32 candidates per warp at a time ----
-        for (int base = warp * 32; base < M; base += nwarps * 32) {
-          const int m = base + lane;
-          int v = -1, u = -1;
-          unsigned p = 0;
-          if (m < M) {
-            if (staged) {
-              v = sm.st_tok[m * D + d - 1];
-              if (v >= 0) { u = d == 1 ? root : sm.st_tok[m * D + d - 2]; p = (unsigned)sm.st_pq[m * D + d - 1]; }
-            } else {
-              const int gpos = mlist[m];
-              const int j = gpos / s.L;
-              if (gpos - j * s.L + d <= s.len[j] - 1) {
-                v = __ldg(s.tok + gpos + d);
-                u = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
-                p = (unsigned)__ldg(s.pq + gpos + d);
-              }
-            }
-            if (v >= 0 && npart > 1 && v % npart != part) v = -1;
+        // ---- accumulate this residue class of follower tokens ----
+        for (int m = tid; m < M; m += blockDim.x) {
+          int v, u;
+          unsigned p;
+          if (staged) {
+            v = sm.st_tok[m * D + d - 1];
+            if (v < 0) continue;
+            u = d == 1 ? root : sm.st_tok[m * D + d - 2];
+            p = (unsigned)sm.st_pq[m * D + d - 1];
+          } else {
+            const int gpos = mlist[m];
+            const int j = gpos / s.L;
+            if (gpos - j * s.L + d > plen[j - poff] - 1) continue;
+            v = __ldg(s.tok + gpos + d);
+            u = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
+            p = (unsigned)__ldg(s.pq + gpos + d);
           }
-          const bool on = v >= 0;
-          const unsigned live = __ballot_sync(FULL, on);
-          if (live == 0) continue;
-          const unsigned gv = __match_any_sync(FULL, v);
-          const unsigned fc = __ballot_sync(FULL, on && u == cur);
-          u64 S_all, S_cur;
-          group_sums(live, gv, gv & fc, p, &S_all, &S_cur);
-          if (on && lane == __ffs(gv) - 1) {                             // one insert per distinct token of the warp
-            unsigned h = slot_hash((unsigned)(v / npart));
-            int slot = -1;
-            for (int probe = 0; probe < CAP; ++probe) {
-              const int old = atomicCAS(&sm.n_key[h], -1, v);
-              if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
-              if (old == -1 || old == v) { slot = (int)h; break; }
-              h = (h + 1) & (CAP - 1);
-            }
-            if (slot < 0) {
-              sh_overflow = 1;
-            } else {
-              add64(&sm.n_Slo[slot], &sm.n_Shi[slot], S_all);
-              atomicAdd(&sm.n_call[slot], (unsigned)__popc(gv));
-              const unsigned cc = __popc(gv & fc);
-              if (cc) { add64(&sm.n_Clo[slot], &sm.n_Chi[slot], S_cur); atomicAdd(&sm.n_ccur[slot], cc); }
-            }
+          if (npart > 1 && v % npart != part) continue;
+          unsigned h = slot_hash((unsigned)(v / npart));
+          int slot = -1;
+          for (int probe = 0; probe < CAP; ++probe) {
+            const int old = atomicCAS(&sm.n_key[h], -1, v);
+            if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
+            if (old == -1 || old == v) { slot = (int)h; break; }
+            h = (h + 1) & (CAP - 1);
           }
+          if (slot < 0) { sh_overflow = 1; continue; }
+          add64(&sm.n_Slo[slot], &sm.n_Shi[slot], p);
+          atomicAdd(&sm.n_call[slot], 1u);
+          if (u == cur) { add64(&sm.n_Clo[slot], &sm.n_Chi[slot], p); atomicAdd(&sm.n_ccur[slot], 1u); }
           if (EXPORT && d > 1) {
             int b = -1;
-            if (on) for (int x = 0; x < nkept; ++x) if (sm.kept[x] == u) { b = x; break; }
-            const bool has_src = b >= 0;
-            const unsigned srcs = __ballot_sync(FULL, has_src);
-            if (srcs) {
-              const unsigned ge = gv & __match_any_sync(FULL, has_src ? u : -1);
-              u64 S_uv, unused;
-              group_sums(srcs, ge, 0u, p, &S_uv, &unused);
-              if (has_src && lane == __ffs(ge) - 1) {
-                const int ekey = v * MAXB + b;                 // (destination, kept source) in one word
-                unsigned he = slot_hash((unsigned)(v / npart) * 37u + (unsigned)b);
-                int es = -1;
-                for (int probe = 0; probe < CAP; ++probe) {
-                  const int old = atomicCAS(&sm.e_key[he], -1, ekey);
-                  if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
-                  if (old == -1 || old == ekey) { es = (int)he; break; }
-                  he = (he + 1) & (CAP - 1);
-                }
-                if (es < 0) {
-                  sh_overflow = 1;
-                } else {
-                  add64(&sm.e_Slo[es], &sm.e_Shi[es], S_uv);
-                  atomicAdd(&sm.e_c[es], (unsigned)__popc(ge));
-                }
+            for (int x = 0; x < nkept; ++x) if (sm.kept[x] == u) { b = x; break; }
+            if (b >= 0) {
+              const int ekey = v * MAXB + b;                 // (destination, kept source) in one word
+              unsigned he = slot_hash((unsigned)(v / npart) * 37u + (unsigned)b);
+              int es = -1;
+              for (int probe = 0; probe < CAP; ++probe) {
+                const int old = atomicCAS(&sm.e_key[he], -1, ekey);
+                if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
+                if (old == -1 || old == ekey) { es = (int)he; break; }
+                he = (he + 1) & (CAP - 1);
               }
+              if (es < 0) { sh_overflow = 1; continue; }
+              add64(&sm.e_Slo[es], &sm.e_Shi[es], p);
+              atomicAdd(&sm.e_c[es], 1u);
             }
           }
         }
@@ -589,10 +564,11 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
 // that follows write_defaults.
 template <bool EXPORT>
 __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                                          int32_t* draft_tok, int32_t* draft_len, float* draft_score,
-                                          float* draft_edge_w) {
-  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, draft_tok, draft_len, draft_score, draft_edge_w);
-  else dag_block<EXPORT>(s, sm, i, M, mlist, draft_tok, draft_len, draft_score, draft_edge_w);
+                                          const int32_t* plen, int poff, int32_t* draft_tok, int32_t* draft_len,
+                                          float* draft_score, float* draft_edge_w) {
+  // plen[j - poff] = length of path j (the prompt's lengths in shared memory, or the global array)
+  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
+  else dag_block<EXPORT>(s, sm, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 template <bool EXPORT>
@@ -610,7 +586,7 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
     return;
   }
   __syncthreads();
-  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], draft_tok, draft_len, draft_score, draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], s.len, 0, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 // Whole draft construction of one query path in one CTA, for prompts whose
@@ -700,29 +676,29 @@ __global__ void __launch_bounds__(kDagThreads) build_fused_kernel(Dev s, int k, 
       my_matches[at] = pos;
     };
     if ((s.L & 3) == 0) {
-      const int per = s.L >> 2, total = s.N * per;
+      // thread t takes the 16-byte chunks t, t + blockDim, ... of every path, eight paths in flight at a time
+      const int per = s.L >> 2;
       const int4* g4 = reinterpret_cast<const int4*>(gtok);
       constexpr int kBatch = 8;
-      for (int x0 = tid; x0 < total; x0 += kBatch * blockDim.x) {
-        int4 w[kBatch];
-        int jn[kBatch], e0[kBatch], e_hi[kBatch];
+      for (int c = tid; c < per; c += blockDim.x) {
+        const int e0 = 4 * c;
+        for (int j0 = 0; j0 < s.N; j0 += kBatch) {
+          int4 w[kBatch];
+          int e_hi[kBatch];
 #pragma unroll
-        for (int r = 0; r < kBatch; ++r) {
-          const int x = x0 + r * blockDim.x;
-          e_hi[r] = -1; e0[r] = 0; jn[r] = 0;
-          if (x < total) {
-            jn[r] = x / per; e0[r] = 4 * (x - jn[r] * per);
-            e_hi[r] = g * s.N + jn[r] == i ? -1 : sh_len[jn[r]] - 2;     // last position with a follower
-            if (e0[r] <= e_hi[r]) w[r] = __ldg(g4 + x);
+          for (int r = 0; r < kBatch; ++r) {
+            const int jn = j0 + r;
+            e_hi[r] = (jn < s.N && g * s.N + jn != i) ? sh_len[jn] - 2 : -1;   // last position with a follower
+            if (e0 <= e_hi[r]) w[r] = __ldg(g4 + (size_t)jn * per + c);
           }
-        }
 #pragma unroll
-        for (int r = 0; r < kBatch; ++r) {
-          if (e0[r] > e_hi[r]) continue;
-          if (w[r].x == last && e0[r] >= k - 1) hit(jn[r], e0[r]);
-          if (w[r].y == last && e0[r] + 1 >= k - 1 && e0[r] + 1 <= e_hi[r]) hit(jn[r], e0[r] + 1);
-          if (w[r].z == last && e0[r] + 2 >= k - 1 && e0[r] + 2 <= e_hi[r]) hit(jn[r], e0[r] + 2);
-          if (w[r].w == last && e0[r] + 3 >= k - 1 && e0[r] + 3 <= e_hi[r]) hit(jn[r], e0[r] + 3);
+          for (int r = 0; r < kBatch; ++r) {
+            if (e0 > e_hi[r]) continue;
+            if (w[r].x == last && e0 >= k - 1) hit(j0 + r, e0);
+            if (w[r].y == last && e0 + 1 >= k - 1 && e0 + 1 <= e_hi[r]) hit(j0 + r, e0 + 1);
+            if (w[r].z == last && e0 + 2 >= k - 1 && e0 + 2 <= e_hi[r]) hit(j0 + r, e0 + 2);
+            if (w[r].w == last && e0 + 3 >= k - 1 && e0 + 3 <= e_hi[r]) hit(j0 + r, e0 + 3);
+          }
         }
       }
     } else {
@@ -741,8 +717,8 @@ __global__ void __launch_bounds__(kDagThreads) build_fused_kernel(Dev s, int k, 
     if (tid == 0) draft_len[i] = 0;
     return;
   }
-  dag_phase<EXPORT>(s, sm, i, M, M <= kListCap ? sm.list : my_matches, draft_tok, draft_len, draft_score,
-                    draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, M, M <= kListCap ? sm.list : my_matches, sh_len, g * s.N, draft_tok, draft_len,
+                    draft_score, draft_edge_w);
 }
 
 }  // namespace

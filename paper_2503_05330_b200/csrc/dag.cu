@@ -572,7 +572,7 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
 }
 
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
+__global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
                                                           int32_t* __restrict__ draft_len,
                                                           float* __restrict__ draft_score,
                                                           float* __restrict__ draft_edge_w) {
@@ -597,7 +597,7 @@ __global__ void __launch_bounds__(kDagThreads) dag_kernel(Dev s, int32_t* __rest
 // gather / DAG / search phase runs on the matches just found.  The matches also
 // go to the path's private slice of the match list for inspection.
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads) build_fused_kernel(Dev s, int k, int32_t* __restrict__ draft_tok,
+__global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int k, int32_t* __restrict__ draft_tok,
                                                                   int32_t* __restrict__ draft_len,
                                                                   float* __restrict__ draft_score,
                                                                   float* __restrict__ draft_edge_w) {

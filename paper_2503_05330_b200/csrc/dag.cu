@@ -41,18 +41,31 @@ struct Cand {            // a node or an edge competing in a selection
   double w; u64 S; unsigned cnt; int tok; int valid;
 };
 
+// Lane holding the first candidate in rank order (largest weight, then smallest
+// token) among the lanes with valid set, or -1.  Weights are non-negative, so
+// their bit patterns order like the values: three full-warp reductions settle it.
+__device__ __forceinline__ int warp_arg_first(bool valid, double w, int tok) {
+  const u64 bits = (u64)__double_as_longlong(w);
+  const unsigned hi = (unsigned)(bits >> 32), lo = (unsigned)bits;
+  if (__ballot_sync(FULL, valid) == 0) return -1;
+  const unsigned mh = __reduce_max_sync(FULL, valid ? hi : 0u);
+  const bool c1 = valid && hi == mh;
+  const unsigned ml = __reduce_max_sync(FULL, c1 ? lo : 0u);
+  const bool c2 = c1 && lo == ml;
+  const unsigned mt = __reduce_min_sync(FULL, c2 ? (unsigned)tok : 0xffffffffu);
+  return __ffs(__ballot_sync(FULL, c2 && (unsigned)tok == mt)) - 1;
+}
+
 __device__ __forceinline__ Cand warp_best(Cand c) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    Cand x;
-    x.w = __shfl_xor_sync(FULL, c.w, o);
-    x.S = __shfl_xor_sync(FULL, c.S, o);
-    x.cnt = __shfl_xor_sync(FULL, c.cnt, o);
-    x.tok = __shfl_xor_sync(FULL, c.tok, o);
-    x.valid = __shfl_xor_sync(FULL, c.valid, o);
-    if (x.valid && (!c.valid || ranks_before(x.w, x.tok, c.w, c.tok))) c = x;
-  }
-  return c;
+  const int src = warp_arg_first(c.valid != 0, c.w, c.tok);
+  const int from = src < 0 ? 0 : src;
+  Cand r;
+  r.valid = src >= 0;
+  r.w = __shfl_sync(FULL, c.w, from);
+  r.S = __shfl_sync(FULL, c.S, from);
+  r.cnt = __shfl_sync(FULL, c.cnt, from);
+  r.tok = __shfl_sync(FULL, c.tok, from);
+  return r;
 }
 
 // The K first candidates in rank order among get(0..ncand-1); lane 0 stores them.
@@ -214,6 +227,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   int* L_u = sm.st_tok + 32 * SDMS_MAX_DRAFT;
   unsigned* L_lead = reinterpret_cast<unsigned*>(sm.st_tok + 2 * 32 * SDMS_MAX_DRAFT);
   unsigned* L_elead = L_lead + SDMS_MAX_DRAFT;
+  unsigned* L_best = L_elead + SDMS_MAX_DRAFT;      // per layer: the best edge out of each source / the best node
   double* L_W = reinterpret_cast<double*>(sm.st_pq);
   double* L_we = L_W + 32 * SDMS_MAX_DRAFT;
 
@@ -241,9 +255,23 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
     const double W = eq5_weight(s.alpha, S_all, c_all);
     const double w_uv = eq5_weight(s.alpha, S_uv, c_uv);
     const unsigned leaders = __ballot_sync(FULL, leader), eleaders = __ballot_sync(FULL, eleader);
+    // is this edge the best way out of its source, judged by the score of its destination?
+    bool beaten = false;
+    for (unsigned rem = eleaders; rem; rem &= rem - 1) {
+      const int src = __ffs(rem) - 1;
+      const int ou = __shfl_sync(FULL, u, src);
+      const int ot = __shfl_sync(FULL, v, src);
+      const double oW = __shfl_sync(FULL, W, src);
+      if (ou == u && ranks_before(oW, ot, W, v)) beaten = true;
+    }
+    const unsigned best_out = __ballot_sync(FULL, eleader && !beaten);
+    const int top = s.mode == 1 ? warp_arg_first(leader, W, v) : -1;   // best node of the layer
     L_v[(d - 1) * 32 + lane] = v; L_u[(d - 1) * 32 + lane] = u;
     L_W[(d - 1) * 32 + lane] = W; L_we[(d - 1) * 32 + lane] = w_uv;
-    if (lane == 0) { L_lead[d - 1] = leaders; L_elead[d - 1] = eleaders; }
+    if (lane == 0) {
+      L_lead[d - 1] = leaders; L_elead[d - 1] = eleaders;
+      L_best[d - 1] = s.mode == 1 ? (top >= 0 ? 1u << top : 0u) : best_out;
+    }
     if (EXPORT && live) {
       int rank = 0;
       for (unsigned rem = leaders; rem; rem &= rem - 1) {
@@ -298,20 +326,21 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   int cur = root, emitted = 0;
   for (int d = 1; d <= D; ++d) {
     const int v = L_v[(d - 1) * 32 + lane], u = L_u[(d - 1) * 32 + lane];
-    const bool el = L_elead[d - 1] >> lane & 1, ld = L_lead[d - 1] >> lane & 1;
-    Cand c;
-    c.valid = s.mode == 1 ? ld : (el && u == cur);
-    c.w = L_W[(d - 1) * 32 + lane]; c.tok = v; c.S = 0; c.cnt = 0;
-    c = warp_best(c);
-    if (!c.valid) break;
-    const unsigned emask = __ballot_sync(FULL, el && u == cur && v == c.tok);   // the edge taken, if it exists
+    const unsigned from_cur = __ballot_sync(FULL, u == cur);
+    const unsigned pick = s.mode == 1 ? L_best[d - 1] : (L_best[d - 1] & from_cur);
+    if (pick == 0) break;
+    const int src = __ffs(pick) - 1;
+    const int tok = __shfl_sync(FULL, v, src);
+    const double W = __shfl_sync(FULL, L_W[(d - 1) * 32 + lane], src);
+    // the edge taken: in mode 0 the picked lane leads it; in mode 1 it may not exist
+    const unsigned emask = L_elead[d - 1] & from_cur & __ballot_sync(FULL, v == tok);
     const double we = __shfl_sync(FULL, L_we[(d - 1) * 32 + lane], emask ? __ffs(emask) - 1 : 0);
     if (lane == 0) {
-      draft_tok[(size_t)i * D + (d - 1)] = c.tok;
-      if (draft_score) draft_score[(size_t)i * D + (d - 1)] = (float)c.w;
+      draft_tok[(size_t)i * D + (d - 1)] = tok;
+      if (draft_score) draft_score[(size_t)i * D + (d - 1)] = (float)W;
       if (draft_edge_w) draft_edge_w[(size_t)i * D + (d - 1)] = emask ? (float)we : 0.0f;
     }
-    cur = c.tok;
+    cur = tok;
     ++emitted;
   }
   if (lane == 0) draft_len[i] = emitted;
@@ -676,10 +705,10 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
       my_matches[at] = pos;
     };
     if ((s.L & 3) == 0) {
-      // thread t takes the 16-byte chunks t, t + blockDim, ... of every path, eight paths in flight at a time
+      // thread t takes the 16-byte chunks t, t + blockDim, ... of every path, sixteen paths in flight at a time
       const int per = s.L >> 2;
       const int4* g4 = reinterpret_cast<const int4*>(gtok);
-      constexpr int kBatch = 8;
+      constexpr int kBatch = 16;
       for (int c = tid; c < per; c += blockDim.x) {
         const int e0 = 4 * c;
         for (int j0 = 0; j0 < s.N; j0 += kBatch) {

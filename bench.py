@@ -216,6 +216,7 @@ class Runner:
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         units = 0
         done = 0
+        ks = []
         if e2e:
             h_acc = torch.empty(w.P, dtype=torch.int32).pin_memory()
             h_tok = torch.empty((w.P, w.D), dtype=torch.int32).pin_memory()
@@ -246,10 +247,16 @@ class Runner:
                     s.accept(plan["sampled"][step], plan["lp"][step])
                     b.record()
                 units += plan["active"][step]
+                ks.append(k_of(step, w.k_max))
                 done += 1
         torch.cuda.synchronize()
-        ms = sum(a.elapsed_time(b) for a, b in ev)
-        return ms, units
+        per_step = [a.elapsed_time(b) for a, b in ev]
+        self.last_by_k = {}
+        for kk in range(1, w.k_max + 1):
+            t = [per_step[x] for x in range(K) if ks[x] == kk]
+            if t:
+                self.last_by_k[str(kk)] = 1e3 * float(np.mean(t))
+        return sum(per_step), units
 
 
 def ours_main(args, w):
@@ -277,6 +284,7 @@ def ours_main(args, w):
     launches0 = binding.sdms_launch_count(run.s.ctx)
     t0 = time.perf_counter()
     ms, units = run.timed_steps(args.steps)
+    by_k = dict(run.last_by_k)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -295,6 +303,21 @@ def ours_main(args, w):
     binding.sdms_profile_enable(run.s.ctx, False)
     # warm-L2 figure for context (no flush between steps)
     ms_warm, units_warm = run.timed_steps(args.steps, flush=False)
+    # the DAG export is an inspection call outside the step: time it once per build on a short replay
+    export_us = None
+    if args.dag_nodes > 0:
+        run.start_run()
+        evs = []
+        for step in range(min(plan["steps"], 200)):
+            run.s.build_drafts(k_of(step, w.k_max))
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            dag = run.s.dag_device()
+            b.record()
+            evs.append((a, b))
+            run.s.accept(plan["sampled"][step], plan["lp"][step])
+        torch.cuda.synchronize()
+        export_us = 1e3 * float(np.mean([a.elapsed_time(b) for a, b in evs]))
 
     if world > 1:
         t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
@@ -341,7 +364,10 @@ def ours_main(args, w):
         "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
         "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
-        "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges},
+        "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
+        "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
+                       "us_per_sdms_get_dag_call": export_us,
+                       "note": "inspection call that re-aggregates the last build's matches; not part of a step"},
     }
     if world == 1 and not args.no_cpu_baseline:
         units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 4 * w.steps, 20.0)

@@ -69,7 +69,7 @@ typedef struct {
   int32_t  k_max;                /* largest query suffix length that will be asked for        */
   int32_t  max_draft_len;        /* D: the paper's maximum draft token length                 */
   int32_t  max_append;           /* most tokens a path may gain per sdms_accept commit        */
-  int32_t  dag_nodes_per_layer;  /* B: nodes kept per layer in the DAG export, 0 = no export  */
+  int32_t  dag_nodes_per_layer;  /* B: nodes kept per layer by sdms_get_dag, 0 = no export     */
   int32_t  dag_edges_per_node;   /* Ke: out-edges kept per exported node                      */
   int32_t  search_mode;          /* 0: walk to the best successor of the current node;
                                     1: best node of each layer regardless of the previous one */
@@ -146,7 +146,10 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
  * d_offsets always holds the true counts. */
 int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t cap, void* stream);
 
-/* DAG export of the last sdms_build_drafts (needs dag_nodes_per_layer > 0).
+/* DAG export of the last sdms_build_drafts (needs dag_nodes_per_layer > 0).  The
+ * call aggregates the same matches once more and this time ranks and writes out
+ * the nodes and edges; the histories must not have changed since that build
+ * (an append or a committing accept in between gives SDMS_ERR_BAD_STATE).
  * Layer index d-1 for d = 1..D.  Per layer the B best nodes by (score desc,
  * token asc): node_tok/node_S/node_cnt [P][D][B] (unused token -1), the true
  * number of nodes node_count [P][D].  Per kept node of layer d its Ke best

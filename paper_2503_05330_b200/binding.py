@@ -262,6 +262,9 @@ class Sdms:
         return offsets.cpu(), gpos[:total].cpu()
 
     def dag(self):
+        return {k: v.cpu().numpy() for k, v in self.dag_device().items()}
+
+    def dag_device(self):
         P, D, B, Ke, dev = self.P, self.D, self.B, self.Ke, self.device
         r = dict(node_tok=torch.empty((P, D, B), dtype=torch.int32, device=dev),
                  node_S=torch.empty((P, D, B), dtype=torch.int64, device=dev),
@@ -273,7 +276,7 @@ class Sdms:
                  out_degree=torch.empty((P, D, B), dtype=torch.int32, device=dev))
         sdms_get_dag(self.ctx, r["node_tok"], r["node_S"], r["node_cnt"], r["node_count"], r["edge_dst"],
                      r["edge_S"], r["edge_cnt"], r["out_degree"])
-        return {k: v.cpu().numpy() for k, v in r.items()}
+        return r
 
     def query_modes(self):
         modes = torch.empty(self.P, dtype=torch.int32, device=self.device)

@@ -13,7 +13,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t tok, pq, len, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, matches;
-  size_t x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
+  size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
   size_t total;
   uint32_t table_cap;
   int64_t match_cap;
@@ -63,6 +63,7 @@ Layout make_layout(const sdms_config* c) {
   l.q_off = take(P * 4); l.q_cursor = take(P * 4);
   l.g_nscan = take((size_t)c->num_groups * 4);
   l.matches = take((size_t)mc * 4);
+  l.x_draft_tok = take(P * D * 4); l.x_draft_len = take(P * 4);
   l.x_node_tok = take(P * D * B * 4); l.x_node_S = take(P * D * B * 8); l.x_node_cnt = take(P * D * B * 4);
   l.x_node_count = take(P * D * 4);
   l.x_edge_dst = take(P * D * B * Ke * 4); l.x_edge_S = take(P * D * B * Ke * 8);
@@ -83,6 +84,7 @@ struct sdms_ctx {
   uint64_t launches;
   bool profiling;
   bool built;
+  int32_t* x_draft_tok; int32_t* x_draft_len;   // where the export pass leaves the drafts it recomputes
   std::vector<EventPair> pending;
   std::vector<EventPair> pool;
   float prof_ms[SDMS_NUM_KERNELS];
@@ -155,6 +157,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.q_reserved = (int32_t*)(w + lay.q_reserved); d.q_off = (int32_t*)(w + lay.q_off);
   d.q_cursor = (int32_t*)(w + lay.q_cursor); d.g_nscan = (int32_t*)(w + lay.g_nscan);
   d.matches = (int32_t*)(w + lay.matches);
+  ctx->x_draft_tok = (int32_t*)(w + lay.x_draft_tok); ctx->x_draft_len = (int32_t*)(w + lay.x_draft_len);
   d.x_node_tok = (int32_t*)(w + lay.x_node_tok); d.x_node_S = (int64_t*)(w + lay.x_node_S);
   d.x_node_cnt = (int32_t*)(w + lay.x_node_cnt); d.x_node_count = (int32_t*)(w + lay.x_node_count);
   d.x_edge_dst = (int32_t*)(w + lay.x_edge_dst); d.x_edge_S = (int64_t*)(w + lay.x_edge_S);
@@ -185,6 +188,7 @@ int sdms_append(sdms_ctx* ctx, const int32_t* d_tokens, const float* d_logprobs,
                 int32_t row_width, void* stream) {
   if (!ctx || !d_tokens || !d_logprobs || !d_counts || row_width < 1) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  ctx->built = false;
   return timed(ctx, SDMS_KERNEL_APPEND, st,
                [&] { return launch_append(ctx->dev, d_tokens, d_logprobs, d_counts, row_width, st); });
 }
@@ -205,7 +209,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
   if (rc != SDMS_OK) return rc;
   rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
-    return launch_dag(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+    return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
   if (rc == SDMS_OK) ctx->built = true;
   return rc;
 }
@@ -214,6 +218,7 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
                 const float* d_sampled_logprobs, int32_t* d_accept_len, void* stream) {
   if (!ctx || !d_draft_tok || !d_draft_len || !d_sampled || !d_accept_len) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  if (d_sampled_logprobs) ctx->built = false;          // the commit changes the histories
   return timed(ctx, SDMS_KERNEL_ACCEPT, st, [&] {
     return launch_accept(ctx->dev, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, st); });
 }
@@ -234,6 +239,10 @@ int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t*
   cudaStream_t st = (cudaStream_t)stream;
   const Dev& d = ctx->dev;
   const size_t nb = (size_t)d.P * d.D * d.B, ne = nb * d.Ke;
+  // aggregate again over the matches of the last build, this time keeping the ranked nodes and edges
+  const int rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
+    return launch_dag(d, true, ctx->x_draft_tok, ctx->x_draft_len, nullptr, nullptr, st); });
+  if (rc != SDMS_OK) return rc;
   bool ok = true;
   auto copy = [&](void* dst, const void* src, size_t bytes) {
     if (dst && bytes) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;

@@ -761,15 +761,12 @@ cudaError_t dag_kernel_setup() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)dag_smem_bytes<false>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(build_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)dag_smem_bytes<true>());
   return e;
 }
 
-cudaError_t launch_dag(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                        float* draft_edge_w, cudaStream_t stream) {
-  if (s.B > 0)
+  if (with_export)
     dag_kernel<true><<<s.P, kDagThreads, dag_smem_bytes<true>(), stream>>>(s, draft_tok, draft_len, draft_score,
                                                                           draft_edge_w);
   else
@@ -780,12 +777,8 @@ cudaError_t launch_dag(const Dev& s, int32_t* draft_tok, int32_t* draft_len, flo
 
 cudaError_t launch_build_fused(const Dev& s, int k, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                                float* draft_edge_w, cudaStream_t stream) {
-  if (s.B > 0)
-    build_fused_kernel<true><<<s.P, kDagThreads, dag_smem_bytes<true>(), stream>>>(s, k, draft_tok, draft_len,
-                                                                                   draft_score, draft_edge_w);
-  else
-    build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, k, draft_tok, draft_len,
-                                                                                    draft_score, draft_edge_w);
+  build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, k, draft_tok, draft_len,
+                                                                                  draft_score, draft_edge_w);
   return cudaGetLastError();
 }
 

@@ -259,6 +259,26 @@ class Runner:
         return sum(per_step), units
 
 
+def rank_seed(w, rank):
+    """Every rank owns its own prompts: same recipe, different seed."""
+    return synth.BASE_SEED + w.index + 7919 * rank
+
+
+def whole_job(times_ms, units, device):
+    """Whole-job figures over all ranks: the slowest rank's time (MAX) and the
+    units of all ranks (SUM).  Works with any initialised process group; without
+    one it returns its inputs."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(times_ms), list(units)
+    t = torch.tensor(times_ms, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    u = torch.tensor(units, dtype=torch.float64, device=device)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return t.tolist(), u.tolist()
+
+
 def ours_main(args, w):
     import torch
     import torch.distributed as dist
@@ -272,7 +292,7 @@ def ours_main(args, w):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     device = f"cuda:{local}"
     # every rank owns its own prompts (different seed): no data-path collective
-    run = Runner(w, synth.BASE_SEED + w.index + 7919 * rank, device, args.dag_nodes, args.dag_edges)
+    run = Runner(w, rank_seed(w, rank), device, args.dag_nodes, args.dag_edges)
     plan = run.dry_run()
 
     run.timed_steps(max(args.warmup, 3))
@@ -319,13 +339,7 @@ def ours_main(args, w):
         torch.cuda.synchronize()
         export_us = 1e3 * float(np.mean([a.elapsed_time(b) for a, b in evs]))
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        u = torch.tensor([units, units_e2e], dtype=torch.float64, device=device)
-        dist.all_reduce(u, op=dist.ReduceOp.SUM)
-        ms, ms_e2e = t.tolist()
-        units, units_e2e = u.tolist()
+    (ms, ms_e2e), (units, units_e2e) = whole_job([ms, ms_e2e], [units, units_e2e], device)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

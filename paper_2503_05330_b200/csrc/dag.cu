@@ -34,6 +34,7 @@ constexpr int CAP = kDagCap;
 constexpr int MAXB = SDMS_MAX_DAG_NODES;
 constexpr int MAXKE = SDMS_MAX_DAG_EDGES;
 constexpr int kStageWords = 8192;      // followers (token, pq) of all matches staged in shared memory when M*D fits
+constexpr int kLoadBatch = 4;          // candidates a thread loads before it touches the tables
 constexpr int kListCap = 2048;         // matches a fused CTA keeps in shared memory besides its global slice
 static_assert(kStageWords >= 4 * 32 * SDMS_MAX_DRAFT, "dag_small keeps its per-layer lanes in the staging area");
 
@@ -391,6 +392,13 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
     if (!walking && !EXPORT) break;
     const int cur = sh_cur;
     const int nkept = EXPORT ? sh_nkept : 0;
+    const bool restricted = !EXPORT && !staged && s.mode == 0 && d > 1;    // staged candidates are cheap to revisit
+    if (!EXPORT) {
+      // first layer (or every layer in mode 1): every distinct follower is a node, guess one per four
+      // candidates; restricted layers only hold the successors of one node
+      npart = 1;
+      if (!restricted) while (npart * (CAP / 2) * 4 < M && npart < npart_max) npart *= 2;
+    }
     bool layer_done = false;
     while (!layer_done) {
       if (tid == 0) { sh_best_valid = 0; sh_nnode_run = 0; sh_node_total = 0; }
@@ -399,53 +407,81 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       bool overflowed = false;
       for (int part = 0; part < npart && !overflowed; ++part) {
         // ---- accumulate this residue class of follower tokens ----
-        for (int m = tid; m < M; m += blockDim.x) {
-          int v, u;
-          unsigned p;
-          if (staged) {
-            v = sm.st_tok[m * D + d - 1];
-            if (v < 0) continue;
-            u = d == 1 ? root : sm.st_tok[m * D + d - 2];
-            p = (unsigned)sm.st_pq[m * D + d - 1];
-          } else {
-            const int gpos = mlist[m];
-            const int j = gpos / s.L;
-            if (gpos - j * s.L + d > plen[j - poff] - 1) continue;
-            v = __ldg(s.tok + gpos + d);
-            u = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
-            p = (unsigned)__ldg(s.pq + gpos + d);
-          }
-          if (npart > 1 && v % npart != part) continue;
-          unsigned h = slot_hash((unsigned)(v / npart));
-          int slot = -1;
-          for (int probe = 0; probe < CAP; ++probe) {
-            const int old = atomicCAS(&sm.n_key[h], -1, v);
-            if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
-            if (old == -1 || old == v) { slot = (int)h; break; }
-            h = (h + 1) & (CAP - 1);
-          }
-          if (slot < 0) { sh_overflow = 1; continue; }
-          add64(&sm.n_Slo[slot], &sm.n_Shi[slot], p);
-          atomicAdd(&sm.n_call[slot], 1u);
-          if (u == cur) { add64(&sm.n_Clo[slot], &sm.n_Chi[slot], p); atomicAdd(&sm.n_ccur[slot], 1u); }
-          if (EXPORT && d > 1) {
-            int b = -1;
-            for (int x = 0; x < nkept; ++x) if (sm.kept[x] == u) { b = x; break; }
-            if (b >= 0) {
-              const int ekey = v * MAXB + b;                 // (destination, kept source) in one word
-              unsigned he = slot_hash((unsigned)(v / npart) * 37u + (unsigned)b);
-              int es = -1;
-              for (int probe = 0; probe < CAP; ++probe) {
-                const int old = atomicCAS(&sm.e_key[he], -1, ekey);
-                if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
-                if (old == -1 || old == ekey) { es = (int)he; break; }
-                he = (he + 1) & (CAP - 1);
+        // Walking in mode 0 past the first layer, only successors of the current node can be chosen:
+        // phase 0 claims a slot for each of them, phase 1 adds every candidate that lands on a claimed
+        // slot.  Otherwise one phase claims and adds.
+        for (int phase = restricted ? 0 : 1; phase < 2; ++phase) {
+          for (int m0 = tid; m0 < M; m0 += kLoadBatch * blockDim.x) {
+            int v[kLoadBatch], u[kLoadBatch];
+            unsigned p[kLoadBatch];
+#pragma unroll
+            for (int r = 0; r < kLoadBatch; ++r) {                    // loads of the whole batch go out together
+              const int m = m0 + r * blockDim.x;
+              v[r] = -1; u[r] = -1; p[r] = 0;
+              if (m >= M) continue;
+              if (staged) {
+                v[r] = sm.st_tok[m * D + d - 1];
+                if (v[r] >= 0) { u[r] = d == 1 ? root : sm.st_tok[m * D + d - 2]; p[r] = (unsigned)sm.st_pq[m * D + d - 1]; }
+              } else {
+                const int gpos = mlist[m];
+                const int j = gpos / s.L;
+                if (gpos - j * s.L + d <= plen[j - poff] - 1) {
+                  v[r] = __ldg(s.tok + gpos + d);
+                  u[r] = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
+                  p[r] = (unsigned)__ldg(s.pq + gpos + d);
+                }
               }
-              if (es < 0) { sh_overflow = 1; continue; }
-              add64(&sm.e_Slo[es], &sm.e_Shi[es], p);
-              atomicAdd(&sm.e_c[es], 1u);
+            }
+#pragma unroll
+            for (int r = 0; r < kLoadBatch; ++r) {
+              const int vv = v[r], uu = u[r];
+              const unsigned pp = p[r];
+              if (vv < 0 || (npart > 1 && vv % npart != part)) continue;
+              if (phase == 0 && uu != cur) continue;
+              unsigned h = slot_hash((unsigned)(vv / npart));
+              int slot = -1;
+              if (phase == 1 && restricted) {                          // read-only: is vv a claimed successor?
+                for (int probe = 0; probe < CAP; ++probe) {
+                  const int key = sm.n_key[h];
+                  if (key == vv) { slot = (int)h; break; }
+                  if (key == -1) break;
+                  h = (h + 1) & (CAP - 1);
+                }
+                if (slot < 0) continue;
+              } else {
+                for (int probe = 0; probe < CAP; ++probe) {
+                  const int old = atomicCAS(&sm.n_key[h], -1, vv);
+                  if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
+                  if (old == -1 || old == vv) { slot = (int)h; break; }
+                  h = (h + 1) & (CAP - 1);
+                }
+                if (slot < 0) { sh_overflow = 1; continue; }
+                if (phase == 0) continue;
+              }
+              add64(&sm.n_Slo[slot], &sm.n_Shi[slot], pp);
+              atomicAdd(&sm.n_call[slot], 1u);
+              if (uu == cur) { add64(&sm.n_Clo[slot], &sm.n_Chi[slot], pp); atomicAdd(&sm.n_ccur[slot], 1u); }
+              if (EXPORT && d > 1) {
+                int b = -1;
+                for (int x = 0; x < nkept; ++x) if (sm.kept[x] == uu) { b = x; break; }
+                if (b >= 0) {
+                  const int ekey = vv * MAXB + b;               // (destination, kept source) in one word
+                  unsigned he = slot_hash((unsigned)(vv / npart) * 37u + (unsigned)b);
+                  int es = -1;
+                  for (int probe = 0; probe < CAP; ++probe) {
+                    const int old = atomicCAS(&sm.e_key[he], -1, ekey);
+                    if (old == -1) sm.e_touch[atomicAdd(&sh_ne, 1)] = (int)he;
+                    if (old == -1 || old == ekey) { es = (int)he; break; }
+                    he = (he + 1) & (CAP - 1);
+                  }
+                  if (es < 0) { sh_overflow = 1; continue; }
+                  add64(&sm.e_Slo[es], &sm.e_Shi[es], pp);
+                  atomicAdd(&sm.e_c[es], 1u);
+                }
+              }
             }
           }
+          if (phase == 0) __syncthreads();
         }
         __syncthreads();
         const int nn = sh_nn, ne = EXPORT ? sh_ne : 0;
@@ -607,6 +643,7 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
                                                           float* __restrict__ draft_edge_w) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
+  __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   const int i = blockIdx.x;
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
   const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
@@ -614,8 +651,11 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
     if (threadIdx.x == 0) draft_len[i] = 0;
     return;
   }
+  const int g = i / s.N;
+  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   __syncthreads();
-  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], s.len, 0, draft_tok, draft_len, draft_score, draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, draft_tok, draft_len, draft_score,
+                    draft_edge_w);
 }
 
 // Whole draft construction of one query path in one CTA, for prompts whose

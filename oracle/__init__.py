@@ -46,6 +46,7 @@ def lib():
         for name in ("orc_append", "orc_append_fixed", "orc_accept_commit"):
             getattr(l, name).restype = C.c_uint32
         l.orc_num_matches.restype = C.c_int
+        l.orc_edit_distance.restype = C.c_int
         l.orc_get_draft.restype = C.c_int
         _lib = l
     return _lib
@@ -55,6 +56,11 @@ def prob_to_fixed(lp: float) -> int:
     return int(lib().orc_prob_to_fixed(C.c_float(lp)))
 
 
+def edit_distance(a, b) -> int:
+    a = np.ascontiguousarray(a, dtype=np.int32); b = np.ascontiguousarray(b, dtype=np.int32)
+    return int(lib().orc_edit_distance(_ptr(a, C.c_int32), C.c_int(len(a)), _ptr(b, C.c_int32), C.c_int(len(b))))
+
+
 def weight(alpha: float, S: int, cnt: int) -> float:
     return float(lib().orc_weight(C.c_float(alpha), C.c_int64(S), C.c_int64(cnt)))
 
@@ -62,12 +68,14 @@ def weight(alpha: float, S: int, cnt: int) -> float:
 class Oracle:
     """State of G prompts x N paths and the per-path draft construction."""
 
-    def __init__(self, G, N, L, V, D, alpha=1.0, mode=0):
+    def __init__(self, G, N, L, V, D, alpha=1.0, mode=0, eps=0):
         self.G, self.N, self.L, self.V, self.D = G, N, L, V, D
+        self.eps = eps
         self.P = G * N
         self.alpha, self.mode = alpha, mode
         self._l = lib()
         self._h = C.c_void_p(self._l.orc_create(G, N, L, V, D, C.c_float(alpha), mode))
+        self._l.orc_set_epsilon(self._h, C.c_int(eps))
 
     def __del__(self):
         if getattr(self, "_h", None):

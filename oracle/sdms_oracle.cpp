@@ -8,7 +8,9 @@
 //                Construction"), with the model probability of every generated
 //                token (the p_theta of Eq. 5).
 //   match      - Eq. 3: every position of every OTHER path of the same prompt
-//                whose prefix ends with the query path's k-token suffix.
+//                whose prefix ends with the query path's k-token suffix; with a
+//                tolerance eps (Eq. 4, "Fuzzy Suffix Matching") every position
+//                where some window s' ends with edit distance delta(q, s') <= eps.
 //   candidates - the tokens following each match (at most D of them).
 //   DAG        - "Consensus-Driven Draft Extraction": layer d holds the distinct
 //                d-th follower tokens; edge (u,v) between layers d-1 and d
@@ -33,7 +35,8 @@
 // Pins (tests/, CPU only): hand-worked example from Eq. 3 / Eq. 5 with dyadic
 // probabilities; match set against regex/numpy searches and closed-form counts;
 // alpha = 0 against collections.Counter; conservation invariants; enumeration
-// of every root-to-node DAG path; pq against 50-digit decimal arithmetic;
+// of every root-to-node DAG path; fuzzy matches against exact search for every
+// string within one edit of the query; pq against 50-digit decimal arithmetic;
 // acceptance against os.path.commonprefix.  Behaviour on real model traces
 // (the paper's Table 1) is "parity unpinned": it needs the models and datasets.
 #include <cmath>
@@ -68,6 +71,7 @@ struct PathResult {
 
 struct Ctx {
   int G, N, L, V, D, mode;
+  int eps = 0;                                  // edit-distance tolerance of the suffix match (Eq. 4)
   double alpha;
   std::vector<std::vector<int32_t>> tok, pq;
   std::vector<PathResult> res;
@@ -114,6 +118,27 @@ uint32_t append_impl(Ctx* c, const int32_t* tokens, const float* logprobs, const
   return st;
 }
 
+// Textbook Levenshtein distance (unit costs) between a[0..na) and b[0..nb).
+int edit_distance(const int32_t* a, int na, const int32_t* b, int nb) {
+  std::vector<std::vector<int>> dp(na + 1, std::vector<int>(nb + 1, 0));
+  for (int x = 0; x <= na; ++x) dp[x][0] = x;
+  for (int y = 0; y <= nb; ++y) dp[0][y] = y;
+  for (int x = 1; x <= na; ++x)
+    for (int y = 1; y <= nb; ++y)
+      dp[x][y] = std::min({dp[x - 1][y] + 1, dp[x][y - 1] + 1, dp[x - 1][y - 1] + (a[x - 1] != b[y - 1] ? 1 : 0)});
+  return dp[na][nb];
+}
+
+// Eq. 4: does some window s' of path y that ends at e satisfy delta(q, s') <= eps?  Windows within eps of
+// the query's length are the only ones that can; the empty window is not a match.
+bool fuzzy_end(const std::vector<int32_t>& y, int e, const int32_t* q, int k, int eps) {
+  for (int n = std::max(1, k - eps); n <= k + eps; ++n) {
+    if (e - n + 1 < 0) continue;
+    if (edit_distance(q, k, y.data() + (e - n + 1), n) <= eps) return true;
+  }
+  return false;
+}
+
 void build_path(Ctx* c, int k, int i) {
   PathResult& r = c->res[i];
   r = PathResult();
@@ -130,6 +155,11 @@ void build_path(Ctx* c, int k, int i) {
     if (j == i) continue;
     const std::vector<int32_t>& yj = c->tok[j];
     int len_j = (int)yj.size();
+    if (c->eps > 0) {                              // "Fuzzy Suffix Matching": each end position counts once
+      for (int e = 0; e <= len_j - 2; ++e)
+        if (fuzzy_end(yj, e, yi.data() + (len_i - k), k, c->eps)) r.matches.push_back({j, e});
+      continue;
+    }
     for (int e = k - 1; e <= len_j - 2; ++e) {
       bool same = true;
       for (int t = 0; t < k; ++t)
@@ -160,11 +190,15 @@ void build_path(Ctx* c, int k, int i) {
       int v = kv.first;
       auto it = r.edges[d - 1].find({cur, v});
       bool succ = it != r.edges[d - 1].end();
-      if (c->mode == 0 && !succ) continue;
+      // fuzzy matches may end in different tokens: the walk then starts from a virtual root that
+      // precedes all of them, so every first-layer node is a successor and the edge taken carries
+      // everything that enters the node
+      const bool from_virtual_root = d == 1 && c->eps > 0;
+      if (c->mode == 0 && !succ && !from_virtual_root) continue;
       double w = weight(c->alpha, kv.second.S, kv.second.cnt);
       if (!found || w > best_w) {                 // strict: ties keep the smaller token
         found = true; best_v = v; best_w = w;
-        best_e = succ ? weight(c->alpha, it->second.S, it->second.cnt) : 0.0;
+        best_e = from_virtual_root ? w : (succ ? weight(c->alpha, it->second.S, it->second.cnt) : 0.0);
       }
     }
     if (!found) break;
@@ -190,6 +224,11 @@ void* orc_create(int G, int N, int L, int V, int D, float alpha, int mode) {
 }
 
 void orc_destroy(void* h) { delete (Ctx*)h; }
+
+// Edit-distance tolerance of the suffix match (Eq. 4); 0 = exact matching.
+void orc_set_epsilon(void* h, int eps) { ((Ctx*)h)->eps = eps; }
+
+int orc_edit_distance(const int32_t* a, int na, const int32_t* b, int nb) { return edit_distance(a, na, b, nb); }
 
 int32_t orc_prob_to_fixed(float lp) { return prob_to_fixed(lp, nullptr); }
 

@@ -455,3 +455,125 @@ def test_append_rules_and_status():
     assert st == 0                                        # the NaN entry was not among the appended
     st = o.append(tok, np.full((4, 4), np.nan, np.float32), np.array([0, 1, 0, 0], np.int32))
     assert st == oracle.ST_BAD_LOGPROB and o.history(1)[1][-1] == 0
+
+
+# ----------------------------------------------------------------------------
+# fuzzy suffix matching (Eq. 4, tolerance 1)
+# ----------------------------------------------------------------------------
+def test_edit_distance_textbook_values_and_properties():
+    enc = lambda w: [ord(ch) for ch in w]
+    assert oracle.edit_distance(enc("kitten"), enc("sitting")) == 3
+    assert oracle.edit_distance(enc("flaw"), enc("lawn")) == 2
+    assert oracle.edit_distance(enc("abc"), enc("abc")) == 0
+    assert oracle.edit_distance(enc("abc"), enc("")) == 3
+    rng = synth.Stream(606)
+    for _ in range(200):
+        a = (rng.uniform(1 + int(rng.one() * 5)) * 3).astype(int).tolist()
+        b = (rng.uniform(1 + int(rng.one() * 5)) * 3).astype(int).tolist()
+        d = oracle.edit_distance(a, b)
+        assert d == oracle.edit_distance(b, a)
+        assert abs(len(a) - len(b)) <= d <= max(len(a), len(b))
+        assert (d == 0) == (a == b)
+
+
+def one_edit_neighbourhood(q, V):
+    """Every non-empty string within one edit of q over the alphabet [0, V)."""
+    out = {tuple(q)}
+    for x in range(len(q)):
+        out.add(tuple(q[:x] + q[x + 1:]))
+        for t in range(V):
+            out.add(tuple(q[:x] + [t] + q[x + 1:]))
+    for x in range(len(q) + 1):
+        for t in range(V):
+            out.add(tuple(q[:x] + [t] + q[x:]))
+    out.discard(())
+    return out
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_fuzzy_match_set_equals_exact_search_of_the_neighbourhood(seed):
+    G, N, L, V = 1, 4, 28, 3
+    tokens, lps = synth.small_random(G * N, L, V, 700 + seed)
+    rng = synth.Stream(7000 + seed)
+    lens = (4 + rng.uniform(N) * (L - 5)).astype(np.int32)
+    exact = Oracle(G, N, L, V, 3)
+    fuzzy = Oracle(G, N, L, V, 3, eps=1)
+    exact.append(tokens, lps, lens)
+    fuzzy.append(tokens, lps, lens)
+    for k in (1, 2, 3, 4):
+        exact.build_all(k)
+        fuzzy.build_all(k)
+        for i in range(N):
+            if lens[i] < k:
+                assert len(fuzzy.matches(i)) == 0
+                continue
+            q = tokens[i, lens[i] - k:lens[i]].tolist()
+            want = set()
+            for var in one_edit_neighbourhood(q, V):
+                pat = re.compile(b"(?=" + re.escape(bytes(var)) + b")")
+                for j in range(N):
+                    if j == i:
+                        continue
+                    for m in pat.finditer(bytes(tokens[j, :lens[j]].tolist())):
+                        e = m.start() + len(var) - 1
+                        if e <= lens[j] - 2:
+                            want.add(j * L + e)
+            got = fuzzy.matches(i).tolist()
+            assert got == sorted(want), (seed, k, i)
+            assert set(exact.matches(i).tolist()) <= set(got)
+
+
+def test_fuzzy_candidates_with_different_last_tokens_share_a_virtual_root():
+    # hand-worked: query (1,2), tolerance 1.  Path 1 = [1,3,7,5,5]: "1" (deletion) ends at 0, "1 3"
+    # (substitution) at 1.  Path 2 = [4,1,2,7,6,6]: "1" ends at 1, "1 2" (exact) at 2, "1 2 7"
+    # (insertion) at 3.  Five candidates whose matched windows end in 1, 3, 1, 2, 7.
+    paths = [[9, 1, 2], [1, 3, 7, 5, 5], [4, 1, 2, 7, 6, 6], [8, 8, 8]]
+    probs = [[0.5] * 3, [0.5, 0.5, 0.25, 0.5, 0.5], [0.5, 0.5, 0.5, 0.5, 0.25, 0.5], [0.5] * 3]
+    o = Oracle(1, 4, 10, 16, 3, eps=1)
+    load_paths(o, paths, probs=probs)
+    o.build_path(2, 0)
+    assert o.matches(0).tolist() == [10, 11, 21, 22, 23]
+    # followers: [3,7,5] [7,5,5] [2,7,6] [7,6,6] [6,6]
+    nodes, edges = o.layer(0, 1)
+    q = lambda x: int(x * Q30)
+    assert nodes == {3: (q(0.5), 1), 7: (q(0.75), 2), 2: (q(0.5), 1), 6: (q(0.25), 1)}
+    assert edges == {(1, 3): (q(0.5), 1), (3, 7): (q(0.25), 1), (1, 2): (q(0.5), 1), (2, 7): (q(0.5), 1),
+                     (7, 6): (q(0.25), 1)}
+    nodes2, edges2 = o.layer(0, 2)
+    assert nodes2 == {7: (q(0.75), 2), 5: (q(0.5), 1), 6: (q(0.75), 2)}
+    tok, score, edge_w = o.draft(0)
+    # layer 1: 7 (0.75) from the virtual root; layer 2: successors of 7 are 5 (0.5) and 6 (0.75);
+    # layer 3: the successor of 6 is 6 (0.5 + 0.25)
+    assert tok.tolist() == [7, 6, 6]
+    assert score.tolist() == [0.75, 0.75, 0.75]
+    assert edge_w.tolist() == [0.75, 0.25, 0.5]    # the virtual-root edge carries the whole node
+    # exact matching sees only the window that ends at (2, 2)
+    o0 = Oracle(1, 4, 10, 16, 3)
+    load_paths(o0, paths, probs=probs)
+    o0.build_path(2, 0)
+    assert o0.matches(0).tolist() == [22] and o0.draft(0)[0].tolist() == [7, 6, 6]
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_fuzzy_draft_is_greedy_walk_from_the_virtual_root(seed):
+    G, N, L, V, D = 1, 4, 24, 3, 4
+    tokens, lps = synth.small_random(N, L, V, 800 + seed)
+    lens = np.full(N, L - 2 - seed, np.int32)
+    o = Oracle(G, N, L, V, D, eps=1)
+    o.append(tokens, lps, lens)
+    o.build_all(2)
+    for i in range(N):
+        layers = [o.layer(i, d) for d in range(1, D + 1)]
+        draft, score, edge_w = o.draft(i)
+        cur = None
+        for d in range(D):
+            nodes, edges = layers[d]
+            succ = sorted(nodes) if d == 0 else sorted(v for (u, v) in edges if u == cur)
+            if not succ:
+                assert len(draft) == d
+                break
+            w = {v: oracle.weight(1.0, *nodes[v]) for v in succ}
+            best = min(v for v in succ if w[v] == max(w.values()))
+            assert draft[d] == best and score[d] == w[best]
+            assert edge_w[d] == (w[best] if d == 0 else oracle.weight(1.0, *edges[(cur, best)]))
+            cur = best

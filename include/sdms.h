@@ -75,6 +75,10 @@ typedef struct {
                                     1: best node of each layer regardless of the previous one */
   float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
   int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
+  int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)
+                                    or 1.  1 needs a small prompt: N*L <= 131072 tokens and
+                                    G*N*N*L <= match_capacity (every path then owns N*L match slots) */
+  int32_t  reserved;             /* must be 0 */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,
@@ -106,10 +110,14 @@ int sdms_append(sdms_ctx* ctx, const int32_t* d_tokens, const float* d_logprobs,
                 const int32_t* d_counts, int32_t row_width, void* stream);
 
 /*
- * One draft per path (Algorithm 1 with exact matching, epsilon = 0):
+ * One draft per path (Algorithm 1):
  *   query      the last k tokens of path i                       (1 <= k <= k_max)
  *   match      Eq. 3: every end position e in every other path j of the same
  *              prompt with y_j[e-k+1..e] equal to the query and e <= len_j - 2
+ *              With epsilon = 1 ("Fuzzy Suffix Matching", Eq. 4): every e <= len_j - 2
+ *              at which some window of k-1, k or k+1 tokens (at least one) ends
+ *              within edit distance 1 of the query; each e counts once.  The walk
+ *              then starts from a virtual root in front of all matched windows.
  *   candidates the up to D tokens that follow each match
  *   DAG        layer d = distinct d-th followers; edge (u,v) between layers d-1
  *              and d accumulates S = sum of fixed-point probabilities of v and

@@ -35,6 +35,7 @@ int check_config(const sdms_config* c) {
   if (c->match_capacity < 0 || c->match_capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;
   const int64_t P = (int64_t)c->num_groups * c->paths_per_group;
   if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
+  if (c->epsilon < 0 || c->epsilon > 1 || c->reserved != 0) return SDMS_ERR_INVALID_ARG;
   return SDMS_OK;
 }
 
@@ -70,6 +71,22 @@ Layout make_layout(const sdms_config* c) {
   l.x_edge_cnt = take(P * D * B * Ke * 4); l.x_out_degree = take(P * D * B * 4);
   l.total = o;
   return l;
+}
+
+// Small prompts: every query path gets a private slice of N*L match slots and one CTA does the whole build.
+bool fits_fused(const sdms_config* c, const Layout& l) {
+  const int64_t group_tokens = (int64_t)c->paths_per_group * c->capacity;
+  return group_tokens <= kFusedMaxTokens &&
+         (int64_t)c->num_groups * c->paths_per_group * group_tokens <= l.match_cap;
+}
+
+// Full check: field ranges, then what depends on the layout (fuzzy matches are not sized by the index).
+int check_all(const sdms_config* c, Layout* out) {
+  const int rc = check_config(c);
+  if (rc != SDMS_OK) return rc;
+  *out = make_layout(c);
+  if (c->epsilon > 0 && !fits_fused(c, *out)) return SDMS_ERR_INVALID_ARG;
+  return SDMS_OK;
 }
 
 struct EventPair { cudaEvent_t a, b; int kernel; };
@@ -114,19 +131,20 @@ extern "C" {
 
 int sdms_workspace_bytes(const sdms_config* cfg, size_t* bytes) {
   if (!bytes) return SDMS_ERR_INVALID_ARG;
-  const int rc = check_config(cfg);
+  Layout lay;
+  const int rc = check_all(cfg, &lay);
   if (rc != SDMS_OK) return rc;
-  *bytes = make_layout(cfg).total;
+  *bytes = lay.total;
   return SDMS_OK;
 }
 
 int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ctx** out) {
   if (!out) return SDMS_ERR_INVALID_ARG;
   *out = nullptr;
-  const int rc = check_config(cfg);
+  Layout lay;
+  const int rc = check_all(cfg, &lay);
   if (rc != SDMS_OK) return rc;
   if (!d_workspace || ((uintptr_t)d_workspace & (kAlign - 1))) return SDMS_ERR_INVALID_ARG;
-  const Layout lay = make_layout(cfg);
   if (bytes < lay.total) return SDMS_ERR_WORKSPACE_TOO_SMALL;
   if (dag_kernel_setup() != cudaSuccess) return SDMS_ERR_CUDA;
   if (cudaMemsetAsync(d_workspace, 0, lay.total, 0) != cudaSuccess) return SDMS_ERR_CUDA;
@@ -148,8 +166,8 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.mode = cfg->search_mode; d.P = d.G * d.N;
   d.alpha = (double)cfg->alpha;
   d.table_cap = lay.table_cap; d.match_cap = lay.match_cap;
-  // small prompts: every query path gets a private slice of N*L match slots and one CTA does the whole build
-  d.fused = (int64_t)d.N * d.L <= kFusedMaxTokens && (int64_t)d.P * d.N * d.L <= lay.match_cap;
+  d.fused = fits_fused(cfg, lay);
+  d.eps = cfg->epsilon;
   unsigned char* w = ctx->ws;
   d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len);
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);

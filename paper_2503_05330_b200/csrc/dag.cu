@@ -686,7 +686,11 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
     const int len_i = s.len[i];
     int mode = Q_NONE;
     uint32_t fp = 0, count = 0;
-    if (len_i >= k && len_i < s.L) {
+    if (len_i >= k && len_i < s.L && s.eps > 0) {      // fuzzy matches are found by scanning only
+      const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
+      for (int t = 0; t < k; ++t) sh_q[t] = q[t];
+      mode = Q_SCAN;
+    } else if (len_i >= k && len_i < s.L) {
       const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
       uint64_t h = gram_init(k);
       for (int t = 0; t < k; ++t) { const int32_t x = q[t]; sh_q[t] = x; h = gram_step(h, x); }
@@ -728,6 +732,36 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
           const int at = atomicAdd(&sh_M, 1);
           sm.list[at] = j * s.L + e;
           my_matches[at] = j * s.L + e;
+        }
+      }
+    }
+  } else if (mode == Q_SCAN && s.eps > 0) {
+    // Eq. 4 with tolerance 1.  A window s' is within one edit of the query q iff, with a = their common
+    // prefix and b = their common suffix (each at most the shorter length), a + b >= max(|q|, |s'|) - 1.
+    // For the windows that end at e, b is shared; a is looked at only as far as it can still decide.
+    const int32_t* gtok = s.tok + (size_t)g * s.N * s.L;
+    for (int jn = 0; jn < s.N; ++jn) {
+      if (g * s.N + jn == i) continue;
+      const int32_t* row = gtok + (size_t)jn * s.L;
+      const int e_hi = sh_len[jn] - 2;
+      for (int e = tid; e <= e_hi; e += blockDim.x) {
+        int b = 0;
+        while (b < k && b <= e && __ldg(row + e - b) == sh_q[k - 1 - b]) ++b;
+        bool found = false;
+        for (int n = max(1, k - 1); n <= k + 1 && !found; ++n) {
+          if (e - n + 1 < 0) break;
+          const int shorter = min(k, n), need = max(k, n) - 1 - min(b, shorter);
+          if (need <= 0) { found = true; break; }
+          if (need > shorter) continue;
+          int a = 0;
+          while (a < need && __ldg(row + e - n + 1 + a) == sh_q[a]) ++a;
+          found = a >= need;
+        }
+        if (found) {
+          const int at = atomicAdd(&sh_M, 1);
+          const int pos = (g * s.N + jn) * s.L + e;
+          if (at < kListCap) sm.list[at] = pos;
+          my_matches[at] = pos;
         }
       }
     }

@@ -173,3 +173,54 @@ def test_config5_sampled_steps(k):
         pair.accept_and_compare(sampled, sampled_lp)
     pair.check_history()
     torch.cuda.synchronize()
+
+
+# ---- fuzzy suffix matching (tolerance 1) ---------------------------------------
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("alpha,mode", [(1.0, 0), (0.5, 0), (1.0, 1)])
+def test_fuzzy_dense_tiny_vocab_every_step(seed, alpha, mode):
+    G, N, L, V, D, k_max = 2, 4, 48, 3 + seed % 2, 4, 4
+    tokens, lps = synth.small_random(G * N, L, V, 1900 + seed)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, B=4, Ke=3, eps=1)
+        start = 2 + (np.arange(G * N) * 5 + seed) % 9          # some paths shorter than k
+        st = run_protocol(pair, tokens, lps, k, steps=30, warm=0, start_lens=start, commit_in_accept=bool(seed % 2))
+        assert st["steps"] > 0
+
+
+def test_fuzzy_hand_worked_case_on_device():
+    paths = [[9, 1, 2], [1, 3, 7, 5, 5], [4, 1, 2, 7, 6, 6], [8, 8, 8]]
+    pair = Pair(1, 4, 10, 16, 2, 3, B=4, Ke=4, eps=1)
+    tok = np.zeros((4, 6), np.int32); lp = np.full((4, 6), -0.7, np.float32)
+    for i, p in enumerate(paths):
+        tok[i, :len(p)] = p
+    pair.append(tok, lp, np.array([len(p) for p in paths], np.int32), expect_status=0)
+    t, ln = pair.build_and_compare(2)
+    assert t[0, :ln[0]].tolist() == [7, 6, 6]
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_fuzzy_config1_protocol(k):
+    w = synth.WORKLOADS[1]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D, eps=1)
+    st = run_protocol(pair, tokens, lps, k, steps=w.steps, warm=w.k_max)
+    assert st["steps"] == w.steps
+
+
+@pytest.mark.parametrize("k", [1, 2, 4])
+def test_fuzzy_config2_protocol(k):
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4, max_append=w.D, eps=1)
+    start = 600 + (np.arange(w.P) * 37) % 300
+    st = run_protocol(pair, tokens, lps, k, steps=60, warm=0, start_lens=start, check_every=5, commit_in_accept=True)
+    assert st["steps"] == 60
+
+
+def test_fuzzy_needs_a_small_prompt():
+    from paper_2503_05330_b200 import binding
+    w = synth.WORKLOADS[5]
+    with pytest.raises(binding.SdmsError) as e:
+        binding.sdms_workspace_bytes(binding.make_config(w.G, w.N, w.L, w.V, w.k_max, w.D, epsilon=1))
+    assert e.value.code == binding.ERR_INVALID_ARG

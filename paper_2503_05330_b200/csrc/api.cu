@@ -12,7 +12,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-  size_t tok, pq, len, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, matches;
+  size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, matches;
   size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
   size_t total;
   uint32_t table_cap;
@@ -58,6 +58,7 @@ Layout make_layout(const sdms_config* c) {
   l.tok = take((P * L + SDMS_MAX_DRAFT + 8) * 4);
   l.pq = take((P * L + SDMS_MAX_DRAFT + 8) * 4);
   l.len = take(P * 4);
+  l.rec = take(P * kRecWords * 4);
   l.status = take(4);
   l.index = take((size_t)c->num_groups * c->k_max * cap * kBucketWords * 4);
   l.q_fp = take(P * 4); l.q_mode = take(P * 4); l.q_reserved = take(P * 4);
@@ -169,7 +170,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.fused = fits_fused(cfg, lay);
   d.eps = cfg->epsilon;
   unsigned char* w = ctx->ws;
-  d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len);
+  d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len); d.rec = (int32_t*)(w + lay.rec);
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);
   d.q_fp = (uint32_t*)(w + lay.q_fp); d.q_mode = (int32_t*)(w + lay.q_mode);
   d.q_reserved = (int32_t*)(w + lay.q_reserved); d.q_off = (int32_t*)(w + lay.q_off);

@@ -106,9 +106,12 @@ __device__ void index_insert(const Dev& s, int g, int n, uint64_t h, uint32_t lp
   *st |= SDMS_STATUS_INDEX_FULL;
 }
 
-// Block-cooperative append of n validated tokens to path p whose length is len0.
+// Block-cooperative append of n validated tokens to path p whose length is len0.  rec is the
+// path's record as it was before the call (shared memory): rec[1 + t] = token at len0 - 1 - t.
+// Ends with a barrier-free write of the new record by the first k_max threads; the caller
+// updates nothing else.
 __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_t* in_tok,
-                              const float* in_lp, uint32_t* st) {
+                              const float* in_lp, const int32_t* rec, uint32_t* st) {
   int32_t* tok = s.tok + (size_t)p * s.L;
   int32_t* pq = s.pq + (size_t)p * s.L;
   for (int a = threadIdx.x; a < n; a += blockDim.x) {
@@ -123,9 +126,16 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
     if (pos + 1 < nn) continue;
     uint64_t h = gram_init(nn);
     for (int t = pos - nn + 1; t <= pos; ++t)
-      h = gram_step(h, t < len0 ? tok[t] : in_tok[t - len0]);   // old tokens from the store, new from the input
+      h = gram_step(h, t < len0 ? rec[len0 - t] : in_tok[t - len0]);   // old tokens from the record, new from the input
     index_insert(s, g, nn, gram_final(h), lbase + (uint32_t)pos, st);
   }
+  // the record after the append: new length, then the newest k_max tokens
+  int32_t* out = s.rec + (size_t)p * kRecWords;
+  if (threadIdx.x < s.k_max) {
+    const int x = len0 + n - 1 - (int)threadIdx.x;                       // position of the token this word holds
+    out[1 + threadIdx.x] = x >= len0 ? in_tok[x - len0] : (x >= 0 ? rec[len0 - x] : 0);
+  }
+  if (threadIdx.x == 0) { out[0] = len0 + n; s.len[p] = len0 + n; }
 }
 
 __global__ void __launch_bounds__(128) append_kernel(Dev s, const int32_t* __restrict__ tokens,
@@ -134,12 +144,14 @@ __global__ void __launch_bounds__(128) append_kernel(Dev s, const int32_t* __res
   const int p = blockIdx.x;
   __shared__ int sh_len0, sh_n, sh_bad;
   __shared__ uint32_t sh_st;
+  __shared__ int32_t sh_rec[kRecWords];
+  if (threadIdx.x < kRecWords) sh_rec[threadIdx.x] = s.rec[(size_t)p * kRecWords + threadIdx.x];
   if (threadIdx.x == 0) {
     uint32_t st = 0;
     int n = counts[p];
     if (n < 0) { st |= SDMS_STATUS_BAD_COUNT; n = 0; }
     if (n > row_width) { st |= SDMS_STATUS_BAD_COUNT; n = row_width; }
-    const int len0 = s.len[p];
+    const int len0 = sh_rec[0];
     if (n > s.L - len0) { st |= SDMS_STATUS_CAPACITY; n = s.L - len0; }
     sh_len0 = len0; sh_n = n; sh_bad = n; sh_st = st;
   }
@@ -154,13 +166,10 @@ __global__ void __launch_bounds__(128) append_kernel(Dev s, const int32_t* __res
   uint32_t st = 0;
   const int n = sh_bad;
   if (threadIdx.x == 0 && n < sh_n) st |= SDMS_STATUS_BAD_TOKEN;
-  append_tokens(s, p, sh_len0, n, in_tok, in_lp, &st);
+  append_tokens(s, p, sh_len0, n, in_tok, in_lp, sh_rec, &st);
   if (st) atomicOr(&sh_st, st);
   __syncthreads();
-  if (threadIdx.x == 0) {
-    s.len[p] = sh_len0 + n;
-    if (sh_st) atomicOr(s.status, sh_st);
-  }
+  if (threadIdx.x == 0 && sh_st) atomicOr(s.status, sh_st);
 }
 
 __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __restrict__ draft_tok,
@@ -171,8 +180,12 @@ __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __res
   const int p = blockIdx.x;
   __shared__ int sh_len0, sh_n, sh_bad;
   __shared__ uint32_t sh_st;
+  __shared__ int32_t sh_rec[kRecWords];
   const int32_t* smp = sampled + (size_t)p * (s.D + 1);
   if (threadIdx.x < 32) {
+    static_assert(kRecWords == 32, "one record word per lane");
+    const int32_t mine = sampled_lp ? s.rec[(size_t)p * kRecWords + threadIdx.x] : 0;   // in flight with the draft
+    sh_rec[threadIdx.x] = mine;
     int dl = draft_len[p];
     dl = dl < 0 ? 0 : (dl > s.D ? s.D : dl);
     const int d = threadIdx.x;
@@ -183,7 +196,7 @@ __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __res
       accept_len[p] = tau;
       int n = 0, len0 = 0;
       if (sampled_lp) {
-        len0 = s.len[p];
+        len0 = mine;                                  // lane 0 holds the length
         n = min(min(tau + 1, s.max_append), s.L - len0);
       }
       sh_len0 = len0; sh_n = n; sh_bad = n; sh_st = 0;
@@ -199,13 +212,10 @@ __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __res
   uint32_t st = 0;
   const int n = sh_bad;
   if (threadIdx.x == 0 && n < sh_n) st |= SDMS_STATUS_BAD_TOKEN;
-  append_tokens(s, p, sh_len0, n, smp, sampled_lp + (size_t)p * (s.D + 1), &st);
+  append_tokens(s, p, sh_len0, n, smp, sampled_lp + (size_t)p * (s.D + 1), sh_rec, &st);
   if (st) atomicOr(&sh_st, st);
   __syncthreads();
-  if (threadIdx.x == 0) {
-    s.len[p] = sh_len0 + n;
-    if (sh_st) atomicOr(s.status, sh_st);
-  }
+  if (threadIdx.x == 0 && sh_st) atomicOr(s.status, sh_st);
 }
 
 }  // namespace

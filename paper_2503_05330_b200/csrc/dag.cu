@@ -218,11 +218,10 @@ __device__ void write_defaults(const Dev& s, int i, int32_t* draft_tok, float* d
 // ---------------------------------------------------------------------------
 template <bool EXPORT>
 __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                          const int32_t* plen, int poff, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          const int32_t* plen, int poff, int root, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                           float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int D = s.D, B = s.B, Ke = s.Ke;
-  const int root = s.tok[(size_t)i * s.L + s.len[i] - 1];
   // per layer and lane: follower token, previous token, node score, edge weight; per layer: leader masks
   int* L_v = sm.st_tok;
   int* L_u = sm.st_tok + 32 * SDMS_MAX_DRAFT;
@@ -352,7 +351,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
 // ---------------------------------------------------------------------------
 template <bool EXPORT>
 __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                          const int32_t* plen, int poff, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          const int32_t* plen, int poff, int root, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                           float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   __shared__ int sh_nn, sh_ne, sh_overflow, sh_found, sh_cur, sh_nkept, sh_nnode_run, sh_node_total;
   __shared__ double sh_best_w, sh_best_ew;
@@ -360,7 +359,6 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int D = s.D, B = s.B, Ke = s.Ke;
-  const int root = s.tok[(size_t)i * s.L + s.len[i] - 1];
 
   // stage every follower once: one round trip to memory instead of one per layer
   const bool staged = M * D <= kStageWords;
@@ -629,11 +627,11 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
 // that follows write_defaults.
 template <bool EXPORT>
 __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist,
-                                          const int32_t* plen, int poff, int32_t* draft_tok, int32_t* draft_len,
-                                          float* draft_score, float* draft_edge_w) {
+                                          const int32_t* plen, int poff, int root, int32_t* draft_tok,
+                                          int32_t* draft_len, float* draft_score, float* draft_edge_w) {
   // plen[j - poff] = length of path j (the prompt's lengths in shared memory, or the global array)
-  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
-  else dag_block<EXPORT>(s, sm, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
+  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
+  else dag_block<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 template <bool EXPORT>
@@ -654,8 +652,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
   const int g = i / s.N;
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   __syncthreads();
-  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, draft_tok, draft_len, draft_score,
-                    draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, s.rec[(size_t)i * kRecWords + 1],
+                    draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 // Whole draft construction of one query path in one CTA, for prompts whose
@@ -683,17 +681,17 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
   int32_t* my_matches = s.matches + (size_t)i * slice;
 
   if (tid == 0) {
-    const int len_i = s.len[i];
+    // the path's record: length and last tokens (newest first) in one 128-byte line
+    const int32_t* rec = s.rec + (size_t)i * kRecWords;
+    const int len_i = rec[0];
     int mode = Q_NONE;
     uint32_t fp = 0, count = 0;
     if (len_i >= k && len_i < s.L && s.eps > 0) {      // fuzzy matches are found by scanning only
-      const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
-      for (int t = 0; t < k; ++t) sh_q[t] = q[t];
+      for (int t = 0; t < k; ++t) sh_q[t] = rec[k - t];
       mode = Q_SCAN;
     } else if (len_i >= k && len_i < s.L) {
-      const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
       uint64_t h = gram_init(k);
-      for (int t = 0; t < k; ++t) { const int32_t x = q[t]; sh_q[t] = x; h = gram_step(h, x); }
+      for (int t = 0; t < k; ++t) { const int32_t x = rec[k - t]; sh_q[t] = x; h = gram_step(h, x); }
       h = gram_final(h);
       fp = gram_fp(h);
       const uint32_t* table = index_table(s, g, k);
@@ -820,8 +818,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
     if (tid == 0) draft_len[i] = 0;
     return;
   }
-  dag_phase<EXPORT>(s, sm, i, M, M <= kListCap ? sm.list : my_matches, sh_len, g * s.N, draft_tok, draft_len,
-                    draft_score, draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, M, M <= kListCap ? sm.list : my_matches, sh_len, g * s.N, sh_q[k - 1], draft_tok,
+                    draft_len, draft_score, draft_edge_w);
 }
 
 }  // namespace

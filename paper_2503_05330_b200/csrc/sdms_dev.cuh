@@ -8,6 +8,7 @@ namespace sdms {
 
 constexpr int kBucketWords = 8;        // one 32-byte sector: fingerprint, count, 6 positions
 constexpr int kInlineSlots = kBucketWords - 2;
+constexpr int kRecWords = 32;          // one 128-byte line per path: what a step needs first, in one load
 constexpr int kHalo = SDMS_MAX_K;      // tokens staged in front of a scan tile
 constexpr int kScanTile = 1024;        // history tokens per scan CTA
 constexpr int kScanThreads = 256;
@@ -29,6 +30,7 @@ struct Dev {
   int32_t* tok;                        // [P][L]
   int32_t* pq;                         // [P][L] fixed-point probabilities
   int32_t* len;                        // [P]
+  int32_t* rec;                        // [P][kRecWords] per path: length, then its last k_max tokens, newest first
   uint32_t* status;
   uint32_t* index;                     // [G][k_max][table_cap][kBucketWords]
   // per-query scratch of the last build

@@ -19,6 +19,8 @@
 //                in-edge weight is highest; stop at length D or at a leaf.
 //   accept     - "Draft acceptance": longest prefix of the draft equal to the
 //                sampled tokens.
+//   tree, list - the two weaker draft pools of the "Ablation Study": a tree merges
+//                candidates only along identical prefixes, a list does not merge.
 //
 // Readings where the paper is silent (all restated in the design notes):
 //   * followers start one position after the matched suffix;
@@ -72,6 +74,7 @@ struct PathResult {
 struct Ctx {
   int G, N, L, V, D, mode;
   int eps = 0;                                  // edit-distance tolerance of the suffix match (Eq. 4)
+  int pool = 0;                                 // draft pool of the ablation: 0 DAG, 1 tree, 2 list
   double alpha;
   std::vector<std::vector<int32_t>> tok, pq;
   std::vector<PathResult> res;
@@ -182,6 +185,55 @@ void build_path(Ctx* c, int k, int i) {
       nd.S += p; nd.cnt += 1;
     }
   }
+  if (c->pool == 1) {
+    // Tree pool (ablation study): candidates merge only while their whole prefix is the same, so a
+    // node is a prefix.  Walk: among the candidates that spell the draft so far, group by next token,
+    // weigh each child by Eq. 5 over its own instances, take the heaviest (ties: smaller token).
+    std::vector<std::pair<int, int>> live(r.matches);
+    for (int d = 1; d <= c->D; ++d) {
+      std::map<int, Acc> child;
+      for (const auto& m : live) {
+        int j = m.first, e = m.second;
+        if (e + d > (int)c->tok[j].size() - 1) continue;
+        Acc& a = child[c->tok[j][e + d]];
+        a.S += c->pq[j][e + d]; a.cnt += 1;
+      }
+      bool found = false; int best_v = -1; double best_w = 0.0;
+      for (const auto& kv : child) {
+        double w = weight(c->alpha, kv.second.S, kv.second.cnt);
+        if (!found || w > best_w) { found = true; best_v = kv.first; best_w = w; }
+      }
+      if (!found) break;
+      r.draft.push_back(best_v); r.score.push_back(best_w); r.edge_w.push_back(best_w);
+      std::vector<std::pair<int, int>> next;
+      for (const auto& m : live)
+        if (m.second + d <= (int)c->tok[m.first].size() - 1 && c->tok[m.first][m.second + d] == best_v) next.push_back(m);
+      live.swap(next);
+    }
+    return;
+  }
+  if (c->pool == 2) {
+    // List pool (ablation study): no merging at all.  The draft is the candidate whose own tokens
+    // weigh most by Eq. 5 (S = sum of its probabilities, Freq = its length); ties go to the
+    // candidate that comes first in (path, position) order.
+    bool found = false; double best_w = 0.0; std::pair<int, int> best;
+    for (const auto& m : r.matches) {
+      int j = m.first, e = m.second;
+      int n_m = std::min(c->D, (int)c->tok[j].size() - 1 - e);
+      int64_t S = 0;
+      for (int d = 1; d <= n_m; ++d) S += c->pq[j][e + d];
+      double w = weight(c->alpha, S, n_m);
+      if (!found || w > best_w) { found = true; best_w = w; best = m; }
+    }
+    if (!found) return;
+    int j = best.first, e = best.second;
+    int n_m = std::min(c->D, (int)c->tok[j].size() - 1 - e);
+    for (int d = 1; d <= n_m; ++d) {
+      double w = weight(c->alpha, c->pq[j][e + d], 1);
+      r.draft.push_back(c->tok[j][e + d]); r.score.push_back(w); r.edge_w.push_back(w);
+    }
+    return;
+  }
   // Greedy extraction.
   int cur = r.root;
   for (int d = 1; d <= c->D; ++d) {
@@ -227,6 +279,9 @@ void orc_destroy(void* h) { delete (Ctx*)h; }
 
 // Edit-distance tolerance of the suffix match (Eq. 4); 0 = exact matching.
 void orc_set_epsilon(void* h, int eps) { ((Ctx*)h)->eps = eps; }
+
+// Draft pool structure of the paper's ablation: 0 = DAG (the method), 1 = tree, 2 = list.
+void orc_set_pool(void* h, int pool) { ((Ctx*)h)->pool = pool; }
 
 int orc_edit_distance(const int32_t* a, int na, const int32_t* b, int nb) { return edit_distance(a, na, b, nb); }
 

@@ -577,3 +577,78 @@ def test_fuzzy_draft_is_greedy_walk_from_the_virtual_root(seed):
             assert draft[d] == best and score[d] == w[best]
             assert edge_w[d] == (w[best] if d == 0 else oracle.weight(1.0, *edges[(cur, best)]))
             cur = best
+
+
+# ----------------------------------------------------------------------------
+# tree and list draft pools (the paper's ablation variants)
+# ----------------------------------------------------------------------------
+def candidate_rows(o, tokens, lens, L, D, i):
+    pqs = [o.history(p)[1] for p in range(o.P)]
+    rows = []
+    for g in o.matches(i):
+        j, e = divmod(int(g), L)
+        n = min(D, lens[j] - 1 - e)
+        rows.append((int(g), [int(t) for t in tokens[j, e + 1:e + 1 + n]], [int(x) for x in pqs[j][e + 1:e + 1 + n]]))
+    return rows
+
+
+@pytest.mark.parametrize("seed,alpha", list(itertools.product(range(4), (1.0, 0.5))))
+def test_tree_pool_is_a_greedy_walk_of_the_trie(seed, alpha):
+    G, N, L, V, D = 1, 5, 40, 3, 5
+    tokens, lps = synth.small_random(N, L, V, 1300 + seed)
+    lens = np.full(N, L - 1 - seed, np.int32)
+    o = Oracle(G, N, L, V, D, alpha=alpha, pool=1)
+    o.append(tokens, lps, lens)
+    o.build_all(1)
+    for i in range(N):
+        rows = candidate_rows(o, tokens, lens, L, D, i)
+        draft, score, _ = o.draft(i)
+        prefix = []
+        for d in range(D + 1):
+            # children of the trie node `prefix`: Counter / sums over the candidates that start with it
+            live = [(t, p) for _, t, p in rows if len(t) > d and t[:d] == prefix]
+            if d == len(draft):
+                assert d == D or not live
+                break
+            w = {}
+            for v in sorted({t[d] for t, _ in live}):
+                w[v] = oracle.weight(alpha, sum(p[d] for t, p in live if t[d] == v), sum(1 for t, _ in live if t[d] == v))
+            best = min(v for v in w if w[v] == max(w.values()))
+            assert draft[d] == best and score[d] == w[best]
+            prefix.append(best)
+
+
+@pytest.mark.parametrize("seed,alpha", list(itertools.product(range(4), (1.0, 0.5))))
+def test_list_pool_picks_the_heaviest_candidate(seed, alpha):
+    G, N, L, V, D = 1, 5, 40, 3, 5
+    tokens, lps = synth.small_random(N, L, V, 1400 + seed)
+    lens = (L - 1 - 3 * np.arange(N)).astype(np.int32)
+    o = Oracle(G, N, L, V, D, alpha=alpha, pool=2)
+    o.append(tokens, lps, lens)
+    o.build_all(2)
+    for i in range(N):
+        rows = candidate_rows(o, tokens, lens, L, D, i)
+        draft, score, _ = o.draft(i)
+        if not rows:
+            assert len(draft) == 0
+            continue
+        w = [oracle.weight(alpha, sum(p), len(p)) for _, _, p in rows]
+        first_best = w.index(max(w))                     # rows are in (path, position) order
+        assert draft.tolist() == rows[first_best][1]
+        assert score.tolist() == [oracle.weight(alpha, x, 1) for x in rows[first_best][2]]
+
+
+def test_pools_agree_when_there_is_one_candidate_and_differ_on_reconvergence():
+    # candidates [2,7,5] and [3,7,6] plus [2,7,6]: after "2 7" the DAG sees 6 twice (via 2 and via 3),
+    # the tree only the continuations of the prefix "2 7"
+    paths = [[9, 1], [1, 2, 7, 5], [1, 3, 7, 6], [1, 2, 7, 6]]
+    probs = [[0.5, 0.5], [0.5, 0.5, 0.5, 0.5], [0.5, 0.25, 0.5, 0.5], [0.5, 0.5, 0.5, 0.25]]
+    drafts = {}
+    for pool in (0, 1, 2):
+        o = Oracle(1, 4, 8, 16, 3, pool=pool)
+        load_paths(o, paths, probs=probs)
+        o.build_path(1, 0)
+        drafts[pool] = (o.draft(0)[0].tolist(), o.draft(0)[1].tolist())
+    assert drafts[0] == ([2, 7, 6], [1.0, 1.5, 0.75])     # DAG: node (3, 6) = 0.5 + 0.25
+    assert drafts[1] == ([2, 7, 5], [1.0, 1.0, 0.5])      # tree: children of "2 7" are 5 (0.5) and 6 (0.25)
+    assert drafts[2] == ([2, 7, 5], [0.5, 0.5, 0.5])      # list: the first candidate sums to 1.5

@@ -78,7 +78,9 @@ typedef struct {
   int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)
                                     or 1.  1 needs a small prompt: N*L <= 131072 tokens and
                                     G*N*N*L <= match_capacity (every path then owns N*L match slots) */
-  int32_t  reserved;             /* must be 0 */
+  int32_t  pool_mode;            /* draft pool: 0 = weighted DAG (the method); the weaker pools of the
+                                    paper's ablation: 1 = tree (merge identical prefixes only),
+                                    2 = list (no merging: the heaviest single candidate)            */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,

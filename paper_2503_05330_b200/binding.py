@@ -38,14 +38,14 @@ class SdmsConfig(C.Structure):
         ("capacity", C.c_int32), ("vocab", C.c_int32), ("k_max", C.c_int32),
         ("max_draft_len", C.c_int32), ("max_append", C.c_int32), ("dag_nodes_per_layer", C.c_int32),
         ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
-        ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("reserved", C.c_int32),
+        ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("pool_mode", C.c_int32),
     ]
 
 
 def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
-                match_capacity=0, epsilon=0) -> SdmsConfig:
+                match_capacity=0, epsilon=0, pool_mode=0) -> SdmsConfig:
     return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
-                      B, Ke, search_mode, alpha, match_capacity, epsilon, 0)
+                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode)
 
 
 _lib = None

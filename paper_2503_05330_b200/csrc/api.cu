@@ -35,7 +35,7 @@ int check_config(const sdms_config* c) {
   if (c->match_capacity < 0 || c->match_capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;
   const int64_t P = (int64_t)c->num_groups * c->paths_per_group;
   if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
-  if (c->epsilon < 0 || c->epsilon > 1 || c->reserved != 0) return SDMS_ERR_INVALID_ARG;
+  if (c->epsilon < 0 || c->epsilon > 1 || c->pool_mode < 0 || c->pool_mode > 2) return SDMS_ERR_INVALID_ARG;
   return SDMS_OK;
 }
 
@@ -169,6 +169,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.table_cap = lay.table_cap; d.match_cap = lay.match_cap;
   d.fused = fits_fused(cfg, lay);
   d.eps = cfg->epsilon;
+  d.pool = cfg->pool_mode;
   unsigned char* w = ctx->ws;
   d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len); d.rec = (int32_t*)(w + lay.rec);
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);

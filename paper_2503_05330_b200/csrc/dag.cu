@@ -228,6 +228,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   unsigned* L_lead = reinterpret_cast<unsigned*>(sm.st_tok + 2 * 32 * SDMS_MAX_DRAFT);
   unsigned* L_elead = L_lead + SDMS_MAX_DRAFT;
   unsigned* L_best = L_elead + SDMS_MAX_DRAFT;      // per layer: the best edge out of each source / the best node
+  int* L_p = sm.st_tok + 3 * 32 * SDMS_MAX_DRAFT;   // fixed-point probability of the follower (tree pool)
   double* L_W = reinterpret_cast<double*>(sm.st_pq);
   double* L_we = L_W + 32 * SDMS_MAX_DRAFT;
 
@@ -266,7 +267,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
     }
     const unsigned best_out = __ballot_sync(FULL, eleader && !beaten);
     const int top = s.mode == 1 ? warp_arg_first(leader, W, v) : -1;   // best node of the layer
-    L_v[(d - 1) * 32 + lane] = v; L_u[(d - 1) * 32 + lane] = u;
+    L_v[(d - 1) * 32 + lane] = v; L_u[(d - 1) * 32 + lane] = u; L_p[(d - 1) * 32 + lane] = (int)p;
     L_W[(d - 1) * 32 + lane] = W; L_we[(d - 1) * 32 + lane] = w_uv;
     if (lane == 0) {
       L_lead[d - 1] = leaders; L_elead[d - 1] = eleaders;
@@ -323,6 +324,33 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   }
   __syncthreads();
   if (warp != 0) return;
+  if (!EXPORT && s.pool == 1) {
+    // tree pool: only the candidates that spell the draft so far stay in play
+    bool in_play = lane < M;
+    int emitted = 0;
+    for (int d = 1; d <= D; ++d) {
+      const int v = L_v[(d - 1) * 32 + lane];
+      const bool on = in_play && v >= 0;
+      const unsigned live = __ballot_sync(FULL, on);
+      if (live == 0) break;
+      const unsigned gv = __match_any_sync(FULL, on ? v : -1);
+      u64 S, unused;
+      group_sums(live, gv, 0u, (unsigned)L_p[(d - 1) * 32 + lane], &S, &unused);
+      const double W = eq5_weight(s.alpha, S, __popc(gv));
+      const int src = warp_arg_first(on && lane == __ffs(gv) - 1, W, v);
+      const int tok = __shfl_sync(FULL, v, src);
+      const double Wb = __shfl_sync(FULL, W, src);
+      if (lane == 0) {
+        draft_tok[(size_t)i * D + (d - 1)] = tok;
+        if (draft_score) draft_score[(size_t)i * D + (d - 1)] = (float)Wb;
+        if (draft_edge_w) draft_edge_w[(size_t)i * D + (d - 1)] = (float)Wb;
+      }
+      in_play = on && v == tok;
+      ++emitted;
+    }
+    if (lane == 0) draft_len[i] = emitted;
+    return;
+  }
   int cur = root, emitted = 0;
   for (int d = 1; d <= D; ++d) {
     const int v = L_v[(d - 1) * 32 + lane], u = L_u[(d - 1) * 32 + lane];
@@ -354,6 +382,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                           const int32_t* plen, int poff, int root, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                           float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   __shared__ int sh_nn, sh_ne, sh_overflow, sh_found, sh_cur, sh_nkept, sh_nnode_run, sh_node_total;
+  __shared__ int sh_draft[SDMS_MAX_DRAFT];
   __shared__ double sh_best_w, sh_best_ew;
   __shared__ int sh_best_tok, sh_best_valid;
 
@@ -390,7 +419,8 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
     if (!walking && !EXPORT) break;
     const int cur = sh_cur;
     const int nkept = EXPORT ? sh_nkept : 0;
-    const bool restricted = !EXPORT && !staged && s.mode == 0 && d > 1;    // staged candidates are cheap to revisit
+    const bool tree = !EXPORT && s.pool == 1;       // only candidates that spell the draft so far take part
+    const bool restricted = !EXPORT && !staged && !tree && s.mode == 0 && d > 1;   // staged candidates are cheap to revisit
     if (!EXPORT) {
       // first layer (or every layer in mode 1): every distinct follower is a node, guess one per four
       // candidates; restricted layers only hold the successors of one node
@@ -420,6 +450,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
               if (staged) {
                 v[r] = sm.st_tok[m * D + d - 1];
                 if (v[r] >= 0) { u[r] = d == 1 ? root : sm.st_tok[m * D + d - 2]; p[r] = (unsigned)sm.st_pq[m * D + d - 1]; }
+                if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (sm.st_tok[m * D + x - 1] != sh_draft[x - 1]) v[r] = -1;
               } else {
                 const int gpos = mlist[m];
                 const int j = gpos / s.L;
@@ -427,6 +458,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                   v[r] = __ldg(s.tok + gpos + d);
                   u[r] = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
                   p[r] = (unsigned)__ldg(s.pq + gpos + d);
+                  if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (__ldg(s.tok + gpos + x) != sh_draft[x - 1]) v[r] = -1;
                 }
               }
             }
@@ -492,7 +524,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
               const int sl = sm.n_touch[x];
               Cand c;
               c.tok = sm.n_key[sl]; c.S = 0;
-              c.valid = s.mode == 1 || sm.n_ccur[sl] > 0;
+              c.valid = s.mode == 1 || tree || sm.n_ccur[sl] > 0;
               c.w = eq5_weight(s.alpha, get64(sm.n_Slo, sm.n_Shi, sl), sm.n_call[sl]);
               c.cnt = (unsigned)sl;                  // carry the slot: the edge weight is read from it below
               if (c.valid && (!best.valid || ranks_before(c.w, c.tok, best.w, best.tok))) best = c;
@@ -502,7 +534,8 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 (!sh_best_valid || ranks_before(best.w, best.tok, sh_best_w, sh_best_tok))) {
               const int sl = (int)best.cnt;
               sh_best_valid = 1; sh_best_w = best.w; sh_best_tok = best.tok;
-              sh_best_ew = sm.n_ccur[sl] ? eq5_weight(s.alpha, get64(sm.n_Clo, sm.n_Chi, sl), sm.n_ccur[sl]) : 0.0;
+              sh_best_ew = tree ? best.w
+                         : sm.n_ccur[sl] ? eq5_weight(s.alpha, get64(sm.n_Clo, sm.n_Chi, sl), sm.n_ccur[sl]) : 0.0;
             }
           }
           if (EXPORT && warp == 1) {
@@ -578,6 +611,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       if (walking && sh_best_valid) {
         sh_found = 1;
         draft_tok[(size_t)i * D + (d - 1)] = sh_best_tok;
+        sh_draft[d - 1] = sh_best_tok;
         if (draft_score) draft_score[(size_t)i * D + (d - 1)] = (float)sh_best_w;
         if (draft_edge_w) draft_edge_w[(size_t)i * D + (d - 1)] = (float)sh_best_ew;
         sh_cur = sh_best_tok;
@@ -622,6 +656,46 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
   if (tid == 0) draft_len[i] = emitted;
 }
 
+// List pool (ablation): no merging; the draft is the single candidate that weighs most by Eq. 5 on
+// its own tokens (S = sum of its probabilities, Freq = its length), ties to the smaller position.
+__device__ void list_pool(const Dev& s, int i, int M, const int32_t* mlist, const int32_t* plen, int poff,
+                          int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                          float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
+  __shared__ double sh_w[kMaxWarps];
+  __shared__ int sh_g[kMaxWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int D = s.D;
+  double best_w = 0.0;
+  int best_g = -1;
+  for (int m = tid; m < M; m += blockDim.x) {
+    const int gpos = mlist[m];
+    const int j = gpos / s.L;
+    const int n_m = min(D, plen[j - poff] - 1 - (gpos - j * s.L));
+    u64 S = 0;
+    for (int d = 1; d <= n_m; ++d) S += (unsigned)__ldg(s.pq + gpos + d);
+    const double w = eq5_weight(s.alpha, S, (unsigned)n_m);
+    if (best_g < 0 || ranks_before(w, gpos, best_w, best_g)) { best_w = w; best_g = gpos; }
+  }
+  int src = warp_arg_first(best_g >= 0, best_w, best_g);
+  if (src < 0) src = 0;
+  best_w = __shfl_sync(FULL, best_w, src); best_g = __shfl_sync(FULL, best_g, src);
+  if (lane == 0) { sh_w[warp] = best_w; sh_g[warp] = best_g; }
+  __syncthreads();
+  if (warp != 0) return;
+  best_w = lane < nwarps ? sh_w[lane] : 0.0; best_g = lane < nwarps ? sh_g[lane] : -1;
+  src = warp_arg_first(best_g >= 0, best_w, best_g);
+  best_g = __shfl_sync(FULL, best_g, src < 0 ? 0 : src);
+  const int j = best_g / s.L;
+  const int n_m = min(D, plen[j - poff] - 1 - (best_g - j * s.L));
+  if (lane < n_m) {
+    const float w = (float)eq5_weight(s.alpha, (unsigned)__ldg(s.pq + best_g + 1 + lane), 1u);
+    draft_tok[(size_t)i * D + lane] = __ldg(s.tok + best_g + 1 + lane);
+    if (draft_score) draft_score[(size_t)i * D + lane] = w;
+    if (draft_edge_w) draft_edge_w[(size_t)i * D + lane] = w;
+  }
+  if (lane == 0) draft_len[i] = n_m;
+}
+
 // Gather + DAG + search for query path i over its M (> 0) matches in mlist
 // (shared or global memory).  Called by all threads of the CTA, after a barrier
 // that follows write_defaults.
@@ -630,7 +704,8 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
                                           const int32_t* plen, int poff, int root, int32_t* draft_tok,
                                           int32_t* draft_len, float* draft_score, float* draft_edge_w) {
   // plen[j - poff] = length of path j (the prompt's lengths in shared memory, or the global array)
-  if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
+  if (!EXPORT && s.pool == 2) list_pool(s, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
+  else if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
   else dag_block<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 

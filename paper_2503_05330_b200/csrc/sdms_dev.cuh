@@ -21,6 +21,7 @@ enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
 // Everything a kernel needs, passed by value.
 struct Dev {
   int32_t G, N, L, V, k_max, D, max_append, B, Ke, mode, P;
+  int32_t pool;                        // 0 DAG, 1 tree, 2 list
   int32_t eps;                         // edit-distance tolerance of the suffix match (0 or 1)
   int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
   double alpha;

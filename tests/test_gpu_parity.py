@@ -224,3 +224,39 @@ def test_fuzzy_needs_a_small_prompt():
     with pytest.raises(binding.SdmsError) as e:
         binding.sdms_workspace_bytes(binding.make_config(w.G, w.N, w.L, w.V, w.k_max, w.D, epsilon=1))
     assert e.value.code == binding.ERR_INVALID_ARG
+
+
+# ---- tree and list draft pools (ablation variants) --------------------------------
+@pytest.mark.parametrize("pool", [1, 2])
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("alpha", [1.0, 0.5])
+def test_pools_dense_tiny_vocab_every_step(pool, seed, alpha):
+    G, N, L, V, D, k_max = 2, 4, 48, 3 + seed % 2, 4, 3
+    tokens, lps = synth.small_random(G * N, L, V, 2300 + seed)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, B=4, Ke=3, pool=pool, eps=seed % 2)
+        start = 3 + (np.arange(G * N) * 5 + seed) % 9
+        st = run_protocol(pair, tokens, lps, k, steps=30, warm=0, start_lens=start, commit_in_accept=bool(seed % 2))
+        assert st["steps"] > 0
+
+
+@pytest.mark.parametrize("pool", [1, 2])
+@pytest.mark.parametrize("k", [1, 3])
+def test_pools_config2_protocol(pool, k):
+    # k = 1 reaches a few hundred matches per query: the block path with its prefix filter
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, pool=pool)
+    start = 700 + (np.arange(w.P) * 37) % 250
+    st = run_protocol(pair, tokens, lps, k, steps=60, warm=0, start_lens=start, check_every=10, commit_in_accept=True)
+    assert st["steps"] == 60
+
+
+@pytest.mark.parametrize("pool", [1, 2])
+def test_pools_config5_heavy_fan_out(pool):
+    w = synth.WORKLOADS[5]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, pool=pool)
+    start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+    pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+    pair.build_and_compare(1, paths=list(range(0, w.P, 16)))

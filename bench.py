@@ -144,12 +144,12 @@ class ClockSampler(threading.Thread):
 class Runner:
     """Device-resident replay of the decode protocol of one workload."""
 
-    def __init__(self, w, seed, device, B, Ke, eps=0):
+    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0):
         import torch
         from paper_2503_05330_b200 import binding
         self.torch, self.binding, self.w, self.device = torch, binding, w, device
         self.tokens, self.logprobs = synth.make_streams(w, seed)
-        self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke, epsilon=eps)
+        self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke, epsilon=eps, pool_mode=pool)
         dev = self.s.device
         self.warm_tok = torch.from_numpy(np.ascontiguousarray(self.tokens[:, :w.k_max])).to(dev)
         self.warm_lp = torch.from_numpy(np.ascontiguousarray(self.logprobs[:, :w.k_max])).to(dev)
@@ -170,6 +170,7 @@ class Runner:
         sampled_all, lp_all, active, bytes_scan, bytes_dag, bytes_io = [], [], [], [], [], []
         bytes_fused, bytes_useful, scan_queries = [], [], []
         matches = []
+        accepted = []
         for step in range(w.steps):
             _, _, lens = s.history()
             live = int((lens < w.L).sum())
@@ -194,6 +195,7 @@ class Runner:
             scan_queries.append(int((modes == 2).sum()))
             s.accept(torch.from_numpy(sm).to(dev), torch.from_numpy(lp).to(dev))
             tau = s.accept_len.cpu().numpy()
+            accepted.append(int(tau[lens < w.L].sum()))
             gained = np.minimum(np.minimum(tau + 1, w.D), w.L - lens)
             bytes_io.append(int(gained.sum()) * (8 + 8 + w.k_max * 32) + w.P * (w.D + 1) * 8)
             sampled_all.append(sm); lp_all.append(lp); active.append(live)
@@ -206,7 +208,8 @@ class Runner:
             bytes={"scan": float(np.mean(bytes_scan)), "dag": float(np.mean(bytes_dag)),
                    "accept": float(np.mean(bytes_io)), "build_fused": float(np.mean(bytes_fused))},
             useful_bytes_build=float(np.mean(bytes_useful)), scan_queries_per_step=float(np.mean(scan_queries)),
-            mean_matches_per_step=float(np.mean(matches)))
+            mean_matches_per_step=float(np.mean(matches)),
+            accept_length=float(np.sum(accepted)) / float(np.sum(active)))
         return self.plan
 
     def timed_steps(self, K, flush=True, e2e=False):
@@ -349,6 +352,17 @@ def ours_main(args, w):
         fuzzy = {"us_per_step": 1e3 * fms / min(args.steps, 1000), "value": funits / (fms * 1e-3), "unit": UNIT,
                  "us_per_step_by_k": dict(frun.last_by_k), "mean_matches_per_step": fplan["mean_matches_per_step"]}
         del frun
+    # accept length (accepted draft tokens per path and step) of the pool structures and of fuzzy
+    # matching on these synthetic streams: the axes of the paper's ablation, as context only
+    ablation = None
+    if world == 1 and not args.no_fuzzy:
+        ablation = {"dag": plan["accept_length"]}
+        if fuzzy is not None:
+            ablation["dag_fuzzy"] = fplan["accept_length"]
+        for name, pool, eps in (("tree", 1, 0), ("list", 2, 0), ("tree_fuzzy", 1, 1), ("list_fuzzy", 2, 1)):
+            arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool)
+            ablation[name] = arun.dry_run()["accept_length"]
+            del arun
     (ms, ms_e2e), (units, units_e2e) = whole_job([ms, ms_e2e], [units, units_e2e], device)
     if rank != 0:
         if world > 1:
@@ -389,7 +403,7 @@ def ours_main(args, w):
         "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
-        "fuzzy_epsilon_1": fuzzy,
+        "fuzzy_epsilon_1": fuzzy, "synthetic_accept_length": ablation,
         "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
                        "us_per_sdms_get_dag_call": export_us,
                        "note": "inspection call that re-aggregates the last build's matches; not part of a step"},

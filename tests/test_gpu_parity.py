@@ -260,3 +260,63 @@ def test_pools_config5_heavy_fan_out(pool):
     start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
     pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
     pair.build_and_compare(1, paths=list(range(0, w.P, 16)))
+
+
+# ---- limits and both match paths ------------------------------------------------------
+@pytest.mark.parametrize("match_capacity", [0, 60000])
+def test_maximum_k_and_draft_length_odd_capacity_both_match_paths(match_capacity):
+    # k_max = 16, D = 32 (the largest supported), capacity not a multiple of 4 (scalar loads),
+    # 40 paths per prompt.  match_capacity = 60000 is below P*N*L, which sends the build through
+    # the probe / tile-scan / dag kernels instead of the single-launch one.
+    G, N, L, V, D, k_max = 2, 40, 71, 3, 32, 16
+    tokens, lps = synth.small_random(G * N, L, V, 3100)
+    for k in (1, 2, 7, 16):
+        pair = Pair(G, N, L, V, k_max, D, B=5, Ke=3, match_capacity=match_capacity, alpha=0.5)
+        start = 20 + (np.arange(G * N) * 7) % 40
+        st = run_protocol(pair, tokens, lps, k, steps=6, warm=0, start_lens=start, commit_in_accept=True)
+        assert st["steps"] == 6
+
+
+def test_one_path_per_prompt_never_matches():
+    pair = Pair(3, 1, 32, 4, 2, 4)
+    tokens, lps = synth.small_random(3, 32, 4, 77)
+    pair.append(tokens[:, :20], lps[:, :20], np.full(3, 20, np.int32), expect_status=0)
+    _, ln = pair.build_and_compare(1)
+    assert ln.sum() == 0
+
+
+def test_many_paths_per_prompt():
+    # 300 paths in one prompt: the per-prompt shared tables of the kernels are sized for 1024
+    G, N, L, V, D = 1, 300, 32, 6, 4
+    tokens, lps = synth.small_random(N, L, V, 91)
+    pair = Pair(G, N, L, V, 3, D, B=4, Ke=2)
+    pair.append(tokens[:, :28], lps[:, :28], (10 + np.arange(N) % 18).astype(np.int32), expect_status=0)
+    for k in (1, 2, 3):
+        pair.build_and_compare(k, paths=list(range(0, N, 7)))
+
+
+def test_repeated_builds_are_bit_identical():
+    # sums are integers and ties have a rule, so atomics and scheduling must not show in any output
+    w = synth.WORKLOADS[3]
+    tokens, lps = synth.make_streams(w)
+    from paper_2503_05330_b200 import binding
+    s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, B=8, Ke=4)
+    dev = s.device
+    n = 1500
+    s.append(harness.t32(tokens[:, :n], dev), harness.t32(lps[:, :n], dev),
+             harness.t32((n - (np.arange(w.P) * 11) % 200).astype(np.int32), dev))
+    for k in (1, 3):
+        snaps = []
+        for _ in range(3):
+            s.build_drafts(k)
+            off, gpos = s.matches()
+            off = off.numpy(); gpos = gpos.numpy()
+            srt = np.concatenate([np.sort(gpos[off[i]:off[i + 1]]) for i in range(w.P)]) if len(gpos) else gpos
+            dag = s.dag()
+            snaps.append([s.draft_tok.cpu().numpy().copy(), s.draft_len.cpu().numpy().copy(),
+                          s.draft_score.cpu().numpy().copy(), s.draft_edge_w.cpu().numpy().copy(), off, srt]
+                         + [dag[key] for key in sorted(dag)])
+        for other in snaps[1:]:
+            for a, b in zip(snaps[0], other):
+                assert np.array_equal(a, b)
+    assert s.status() == 0

@@ -137,6 +137,17 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
                       float* d_draft_score, float* d_draft_edge_w, void* stream);
 
 /*
+ * The same with a suffix length that backs off: every path uses the longest k in
+ * [1, k_hi] for which it has at least one match (the paper names k but never fixes
+ * it; longer suffixes give fewer, more specific candidates).  d_used_k [P] (may be
+ * NULL) receives that k, 0 for paths without a draft.  One launch; only for
+ * prompts small enough for the single-launch build (N*L <= 131072 tokens and
+ * G*N*N*L <= match_capacity), otherwise SDMS_ERR_BAD_STATE.
+ */
+int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok, int32_t* d_draft_len,
+                              float* d_draft_score, float* d_draft_edge_w, int32_t* d_used_k, void* stream);
+
+/*
  * "Draft acceptance": d_accept_len[p] = longest t <= d_draft_len[p] with
  * d_draft_tok[p][0..t) == d_sampled[p][0..t), d_sampled being [P][D+1] tokens
  * sampled by the model at the draft positions plus one more.

@@ -26,7 +26,7 @@ KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused")
 
 EXPORTS = (
     "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
-    "sdms_build_drafts", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
+    "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc",
 )
@@ -66,6 +66,7 @@ def lib():
         l.sdms_destroy.argtypes = [vp]
         l.sdms_append.argtypes = [vp, vp, vp, vp, i32, vp]
         l.sdms_build_drafts.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+        l.sdms_build_drafts_backoff.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         l.sdms_accept.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
         l.sdms_get_dag.argtypes = [vp] * 10
@@ -140,6 +141,12 @@ def sdms_append(ctx, tokens, logprobs, counts, stream=None):
 def sdms_build_drafts(ctx, k, draft_tok, draft_len, draft_score=None, draft_edge_w=None, stream=None):
     _check(lib().sdms_build_drafts(ctx, k, _dp(draft_tok), _dp(draft_len), _dp(draft_score), _dp(draft_edge_w),
                                    _sp(stream)), "sdms_build_drafts")
+
+
+def sdms_build_drafts_backoff(ctx, k_hi, draft_tok, draft_len, draft_score=None, draft_edge_w=None, used_k=None,
+                              stream=None):
+    _check(lib().sdms_build_drafts_backoff(ctx, k_hi, _dp(draft_tok), _dp(draft_len), _dp(draft_score),
+                                           _dp(draft_edge_w), _dp(used_k), _sp(stream)), "sdms_build_drafts_backoff")
 
 
 def sdms_accept(ctx, draft_tok, draft_len, sampled, sampled_logprobs, accept_len, stream=None):
@@ -243,6 +250,13 @@ class Sdms:
     def build_drafts(self, k, stream=None):
         sdms_build_drafts(self.ctx, k, self.draft_tok, self.draft_len, self.draft_score, self.draft_edge_w, stream)
         return self.draft_tok, self.draft_len
+
+    def build_drafts_backoff(self, k_hi, stream=None):
+        if not hasattr(self, "used_k"):
+            self.used_k = torch.empty(self.P, dtype=torch.int32, device=self.device)
+        sdms_build_drafts_backoff(self.ctx, k_hi, self.draft_tok, self.draft_len, self.draft_score, self.draft_edge_w,
+                                  self.used_k, stream)
+        return self.draft_tok, self.draft_len, self.used_k
 
     def accept(self, sampled, sampled_logprobs=None, stream=None):
         sdms_accept(self.ctx, self.draft_tok, self.draft_len, sampled, sampled_logprobs, self.accept_len, stream)

@@ -220,7 +220,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->dev.fused) {
     const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
-      return launch_build_fused(ctx->dev, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+      return launch_build_fused(ctx->dev, k, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, nullptr, st); });
     if (rc == SDMS_OK) ctx->built = true;
     return rc;
   }
@@ -230,6 +230,18 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (rc != SDMS_OK) return rc;
   rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
     return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+  if (rc == SDMS_OK) ctx->built = true;
+  return rc;
+}
+
+int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok, int32_t* d_draft_len,
+                              float* d_draft_score, float* d_draft_edge_w, int32_t* d_used_k, void* stream) {
+  if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
+  if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->dev.fused) return SDMS_ERR_BAD_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
+    return launch_build_fused(ctx->dev, k_hi, 1, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, d_used_k, st); });
   if (rc == SDMS_OK) ctx->built = true;
   return rc;
 }

@@ -739,10 +739,12 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
 // gather / DAG / search phase runs on the matches just found.  The matches also
 // go to the path's private slice of the match list for inspection.
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int k, int32_t* __restrict__ draft_tok,
+__global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo,
+                                                                  int32_t* __restrict__ draft_tok,
                                                                   int32_t* __restrict__ draft_len,
                                                                   float* __restrict__ draft_score,
-                                                                  float* __restrict__ draft_edge_w) {
+                                                                  float* __restrict__ draft_edge_w,
+                                                                  int32_t* __restrict__ used_k) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
   __shared__ int sh_mode, sh_M;
@@ -755,6 +757,10 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
   const int slice = s.N * s.L;
   int32_t* my_matches = s.matches + (size_t)i * slice;
 
+  write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
+  // With k_lo < k_hi the suffix length backs off: the longest k in [k_lo, k_hi] that has a match wins.
+  int k = k_hi;
+  for (;; --k) {
   if (tid == 0) {
     // the path's record: length and last tokens (newest first) in one 128-byte line
     const int32_t* rec = s.rec + (size_t)i * kRecWords;
@@ -788,7 +794,6 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
     sh_mode = mode; sh_count = count; sh_M = 0;
     s.q_fp[i] = fp; s.q_mode[i] = mode; s.q_reserved[i] = mode == Q_NONE ? 0 : slice; s.q_off[i] = i * slice;
   }
-  write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
   __syncthreads();
   const int mode = sh_mode;
   if (mode == Q_INLINE) {
@@ -887,8 +892,11 @@ __global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int 
     }
   }
   __syncthreads();
+  if (sh_M > 0 || k <= k_lo) break;
+  __syncthreads();                                   // everybody has read sh_M before the next probe resets it
+  }
   const int M = sh_M;
-  if (tid == 0) s.q_cursor[i] = M;
+  if (tid == 0) { s.q_cursor[i] = M; if (used_k) used_k[i] = M > 0 ? k : 0; }
   if (M == 0) {
     if (tid == 0) draft_len[i] = 0;
     return;
@@ -922,10 +930,10 @@ cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32
   return cudaGetLastError();
 }
 
-cudaError_t launch_build_fused(const Dev& s, int k, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
-                               float* draft_edge_w, cudaStream_t stream) {
-  build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, k, draft_tok, draft_len,
-                                                                                  draft_score, draft_edge_w);
+cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
+                               float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
+  build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(
+      s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
   return cudaGetLastError();
 }
 

@@ -77,6 +77,29 @@ class Pair:
                     assert np.array_equal(dag[key][i], ex[key]), (k, i, key, dag[key][i], ex[key])
         return tok, ln
 
+    def backoff_and_compare(self, k_hi):
+        """Back-off build: per path the longest k <= k_hi with a match (oracle: fixed-k builds composed)."""
+        used = np.zeros(self.P, np.int32)
+        for i in range(self.P):
+            for k in range(k_hi, 0, -1):
+                self.o.build_path(k, i)
+                if len(self.o.matches(i)) > 0:
+                    used[i] = k
+                    break
+        self.g.build_drafts_backoff(k_hi)
+        assert self.g.status() == 0
+        tok, ln, sc, ew = self.o.drafts()
+        assert np.array_equal(self.g.used_k.cpu().numpy(), used), (self.g.used_k.cpu().numpy(), used)
+        assert np.array_equal(self.g.draft_len.cpu().numpy(), ln)
+        assert np.array_equal(self.g.draft_tok.cpu().numpy(), tok)
+        np.testing.assert_allclose(self.g.draft_score.cpu().numpy(), sc, rtol=RTOL, atol=0)
+        np.testing.assert_allclose(self.g.draft_edge_w.cpu().numpy(), ew, rtol=RTOL, atol=0)
+        off, gpos = self.g.matches()
+        off, gpos = off.numpy(), gpos.numpy()
+        for i in range(self.P):
+            assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), self.o.matches(i)), i
+        return tok, ln, used
+
     def accept_and_compare(self, sampled, sampled_lp=None):
         tok, ln, _, _ = self.o.drafts()
         if sampled_lp is None:

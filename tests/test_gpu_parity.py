@@ -320,3 +320,31 @@ def test_repeated_builds_are_bit_identical():
             for a, b in zip(snaps[0], other):
                 assert np.array_equal(a, b)
     assert s.status() == 0
+
+
+# ---- suffix length with back-off ------------------------------------------------------------
+@pytest.mark.parametrize("eps", [0, 1])
+def test_backoff_picks_the_longest_matching_suffix(eps):
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, eps=eps)
+    lens = (500 + (np.arange(w.P) * 37) % 400).astype(np.int32)
+    pair.append(tokens[:, :int(lens.max())], lps[:, :int(lens.max())], lens, expect_status=0)
+    seen = set()
+    for step in range(25):
+        lens = pair.o.lengths()
+        _, ln, used = pair.backoff_and_compare(w.k_max)
+        seen |= set(used.tolist())
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
+        pair.accept_and_compare(sampled, sampled_lp)
+    assert len(seen) >= 3                      # different paths really end up with different k
+    pair.check_history()
+
+
+def test_backoff_dense_tiny_vocab_and_short_paths():
+    G, N, L, V, D, k_max = 2, 4, 40, 3, 4, 4
+    tokens, lps = synth.small_random(G * N, L, V, 4100)
+    pair = Pair(G, N, L, V, k_max, D)
+    pair.append(tokens[:, :12], lps[:, :12], np.array([12, 1, 2, 3, 0, 7, 12, 5], np.int32), expect_status=0)
+    for k_hi in (4, 2, 1):
+        pair.backoff_and_compare(k_hi)

@@ -262,6 +262,46 @@ class Runner:
         return sum(per_step), units
 
 
+def steady_state(wl, device, iters=20):
+    """Build latency of another workload at 97 % full histories: per k the median time of
+    sdms_build_drafts (CUDA events on the launch stream, L2 flushed before every call), the
+    matches it found and the kernel's own byte count per call.  Context for the headline."""
+    import torch
+    from paper_2503_05330_b200 import binding
+    tokens, logprobs = synth.make_streams(wl)
+    s = binding.Sdms(wl.G, wl.N, wl.L, wl.V, wl.k_max, wl.D, device=device, max_append=wl.D)
+    dev = s.device
+    n = int(wl.L * 0.97)
+    lens = (n - (np.arange(wl.P) * 13) % 97).astype(np.int32)
+    s.append(torch.from_numpy(np.ascontiguousarray(tokens[:, :n])).to(dev),
+             torch.from_numpy(np.ascontiguousarray(logprobs[:, :n])).to(dev), torch.from_numpy(lens).to(dev))
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    out = {}
+    for k in range(1, wl.k_max + 1):
+        for _ in range(3):
+            s.build_drafts(k)
+        evs = []
+        for _ in range(iters):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); s.build_drafts(k); b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        us = 1e3 * float(np.median([a.elapsed_time(b) for a, b in evs]))
+        off, _ = s.matches()
+        m = np.diff(off.numpy())
+        modes = s.query_modes()
+        glen = lens.reshape(wl.G, wl.N).sum(1).repeat(wl.N)
+        fused = wl.N * wl.L <= 131072
+        scan_bytes = int(4 * (glen - lens)[modes == 2].sum()) if fused else (4 * int(lens.sum()) if (modes == 2).any() else 0)
+        nbytes = scan_bytes + int((modes > 0).sum()) * (32 + 4 * k) + int(m.sum()) * (4 + 8 * wl.D) + wl.P * (12 * wl.D + 4)
+        out[str(k)] = {"us": us, "paths_per_s": wl.P / (us * 1e-6), "matches": int(m.sum()), "max_matches": int(m.max()),
+                       "scanned_queries": int((modes == 2).sum()), "bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9}
+    assert s.status() == 0
+    return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
+            "launches_per_build": 1 if fused else 3, "build_by_k": out}
+
+
 def rank_seed(w, rank):
     """Every rank owns its own prompts: same recipe, different seed."""
     return synth.BASE_SEED + w.index + 7919 * rank
@@ -363,6 +403,11 @@ def ours_main(args, w):
             arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool)
             ablation[name] = arun.dry_run()["accept_length"]
             del arun
+    others = None
+    if world == 1 and not args.no_others:
+        del run.flush
+        torch.cuda.empty_cache()
+        others = {synth.WORKLOADS[c].name: steady_state(synth.WORKLOADS[c], device) for c in (1, 3, 4, 5)}
     (ms, ms_e2e), (units, units_e2e) = whole_job([ms, ms_e2e], [units, units_e2e], device)
     if rank != 0:
         if world > 1:
@@ -404,12 +449,13 @@ def ours_main(args, w):
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
         "fuzzy_epsilon_1": fuzzy, "synthetic_accept_length": ablation,
+        "other_workloads_build_only": others,
         "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
                        "us_per_sdms_get_dag_call": export_us,
                        "note": "inspection call that re-aggregates the last build's matches; not part of a step"},
     }
     if world == 1 and not args.no_cpu_baseline:
-        units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 4 * w.steps, 20.0)
+        units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 10 ** 9, 10.0)
         line["cpu_baseline"] = {"value": units_c / secs_c, "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "us_per_step": 1e6 * secs_c / steps_c,
                                 "sample": f"{steps_c} decode steps of {w.name} ({runs_c} run(s) from the warm start)"}
@@ -429,6 +475,7 @@ def main():
     ap.add_argument("--dag-edges", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fuzzy", action="store_true", help="skip the extra pass with tolerance 1")
+    ap.add_argument("--no-others", action="store_true", help="skip the build-only figures of the other workloads")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -739,7 +739,7 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
 // gather / DAG / search phase runs on the matches just found.  The matches also
 // go to the path's private slice of the match list for inspection.
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo,
+__global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo,
                                                                   int32_t* __restrict__ draft_tok,
                                                                   int32_t* __restrict__ draft_len,
                                                                   float* __restrict__ draft_score,
@@ -932,7 +932,7 @@ cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32
 
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
-  build_fused_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(
+  build_fused_kernel<false><<<s.P, kFusedThreads, dag_smem_bytes<false>(), stream>>>(
       s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
   return cudaGetLastError();
 }

@@ -12,7 +12,7 @@ constexpr int kRecWords = 32;          // one 128-byte line per path: what a ste
 constexpr int kHalo = SDMS_MAX_K;      // tokens staged in front of a scan tile
 constexpr int kScanTile = 1024;        // history tokens per scan CTA
 constexpr int kScanThreads = 256;
-constexpr int kDagThreads = 256;
+constexpr int kDagThreads = 512;
 constexpr int kFusedThreads = 512;     // the single-launch build: more loads in flight while it scans
 constexpr int kDagCap = 1024;          // entries of the shared-memory node / edge tables
 constexpr int kFusedMaxTokens = 131072; // largest N*L a CTA scans on its own

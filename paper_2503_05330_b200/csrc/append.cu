@@ -141,6 +141,8 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
 __global__ void __launch_bounds__(128) append_kernel(Dev s, const int32_t* __restrict__ tokens,
                                                      const float* __restrict__ logprobs,
                                                      const int32_t* __restrict__ counts, int row_width) {
+  grid_wait();
+  grid_release();
   const int p = blockIdx.x;
   __shared__ int sh_len0, sh_n, sh_bad;
   __shared__ uint32_t sh_st;
@@ -177,6 +179,8 @@ __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __res
                                                      const int32_t* __restrict__ sampled,
                                                      const float* __restrict__ sampled_lp,
                                                      int32_t* __restrict__ accept_len) {
+  grid_wait();
+  grid_release();
   const int p = blockIdx.x;
   __shared__ int sh_len0, sh_n, sh_bad;
   __shared__ uint32_t sh_st;
@@ -222,15 +226,14 @@ __global__ void __launch_bounds__(128) accept_kernel(Dev s, const int32_t* __res
 
 cudaError_t launch_append(const Dev& s, const int32_t* tokens, const float* logprobs, const int32_t* counts,
                           int row_width, cudaStream_t stream) {
-  append_kernel<<<s.P, 128, 0, stream>>>(s, tokens, logprobs, counts, row_width);
-  return cudaGetLastError();
+  return launch_overlapped(append_kernel, dim3(s.P), dim3(128), 0, stream, s, tokens, logprobs, counts, row_width);
 }
 
 cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t* draft_len,
                           const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
                           cudaStream_t stream) {
-  accept_kernel<<<s.P, 128, 0, stream>>>(s, draft_tok, draft_len, sampled, sampled_lp, accept_len);
-  return cudaGetLastError();
+  return launch_overlapped(accept_kernel, dim3(s.P), dim3(128), 0, stream, s, draft_tok, draft_len, sampled, sampled_lp,
+                           accept_len);
 }
 
 }  // namespace sdms

@@ -714,6 +714,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
                                                           int32_t* __restrict__ draft_len,
                                                           float* __restrict__ draft_score,
                                                           float* __restrict__ draft_edge_w) {
+  grid_wait();
+  grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
@@ -745,6 +747,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
                                                                   float* __restrict__ draft_score,
                                                                   float* __restrict__ draft_edge_w,
                                                                   int32_t* __restrict__ used_k) {
+  grid_wait();
+  grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
   __shared__ int sh_mode, sh_M;
@@ -922,19 +926,16 @@ cudaError_t dag_kernel_setup() {
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                        float* draft_edge_w, cudaStream_t stream) {
   if (with_export)
-    dag_kernel<true><<<s.P, kDagThreads, dag_smem_bytes<true>(), stream>>>(s, draft_tok, draft_len, draft_score,
-                                                                          draft_edge_w);
-  else
-    dag_kernel<false><<<s.P, kDagThreads, dag_smem_bytes<false>(), stream>>>(s, draft_tok, draft_len, draft_score,
-                                                                            draft_edge_w);
-  return cudaGetLastError();
+    return launch_overlapped(dag_kernel<true>, dim3(s.P), dim3(kDagThreads), dag_smem_bytes<true>(), stream, s,
+                             draft_tok, draft_len, draft_score, draft_edge_w);
+  return launch_overlapped(dag_kernel<false>, dim3(s.P), dim3(kDagThreads), dag_smem_bytes<false>(), stream, s,
+                           draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
-  build_fused_kernel<false><<<s.P, kFusedThreads, dag_smem_bytes<false>(), stream>>>(
-      s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
-  return cudaGetLastError();
+  return launch_overlapped(build_fused_kernel<false>, dim3(s.P), dim3(kFusedThreads), dag_smem_bytes<false>(), stream,
+                           s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
 }
 
 }  // namespace sdms

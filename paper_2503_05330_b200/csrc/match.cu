@@ -48,6 +48,8 @@ __device__ __forceinline__ long long block_exclusive_scan(long long v, long long
 }
 
 __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
+  grid_wait();
+  grid_release();
   __shared__ long long warp_tot[32];
   __shared__ long long sh_carry;
   for (int g = threadIdx.x; g < s.G; g += blockDim.x) s.g_nscan[g] = 0;
@@ -121,6 +123,8 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
 
 __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
+  grid_wait();
+  grid_release();
   const int j = blockIdx.y;                    // path whose history is scanned
   const int g = j / s.N;
   if (s.g_nscan[g] == 0) return;
@@ -253,14 +257,12 @@ __global__ void __launch_bounds__(kProbeThreads) compact_matches_kernel(Dev s, i
 }  // namespace
 
 cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
-  probe_kernel<<<1, kProbeThreads, 0, stream>>>(s, k);
-  return cudaGetLastError();
+  return launch_overlapped(probe_kernel, dim3(1), dim3(kProbeThreads), 0, stream, s, k);
 }
 
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   dim3 grid((s.L + kScanTile - 1) / kScanTile, s.P);
-  scan_kernel<<<grid, kScanThreads, 0, stream>>>(s, k);
-  return cudaGetLastError();
+  return launch_overlapped(scan_kernel, grid, dim3(kScanThreads), 0, stream, s, k);
 }
 
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream) {

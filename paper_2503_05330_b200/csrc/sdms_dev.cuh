@@ -78,6 +78,13 @@ __device__ __forceinline__ double eq5_weight(double alpha, unsigned long long S,
   return __dadd_rn(t1, t2);
 }
 
+// Programmatic dependent launch: a kernel launched with launch_overlapped() may be scheduled while
+// the kernel before it on the stream is still draining.  grid_wait() returns once that kernel has
+// completed and its writes are visible; everything that touches memory comes after it.
+// grid_release() lets the next kernel on the stream start being scheduled.
+__device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Total order of the export and of the search: larger weight first, then smaller token.
 __device__ __forceinline__ bool ranks_before(double wa, int ta, double wb, int tb) {
   return wa > wb || (wa == wb && ta < tb);

@@ -4,6 +4,21 @@
 
 namespace sdms {
 
+// Launch with programmatic stream serialization: the kernel's CTAs may be scheduled before the
+// previous kernel on the stream has finished; the kernel itself waits (grid_wait) before it reads
+// or writes anything.
+template <class... KArgs, class... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 cudaError_t launch_append(const Dev& s, const int32_t* tokens, const float* logprobs, const int32_t* counts,
                           int row_width, cudaStream_t stream);
 cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t* draft_len,

@@ -202,8 +202,9 @@ class Runner:
         assert s.status() == 0
         self.plan = dict(
             sampled=torch.from_numpy(np.stack(sampled_all)).to(dev), lp=torch.from_numpy(np.stack(lp_all)).to(dev),
-            sampled_host=torch.from_numpy(np.stack(sampled_all)).pin_memory(),
-            lp_host=torch.from_numpy(np.stack(lp_all)).pin_memory(),
+            step_in_host=torch.from_numpy(np.concatenate(
+                [np.stack(sampled_all).reshape(len(active), -1),
+                 np.stack(lp_all).view(np.int32).reshape(len(active), -1)], axis=1)).pin_memory(),
             active=active, steps=len(active),
             bytes={"scan": float(np.mean(bytes_scan)), "dag": float(np.mean(bytes_dag)),
                    "accept": float(np.mean(bytes_io)), "build_fused": float(np.mean(bytes_fused))},
@@ -221,11 +222,8 @@ class Runner:
         done = 0
         ks = []
         if e2e:
-            h_acc = torch.empty(w.P, dtype=torch.int32).pin_memory()
-            h_tok = torch.empty((w.P, w.D), dtype=torch.int32).pin_memory()
-            h_len = torch.empty(w.P, dtype=torch.int32).pin_memory()
-            d_sm = torch.empty((w.P, w.D + 1), dtype=torch.int32, device=s.device)
-            d_lp = torch.empty((w.P, w.D + 1), dtype=torch.float32, device=s.device)
+            h_res = torch.empty_like(s.results, device="cpu").pin_memory()     # drafts + accept lengths
+            h_in = plan["step_in_host"]                                        # [steps][sampled | logprobs]
         while done < K:
             self.start_run()
             for step in range(plan["steps"]):
@@ -236,13 +234,10 @@ class Runner:
                 a, b = ev[done]
                 a.record()
                 if e2e:
-                    d_sm.copy_(plan["sampled_host"][step], non_blocking=True)
-                    d_lp.copy_(plan["lp_host"][step], non_blocking=True)
+                    s.step_in.copy_(h_in[step], non_blocking=True)
                     s.build_drafts(k_of(step, w.k_max))
-                    s.accept(d_sm, d_lp)
-                    h_acc.copy_(s.accept_len, non_blocking=True)
-                    h_tok.copy_(s.draft_tok, non_blocking=True)
-                    h_len.copy_(s.draft_len, non_blocking=True)
+                    s.accept(s.sampled_in, s.sampled_lp_in)
+                    h_res.copy_(s.results, non_blocking=True)
                     b.record()
                     b.synchronize()                 # the caller reads the result before its next step
                 else:

@@ -224,11 +224,18 @@ class Sdms:
             self.ctx = sdms_create(self.cfg, self.workspace)
         P, D_ = self.P, D
         dev = self.device
-        self.draft_tok = torch.empty((P, D_), dtype=torch.int32, device=dev)
-        self.draft_len = torch.empty(P, dtype=torch.int32, device=dev)
+        # integer results side by side, so that a caller can fetch them with one copy:
+        # [draft_tok P*D | draft_len P | accept_len P]
+        self.results = torch.empty(P * (D_ + 2), dtype=torch.int32, device=dev)
+        self.draft_tok = self.results[:P * D_].view(P, D_)
+        self.draft_len = self.results[P * D_:P * D_ + P]
+        self.accept_len = self.results[P * D_ + P:]
         self.draft_score = torch.empty((P, D_), dtype=torch.float32, device=dev)
         self.draft_edge_w = torch.empty((P, D_), dtype=torch.float32, device=dev)
-        self.accept_len = torch.empty(P, dtype=torch.int32, device=dev)
+        # the model's answer of a step, likewise one buffer: [sampled P*(D+1) int32 | logprobs P*(D+1) float32]
+        self.step_in = torch.empty(2 * P * (D_ + 1), dtype=torch.int32, device=dev)
+        self.sampled_in = self.step_in[:P * (D_ + 1)].view(P, D_ + 1)
+        self.sampled_lp_in = self.step_in[P * (D_ + 1):].view(torch.float32).view(P, D_ + 1)
 
     def close(self):
         if getattr(self, "ctx", None):

@@ -12,16 +12,22 @@
 //     each WARP owns a layer, so all layers aggregate at the same time.  Lanes
 //     with the same follower token (__match_any_sync) form a node, lanes that
 //     also share the previous token form an edge; sums run over the lanes of a
-//     group, ranks over the group leaders.  One barrier, then one warp walks the
-//     layers (a warp-wide arg-max per layer).
-//   dag_block (any M): layers in sequence; every warp takes 32 candidates at a
-//     time, pre-aggregates equal tokens with the same warp primitives and lets
-//     the group leaders add into shared-memory hash tables (32-bit atomics with
-//     explicit carry).  After the pass one warp picks the best successor; with
-//     the export enabled other warps select the B best nodes of the layer and the
-//     Ke best out-edges of the nodes kept one layer up.  A layer with more
-//     distinct tokens than the table holds is processed in several passes, each
-//     over the tokens of one residue class, so any fan-out fits the same tables.
+//     group, ranks over the group leaders, and each layer also decides the best
+//     way out of every source node.  One barrier, then one warp walks the layers
+//     by looking those decisions up.
+//   dag_block (any M): layers in sequence.  Followers are staged in shared memory
+//     when they fit; every candidate adds into a shared-memory hash table keyed
+//     by token (32-bit atomics with explicit carry).  Unstaged fan-out past the
+//     first layer runs in two phases - claim a slot for every successor of the
+//     current node, then add only the candidates that land on a claimed slot -
+//     so the table holds the successors of one node instead of a whole layer.
+//     One warp then picks the best successor.  A layer with more distinct tokens
+//     than the table holds is processed in several passes, each over the tokens
+//     of one residue class, so any fan-out fits the same tables.
+//   The EXPORT instantiation (sdms_get_dag) also keeps an edge table and lets
+//   other warps rank the B best nodes of the layer and the Ke best out-edges of
+//   the nodes kept one layer up.  tree / list pools reuse the same passes with a
+//   prefix filter / a single arg-max over candidates.
 #include "sdms_internal.h"
 
 namespace sdms {

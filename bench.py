@@ -471,7 +471,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fuzzy", action="store_true", help="skip the extra pass with tolerance 1")
     ap.add_argument("--no-others", action="store_true", help="skip the build-only figures of the other workloads")
+    ap.add_argument("--steady", type=int, default=0,
+                    help="only print the build-only figures of this workload at 97 %% full histories (for profiling)")
     args = ap.parse_args()
+    if args.steady:
+        import torch
+        torch.cuda.set_device(0)
+        wl = synth.WORKLOADS[args.steady]
+        print(json.dumps({"steady_state": wl.name, **steady_state(wl, "cuda:0", iters=max(args.steps, 1))}), flush=True)
+        return
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
         reference_main(args, w)

@@ -283,6 +283,12 @@ def steady_state(wl, device, iters=20):
             evs.append((a, b))
         torch.cuda.synchronize()
         us = 1e3 * float(np.median([a.elapsed_time(b) for a, b in evs]))
+        binding.sdms_profile_enable(s.ctx, True)                 # per-kernel split (events between the launches)
+        for _ in range(5):
+            flush.zero_()
+            s.build_drafts(k)
+        split = {n: 1e3 * ms / c for n, (ms, c) in binding.sdms_profile_read(s.ctx).items() if c}
+        binding.sdms_profile_enable(s.ctx, False)
         off, _ = s.matches()
         m = np.diff(off.numpy())
         modes = s.query_modes()
@@ -291,7 +297,8 @@ def steady_state(wl, device, iters=20):
         scan_bytes = int(4 * (glen - lens)[modes == 2].sum()) if fused else (4 * int(lens.sum()) if (modes == 2).any() else 0)
         nbytes = scan_bytes + int((modes > 0).sum()) * (32 + 4 * k) + int(m.sum()) * (4 + 8 * wl.D) + wl.P * (12 * wl.D + 4)
         out[str(k)] = {"us": us, "paths_per_s": wl.P / (us * 1e-6), "matches": int(m.sum()), "max_matches": int(m.max()),
-                       "scanned_queries": int((modes == 2).sum()), "bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9}
+                       "scanned_queries": int((modes == 2).sum()), "bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9,
+                       "kernel_us": split}
     assert s.status() == 0
     return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
             "launches_per_build": 1 if fused else 3, "build_by_k": out}

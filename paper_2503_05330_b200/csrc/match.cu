@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 }
 
 constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
+constexpr int kLastBits = 4096;
+__device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 20; }
 
 __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
   grid_wait();
@@ -140,10 +142,12 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
   __shared__ int32_t sh_cnt[SDMS_MAX_PATHS_PER_GROUP];
   __shared__ int32_t sh_base[SDMS_MAX_PATHS_PER_GROUP];
   __shared__ int32_t sh_set[kSetSlots];
+  __shared__ uint32_t sh_last[kLastBits / 32];   // which last tokens (hashed to 12 bits) any scan query ends in
   __shared__ int sh_nq;
 
   if (threadIdx.x == 0) sh_nq = 0;
   for (int x = threadIdx.x; x < kSetSlots; x += blockDim.x) sh_set[x] = -1;
+  for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
   // stage the tile (and the tokens just before it)
   const int32_t* row = s.tok + (size_t)j * s.L;
   const int hi = min(t0 + kScanTile, s.L);
@@ -170,6 +174,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
       sh_cnt[sl] = 0;
       uint32_t hs = (fp >> 1) & (kSetSlots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (kSetSlots - 1);
+      const uint32_t lb = last_bit(s.rec[(size_t)i * kRecWords + 1]);
+      atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
     }
   }
   __syncthreads();
@@ -185,19 +191,22 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
     fps[r] = 0;
     if (e < e_lo || e > e_hi) continue;
     const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
+    const uint32_t lb = last_bit(w[k - 1]);
+    if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) continue;       // no query ends in this token: nothing to hash
     uint64_t h = gram_init(k);
     for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
     const uint32_t fp = gram_fp(gram_final(h));
-    fps[r] = fp;
     uint32_t hs = (fp >> 1) & (kSetSlots - 1);
+    bool mine = false;
     for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
       if (sh_qfp[sl] != fp) continue;
       const int i = sh_qid[sl];
       const int32_t* q = s.tok + (size_t)i * s.L + (s.len[i] - k);
       bool same = true;
       for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(q + t));
-      if (same) { atomicAdd(&sh_cnt[sl], 1); any = true; }
+      if (same) { atomicAdd(&sh_cnt[sl], 1); mine = true; }
     }
+    if (mine) { fps[r] = fp; any = true; }                     // the second pass revisits matching positions only
   }
   if (!__syncthreads_or(any)) return;
   for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {

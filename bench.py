@@ -6,7 +6,7 @@
 One step = one pass of the whole path for all paths of the workload:
 sdms_build_drafts (query, match, gather, DAG, search) followed by sdms_accept
 with commit (acceptance check and state update with index insertion).  The
-suffix length cycles k = 1..k_max over the steps.  Prints one JSON line.
+suffix length takes every value 1..k_max equally often over the steps.  Prints one JSON line.
 """
 from __future__ import annotations
 
@@ -30,7 +30,11 @@ L2_FLUSH_BYTES = 256 << 20
 
 
 def k_of(step, k_max):
-    return 1 + step % k_max
+    """Suffix length of a step: every k in 1..k_max equally often, in a fixed scrambled order (so that
+    evenly spaced timed steps do not always meet the same k)."""
+    h = ((step + 1) * 0x9E3779B1) & 0xFFFFFFFF
+    h = ((h ^ (h >> 15)) * 0x85EBCA77) & 0xFFFFFFFF
+    return 1 + (h ^ (h >> 13)) % k_max
 
 
 # ----------------------------------------------------------------------------
@@ -88,7 +92,7 @@ def reference_main(args, w):
 
 def workload_config(w):
     return {"workload": w.name, "groups": w.G, "paths_per_group": w.N, "capacity": w.L, "vocab": w.V,
-            "k": f"cycles 1..{w.k_max} over the steps", "max_draft_len": w.D,
+            "k": f"1..{w.k_max}, equally often, fixed scrambled order over the steps", "timed_steps": "spread evenly over whole decode runs", "max_draft_len": w.D,
             "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)"}
 
 
@@ -224,16 +228,23 @@ class Runner:
         if e2e:
             h_res = torch.empty_like(s.results, device="cpu").pin_memory()     # drafts + accept lengths
             h_in = plan["step_in_host"]                                        # [steps][sampled | logprobs]
-        while done < K:
+        # K timed steps spread evenly over whole runs (warm start .. histories full), so that a
+        # small K still sees short and long histories and every k alike; the steps in between run
+        # untimed because the state has to evolve
+        S = plan["steps"]
+        runs = -(-K // S)
+        for r in range(runs):
+            quota = K // runs + (1 if r < K % runs else 0)
+            timed = set(int((x + 0.5) * S / quota) for x in range(quota)) if quota < S else set(range(S))
             self.start_run()
-            for step in range(plan["steps"]):
-                if done == K:
-                    break
-                if flush:
+            for step in range(S):
+                on = step in timed
+                if on and flush:
                     self.flush.zero_()
-                a, b = ev[done]
-                a.record()
-                if e2e:
+                if on:
+                    a, b = ev[done]
+                    a.record()
+                if e2e and on:
                     s.step_in.copy_(h_in[step], non_blocking=True)
                     s.build_drafts(k_of(step, w.k_max))
                     s.accept(s.sampled_in, s.sampled_lp_in)
@@ -243,10 +254,13 @@ class Runner:
                 else:
                     s.build_drafts(k_of(step, w.k_max))
                     s.accept(plan["sampled"][step], plan["lp"][step])
-                    b.record()
-                units += plan["active"][step]
-                ks.append(k_of(step, w.k_max))
-                done += 1
+                    if on:
+                        b.record()
+                if on:
+                    units += plan["active"][step]
+                    ks.append(k_of(step, w.k_max))
+                    done += 1
+        assert done == K
         torch.cuda.synchronize()
         per_step = [a.elapsed_time(b) for a, b in ev]
         self.last_by_k = {}

@@ -44,6 +44,12 @@ constexpr int kLoadBatch = 4;          // candidates a thread loads before it to
 constexpr int kListCap = 2048;         // matches a fused CTA keeps in shared memory besides its global slice
 static_assert(kStageWords >= 4 * 32 * SDMS_MAX_DRAFT, "dag_small keeps its per-layer lanes in the staging area");
 
+// Loads of path state (tokens, probabilities, lengths, records, index buckets).  In the one-launch
+// step other CTAs write this state earlier in the same launch, so it is read with ordinary loads,
+// which a cluster-scope acquire keeps coherent, never through the read-only (non-coherent) path.
+template <class T>
+__device__ __forceinline__ T ldm(const T* p) { return *p; }
+
 struct Cand {            // a node or an edge competing in a selection
   double w; u64 S; unsigned cnt; int tok; int valid;
 };
@@ -247,9 +253,9 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   for (int d = warp + 1; d <= D; d += nwarps) {
     const bool alive = d <= n_m;                        // candidate reaches layer d
     const bool alive_prev = lane < M && d - 1 <= n_m;   // ... reached layer d-1 (layer 0 is the root)
-    const int v = alive ? __ldg(s.tok + gpos + d) : -1;
-    const unsigned p = alive ? (unsigned)__ldg(s.pq + gpos + d) : 0u;
-    const int u = !alive_prev ? -1 : (d == 1 ? root : __ldg(s.tok + gpos + d - 1));
+    const int v = alive ? ldm(s.tok + gpos + d) : -1;
+    const unsigned p = alive ? (unsigned)ldm(s.pq + gpos + d) : 0u;
+    const int u = !alive_prev ? -1 : (d == 1 ? root : ldm(s.tok + gpos + d - 1));
     const unsigned live = __ballot_sync(FULL, alive);
     const unsigned gv = __match_any_sync(FULL, v);                     // lanes on the same node
     const unsigned gu = __match_any_sync(FULL, u);                     // lanes with the same previous node
@@ -294,7 +300,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
       if (lane == 0) s.x_node_count[(size_t)i * D + (d - 1)] = __popc(leaders);
       if (d > 1) {
         // rank of each previous-layer node, recomputed here so that layers stay independent
-        const unsigned pu = alive_prev ? (unsigned)__ldg(s.pq + gpos + d - 1) : 0u;
+        const unsigned pu = alive_prev ? (unsigned)ldm(s.pq + gpos + d - 1) : 0u;
         const unsigned live_prev = __ballot_sync(FULL, alive_prev);
         u64 S_u, unused;
         group_sums(live_prev, gu, 0u, pu, &S_u, &unused);
@@ -404,8 +410,8 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       const int j = gpos / s.L;
       const int e = gpos - j * s.L;
       const bool on = e + dd <= plen[j - poff] - 1;
-      sm.st_tok[x] = on ? __ldg(s.tok + gpos + dd) : -1;
-      sm.st_pq[x] = on ? __ldg(s.pq + gpos + dd) : 0;
+      sm.st_tok[x] = on ? ldm(s.tok + gpos + dd) : -1;
+      sm.st_pq[x] = on ? ldm(s.pq + gpos + dd) : 0;
     }
   }
   for (int x = tid; x < CAP; x += blockDim.x) {
@@ -461,10 +467,10 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 const int gpos = mlist[m];
                 const int j = gpos / s.L;
                 if (gpos - j * s.L + d <= plen[j - poff] - 1) {
-                  v[r] = __ldg(s.tok + gpos + d);
-                  u[r] = d == 1 ? root : __ldg(s.tok + gpos + d - 1);
-                  p[r] = (unsigned)__ldg(s.pq + gpos + d);
-                  if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (__ldg(s.tok + gpos + x) != sh_draft[x - 1]) v[r] = -1;
+                  v[r] = ldm(s.tok + gpos + d);
+                  u[r] = d == 1 ? root : ldm(s.tok + gpos + d - 1);
+                  p[r] = (unsigned)ldm(s.pq + gpos + d);
+                  if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (ldm(s.tok + gpos + x) != sh_draft[x - 1]) v[r] = -1;
                 }
               }
             }
@@ -678,7 +684,7 @@ __device__ void list_pool(const Dev& s, int i, int M, const int32_t* mlist, cons
     const int j = gpos / s.L;
     const int n_m = min(D, plen[j - poff] - 1 - (gpos - j * s.L));
     u64 S = 0;
-    for (int d = 1; d <= n_m; ++d) S += (unsigned)__ldg(s.pq + gpos + d);
+    for (int d = 1; d <= n_m; ++d) S += (unsigned)ldm(s.pq + gpos + d);
     const double w = eq5_weight(s.alpha, S, (unsigned)n_m);
     if (best_g < 0 || ranks_before(w, gpos, best_w, best_g)) { best_w = w; best_g = gpos; }
   }
@@ -694,8 +700,8 @@ __device__ void list_pool(const Dev& s, int i, int M, const int32_t* mlist, cons
   const int j = best_g / s.L;
   const int n_m = min(D, plen[j - poff] - 1 - (best_g - j * s.L));
   if (lane < n_m) {
-    const float w = (float)eq5_weight(s.alpha, (unsigned)__ldg(s.pq + best_g + 1 + lane), 1u);
-    draft_tok[(size_t)i * D + lane] = __ldg(s.tok + best_g + 1 + lane);
+    const float w = (float)eq5_weight(s.alpha, (unsigned)ldm(s.pq + best_g + 1 + lane), 1u);
+    draft_tok[(size_t)i * D + lane] = ldm(s.tok + best_g + 1 + lane);
     if (draft_score) draft_score[(size_t)i * D + lane] = w;
     if (draft_edge_w) draft_edge_w[(size_t)i * D + lane] = w;
   }
@@ -733,9 +739,9 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
     return;
   }
   const int g = i / s.N;
-  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
+  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + g * s.N + n);
   __syncthreads();
-  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, s.rec[(size_t)i * kRecWords + 1],
+  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, ldm(s.rec + (size_t)i * kRecWords + 1),
                     draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
@@ -763,7 +769,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   const int i = blockIdx.x, tid = threadIdx.x;
   const int g = i / s.N;
-  for (int n = tid; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
+  for (int n = tid; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + g * s.N + n);
   const int slice = s.N * s.L;
   int32_t* my_matches = s.matches + (size_t)i * slice;
 
@@ -774,24 +780,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
   if (tid == 0) {
     // the path's record: length and last tokens (newest first) in one 128-byte line
     const int32_t* rec = s.rec + (size_t)i * kRecWords;
-    const int len_i = rec[0];
+    const int len_i = ldm(rec);
     int mode = Q_NONE;
     uint32_t fp = 0, count = 0;
     if (len_i >= k && len_i < s.L && s.eps > 0) {      // fuzzy matches are found by scanning only
-      for (int t = 0; t < k; ++t) sh_q[t] = rec[k - t];
+      for (int t = 0; t < k; ++t) sh_q[t] = ldm(rec + k - t);
       mode = Q_SCAN;
     } else if (len_i >= k && len_i < s.L) {
       uint64_t h = gram_init(k);
-      for (int t = 0; t < k; ++t) { const int32_t x = rec[k - t]; sh_q[t] = x; h = gram_step(h, x); }
+      for (int t = 0; t < k; ++t) { const int32_t x = ldm(rec + k - t); sh_q[t] = x; h = gram_step(h, x); }
       h = gram_final(h);
       fp = gram_fp(h);
       const uint32_t* table = index_table(s, g, k);
       uint32_t b = gram_bucket(h, s.table_cap);
       for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
         const uint4* cand = reinterpret_cast<const uint4*>(table + (size_t)b * kBucketWords);
-        const uint4 lo = cand[0];
+        const uint4 lo = ldm(cand);
         if (lo.x == fp) {
-          const uint4 hi = cand[1];
+          const uint4 hi = ldm(cand + 1);
           count = lo.y;
           sh_pos[0] = lo.z; sh_pos[1] = lo.w; sh_pos[2] = hi.x; sh_pos[3] = hi.y; sh_pos[4] = hi.z; sh_pos[5] = hi.w;
           mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
@@ -815,7 +821,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
       if (j != i && e <= sh_len[jn] - 2) {
         const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
         bool same = true;
-        for (int t = 0; t < k; ++t) same = same && (c[t] == sh_q[t]);
+        for (int t = 0; t < k; ++t) same = same && (ldm(c + t) == sh_q[t]);
         if (same) {
           const int at = atomicAdd(&sh_M, 1);
           sm.list[at] = j * s.L + e;
@@ -834,7 +840,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
       const int e_hi = sh_len[jn] - 2;
       for (int e = tid; e <= e_hi; e += blockDim.x) {
         int b = 0;
-        while (b < k && b <= e && __ldg(row + e - b) == sh_q[k - 1 - b]) ++b;
+        while (b < k && b <= e && ldm(row + e - b) == sh_q[k - 1 - b]) ++b;
         bool found = false;
         for (int n = max(1, k - 1); n <= k + 1 && !found; ++n) {
           if (e - n + 1 < 0) break;
@@ -842,7 +848,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
           if (need <= 0) { found = true; break; }
           if (need > shorter) continue;
           int a = 0;
-          while (a < need && __ldg(row + e - n + 1 + a) == sh_q[a]) ++a;
+          while (a < need && ldm(row + e - n + 1 + a) == sh_q[a]) ++a;
           found = a >= need;
         }
         if (found) {
@@ -860,7 +866,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
     const int32_t* gtok = s.tok + (size_t)g * s.N * s.L;
     auto hit = [&](int jn, int e) {
       const int32_t* row = gtok + (size_t)jn * s.L;
-      for (int t = 0; t < k - 1; ++t) if (__ldg(row + e - (k - 1) + t) != sh_q[t]) return;
+      for (int t = 0; t < k - 1; ++t) if (ldm(row + e - (k - 1) + t) != sh_q[t]) return;
       const int at = atomicAdd(&sh_M, 1);
       const int pos = (g * s.N + jn) * s.L + e;
       if (at < kListCap) sm.list[at] = pos;
@@ -880,7 +886,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
           for (int r = 0; r < kBatch; ++r) {
             const int jn = j0 + r;
             e_hi[r] = (jn < s.N && g * s.N + jn != i) ? sh_len[jn] - 2 : -1;   // last position with a follower
-            if (e0 <= e_hi[r]) w[r] = __ldg(g4 + (size_t)jn * per + c);
+            if (e0 <= e_hi[r]) w[r] = ldm(g4 + (size_t)jn * per + c);
           }
 #pragma unroll
           for (int r = 0; r < kBatch; ++r) {
@@ -897,7 +903,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
       for (int x = tid; x < total; x += blockDim.x) {
         const int jn = x / s.L, e = x - jn * s.L;
         if (g * s.N + jn == i || e < k - 1 || e > sh_len[jn] - 2) continue;
-        if (__ldg(gtok + x) == last) hit(jn, e);
+        if (ldm(gtok + x) == last) hit(jn, e);
       }
     }
   }

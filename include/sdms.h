@@ -159,6 +159,24 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
                 const int32_t* d_sampled, const float* d_sampled_logprobs,
                 int32_t* d_accept_len, void* stream);
 
+/*
+ * One decode step in one call: sdms_accept with commit on the drafts that
+ * d_draft_tok / d_draft_len hold on entry (the previous call's output), then
+ * sdms_build_drafts(k) into the same arrays ("Draft acceptance" followed by
+ * Eq. 3, Eq. 5 and the greedy search on the extended histories).  The results
+ * are identical to those two calls made one after the other.
+ * d_sampled and d_sampled_logprobs ([P][D+1]) are both required.
+ * When a prompt's paths fit one thread-block cluster (paths_per_group <= 16, the
+ * single-launch build applies and the device can co-schedule such a cluster) the
+ * step is ONE kernel launch: the paths of a prompt commit, meet at a cluster
+ * barrier, and build.  Otherwise the call issues the separate launches.
+ * sdms_step_is_single_launch reports which (1 / 0).
+ */
+int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,
+              int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
+              float* d_draft_edge_w, void* stream);
+int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes);
+
 /* ---- inspection (used by the parity tests; not part of a decode step) ------- */
 
 /* Matches of the last sdms_build_drafts: d_offsets [P+1] (exclusive prefix sums)
@@ -231,7 +249,8 @@ int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, int32_t num_g
 #define SDMS_KERNEL_DAG    3
 #define SDMS_KERNEL_ACCEPT 4
 #define SDMS_KERNEL_BUILD_FUSED 5   /* probe + scan + dag in one launch (small prompts) */
-#define SDMS_NUM_KERNELS   6
+#define SDMS_KERNEL_STEP   6        /* accept + commit + build in one launch (sdms_step) */
+#define SDMS_NUM_KERNELS   7
 
 /* Number of kernels this context has launched since creation. */
 int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches);

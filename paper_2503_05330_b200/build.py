@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdms.so")
 SOURCES = ["api.cu", "append.cu", "match.cu", "dag.cu", "match_static.cu"]
-HEADERS = ["sdms_dev.cuh", "sdms_internal.h"]
+HEADERS = ["sdms_dev.cuh", "sdms_internal.h", "append_dev.cuh"]
 
 
 def _newest_source() -> float:

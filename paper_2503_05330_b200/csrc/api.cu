@@ -102,6 +102,7 @@ struct sdms_ctx {
   uint64_t launches;
   bool profiling;
   bool built;
+  bool step_fits;                                // sdms_step runs as one cluster launch
   int32_t* x_draft_tok; int32_t* x_draft_len;   // where the export pass leaves the drafts it recomputes
   std::vector<EventPair> pending;
   std::vector<EventPair> pool;
@@ -170,6 +171,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.fused = fits_fused(cfg, lay);
   d.eps = cfg->epsilon;
   d.pool = cfg->pool_mode;
+  ctx->step_fits = false;                        // decided below, once the kernels' attributes are set
   unsigned char* w = ctx->ws;
   d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len); d.rec = (int32_t*)(w + lay.rec);
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);
@@ -182,6 +184,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.x_node_cnt = (int32_t*)(w + lay.x_node_cnt); d.x_node_count = (int32_t*)(w + lay.x_node_count);
   d.x_edge_dst = (int32_t*)(w + lay.x_edge_dst); d.x_edge_S = (int64_t*)(w + lay.x_edge_S);
   d.x_edge_cnt = (int32_t*)(w + lay.x_edge_cnt); d.x_out_degree = (int32_t*)(w + lay.x_out_degree);
+  ctx->step_fits = step_kernel_fits(d);
   *out = ctx;
   return SDMS_OK;
 }
@@ -253,6 +256,32 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
   if (d_sampled_logprobs) ctx->built = false;          // the commit changes the histories
   return timed(ctx, SDMS_KERNEL_ACCEPT, st, [&] {
     return launch_accept(ctx->dev, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, st); });
+}
+
+int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,
+              int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
+              float* d_draft_edge_w, void* stream) {
+  if (!ctx || !d_sampled || !d_sampled_logprobs || !d_accept_len || !d_draft_tok || !d_draft_len)
+    return SDMS_ERR_INVALID_ARG;
+  if (k < 1 || k > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->step_fits) {
+    const int rc = sdms_accept(ctx, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, stream);
+    if (rc != SDMS_OK) return rc;
+    return sdms_build_drafts(ctx, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, stream);
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->built = false;
+  const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
+    return launch_step(ctx->dev, k, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
+                       d_draft_score, d_draft_edge_w, st); });
+  if (rc == SDMS_OK) ctx->built = true;
+  return rc;
+}
+
+int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes) {
+  if (!ctx || !yes) return SDMS_ERR_INVALID_ARG;
+  *yes = ctx->step_fits ? 1 : 0;
+  return SDMS_OK;
 }
 
 int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t cap, void* stream) {
@@ -357,7 +386,7 @@ const char* sdms_strerror(int code) {
 }
 
 const char* sdms_kernel_name(int kernel) {
-  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept", "build_fused"};
+  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept", "build_fused", "step"};
   return kernel >= 0 && kernel < SDMS_NUM_KERNELS ? names[kernel] : "?";
 }
 

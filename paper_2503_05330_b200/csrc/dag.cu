@@ -29,6 +29,7 @@
 //   the nodes kept one layer up.  tree / list pools reuse the same passes with a
 //   prefix filter / a single arg-max over candidates.
 #include "sdms_internal.h"
+#include "append_dev.cuh"
 
 namespace sdms {
 
@@ -753,16 +754,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
 // gather / DAG / search phase runs on the matches just found.  The matches also
 // go to the path's private slice of the match list for inspection.
 template <bool EXPORT>
-__global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo,
-                                                                  int32_t* __restrict__ draft_tok,
-                                                                  int32_t* __restrict__ draft_len,
-                                                                  float* __restrict__ draft_score,
-                                                                  float* __restrict__ draft_edge_w,
-                                                                  int32_t* __restrict__ used_k) {
-  grid_wait();
-  grid_release();
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const Smem sm = carve<EXPORT>(smem_raw);
+__device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
+                            float* draft_score, float* draft_edge_w, int32_t* used_k) {
   __shared__ int sh_mode, sh_M;
   __shared__ uint32_t sh_count, sh_pos[kInlineSlots];
   __shared__ int32_t sh_q[SDMS_MAX_K];
@@ -921,6 +914,37 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
                     draft_len, draft_score, draft_edge_w);
 }
 
+template <bool EXPORT>
+__global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo, int32_t* draft_tok,
+                                                                  int32_t* draft_len, float* draft_score,
+                                                                  float* draft_edge_w, int32_t* used_k) {
+  grid_wait();
+  grid_release();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Smem sm = carve<EXPORT>(smem_raw);
+  build_phase<EXPORT>(s, sm, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
+}
+
+// One launch per decode step.  The CTAs of a prompt form a thread-block cluster.  Each CTA first
+// checks its path's previous draft against the sampled tokens and appends what was accepted (tokens,
+// probabilities, index entries); after a cluster-wide barrier with release/acquire semantics every
+// path of the prompt is up to date and each CTA builds its path's next draft.  draft_tok / draft_len
+// hold the previous drafts on entry and the new ones on exit.
+__global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, const int32_t* sampled,
+                                                           const float* sampled_lp, int32_t* accept_len,
+                                                           int32_t* draft_tok, int32_t* draft_len,
+                                                           float* draft_score, float* draft_edge_w) {
+  grid_wait();
+  grid_release();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Smem sm = carve<false>(smem_raw);
+  accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len);
+  __threadfence();
+  // every thread of every CTA of the cluster gets here exactly once (no early exit above)
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  build_phase<false>(s, sm, k, k, draft_tok, draft_len, draft_score, draft_edge_w, nullptr);
+}
+
 }  // namespace
 
 cudaError_t dag_kernel_setup() {
@@ -932,7 +956,43 @@ cudaError_t dag_kernel_setup() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
+}
+
+namespace {
+void step_launch_config(const Dev& s, cudaStream_t stream, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr) {
+  *cfg = cudaLaunchConfig_t{};
+  cfg->gridDim = dim3(s.P); cfg->blockDim = dim3(kFusedThreads);
+  cfg->dynamicSmemBytes = dag_smem_bytes<false>(); cfg->stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = s.N; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg->attrs = attr; cfg->numAttrs = 2;
+}
+}  // namespace
+
+// Can the prompts of this context run as clusters (one CTA per path) on this device?
+bool step_kernel_fits(const Dev& s) {
+  if (!s.fused || s.N > kMaxClusterPaths) return false;
+  cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
+  step_launch_config(s, 0, &cfg, attr);
+  cfg.numAttrs = 1;                                   // occupancy only looks at the cluster shape
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, step_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
+  return clusters >= 1;
+}
+
+cudaError_t launch_step(const Dev& s, int k, const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
+                        int32_t* draft_tok, int32_t* draft_len, float* draft_score, float* draft_edge_w,
+                        cudaStream_t stream) {
+  cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
+  step_launch_config(s, stream, &cfg, attr);
+  return cudaLaunchKernelEx(&cfg, step_kernel, s, k, sampled, sampled_lp, accept_len, draft_tok, draft_len,
+                            draft_score, draft_edge_w);
 }
 
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,

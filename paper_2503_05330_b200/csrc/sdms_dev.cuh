@@ -13,6 +13,7 @@ constexpr int kHalo = SDMS_MAX_K;      // tokens staged in front of a scan tile
 constexpr int kScanTile = 1024;        // history tokens per scan CTA
 constexpr int kScanThreads = 256;
 constexpr int kDagThreads = 512;
+constexpr int kMaxClusterPaths = 16;    // largest thread-block cluster (one CTA per path of a prompt)
 constexpr int kFusedThreads = 512;     // the single-launch build: more loads in flight while it scans
 constexpr int kDagCap = 1024;          // entries of the shared-memory node / edge tables
 constexpr int kFusedMaxTokens = 131072; // largest N*L a CTA scans on its own

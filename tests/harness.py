@@ -143,3 +143,42 @@ def run_protocol(pair: Pair, tokens, logprobs, k, steps, warm, commit_in_accept=
         done_steps += 1
     pair.check_history()
     return dict(steps=done_steps, accepted=accepted, drafted=drafted)
+
+
+def run_step_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, start_lens=None, check_matches=True):
+    """The same decode protocol through the one-call step: after a first build,
+    every step is accept + commit + the next build (suffix length ks[step % len(ks)])
+    in one call, compared with the oracle's accept_commit followed by build_all."""
+    P, L, D = pair.P, pair.L, pair.D
+    lens = np.full(P, warm, np.int32) if start_lens is None else np.asarray(start_lens, np.int32)
+    w = int(lens.max())
+    pair.append(tokens[:, :w], logprobs[:, :w], lens, expect_status=0)
+    pair.build_and_compare(ks[0], check_matches=check_matches, check_dag=False)
+    accepted = 0
+    done_steps = 0
+    for step in range(steps):
+        lens = pair.o.lengths()
+        if (lens >= L).all():
+            break
+        k = ks[(step + 1) % len(ks)]
+        sampled, sampled_lp = synth.sampled_window(tokens, logprobs, lens, D + 1)
+        tok, ln, _, _ = pair.o.drafts()
+        tau_o, st_o = pair.o.accept_commit(tok, ln, sampled, sampled_lp, pair.max_append)
+        pair.o.build_all(k, nthreads=min(8, os.cpu_count() or 1))
+        tau_g, gt, gl = pair.g.step(k, t32(sampled, pair.dev), t32(sampled_lp, pair.dev))
+        assert pair.g.status() == st_o
+        assert np.array_equal(tau_g.cpu().numpy(), tau_o), (step, tau_g, tau_o)
+        tok, ln, sc, ew = pair.o.drafts()
+        assert np.array_equal(gl.cpu().numpy(), ln), (step, k, gl, ln)
+        assert np.array_equal(gt.cpu().numpy(), tok), (step, k)
+        np.testing.assert_allclose(pair.g.draft_score.cpu().numpy(), sc, rtol=RTOL, atol=0)
+        np.testing.assert_allclose(pair.g.draft_edge_w.cpu().numpy(), ew, rtol=RTOL, atol=0)
+        if check_matches:
+            off, gpos = pair.g.matches()
+            off, gpos = off.numpy(), gpos.numpy()
+            for i in range(P):
+                assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), pair.o.matches(i)), (step, k, i)
+        accepted += int(tau_o.sum())
+        done_steps += 1
+    pair.check_history()
+    return dict(steps=done_steps, accepted=accepted)

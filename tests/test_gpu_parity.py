@@ -348,3 +348,54 @@ def test_backoff_dense_tiny_vocab_and_short_paths():
     pair.append(tokens[:, :12], lps[:, :12], np.array([12, 1, 2, 3, 0, 7, 12, 5], np.int32), expect_status=0)
     for k_hi in (4, 2, 1):
         pair.backoff_and_compare(k_hi)
+
+
+# ---- the whole decode step in one call -------------------------------------------------------
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("alpha,mode,pool,eps", [(1.0, 0, 0, 0), (0.5, 0, 0, 0), (1.0, 1, 0, 0), (0.5, 0, 1, 0),
+                                                 (1.0, 0, 2, 0), (0.5, 0, 0, 1)])
+def test_step_dense_tiny_vocab(seed, alpha, mode, pool, eps):
+    G, N, L, V, D, k_max = 3, 4, 48, 3 + seed % 2, 4, 3
+    tokens, lps = synth.small_random(G * N, L, V, 5200 + seed)
+    pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, eps=eps, pool=pool, max_append=D - seed % 2)
+    assert pair.g.step_is_single_launch()
+    start = 3 + (np.arange(G * N) * 5 + seed) % 9
+    st = harness.run_step_protocol(pair, tokens, lps, [1, 3, 2], steps=40, warm=0, start_lens=start)
+    assert st["steps"] > 5
+
+
+@pytest.mark.parametrize("wid", [1, 2])
+def test_step_config_full_protocol(wid):
+    w = synth.WORKLOADS[wid]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    assert pair.g.step_is_single_launch()
+    st = harness.run_step_protocol(pair, tokens, lps, list(range(w.k_max, 0, -1)), steps=w.steps, warm=w.k_max,
+                                   check_matches=False)
+    assert st["steps"] > 40 and st["accepted"] > 0
+    from paper_2503_05330_b200 import binding
+    lens = pair.o.lengths()
+    sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
+    n0 = binding.sdms_launch_count(pair.g.ctx)
+    pair.g.step(2, harness.t32(sampled, pair.dev), harness.t32(sampled_lp, pair.dev))
+    assert binding.sdms_launch_count(pair.g.ctx) == n0 + 1
+
+
+def test_step_many_prompts_ragged():
+    w = synth.WORKLOADS[4]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    assert pair.g.step_is_single_launch()
+    start = (int(w.L * 0.98) - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    st = harness.run_step_protocol(pair, tokens, lps, [5, 1, 3], steps=12, warm=0, start_lens=start,
+                                   check_matches=False)
+    assert st["steps"] == 12                   # runs into full paths: those stop drafting and committing
+
+
+def test_step_falls_back_to_separate_launches_for_wide_prompts():
+    G, N, L, V, D, k_max = 1, 24, 64, 5, 4, 3
+    tokens, lps = synth.small_random(G * N, L, V, 77)
+    pair = Pair(G, N, L, V, k_max, D)
+    assert not pair.g.step_is_single_launch()
+    st = harness.run_step_protocol(pair, tokens, lps, [2, 1, 3], steps=20, warm=4)
+    assert st["steps"] > 5

@@ -37,7 +37,7 @@ def kernel_sources_sha():
     import hashlib
     h = hashlib.sha256()
     base = os.path.join(ROOT, "paper_2503_05330_b200", "csrc")
-    for name in ("dag.cu", "sdms_dev.cuh"):
+    for name in ("dag.cu", "sdms_dev.cuh", "append_dev.cuh"):
         h.update(open(os.path.join(base, name), "rb").read())
     return h.hexdigest()
 
@@ -174,9 +174,11 @@ class Runner:
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
         self.plan = None
 
-    def start_run(self):
+    def start_run(self, first_drafts=False):
         self.s.reset()
         self.s.append(self.warm_tok, self.warm_lp, self.warm_cnt)
+        if first_drafts:                 # the drafts the first sdms_step of a run checks
+            self.s.build_drafts(k_of(0, self.w.k_max))
 
     def dry_run(self):
         """Plays one run to record, per step, the sampled windows (what the model
@@ -224,7 +226,8 @@ class Runner:
                  np.stack(lp_all).view(np.int32).reshape(len(active), -1)], axis=1)).pin_memory(),
             active=active, steps=len(active),
             bytes={"scan": float(np.mean(bytes_scan)), "dag": float(np.mean(bytes_dag)),
-                   "accept": float(np.mean(bytes_io)), "build_fused": float(np.mean(bytes_fused))},
+                   "accept": float(np.mean(bytes_io)), "build_fused": float(np.mean(bytes_fused)),
+                   "step": float(np.mean(bytes_fused)) + float(np.mean(bytes_io))},
             useful_bytes_build=float(np.mean(bytes_useful)), scan_queries_per_step=float(np.mean(scan_queries)),
             mean_matches_per_step=float(np.mean(matches)),
             accept_length=float(np.sum(accepted)) / float(np.sum(active)))
@@ -232,7 +235,9 @@ class Runner:
 
     def timed_steps(self, K, flush=True, e2e=False):
         """Times exactly K steps (CUDA events around each step on the launch
-        stream), restarting the run when it ends.  Returns (ms, paths*steps)."""
+        stream), restarting the run when it ends.  A step is one sdms_step call: acceptance check
+        and commit of the drafts of decode step t, then the drafts of step t + 1.
+        Returns (ms, paths*steps)."""
         torch, w, s, plan = self.torch, self.w, self.s, self.plan
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         units = 0
@@ -249,9 +254,10 @@ class Runner:
         for r in range(runs):
             quota = K // runs + (1 if r < K % runs else 0)
             timed = set(int((x + 0.5) * S / quota) for x in range(quota)) if quota < S else set(range(S))
-            self.start_run()
+            self.start_run(first_drafts=True)
             for step in range(S):
                 on = step in timed
+                k_next = k_of(step + 1, w.k_max)
                 if on and flush:
                     self.flush.zero_()
                 if on:
@@ -259,19 +265,17 @@ class Runner:
                     a.record()
                 if e2e and on:
                     s.step_in.copy_(h_in[step], non_blocking=True)
-                    s.build_drafts(k_of(step, w.k_max))
-                    s.accept(s.sampled_in, s.sampled_lp_in)
+                    s.step(k_next, s.sampled_in, s.sampled_lp_in)
                     h_res.copy_(s.results, non_blocking=True)
                     b.record()
                     b.synchronize()                 # the caller reads the result before its next step
                 else:
-                    s.build_drafts(k_of(step, w.k_max))
-                    s.accept(plan["sampled"][step], plan["lp"][step])
+                    s.step(k_next, plan["sampled"][step], plan["lp"][step])
                     if on:
                         b.record()
                 if on:
                     units += plan["active"][step]
-                    ks.append(k_of(step, w.k_max))
+                    ks.append(k_next)
                     done += 1
         assert done == K
         torch.cuda.synchronize()
@@ -475,7 +479,7 @@ def ours_main(args, w):
         "dtype": "int32/int64 (f64 weights)", "data": "synthetic", "config": workload_config(w),
         "e2e": {"value": units_e2e / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": 1e3 * ms_e2e / args.steps,
                 "h2d_bytes_per_step": w.P * (w.D + 1) * 8, "d2h_bytes_per_step": w.P * (w.D + 2) * 4},
-        "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
+        "gpu_launches": launches, "single_launch_step": run.s.step_is_single_launch(), "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
         "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,

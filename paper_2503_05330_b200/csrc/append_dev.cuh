@@ -90,9 +90,12 @@ __device__ void index_insert(const Dev& s, int g, int n, uint64_t h, uint32_t lp
   uint32_t b = gram_bucket(h, s.table_cap);
   for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
     uint32_t* bucket = table + (size_t)b * kBucketWords;
-    const uint32_t old = atomicCAS(&bucket[0], 0u, fp);
-    if (old == 0u || old == fp) {
-      const uint32_t slot = atomicAdd(&bucket[1], 1u);
+    // {fingerprint, count} is one 64-bit word: an empty bucket is claimed and counted in one atomic
+    unsigned long long* head = reinterpret_cast<unsigned long long*>(bucket);
+    const unsigned long long old = atomicCAS(head, 0ull, (1ull << 32) | fp);
+    if (old == 0ull) { bucket[2] = lpos; return; }
+    if ((uint32_t)old == fp) {
+      const uint32_t slot = (uint32_t)(atomicAdd(head, 1ull << 32) >> 32);
       if (slot < (uint32_t)kInlineSlots) bucket[2 + slot] = lpos;
       return;
     }
@@ -103,10 +106,10 @@ __device__ void index_insert(const Dev& s, int g, int n, uint64_t h, uint32_t lp
 
 // Block-cooperative append of n validated tokens to path p whose length is len0.  rec is the
 // path's record as it was before the call (shared memory): rec[1 + t] = token at len0 - 1 - t.
-// Ends with a barrier-free write of the new record by the first k_max threads; the caller
-// updates nothing else.
+// Also writes the path's new record and length (and a copy of the record to rec_out, shared
+// memory, if given); no barrier inside.
 __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_t* in_tok,
-                              const float* in_lp, const int32_t* rec, uint32_t* st) {
+                              const float* in_lp, const int32_t* rec, uint32_t* st, int32_t* rec_out = nullptr) {
   int32_t* tok = s.tok + (size_t)p * s.L;
   int32_t* pq = s.pq + (size_t)p * s.L;
   for (int a = threadIdx.x; a < n; a += blockDim.x) {
@@ -126,53 +129,73 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
   }
   // the record after the append: new length, then the newest k_max tokens
   int32_t* out = s.rec + (size_t)p * kRecWords;
-  if (threadIdx.x < s.k_max) {
-    const int x = len0 + n - 1 - (int)threadIdx.x;                       // position of the token this word holds
-    out[1 + threadIdx.x] = x >= len0 ? in_tok[x - len0] : (x >= 0 ? rec[len0 - x] : 0);
+  // (the last warp writes it, so that the warps with inserts to do are not held up)
+  const int r = (int)blockDim.x - 1 - (int)threadIdx.x;
+  if (r < s.k_max) {
+    const int x = len0 + n - 1 - r;                                      // position of the token this word holds
+    const int32_t v = x >= len0 ? in_tok[x - len0] : (x >= 0 ? rec[len0 - x] : 0);
+    out[1 + r] = v;
+    if (rec_out) rec_out[1 + r] = v;
   }
-  if (threadIdx.x == 0) { out[0] = len0 + n; s.len[p] = len0 + n; }
+  if (r == s.k_max) {
+    out[0] = len0 + n; s.len[p] = len0 + n;
+    if (rec_out) rec_out[0] = len0 + n;
+  }
 }
 
 // "Draft acceptance" for path p, then (if sampled_lp is given) the commit: the path appends
-// sampled[0 .. min(tau + 1, max_append)).  Block-cooperative, any block size >= 32; every thread of
-// the CTA must call it.  draft_tok / draft_len are only read.
+// sampled[0 .. min(tau + 1, max_append)).  Block-cooperative, any block size >= 64; every thread of
+// the CTA must call it.  draft_tok / draft_len are only read.  If rec_out is given (shared memory,
+// kRecWords words) it receives the path's record as it is after the call.
 __device__ void accept_commit_phase(const Dev& s, int p, const int32_t* draft_tok, const int32_t* draft_len,
-                                    const int32_t* sampled, const float* sampled_lp, int32_t* accept_len) {
-  __shared__ int sh_len0, sh_n, sh_bad;
+                                    const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
+                                    int32_t* rec_out = nullptr) {
+  __shared__ int sh_len0, sh_n;
   __shared__ uint32_t sh_st;
   __shared__ int32_t sh_rec[kRecWords];
+  __shared__ int32_t sh_smp[SDMS_MAX_DRAFT + 1];
+  __shared__ float sh_lp[SDMS_MAX_DRAFT + 1];
   const int32_t* smp = sampled + (size_t)p * (s.D + 1);
-  if (threadIdx.x < 32) {
-    static_assert(kRecWords == 32, "one record word per lane");
-    const int32_t mine = sampled_lp ? s.rec[(size_t)p * kRecWords + threadIdx.x] : 0;   // in flight with the draft
-    sh_rec[threadIdx.x] = mine;
+  const int lane = threadIdx.x;
+  if (lane < 32) {
+    static_assert(kRecWords == 32 && SDMS_MAX_DRAFT <= 32, "one record word, one draft position per lane");
+    // every load of this phase is issued before the first use: one round trip to memory
+    const int32_t mine = sampled_lp ? s.rec[(size_t)p * kRecWords + lane] : 0;
     int dl = draft_len[p];
+    const int32_t drafted = lane < s.D ? draft_tok[(size_t)p * s.D + lane] : -1;
+    const int32_t got = lane <= s.D ? smp[lane] : -1;
+    const int32_t got_last = lane == 0 && s.D == 32 ? smp[32] : -1;       // position D when D fills the warp
+    float lp = 0.0f, lp_last = 0.0f;
+    if (sampled_lp) {
+      const float* slp = sampled_lp + (size_t)p * (s.D + 1);
+      if (lane <= s.D) lp = slp[lane];
+      if (lane == 0 && s.D == 32) lp_last = slp[32];
+    }
+    sh_rec[lane] = mine;
+    sh_smp[lane] = got; sh_lp[lane] = lp;
+    if (lane == 0) { sh_smp[32] = got_last; sh_lp[32] = lp_last; }
     dl = dl < 0 ? 0 : (dl > s.D ? s.D : dl);
-    const int d = threadIdx.x;
-    const bool differs = d >= dl || draft_tok[(size_t)p * s.D + d] != smp[d];
+    const bool differs = lane >= dl || drafted != got;
     const unsigned first = __ffs(__ballot_sync(0xffffffffu, differs));   // 0 only if all 32 lanes agree
     const int tau = first ? (int)first - 1 : 32;
-    if (d == 0) {
-      accept_len[p] = tau;
-      int n = 0, len0 = 0;
-      if (sampled_lp) {
-        len0 = mine;                                  // lane 0 holds the length
-        n = min(min(tau + 1, s.max_append), s.L - len0);
-      }
-      sh_len0 = len0; sh_n = n; sh_bad = n; sh_st = 0;
+    int n = 0, len0 = 0;
+    if (sampled_lp) {
+      len0 = __shfl_sync(0xffffffffu, mine, 0);         // lane 0 holds the length
+      n = min(min(tau + 1, s.max_append), s.L - len0);
+      // the commit stops before the first token outside the vocabulary
+      const bool bad = lane < n && (got < 0 || got >= s.V);
+      const bool bad_last = lane == 0 && n == 33 && (got_last < 0 || got_last >= s.V);      // only lane 0 can see it
+      const unsigned bad_mask = __ballot_sync(0xffffffffu, bad);
+      const unsigned bad_last_any = __ballot_sync(0xffffffffu, bad_last);
+      int ok = bad_mask ? __ffs(bad_mask) - 1 : (bad_last_any ? 32 : n);
+      if (lane == 0) { sh_st = ok < n ? SDMS_STATUS_BAD_TOKEN : 0u; sh_len0 = len0; sh_n = ok; }
     }
+    if (lane == 0) accept_len[p] = tau;
   }
   if (!sampled_lp) return;                            // uniform: check only
   __syncthreads();
-  for (int a = threadIdx.x; a < sh_n; a += blockDim.x) {
-    const int32_t t = smp[a];
-    if (t < 0 || t >= s.V) atomicMin(&sh_bad, a);
-  }
-  __syncthreads();
   uint32_t st = 0;
-  const int n = sh_bad;
-  if (threadIdx.x == 0 && n < sh_n) st |= SDMS_STATUS_BAD_TOKEN;
-  append_tokens(s, p, sh_len0, n, smp, sampled_lp + (size_t)p * (s.D + 1), sh_rec, &st);
+  append_tokens(s, p, sh_len0, sh_n, sh_smp, sh_lp, sh_rec, &st, rec_out);
   if (st) atomicOr(&sh_st, st);
   __syncthreads();
   if (threadIdx.x == 0 && sh_st) atomicOr(s.status, sh_st);

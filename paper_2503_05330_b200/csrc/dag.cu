@@ -755,7 +755,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
 // go to the path's private slice of the match list for inspection.
 template <bool EXPORT>
 __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
-                            float* draft_score, float* draft_edge_w, int32_t* used_k) {
+                            float* draft_score, float* draft_edge_w, int32_t* used_k,
+                            const int32_t* own_rec = nullptr) {
   __shared__ int sh_mode, sh_M;
   __shared__ uint32_t sh_count, sh_pos[kInlineSlots];
   __shared__ int32_t sh_q[SDMS_MAX_K];
@@ -771,8 +772,9 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
   int k = k_hi;
   for (;; --k) {
   if (tid == 0) {
-    // the path's record: length and last tokens (newest first) in one 128-byte line
-    const int32_t* rec = s.rec + (size_t)i * kRecWords;
+    // the path's record: length and last tokens (newest first) in one 128-byte line (or the copy
+    // the caller already holds in shared memory)
+    const int32_t* rec = own_rec ? own_rec : s.rec + (size_t)i * kRecWords;
     const int len_i = ldm(rec);
     int mode = Q_NONE;
     uint32_t fp = 0, count = 0;
@@ -788,9 +790,8 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
       uint32_t b = gram_bucket(h, s.table_cap);
       for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
         const uint4* cand = reinterpret_cast<const uint4*>(table + (size_t)b * kBucketWords);
-        const uint4 lo = ldm(cand);
+        const uint4 lo = ldm(cand), hi = ldm(cand + 1);      // both halves in flight together
         if (lo.x == fp) {
-          const uint4 hi = ldm(cand + 1);
           count = lo.y;
           sh_pos[0] = lo.z; sh_pos[1] = lo.w; sh_pos[2] = hi.x; sh_pos[3] = hi.y; sh_pos[4] = hi.z; sh_pos[5] = hi.w;
           mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
@@ -938,11 +939,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, co
   grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<false>(smem_raw);
-  accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len);
+  __shared__ int32_t sh_own_rec[kRecWords];
+  accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec);
   __threadfence();
   // every thread of every CTA of the cluster gets here exactly once (no early exit above)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  build_phase<false>(s, sm, k, k, draft_tok, draft_len, draft_score, draft_edge_w, nullptr);
+  build_phase<false>(s, sm, k, k, draft_tok, draft_len, draft_score, draft_edge_w, nullptr, sh_own_rec);
 }
 
 }  // namespace

@@ -112,7 +112,10 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
                               const float* in_lp, const int32_t* rec, uint32_t* st, int32_t* rec_out = nullptr) {
   int32_t* tok = s.tok + (size_t)p * s.L;
   int32_t* pq = s.pq + (size_t)p * s.L;
-  for (int a = threadIdx.x; a < n; a += blockDim.x) {
+  // the stores start from the last thread, the index inserts (below) from the first: with few new
+  // tokens different warps do the two and the atomics are in flight during the exponentials
+  const int r = (int)blockDim.x - 1 - (int)threadIdx.x;
+  for (int a = r; a < n; a += blockDim.x) {
     tok[len0 + a] = in_tok[a];
     pq[len0 + a] = prob_to_fixed(in_lp[a], st);
   }
@@ -129,8 +132,7 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
   }
   // the record after the append: new length, then the newest k_max tokens
   int32_t* out = s.rec + (size_t)p * kRecWords;
-  // (the last warp writes it, so that the warps with inserts to do are not held up)
-  const int r = (int)blockDim.x - 1 - (int)threadIdx.x;
+  // (the last threads write it, so that the warps with inserts to do are not held up)
   if (r < s.k_max) {
     const int x = len0 + n - 1 - r;                                      // position of the token this word holds
     const int32_t v = x >= len0 ? in_tok[x - len0] : (x >= 0 ? rec[len0 - x] : 0);
@@ -146,10 +148,11 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
 // "Draft acceptance" for path p, then (if sampled_lp is given) the commit: the path appends
 // sampled[0 .. min(tau + 1, max_append)).  Block-cooperative, any block size >= 64; every thread of
 // the CTA must call it.  draft_tok / draft_len are only read.  If rec_out is given (shared memory,
-// kRecWords words) it receives the path's record as it is after the call.
+// kRecWords words) it receives the path's record as it is after the call.  next_k > 0 announces
+// the suffix length of the query the path makes next: its index bucket is prefetched into L2.
 __device__ void accept_commit_phase(const Dev& s, int p, const int32_t* draft_tok, const int32_t* draft_len,
                                     const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
-                                    int32_t* rec_out = nullptr) {
+                                    int32_t* rec_out = nullptr, int next_k = 0) {
   __shared__ int sh_len0, sh_n;
   __shared__ uint32_t sh_st;
   __shared__ int32_t sh_rec[kRecWords];
@@ -195,6 +198,16 @@ __device__ void accept_commit_phase(const Dev& s, int p, const int32_t* draft_to
   if (!sampled_lp) return;                            // uniform: check only
   __syncthreads();
   uint32_t st = 0;
+  if (next_k > 0 && s.eps == 0 && threadIdx.x == blockDim.x - 64) {
+    const int len0 = sh_len0, len1 = len0 + sh_n;
+    if (len1 >= next_k && len1 < s.L) {
+      uint64_t h = gram_init(next_k);
+      for (int x = len1 - next_k; x < len1; ++x) h = gram_step(h, x >= len0 ? sh_smp[x - len0] : sh_rec[len0 - x]);
+      const uint32_t* bucket =
+          index_table(s, p / s.N, next_k) + (size_t)gram_bucket(gram_final(h), s.table_cap) * kBucketWords;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(bucket));
+    }
+  }
   append_tokens(s, p, sh_len0, sh_n, sh_smp, sh_lp, sh_rec, &st, rec_out);
   if (st) atomicOr(&sh_st, st);
   __syncthreads();

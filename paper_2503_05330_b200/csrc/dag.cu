@@ -940,8 +940,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, co
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<false>(smem_raw);
   __shared__ int32_t sh_own_rec[kRecWords];
-  accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec);
-  __threadfence();
+  accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec, k);
   // every thread of every CTA of the cluster gets here exactly once (no early exit above)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   build_phase<false>(s, sm, k, k, draft_tok, draft_len, draft_score, draft_edge_w, nullptr, sh_own_rec);

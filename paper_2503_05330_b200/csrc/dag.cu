@@ -753,6 +753,14 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
 // 128-bit loads (last token first, the rest of the window on a hit); then the
 // gather / DAG / search phase runs on the matches just found.  The matches also
 // go to the path's private slice of the match list for inspection.
+// Do the first k - 2 tokens of the window that ends at `at` equal the query's?  (The last two have been
+// compared by the caller.)
+__device__ __forceinline__ bool window_head_equal(const int32_t* at, int k, const int32_t* q) {
+  for (int t = 0; t < k - 2; ++t)
+    if (ldm(at - (k - 1) + t) != q[t]) return false;
+  return true;
+}
+
 template <bool EXPORT>
 __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                             float* draft_score, float* draft_edge_w, int32_t* used_k,
@@ -858,46 +866,62 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
     // compare the last token of the query first, the rest of the window on a hit
     const int last = sh_q[k - 1];
     const int32_t* gtok = s.tok + (size_t)g * s.N * s.L;
-    auto hit = [&](int jn, int e) {
-      const int32_t* row = gtok + (size_t)jn * s.L;
-      for (int t = 0; t < k - 1; ++t) if (ldm(row + e - (k - 1) + t) != sh_q[t]) return;
-      const int at = atomicAdd(&sh_M, 1);
-      const int pos = (g * s.N + jn) * s.L + e;
-      if (at < kListCap) sm.list[at] = pos;
-      my_matches[at] = pos;
-    };
+    const int own = i - g * s.N;
+    const int pos0 = g * s.N * s.L;
     if ((s.L & 3) == 0) {
-      // thread t takes the 16-byte chunks t, t + blockDim, ... of every path, sixteen paths in flight at a time
-      const int per = s.L >> 2;
+      // 16-byte chunks, chunk x = path x / per, tokens 4 * (x % per) ..; a thread keeps eight loads in flight.
+      // A position passes on to the full comparison only if the token before it fits as well: that token
+      // sits in the same chunk or in the neighbouring lane's, so the filter costs no dependent load.
+      const int per = s.L >> 2, total = s.N * per;
       const int4* g4 = reinterpret_cast<const int4*>(gtok);
-      constexpr int kBatch = 16;
-      for (int c = tid; c < per; c += blockDim.x) {
-        const int e0 = 4 * c;
-        for (int j0 = 0; j0 < s.N; j0 += kBatch) {
-          int4 w[kBatch];
-          int e_hi[kBatch];
+      const int before_last = k >= 2 ? sh_q[k - 2] : -1;
+      constexpr int kBatch = 8;
+      for (int base = 0; base < total; base += kBatch * blockDim.x) {       // same trip count for every thread
+        int4 w[kBatch];
+        int e0[kBatch], e_hi[kBatch];
 #pragma unroll
-          for (int r = 0; r < kBatch; ++r) {
-            const int jn = j0 + r;
-            e_hi[r] = (jn < s.N && g * s.N + jn != i) ? sh_len[jn] - 2 : -1;   // last position with a follower
-            if (e0 <= e_hi[r]) w[r] = ldm(g4 + (size_t)jn * per + c);
-          }
+        for (int r = 0; r < kBatch; ++r) {
+          const int x = base + r * blockDim.x + tid;
+          const int jn = x < total ? x / per : own;
+          e0[r] = 4 * x - jn * s.L;                                   // 4 * (x % per)
+          e_hi[r] = jn != own ? sh_len[jn] - 2 : -1;                  // last position with a follower
+          w[r] = make_int4(-1, -1, -1, -1);
+          if (e0[r] <= e_hi[r]) w[r] = ldm(g4 + x);
+        }
+        unsigned cand = 0;                                            // bit 4 r + u: position u of chunk r is a candidate
 #pragma unroll
-          for (int r = 0; r < kBatch; ++r) {
-            if (e0 > e_hi[r]) continue;
-            if (w[r].x == last && e0 >= k - 1) hit(j0 + r, e0);
-            if (w[r].y == last && e0 + 1 >= k - 1 && e0 + 1 <= e_hi[r]) hit(j0 + r, e0 + 1);
-            if (w[r].z == last && e0 + 2 >= k - 1 && e0 + 2 <= e_hi[r]) hit(j0 + r, e0 + 2);
-            if (w[r].w == last && e0 + 3 >= k - 1 && e0 + 3 <= e_hi[r]) hit(j0 + r, e0 + 3);
+        for (int r = 0; r < kBatch; ++r) {
+          const int left = __shfl_up_sync(FULL, w[r].w, 1);           // last token of the chunk before this one
+          const int v[5] = {left, w[r].x, w[r].y, w[r].z, w[r].w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const bool ok = v[u + 1] == last && e0[r] + u >= k - 1 && e0[r] + u <= e_hi[r] &&
+                            (k < 2 || v[u] == before_last || (u == 0 && (tid & 31) == 0));
+            cand |= (unsigned)ok << (4 * r + u);
           }
+        }
+        // one copy of the code that looks closer, run once per candidate
+        while (cand) {
+          const int bit = __ffs(cand) - 1;
+          cand &= cand - 1;
+          const int at = 4 * (base + (bit >> 2) * (int)blockDim.x + tid) + (bit & 3);   // position within the prompt
+          if (k >= 2 && (bit & 3) == 0 && (tid & 31) == 0 && ldm(gtok + at - 1) != before_last) continue;
+          if (k >= 3 && !window_head_equal(gtok + at, k, sh_q)) continue;
+          const int n = atomicAdd(&sh_M, 1);
+          if (n < kListCap) sm.list[n] = pos0 + at;
+          my_matches[n] = pos0 + at;
         }
       }
     } else {
       const int total = s.N * s.L;
       for (int x = tid; x < total; x += blockDim.x) {
         const int jn = x / s.L, e = x - jn * s.L;
-        if (g * s.N + jn == i || e < k - 1 || e > sh_len[jn] - 2) continue;
-        if (ldm(gtok + x) == last) hit(jn, e);
+        if (jn == own || e < k - 1 || e > sh_len[jn] - 2) continue;
+        if (ldm(gtok + x) != last) continue;
+        if (k >= 2 && (ldm(gtok + x - 1) != sh_q[k - 2] || !window_head_equal(gtok + x, k, sh_q))) continue;
+        const int n = atomicAdd(&sh_M, 1);
+        if (n < kListCap) sm.list[n] = pos0 + x;
+        my_matches[n] = pos0 + x;
       }
     }
   }

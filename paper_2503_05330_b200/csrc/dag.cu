@@ -709,6 +709,165 @@ __device__ void list_pool(const Dev& s, int i, int M, const int32_t* mlist, cons
   if (lane == 0) draft_len[i] = n_m;
 }
 
+// ---- all layers at once (DAG pool, no export, a few hundred matches) ------------------------------
+// dag_block takes the layers one after the other because the walk decides which node's successors
+// count; each layer then costs a few barriers and a chain of shared-memory atomics whatever M is.
+// Here every layer is aggregated at the same time into tables of its own:
+//   node table of layer d : follower token v -> sum of probabilities, count          (Eq. 5 inputs)
+//   pred table of layer d : token u of layer d - 1 -> its best successor v at layer d
+// and the walk is D table look-ups.  The pool of shared words (staging area and dag_block's tables,
+// kPoolWords in a row) holds the staged followers and as many layers' tables as fit; more layers
+// take more rounds.
+constexpr int kPoolWords = 2 * kStageWords + 8 * CAP;
+constexpr int kLayerWords = 8;                    // per table slot: pred weight (2), node key/Slo/Shi/cnt, pred key/token
+
+struct LayerTables {
+  u64* p_w; int* n_key; unsigned* n_Slo; unsigned* n_Shi; unsigned* n_cnt; int* p_key; int* p_tok;
+};
+__device__ __forceinline__ LayerTables layer_tables(int* pool, int cap, int l) {
+  int* b = pool + (size_t)l * kLayerWords * cap;
+  LayerTables t;
+  t.p_w = reinterpret_cast<u64*>(b);
+  t.n_key = b + 2 * cap; t.n_Slo = reinterpret_cast<unsigned*>(b + 3 * cap); t.n_Shi = reinterpret_cast<unsigned*>(b + 4 * cap);
+  t.n_cnt = reinterpret_cast<unsigned*>(b + 5 * cap); t.p_key = b + 6 * cap; t.p_tok = b + 7 * cap;
+  return t;
+}
+// slot of `key` in an open-addressing table of `cap` (power of two) slots; claims one if INSERT
+template <bool INSERT>
+__device__ __forceinline__ int table_slot(int* keys, int cap, int shift, int key) {
+  unsigned h = ((unsigned)key * 2654435761u) >> shift;
+  for (int probe = 0; probe < cap; ++probe) {
+    const int old = INSERT ? atomicCAS(&keys[h], -1, key) : keys[h];
+    if (old == key || (INSERT && old == -1)) return (int)h;
+    if (!INSERT && old == -1) return -1;
+    h = (h + 1) & (cap - 1);
+  }
+  return -1;
+}
+
+// How many layers' tables fit beside the staged followers (0: use dag_block).
+__device__ __forceinline__ int layers_per_round(int M, int D, int* cap_out) {
+  int cap = 64;                                    // more slots than keys: a probe always ends at a free slot
+  while (cap <= M) cap *= 2;
+  *cap_out = cap;
+  const int staged = (2 * M * D + 1) & ~1;
+  return (kPoolWords - staged) / (kLayerWords * cap);
+}
+
+__device__ __forceinline__ bool layers_in_round_ok(int M, int D) {
+  int cap;
+  return layers_per_round(M, D, &cap) >= min(D, 2);
+}
+
+__device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int32_t* mlist, const int32_t* plen,
+                           int poff, int root, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                           float* draft_edge_w) {
+  __shared__ int sh_draft[SDMS_MAX_DRAFT];
+  __shared__ u64 sh_lw[SDMS_MAX_DRAFT];            // mode 1: heaviest node of the layer
+  __shared__ int sh_lt[SDMS_MAX_DRAFT];
+  __shared__ unsigned sh_eSlo[SDMS_MAX_DRAFT], sh_eShi[SDMS_MAX_DRAFT], sh_ec[SDMS_MAX_DRAFT];
+  __shared__ int sh_cur, sh_emitted, sh_walking;
+  const int tid = threadIdx.x, D = s.D;
+  int cap;
+  const int per_round = min(D, layers_per_round(M, D, &cap));
+  const int shift = 32 - (31 - __clz(cap));
+  int* st_tok = sm.st_tok;                         // [m * D + d - 1], -1 past the end of the path
+  int* st_pq = sm.st_tok + M * D;
+  int* pool = sm.st_tok + ((2 * M * D + 1) & ~1);
+
+  for (int x = tid; x < M * D; x += blockDim.x) {
+    const int m = x / D, dd = x - m * D + 1;
+    const int gpos = mlist[m];
+    const int j = gpos / s.L;
+    const bool on = gpos - j * s.L + dd <= plen[j - poff] - 1;
+    st_tok[x] = on ? ldm(s.tok + gpos + dd) : -1;
+    st_pq[x] = on ? ldm(s.pq + gpos + dd) : 0;
+  }
+  if (tid < D) { sh_lw[tid] = 0; sh_lt[tid] = INT_MAX; sh_eSlo[tid] = 0; sh_eShi[tid] = 0; sh_ec[tid] = 0; }
+  if (tid == 0) { sh_cur = root; sh_emitted = 0; sh_walking = 1; }
+
+  for (int d0 = 1; d0 <= D; d0 += per_round) {
+    const int nl = min(per_round, D - d0 + 1);
+    // empty tables: keys -1, sums 0, best weight 0, best token "none"
+    for (int x = tid; x < nl * kLayerWords * cap; x += blockDim.x) {
+      const int w = (x / cap) % kLayerWords;
+      pool[x] = (w == 2 || w == 6) ? -1 : (w == 7 ? INT_MAX : 0);
+    }
+    __syncthreads();
+    if (!sh_walking) break;
+    // node sums
+    for (int x = tid; x < M * nl; x += blockDim.x) {
+      const int m = x / nl, l = x - m * nl, at = m * D + d0 + l - 1;
+      const int v = st_tok[at];
+      if (v < 0) continue;
+      const LayerTables t = layer_tables(pool, cap, l);
+      const int sl = table_slot<true>(t.n_key, cap, shift, v);
+      add64(&t.n_Slo[sl], &t.n_Shi[sl], (unsigned)st_pq[at]);
+      atomicAdd(&t.n_cnt[sl], 1u);
+    }
+    __syncthreads();
+    // heaviest successor of every predecessor: first the weight, then the smallest token that has it
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int x = tid; x < M * nl; x += blockDim.x) {
+        const int m = x / nl, l = x - m * nl, d = d0 + l, at = m * D + d - 1;
+        const int v = st_tok[at];
+        if (v < 0) continue;
+        const int u = d == 1 ? root : st_tok[at - 1];
+        const LayerTables t = layer_tables(pool, cap, l);
+        const int sl = table_slot<false>(t.n_key, cap, shift, v);
+        const u64 w = (u64)__double_as_longlong(eq5_weight(s.alpha, get64(t.n_Slo, t.n_Shi, sl), t.n_cnt[sl]));
+        if (pass == 0) {
+          const int ps = table_slot<true>(t.p_key, cap, shift, u);
+          atomicMax(&t.p_w[ps], w);                 // weights are >= 0: their bit patterns order like the values
+          if (s.mode == 1) atomicMax(&sh_lw[d - 1], w);
+        } else {
+          const int ps = table_slot<false>(t.p_key, cap, shift, u);
+          if (t.p_w[ps] == w) atomicMin(&t.p_tok[ps], v);
+          if (s.mode == 1 && sh_lw[d - 1] == w) atomicMin(&sh_lt[d - 1], v);
+        }
+      }
+      __syncthreads();
+    }
+    // the walk through this round's layers
+    if (tid == 0) {
+      int cur = sh_cur, emitted = sh_emitted;
+      for (int l = 0; l < nl; ++l) {
+        const int d = d0 + l;
+        const LayerTables t = layer_tables(pool, cap, l);
+        int next;
+        u64 w;
+        if (s.mode == 1) {
+          next = sh_lt[d - 1]; w = sh_lw[d - 1];
+          if (next == INT_MAX) { sh_walking = 0; break; }
+        } else {
+          const int ps = table_slot<false>(t.p_key, cap, shift, cur);
+          if (ps < 0) { sh_walking = 0; break; }
+          next = t.p_tok[ps]; w = t.p_w[ps];
+        }
+        draft_tok[(size_t)i * D + d - 1] = next;
+        if (draft_score) draft_score[(size_t)i * D + d - 1] = (float)__longlong_as_double((long long)w);
+        sh_draft[d - 1] = next;
+        cur = next; ++emitted;
+      }
+      sh_cur = cur; sh_emitted = emitted;
+    }
+    __syncthreads();
+  }
+  // weight of the edges the draft took (Eq. 5 over the candidates that contain the edge)
+  const int emitted = sh_emitted;
+  for (int x = tid; x < M * emitted; x += blockDim.x) {
+    const int m = x / emitted, d = x - m * emitted + 1, at = m * D + d - 1;
+    if (st_tok[at] != sh_draft[d - 1] || (d > 1 && st_tok[at - 1] != sh_draft[d - 2])) continue;
+    add64(&sh_eSlo[d - 1], &sh_eShi[d - 1], (unsigned)st_pq[at]);
+    atomicAdd(&sh_ec[d - 1], 1u);
+  }
+  __syncthreads();
+  if (tid < emitted && draft_edge_w)
+    draft_edge_w[(size_t)i * D + tid] =
+        sh_ec[tid] ? (float)eq5_weight(s.alpha, get64(sh_eSlo, sh_eShi, tid), sh_ec[tid]) : 0.0f;
+  if (tid == 0) draft_len[i] = emitted;
+}
+
 // Gather + DAG + search for query path i over its M (> 0) matches in mlist
 // (shared or global memory).  Called by all threads of the CTA, after a barrier
 // that follows write_defaults.
@@ -719,6 +878,8 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
   // plen[j - poff] = length of path j (the prompt's lengths in shared memory, or the global array)
   if (!EXPORT && s.pool == 2) list_pool(s, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
   else if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
+  else if (!EXPORT && s.pool == 0 && M * s.D <= kStageWords && layers_in_round_ok(M, s.D))
+    dag_layers(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
   else dag_block<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 

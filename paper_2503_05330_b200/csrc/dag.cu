@@ -722,12 +722,12 @@ constexpr int kPoolWords = 2 * kStageWords + 8 * CAP;
 constexpr int kLayerWords = 8;                    // per table slot: pred weight (2), node key/Slo/Shi/cnt, pred key/token
 
 struct LayerTables {
-  u64* p_w; int* n_key; unsigned* n_Slo; unsigned* n_Shi; unsigned* n_cnt; int* p_key; int* p_tok;
+  unsigned* p_whi; unsigned* p_wlo; int* n_key; unsigned* n_Slo; unsigned* n_Shi; unsigned* n_cnt; int* p_key; int* p_tok;
 };
 __device__ __forceinline__ LayerTables layer_tables(int* pool, int cap, int l) {
   int* b = pool + (size_t)l * kLayerWords * cap;
   LayerTables t;
-  t.p_w = reinterpret_cast<u64*>(b);
+  t.p_whi = reinterpret_cast<unsigned*>(b); t.p_wlo = reinterpret_cast<unsigned*>(b + cap);
   t.n_key = b + 2 * cap; t.n_Slo = reinterpret_cast<unsigned*>(b + 3 * cap); t.n_Shi = reinterpret_cast<unsigned*>(b + 4 * cap);
   t.n_cnt = reinterpret_cast<unsigned*>(b + 5 * cap); t.p_key = b + 6 * cap; t.p_tok = b + 7 * cap;
   return t;
@@ -736,6 +736,7 @@ __device__ __forceinline__ LayerTables layer_tables(int* pool, int cap, int l) {
 template <bool INSERT>
 __device__ __forceinline__ int table_slot(int* keys, int cap, int shift, int key) {
   unsigned h = ((unsigned)key * 2654435761u) >> shift;
+#pragma unroll 1
   for (int probe = 0; probe < cap; ++probe) {
     const int old = INSERT ? atomicCAS(&keys[h], -1, key) : keys[h];
     if (old == key || (INSERT && old == -1)) return (int)h;
@@ -743,6 +744,17 @@ __device__ __forceinline__ int table_slot(int* keys, int cap, int shift, int key
     h = (h + 1) & (cap - 1);
   }
   return -1;
+}
+// Sums of 30-bit probabilities are kept as two 32-bit sums, of the low 16 bits and of the rest: each
+// stays below 2^32 for any number of candidates a CTA handles, and an add needs no result back (no
+// carry to pass on), so the adds do not stall their thread.
+__device__ __forceinline__ void add_split(unsigned* lo16, unsigned* hi, unsigned* cnt, unsigned pq) {
+  atomicAdd(lo16, pq & 0xffffu);
+  atomicAdd(hi, pq >> 16);
+  atomicAdd(cnt, 1u);
+}
+__device__ __forceinline__ u64 weight_bits(double alpha, const unsigned* lo16, const unsigned* hi, const unsigned* cnt, int x) {
+  return (u64)__double_as_longlong(eq5_weight(alpha, ((u64)hi[x] << 16) + lo16[x], cnt[x]));
 }
 
 // How many layers' tables fit beside the staged followers (0: use dag_block).
@@ -763,67 +775,92 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
                            int poff, int root, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                            float* draft_edge_w) {
   __shared__ int sh_draft[SDMS_MAX_DRAFT];
-  __shared__ u64 sh_lw[SDMS_MAX_DRAFT];            // mode 1: heaviest node of the layer
+  __shared__ unsigned sh_lwhi[SDMS_MAX_DRAFT], sh_lwlo[SDMS_MAX_DRAFT];   // mode 1: heaviest node of the layer
   __shared__ int sh_lt[SDMS_MAX_DRAFT];
   __shared__ unsigned sh_eSlo[SDMS_MAX_DRAFT], sh_eShi[SDMS_MAX_DRAFT], sh_ec[SDMS_MAX_DRAFT];
   __shared__ int sh_cur, sh_emitted, sh_walking;
   const int tid = threadIdx.x, D = s.D;
   int cap;
   const int per_round = min(D, layers_per_round(M, D, &cap));
-  const int shift = 32 - (31 - __clz(cap));
+  const int lcap = 31 - __clz(cap), shift = 32 - lcap;
   int* st_tok = sm.st_tok;                         // [m * D + d - 1], -1 past the end of the path
   int* st_pq = sm.st_tok + M * D;
   int* pool = sm.st_tok + ((2 * M * D + 1) & ~1);
+  const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int nchunk = (M + 31) >> 5;                // a warp takes 32 matches of one layer at a time
 
-  for (int x = tid; x < M * D; x += blockDim.x) {
-    const int m = x / D, dd = x - m * D + 1;
-    const int gpos = mlist[m];
-    const int j = gpos / s.L;
-    const bool on = gpos - j * s.L + dd <= plen[j - poff] - 1;
-    st_tok[x] = on ? ldm(s.tok + gpos + dd) : -1;
-    st_pq[x] = on ? ldm(s.pq + gpos + dd) : 0;
-  }
-  if (tid < D) { sh_lw[tid] = 0; sh_lt[tid] = INT_MAX; sh_eSlo[tid] = 0; sh_eShi[tid] = 0; sh_ec[tid] = 0; }
+  if (tid < D) { sh_lwhi[tid] = 0; sh_lwlo[tid] = 0; sh_lt[tid] = INT_MAX; sh_eSlo[tid] = 0; sh_eShi[tid] = 0; sh_ec[tid] = 0; }
   if (tid == 0) { sh_cur = root; sh_emitted = 0; sh_walking = 1; }
+  // stage the followers: a thread asks for four entries before it stores the first
+  {
+    int lD = 0;
+    while ((1 << lD) < D) ++lD;                    // entries are numbered m << lD | d - 1: no division
+    constexpr int kBatch = 4;
+#pragma unroll 1
+    for (int x0 = tid; x0 < (M << lD); x0 += kBatch * blockDim.x) {
+      int tk[kBatch], pr[kBatch];
+#pragma unroll
+      for (int r = 0; r < kBatch; ++r) {
+        const int x = x0 + r * blockDim.x;
+        const int m = x >> lD, dd = (x & ((1 << lD) - 1)) + 1;
+        tk[r] = -1; pr[r] = 0;
+        if (m >= M || dd > D) continue;
+        const int gpos = mlist[m];
+        const int j = gpos / s.L;
+        if (gpos - j * s.L + dd <= plen[j - poff] - 1) { tk[r] = ldm(s.tok + gpos + dd); pr[r] = ldm(s.pq + gpos + dd); }
+      }
+#pragma unroll
+      for (int r = 0; r < kBatch; ++r) {
+        const int x = x0 + r * blockDim.x;
+        const int m = x >> lD, dd = (x & ((1 << lD) - 1)) + 1;
+        if (m < M && dd <= D) { st_tok[m * D + dd - 1] = tk[r]; st_pq[m * D + dd - 1] = pr[r]; }
+      }
+    }
+  }
 
+#pragma unroll 1
   for (int d0 = 1; d0 <= D; d0 += per_round) {
     const int nl = min(per_round, D - d0 + 1);
     // empty tables: keys -1, sums 0, best weight 0, best token "none"
-    for (int x = tid; x < nl * kLayerWords * cap; x += blockDim.x) {
-      const int w = (x / cap) % kLayerWords;
+#pragma unroll 1
+    for (int x = tid; x < ((nl * kLayerWords) << lcap); x += blockDim.x) {
+      const int w = (x >> lcap) & (kLayerWords - 1);
       pool[x] = (w == 2 || w == 6) ? -1 : (w == 7 ? INT_MAX : 0);
     }
     __syncthreads();
     if (!sh_walking) break;
-    // node sums
-    for (int x = tid; x < M * nl; x += blockDim.x) {
-      const int m = x / nl, l = x - m * nl, at = m * D + d0 + l - 1;
-      const int v = st_tok[at];
-      if (v < 0) continue;
-      const LayerTables t = layer_tables(pool, cap, l);
-      const int sl = table_slot<true>(t.n_key, cap, shift, v);
-      add64(&t.n_Slo[sl], &t.n_Shi[sl], (unsigned)st_pq[at]);
-      atomicAdd(&t.n_cnt[sl], 1u);
-    }
-    __syncthreads();
-    // heaviest successor of every predecessor: first the weight, then the smallest token that has it
-    for (int pass = 0; pass < 2; ++pass) {
-      for (int x = tid; x < M * nl; x += blockDim.x) {
-        const int m = x / nl, l = x - m * nl, d = d0 + l, at = m * D + d - 1;
-        const int v = st_tok[at];
+    // pass 0: node sums; passes 1, 2: heaviest successor weight of every predecessor, the upper half of
+    // the weight's bit pattern first, then the lower half among those (weights are >= 0, so the
+    // patterns order like the values); pass 3: the smallest token that has this weight
+#pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+#pragma unroll 1
+      for (int task = warp; task < nl * nchunk; task += nwarps) {
+        const int l = task / nchunk, m = ((task - l * nchunk) << 5) + lane;
+        const int d = d0 + l, at = m * D + d - 1;
+        const int v = m < M ? st_tok[at] : -1;
         if (v < 0) continue;
-        const int u = d == 1 ? root : st_tok[at - 1];
         const LayerTables t = layer_tables(pool, cap, l);
-        const int sl = table_slot<false>(t.n_key, cap, shift, v);
-        const u64 w = (u64)__double_as_longlong(eq5_weight(s.alpha, get64(t.n_Slo, t.n_Shi, sl), t.n_cnt[sl]));
         if (pass == 0) {
-          const int ps = table_slot<true>(t.p_key, cap, shift, u);
-          atomicMax(&t.p_w[ps], w);                 // weights are >= 0: their bit patterns order like the values
-          if (s.mode == 1) atomicMax(&sh_lw[d - 1], w);
+          const int sl = table_slot<true>(t.n_key, cap, shift, v);
+          add_split(&t.n_Slo[sl], &t.n_Shi[sl], &t.n_cnt[sl], (unsigned)st_pq[at]);
+          continue;
+        }
+        const int u = d == 1 ? root : st_tok[at - 1];
+        const u64 w = weight_bits(s.alpha, t.n_Slo, t.n_Shi, t.n_cnt, table_slot<false>(t.n_key, cap, shift, v));
+        const unsigned whi = (unsigned)(w >> 32), wlo = (unsigned)w;
+        if (pass == 1) {
+          atomicMax(&t.p_whi[table_slot<true>(t.p_key, cap, shift, u)], whi);
+          if (s.mode == 1) atomicMax(&sh_lwhi[d - 1], whi);
+          continue;
+        }
+        const int ps = table_slot<false>(t.p_key, cap, shift, u);
+        if (pass == 2) {
+          if (t.p_whi[ps] == whi) atomicMax(&t.p_wlo[ps], wlo);
+          if (s.mode == 1 && sh_lwhi[d - 1] == whi) atomicMax(&sh_lwlo[d - 1], wlo);
         } else {
-          const int ps = table_slot<false>(t.p_key, cap, shift, u);
-          if (t.p_w[ps] == w) atomicMin(&t.p_tok[ps], v);
-          if (s.mode == 1 && sh_lw[d - 1] == w) atomicMin(&sh_lt[d - 1], v);
+          if (t.p_whi[ps] == whi && t.p_wlo[ps] == wlo) atomicMin(&t.p_tok[ps], v);
+          if (s.mode == 1 && sh_lwhi[d - 1] == whi && sh_lwlo[d - 1] == wlo) atomicMin(&sh_lt[d - 1], v);
         }
       }
       __syncthreads();
@@ -831,18 +868,19 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
     // the walk through this round's layers
     if (tid == 0) {
       int cur = sh_cur, emitted = sh_emitted;
+#pragma unroll 1
       for (int l = 0; l < nl; ++l) {
         const int d = d0 + l;
         const LayerTables t = layer_tables(pool, cap, l);
         int next;
         u64 w;
         if (s.mode == 1) {
-          next = sh_lt[d - 1]; w = sh_lw[d - 1];
+          next = sh_lt[d - 1]; w = ((u64)sh_lwhi[d - 1] << 32) | sh_lwlo[d - 1];
           if (next == INT_MAX) { sh_walking = 0; break; }
         } else {
           const int ps = table_slot<false>(t.p_key, cap, shift, cur);
           if (ps < 0) { sh_walking = 0; break; }
-          next = t.p_tok[ps]; w = t.p_w[ps];
+          next = t.p_tok[ps]; w = ((u64)t.p_whi[ps] << 32) | t.p_wlo[ps];
         }
         draft_tok[(size_t)i * D + d - 1] = next;
         if (draft_score) draft_score[(size_t)i * D + d - 1] = (float)__longlong_as_double((long long)w);
@@ -855,16 +893,17 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
   }
   // weight of the edges the draft took (Eq. 5 over the candidates that contain the edge)
   const int emitted = sh_emitted;
-  for (int x = tid; x < M * emitted; x += blockDim.x) {
-    const int m = x / emitted, d = x - m * emitted + 1, at = m * D + d - 1;
-    if (st_tok[at] != sh_draft[d - 1] || (d > 1 && st_tok[at - 1] != sh_draft[d - 2])) continue;
-    add64(&sh_eSlo[d - 1], &sh_eShi[d - 1], (unsigned)st_pq[at]);
-    atomicAdd(&sh_ec[d - 1], 1u);
+#pragma unroll 1
+  for (int task = warp; task < emitted * nchunk; task += nwarps) {
+    const int l = task / nchunk, m = ((task - l * nchunk) << 5) + lane;
+    const int d = l + 1, at = m * D + d - 1;
+    if (m < M && st_tok[at] == sh_draft[d - 1] && (d == 1 || st_tok[at - 1] == sh_draft[d - 2]))
+      add_split(&sh_eSlo[d - 1], &sh_eShi[d - 1], &sh_ec[d - 1], (unsigned)st_pq[at]);
   }
   __syncthreads();
   if (tid < emitted && draft_edge_w)
     draft_edge_w[(size_t)i * D + tid] =
-        sh_ec[tid] ? (float)eq5_weight(s.alpha, get64(sh_eSlo, sh_eShi, tid), sh_ec[tid]) : 0.0f;
+        sh_ec[tid] ? (float)__longlong_as_double((long long)weight_bits(s.alpha, sh_eSlo, sh_eShi, sh_ec, tid)) : 0.0f;
   if (tid == 0) draft_len[i] = emitted;
 }
 

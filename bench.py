@@ -28,9 +28,9 @@ METRIC = "draft-construction paths*steps/sec at N=16 (and us/step)"
 UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
-# profiles/build_fused_accept_cfg2_ncu_full.md; only quoted while the kernel sources are the ones profiled
-NCU_TRAFFIC = {"kernel": "build_fused", "bytes_per_launch": 102741,
-               "sources_sha256": "7507411f5813335b0920e3b241af443b06b848142bf8055f2bc6af493b3ca362"}
+# profiles/step_kernel_cfg2_ncu_full.md; only quoted while the kernel sources are the ones profiled
+NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76096,
+               "sources_sha256": "2c8252296152901e045367f6a12463d549ce639c1626fa70ef97c0a85ee8d5b8"}
 
 
 def kernel_sources_sha():

@@ -32,6 +32,8 @@
 //     operation rounded separately (build with -ffp-contract=off);
 //   * the walk only moves to successors of the node it stands on (mode 0);
 //     mode 1 takes the best node of each layer regardless of the previous one;
+//     mode 2 replaces the greedy walk by the path of the DAG with the largest sum of
+//     node weights (not in the paper's method; its introduction motivates it);
 //   * ties go to the smallest token id.
 //
 // Pins (tests/, CPU only): hand-worked example from Eq. 3 / Eq. 5 with dyadic
@@ -231,6 +233,44 @@ void build_path(Ctx* c, int k, int i) {
     for (int d = 1; d <= n_m; ++d) {
       double w = weight(c->alpha, c->pq[j][e + d], 1);
       r.draft.push_back(c->tok[j][e + d]); r.score.push_back(w); r.edge_w.push_back(w);
+    }
+    return;
+  }
+  if (c->mode == 2) {
+    // Best path instead of the greedy walk (the introduction asks for the highest-likelihood
+    // sequence of the pool; the greedy rule of "Consensus-Driven Draft Extraction" only looks one
+    // layer ahead).  Value of a path = sum of its nodes' in-weights (the greedy rule's own score),
+    // added from the path's end towards its start:  best(d, v) = w(d, v) + max over successors v'
+    // of best(d+1, v'), and 0 for the max of nothing.  Weights are >= 0, so a path is never cut
+    // short of a leaf.  The walk takes, among the successors of the node it stands on, the one with
+    // the highest best(); ties go to the smaller token.
+    const bool virtual_root = c->eps > 0;
+    std::vector<std::map<int, double>> best(c->D);
+    for (int d = c->D; d >= 1; --d) {
+      for (const auto& kv : r.nodes[d - 1]) {
+        double succ = 0.0;
+        if (d < c->D)
+          for (const auto& e : r.edges[d])          // edges between layer d and layer d + 1
+            if (e.first.first == kv.first) succ = std::max(succ, best[d].at(e.first.second));
+        best[d - 1][kv.first] = weight(c->alpha, kv.second.S, kv.second.cnt) + succ;
+      }
+    }
+    int cur = r.root;
+    for (int d = 1; d <= c->D; ++d) {
+      bool found = false; int best_v = -1; double best_b = 0.0;
+      for (const auto& kv : r.nodes[d - 1]) {       // ascending token id
+        const bool succ = (d == 1 && virtual_root) || r.edges[d - 1].count({cur, kv.first});
+        if (!succ) continue;
+        const double b = best[d - 1].at(kv.first);
+        if (!found || b > best_b) { found = true; best_v = kv.first; best_b = b; }
+      }
+      if (!found) break;
+      const Acc& nd = r.nodes[d - 1].at(best_v);
+      r.draft.push_back(best_v);
+      r.score.push_back(weight(c->alpha, nd.S, nd.cnt));
+      if (d == 1 && virtual_root) r.edge_w.push_back(r.score.back());
+      else { const Acc& ed = r.edges[d - 1].at({cur, best_v}); r.edge_w.push_back(weight(c->alpha, ed.S, ed.cnt)); }
+      cur = best_v;
     }
     return;
   }

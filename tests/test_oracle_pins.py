@@ -652,3 +652,115 @@ def test_pools_agree_when_there_is_one_candidate_and_differ_on_reconvergence():
     assert drafts[0] == ([2, 7, 6], [1.0, 1.5, 0.75])     # DAG: node (3, 6) = 0.5 + 0.25
     assert drafts[1] == ([2, 7, 5], [1.0, 1.0, 0.5])      # tree: children of "2 7" are 5 (0.5) and 6 (0.25)
     assert drafts[2] == ([2, 7, 5], [0.5, 0.5, 0.5])      # list: the first candidate sums to 1.5
+
+
+# ----------------------------------------------------------------------------
+# best-path search (search mode 2): brute force over every path of the DAG
+# ----------------------------------------------------------------------------
+def py_weight(alpha, S, cnt):
+    return alpha * float(S) * (1.0 / Q30) + (1.0 - alpha) * float(cnt)
+
+
+def brute_force_best_path(paths, layers, alpha, D):
+    """Among the paths that end at a leaf or at depth D: the largest sum of node weights, added from
+    the last node towards the first; ties go to the lexicographically smallest token sequence."""
+    maximal = [p for p in paths if p and (len(p) == D or not any(len(q) == len(p) + 1 and q[:len(p)] == p for q in paths))]
+    best, best_total = None, None
+    for p in sorted(maximal):
+        total = 0.0
+        for d in range(len(p) - 1, -1, -1):
+            total = py_weight(alpha, *layers[d][0][p[d]]) + total
+        if best is None or total > best_total:
+            best, best_total = p, total
+    return best, best_total
+
+
+def test_best_path_differs_from_greedy_on_a_hand_worked_pool():
+    # query path ends in 9.  Candidates: 9 -> 1 (.5) -> 3 (.125)   and   9 -> 2 (.25) -> 4 (.75).
+    # Greedy takes 1 (.5 > .25) and is stuck with 3: total .625.  The best path is 2, 4: total 1.0.
+    paths = [[5, 9], [9, 1, 3, 7], [9, 2, 4, 7]]
+    probs = [[.5, .5], [.5, .5, .125, .5], [.5, .25, .75, .5]]
+    for mode, expect, scores in ((0, [1, 3], [.5, .125]), (2, [2, 4], [.25, .75])):
+        o = Oracle(1, 3, 8, 10, 2, alpha=1.0, mode=mode)
+        assert load_paths(o, paths, probs=probs) == 0
+        o.build_all(1)
+        draft, score, edge_w = o.draft(0)
+        assert list(draft) == expect
+        assert list(score) == scores and list(edge_w) == scores
+
+
+def test_best_path_tie_goes_to_the_smaller_token_and_extends_to_a_leaf():
+    # two paths of equal total (.5 + .25 = .25 + .5): the one that starts with the smaller token wins;
+    # a zero-weight tail is still followed to the leaf
+    paths = [[5, 9], [9, 2, 4, 6], [9, 1, 3, 8]]
+    probs = [[.5, .5], [.5, .5, .25, 0.0], [.5, .25, .5, 0.0]]
+    o = Oracle(1, 3, 8, 10, 3, alpha=1.0, mode=2)
+    assert load_paths(o, paths, probs=probs) == 0
+    o.build_all(1)
+    draft, score, _ = o.draft(0)
+    assert list(draft) == [1, 3, 8] and list(score) == [.25, .5, 0.0]
+
+
+@pytest.mark.parametrize("seed,alpha,k", list(itertools.product(range(6), (1.0, 0.5, 0.0), (1, 2))))
+def test_best_path_equals_brute_force_over_all_dag_paths(seed, alpha, k):
+    G, N, L, V, D = 1, 5, 28, 3, 4
+    tokens, lps = synth.small_random(N, L, V, 7300 + seed)
+    rng = synth.Stream(7400 + seed)
+    lens = (5 + rng.uniform(N) * (L - 6)).astype(np.int32)
+    o = Oracle(G, N, L, V, D, alpha=alpha, mode=2)
+    g = Oracle(G, N, L, V, D, alpha=alpha, mode=0)
+    o.append(tokens, lps, lens)
+    g.append(tokens, lps, lens)
+    o.build_all(k)
+    g.build_all(k)
+    for i in range(N):
+        root = int(tokens[i, lens[i] - 1])
+        paths, layers = all_dag_paths(o, i, root, D)
+        draft, score, edge_w = o.draft(i)
+        draft = tuple(int(x) for x in draft)
+        if len(paths) == 1:
+            assert draft == ()
+            continue
+        want, total = brute_force_best_path(paths, layers, alpha, D)
+        assert draft == want
+        for d, v in enumerate(draft):
+            assert score[d] == py_weight(alpha, *layers[d][0][v])
+            u = root if d == 0 else draft[d - 1]
+            assert edge_w[d] == py_weight(alpha, *layers[d][1][(u, v)])
+        # never worse than the greedy walk over the same DAG
+        gd, gs, _ = g.draft(i)
+        gtot = 0.0
+        for x in reversed([float(x) for x in gs]):
+            gtot = x + gtot
+        assert total >= gtot
+
+
+def test_best_path_and_greedy_agree_on_a_chain_and_at_depth_one():
+    tokens, lps = synth.small_random(4, 24, 3, 7777)
+    lens = np.array([20, 18, 22, 19], np.int32)
+    for D in (1,):
+        a, b = Oracle(1, 4, 24, 3, D, alpha=0.5, mode=0), Oracle(1, 4, 24, 3, D, alpha=0.5, mode=2)
+        a.append(tokens, lps, lens); b.append(tokens, lps, lens)
+        a.build_all(1); b.build_all(1)
+        for i in range(4):
+            assert list(a.draft(i)[0]) == list(b.draft(i)[0])
+    # one candidate only: the pool is a chain
+    paths = [[5, 9], [9, 2, 4, 6, 1]]
+    probs = [[.5, .5], [.5, .5, .25, .125, .5]]
+    for mode in (0, 2):
+        o = Oracle(1, 2, 8, 10, 4, alpha=1.0, mode=mode)
+        assert load_paths(o, paths, probs=probs) == 0
+        o.build_all(1)
+        assert list(o.draft(0)[0]) == [2, 4, 6, 1]
+
+
+def test_best_path_really_departs_from_greedy_on_random_pools():
+    differ = 0
+    for seed in range(6):
+        tokens, lps = synth.small_random(5, 28, 3, 7300 + seed)
+        lens = np.full(5, 26, np.int32)
+        a, b = Oracle(1, 5, 28, 3, 4, alpha=1.0, mode=0), Oracle(1, 5, 28, 3, 4, alpha=1.0, mode=2)
+        a.append(tokens, lps, lens); b.append(tokens, lps, lens)
+        a.build_all(1); b.build_all(1)
+        differ += sum(list(a.draft(i)[0]) != list(b.draft(i)[0]) for i in range(5))
+    assert differ > 0

@@ -50,6 +50,8 @@ extern "C" {
 #define SDMS_STATUS_BAD_LOGPROB    0x08u /* NaN logprob: stored as probability 0                  */
 #define SDMS_STATUS_INDEX_FULL     0x10u /* n-gram table had no free bucket (cannot happen with the sized workspace) */
 #define SDMS_STATUS_MATCH_OVERFLOW 0x20u /* match workspace exhausted: the affected paths get draft_len 0 */
+#define SDMS_STATUS_SEARCH_FALLBACK 0x40u /* search_mode 2: a path had too many matches for the best-path tables
+                                            (more than about 24576 / (11 * max_draft_len)); it got the greedy draft */
 
 #define SDMS_MAX_K      16   /* largest supported k_max           */
 #define SDMS_MAX_DRAFT  32   /* largest supported max_draft_len   */
@@ -72,7 +74,14 @@ typedef struct {
   int32_t  dag_nodes_per_layer;  /* B: nodes kept per layer by sdms_get_dag, 0 = no export     */
   int32_t  dag_edges_per_node;   /* Ke: out-edges kept per exported node                      */
   int32_t  search_mode;          /* 0: walk to the best successor of the current node;
-                                    1: best node of each layer regardless of the previous one */
+                                    1: best node of each layer regardless of the previous one;
+                                    2: not the paper's greedy walk but the path of the DAG with the
+                                       largest sum of node weights (its introduction asks for the
+                                       highest-likelihood sequence): best(d,v) = w(d,v) + max over
+                                       successors of best(d+1,.), summed from the path's end; the
+                                       walk follows the largest best(), ties to the smaller token.
+                                       DAG pool only.  Paths with more matches than the tables hold
+                                       get the mode-0 draft and raise SDMS_STATUS_SEARCH_FALLBACK */
   float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
   int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
   int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)

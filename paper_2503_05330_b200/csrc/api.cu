@@ -30,12 +30,13 @@ int check_config(const sdms_config* c) {
   if (c->dag_nodes_per_layer < 0 || c->dag_nodes_per_layer > SDMS_MAX_DAG_NODES) return SDMS_ERR_INVALID_ARG;
   if (c->dag_nodes_per_layer > 0 && (c->dag_edges_per_node < 1 || c->dag_edges_per_node > SDMS_MAX_DAG_EDGES))
     return SDMS_ERR_INVALID_ARG;
-  if (c->search_mode != 0 && c->search_mode != 1) return SDMS_ERR_INVALID_ARG;
+  if (c->search_mode < 0 || c->search_mode > 2) return SDMS_ERR_INVALID_ARG;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f)) return SDMS_ERR_INVALID_ARG;
   if (c->match_capacity < 0 || c->match_capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;
   const int64_t P = (int64_t)c->num_groups * c->paths_per_group;
   if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
   if (c->epsilon < 0 || c->epsilon > 1 || c->pool_mode < 0 || c->pool_mode > 2) return SDMS_ERR_INVALID_ARG;
+  if (c->search_mode == 2 && c->pool_mode != 0) return SDMS_ERR_INVALID_ARG;     // the best path is a path of the DAG
   return SDMS_OK;
 }
 

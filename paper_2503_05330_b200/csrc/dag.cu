@@ -433,7 +433,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
     const int cur = sh_cur;
     const int nkept = EXPORT ? sh_nkept : 0;
     const bool tree = !EXPORT && s.pool == 1;       // only candidates that spell the draft so far take part
-    const bool restricted = !EXPORT && !staged && !tree && s.mode == 0 && d > 1;   // staged candidates are cheap to revisit
+    const bool restricted = !EXPORT && !staged && !tree && s.mode != 1 && d > 1;   // staged candidates are cheap to revisit
     if (!EXPORT) {
       // first layer (or every layer in mode 1): every distinct follower is a node, guess one per four
       // candidates; restricted layers only hold the successors of one node
@@ -907,6 +907,147 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
   if (tid == 0) draft_len[i] = emitted;
 }
 
+// ---- best path instead of the greedy walk (search mode 2) ------------------------------------------
+// best(d, v) = w(d, v) + max over the successors v' of v of best(d + 1, v')  (0 for no successor), w the
+// node's Eq. 5 in-weight; the draft follows, from the root, the successor with the largest best(), ties
+// to the smaller token.  All D layers' node tables stay in shared memory at once; the layers are
+// taken from the last to the first for best(), then every node's choice of successor is made for
+// all layers together, and the walk is D look-ups.
+constexpr int kPathWords = 9;     // per slot: best (2), largest successor best (2), key, sum lo16 / hi, count, chosen successor
+
+struct PathTables {
+  u64* best; u64* succ; int* key; unsigned* Slo; unsigned* Shi; unsigned* cnt; int* next;
+};
+__device__ __forceinline__ PathTables path_tables(int* pool, int cap, int l) {
+  int* b = pool + (size_t)l * kPathWords * cap;
+  PathTables t;
+  t.best = reinterpret_cast<u64*>(b); t.succ = reinterpret_cast<u64*>(b + 2 * cap);
+  t.key = b + 4 * cap; t.Slo = reinterpret_cast<unsigned*>(b + 5 * cap); t.Shi = reinterpret_cast<unsigned*>(b + 6 * cap);
+  t.cnt = reinterpret_cast<unsigned*>(b + 7 * cap); t.next = b + 8 * cap;
+  return t;
+}
+// Do the tables of all D layers fit beside the staged followers?
+__device__ __forceinline__ bool best_path_fits(int M, int D, int* cap_out) {
+  int cap = 64;
+  while (cap <= M) cap *= 2;
+  *cap_out = cap;
+  return (long long)((2 * M * D + 1) & ~1) + (long long)D * kPathWords * cap <= kPoolWords;
+}
+
+__device__ void dag_best_path(const Dev& s, const Smem& sm, int i, int M, int cap, const int32_t* mlist,
+                              const int32_t* plen, int poff, int32_t* draft_tok, int32_t* draft_len,
+                              float* draft_score, float* draft_edge_w) {
+  __shared__ int sh_draft[SDMS_MAX_DRAFT];
+  __shared__ unsigned sh_eSlo[SDMS_MAX_DRAFT], sh_eShi[SDMS_MAX_DRAFT], sh_ec[SDMS_MAX_DRAFT];
+  __shared__ u64 sh_root_succ;
+  __shared__ int sh_root_next, sh_emitted;
+  const int tid = threadIdx.x, D = s.D;
+  const int lcap = 31 - __clz(cap), shift = 32 - lcap;
+  int* st_tok = sm.st_tok;                         // [m * D + d - 1], -1 past the end of the path
+  int* st_pq = sm.st_tok + M * D;
+  int* pool = sm.st_tok + ((2 * M * D + 1) & ~1);
+  int lD = 0;
+  while ((1 << lD) < D) ++lD;                      // items are numbered m << lD | d - 1
+
+  for (int x = tid; x < (M << lD); x += blockDim.x) {
+    const int m = x >> lD, dd = (x & ((1 << lD) - 1)) + 1;
+    if (dd > D) continue;
+    const int gpos = mlist[m];
+    const int j = gpos / s.L;
+    const bool on = gpos - j * s.L + dd <= plen[j - poff] - 1;
+    st_tok[m * D + dd - 1] = on ? ldm(s.tok + gpos + dd) : -1;
+    st_pq[m * D + dd - 1] = on ? ldm(s.pq + gpos + dd) : 0;
+  }
+  for (int x = tid; x < D * kPathWords * cap; x += blockDim.x) {
+    const int w = (x >> lcap) % kPathWords;
+    pool[x] = w == 4 ? -1 : (w == 8 ? INT_MAX : 0);
+  }
+  if (tid < D) { sh_eSlo[tid] = 0; sh_eShi[tid] = 0; sh_ec[tid] = 0; }
+  if (tid == 0) { sh_root_succ = 0; sh_root_next = INT_MAX; sh_emitted = 0; }
+  __syncthreads();
+  // node sums of every layer
+  for (int x = tid; x < (M << lD); x += blockDim.x) {
+    const int m = x >> lD, l = x & ((1 << lD) - 1);
+    if (l >= D) continue;
+    const int v = st_tok[m * D + l];
+    if (v < 0) continue;
+    const PathTables t = path_tables(pool, cap, l);
+    const int sl = table_slot<true>(t.key, cap, shift, v);
+    add_split(&t.Slo[sl], &t.Shi[sl], &t.cnt[sl], (unsigned)st_pq[m * D + l]);
+  }
+  __syncthreads();
+  // best(), last layer first: a candidate hands the best() of its next node to its node of this layer
+  for (int d = D; d >= 1; --d) {
+    const PathTables t = path_tables(pool, cap, d - 1);
+    if (d < D) {
+      const PathTables tn = path_tables(pool, cap, d);
+      for (int m = tid; m < M; m += blockDim.x) {
+        const int v = st_tok[m * D + d - 1], vn = st_tok[m * D + d];
+        if (v < 0 || vn < 0) continue;
+        atomicMax(&t.succ[table_slot<false>(t.key, cap, shift, v)], tn.best[table_slot<false>(tn.key, cap, shift, vn)]);
+      }
+      __syncthreads();
+    }
+    for (int x = tid; x < cap; x += blockDim.x)     // sums are only added to once per key: every slot on its own
+      if (t.key[x] >= 0) {
+        const double w = eq5_weight(s.alpha, ((u64)t.Shi[x] << 16) + t.Slo[x], t.cnt[x]);
+        t.best[x] = (u64)__double_as_longlong(__dadd_rn(w, __longlong_as_double((long long)t.succ[x])));
+      }
+    __syncthreads();
+  }
+  // the root's best successor value (every first-layer node follows the root), then every node's
+  // choice: the smallest successor token whose best() is the largest
+  {
+    const PathTables t = path_tables(pool, cap, 0);
+    for (int x = tid; x < cap; x += blockDim.x)
+      if (t.key[x] >= 0) atomicMax(&sh_root_succ, t.best[x]);
+  }
+  __syncthreads();
+  for (int x = tid; x < (M << lD); x += blockDim.x) {
+    const int m = x >> lD, l = x & ((1 << lD) - 1);
+    if (l >= D) continue;
+    const int v = st_tok[m * D + l];
+    if (v < 0) continue;
+    const PathTables t = path_tables(pool, cap, l);
+    const u64 b = t.best[table_slot<false>(t.key, cap, shift, v)];
+    if (l == 0) {
+      if (b == sh_root_succ) atomicMin(&sh_root_next, v);
+    } else {
+      const PathTables tp = path_tables(pool, cap, l - 1);
+      const int ps = table_slot<false>(tp.key, cap, shift, st_tok[m * D + l - 1]);
+      if (b == tp.succ[ps]) atomicMin(&tp.next[ps], v);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int next = sh_root_next, emitted = 0;
+    for (int d = 1; d <= D && next != INT_MAX; ++d) {
+      const PathTables t = path_tables(pool, cap, d - 1);
+      const int sl = table_slot<false>(t.key, cap, shift, next);
+      draft_tok[(size_t)i * D + d - 1] = next;
+      if (draft_score)
+        draft_score[(size_t)i * D + d - 1] = (float)eq5_weight(s.alpha, ((u64)t.Shi[sl] << 16) + t.Slo[sl], t.cnt[sl]);
+      sh_draft[d - 1] = next;
+      ++emitted;
+      next = t.next[sl];
+    }
+    sh_emitted = emitted;
+  }
+  __syncthreads();
+  // weight of the edges the draft took (Eq. 5 over the candidates that contain the edge)
+  const int emitted = sh_emitted;
+  for (int x = tid; x < (M << lD); x += blockDim.x) {
+    const int m = x >> lD, d = (x & ((1 << lD) - 1)) + 1, at = m * D + d - 1;
+    if (d > emitted || st_tok[at] != sh_draft[d - 1] || (d > 1 && st_tok[at - 1] != sh_draft[d - 2])) continue;
+    add_split(&sh_eSlo[d - 1], &sh_eShi[d - 1], &sh_ec[d - 1], (unsigned)st_pq[at]);
+  }
+  __syncthreads();
+  if (tid < emitted && draft_edge_w)
+    draft_edge_w[(size_t)i * D + tid] =
+        (float)eq5_weight(s.alpha, ((u64)sh_eShi[tid] << 16) + sh_eSlo[tid], sh_ec[tid]);
+  if (tid == 0) draft_len[i] = emitted;
+}
+
 // Gather + DAG + search for query path i over its M (> 0) matches in mlist
 // (shared or global memory).  Called by all threads of the CTA, after a barrier
 // that follows write_defaults.
@@ -915,6 +1056,15 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
                                           const int32_t* plen, int poff, int root, int32_t* draft_tok,
                                           int32_t* draft_len, float* draft_score, float* draft_edge_w) {
   // plen[j - poff] = length of path j (the prompt's lengths in shared memory, or the global array)
+  if (!EXPORT && s.mode == 2) {
+    int cap;
+    if (best_path_fits(M, s.D, &cap)) {
+      dag_best_path(s, sm, i, M, cap, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
+      return;
+    }
+    // too many matches for the tables of all layers: this path gets the greedy walk, and says so
+    if (threadIdx.x == 0) atomicOr(s.status, SDMS_STATUS_SEARCH_FALLBACK);
+  }
   if (!EXPORT && s.pool == 2) list_pool(s, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
   else if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);
   else if (!EXPORT && s.pool == 0 && M * s.D <= kStageWords && layers_in_round_ok(M, s.D))

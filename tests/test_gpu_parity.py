@@ -399,3 +399,75 @@ def test_step_falls_back_to_separate_launches_for_wide_prompts():
     assert not pair.g.step_is_single_launch()
     st = harness.run_step_protocol(pair, tokens, lps, [2, 1, 3], steps=20, warm=4)
     assert st["steps"] > 5
+
+
+# ---- best-path search (search mode 2) --------------------------------------------------------
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("alpha,eps", [(1.0, 0), (0.5, 0), (0.0, 0), (1.0, 1)])
+def test_best_path_dense_small_vocab_every_step(seed, alpha, eps):
+    G, N, L, V, D, k_max = 2, 5, 56, 4 + seed, 6, 3
+    tokens, lps = synth.small_random(G * N, L, V, 6100 + seed)
+    for k in (1, 2):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=2, eps=eps)
+        start = 4 + (np.arange(G * N) * 5 + seed) % 9
+        st = run_protocol(pair, tokens, lps, k, steps=30, warm=0, start_lens=start, commit_in_accept=bool(seed % 2))
+        assert st["steps"] > 5
+
+
+def test_best_path_through_the_single_launch_step():
+    G, N, L, V, D, k_max = 2, 6, 64, 6, 6, 3
+    tokens, lps = synth.small_random(G * N, L, V, 6200)
+    pair = Pair(G, N, L, V, k_max, D, alpha=1.0, mode=2)
+    st = harness.run_step_protocol(pair, tokens, lps, [2, 1, 3], steps=40, warm=4)
+    assert st["steps"] > 5
+
+
+def best_path_fits(M, D):
+    cap = 64
+    while cap <= M:
+        cap *= 2
+    return ((2 * M * D + 1) & ~1) + D * 9 * cap <= 2 * 8192 + 8 * 1024
+
+
+def test_best_path_config2_and_the_fallback_for_heavy_queries():
+    # k = 1 queries on frequent tokens find more matches than the best-path tables of a CTA hold:
+    # those paths get the greedy draft and the status word says so; every other path the best path
+    from oracle import Oracle
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D)
+    greedy = Oracle(w.G, w.N, w.L, w.V, w.D, alpha=1.0, mode=0)
+    n = 1000
+    lens = (n - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    pair.append(tokens[:, :n], lps[:, :n], lens, expect_status=0)
+    greedy.append(tokens[:, :n], lps[:, :n], lens)
+    fell_back = 0
+    for k in (1, 2, 3, 4, 1):
+        pair.o.build_all(k, nthreads=8)
+        greedy.build_all(k, nthreads=8)
+        pair.g.build_drafts(k)
+        status = pair.g.status()
+        gt, gl = pair.g.draft_tok.cpu().numpy(), pair.g.draft_len.cpu().numpy()
+        gs = pair.g.draft_score.cpu().numpy()
+        heavy = 0
+        for i in range(w.P):
+            M = len(pair.o.matches(i))
+            src = pair.o if best_path_fits(M, w.D) else greedy
+            heavy += not best_path_fits(M, w.D)
+            d, sc, _ = src.draft(i)
+            assert gl[i] == len(d) and np.array_equal(gt[i, :len(d)], d), (k, i, M)
+            np.testing.assert_allclose(gs[i, :len(d)], sc, rtol=harness.RTOL, atol=0)
+        assert status == (0x40 if heavy else 0), (k, heavy, status)
+        fell_back += heavy
+        lens = pair.o.lengths()
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
+        tok, ln, _, _ = pair.o.drafts()
+        pair.o.accept_commit(tok, ln, sampled, sampled_lp, w.D)
+        greedy.accept_commit(tok, ln, sampled, sampled_lp, w.D)
+        # the library commits its own drafts, which differ from the oracle's on the fallback paths:
+        # feed it the oracle's instead so that both histories stay the same
+        pair.g.draft_tok.copy_(torch.from_numpy(tok)); pair.g.draft_len.copy_(torch.from_numpy(ln))
+        pair.g.accept(harness.t32(sampled, pair.dev), harness.t32(sampled_lp, pair.dev))
+        assert pair.g.status() == 0
+    pair.check_history()
+    assert fell_back > 0

@@ -43,7 +43,7 @@ def lib():
         l.orc_prob_to_fixed.argtypes = [C.c_float]
         l.orc_weight.restype = C.c_double
         l.orc_weight.argtypes = [C.c_float, C.c_int64, C.c_int64]
-        for name in ("orc_append", "orc_append_fixed", "orc_accept_commit"):
+        for name in ("orc_append", "orc_append_fixed", "orc_accept_commit", "orc_trim"):
             getattr(l, name).restype = C.c_uint32
         l.orc_num_matches.restype = C.c_int
         l.orc_edit_distance.restype = C.c_int
@@ -98,6 +98,11 @@ class Oracle:
         counts = np.ascontiguousarray(counts, dtype=np.int32)
         return int(self._l.orc_append_fixed(self._h, _ptr(tokens, C.c_int32), _ptr(pq, C.c_int32),
                                             _ptr(counts, C.c_int32), C.c_int(tokens.shape[1])))
+
+    def trim(self, keep) -> int:
+        keep = np.ascontiguousarray(keep, dtype=np.int32)
+        assert keep.shape == (self.P,)
+        return int(self._l.orc_trim(self._h, _ptr(keep, C.c_int32)))
 
     def lengths(self) -> np.ndarray:
         out = np.zeros(self.P, dtype=np.int32)

@@ -19,6 +19,8 @@
 //                in-edge weight is highest; stop at length D or at a leaf.
 //   accept     - "Draft acceptance": longest prefix of the draft equal to the
 //                sampled tokens.
+//   trim       - a sliding window for runs longer than the capacity: a path forgets
+//                its oldest tokens (the paper's runs are short; not part of its method).
 //   tree, list - the two weaker draft pools of the "Ablation Study": a tree merges
 //                candidates only along identical prefixes, a list does not merge.
 //
@@ -337,6 +339,23 @@ uint32_t orc_append(void* h, const int32_t* tokens, const float* logprobs, const
 // (used by the hand-worked examples, whose probabilities are dyadic).
 uint32_t orc_append_fixed(void* h, const int32_t* tokens, const int32_t* pq, const int32_t* counts, int a_max) {
   return append_impl((Ctx*)h, tokens, nullptr, pq, counts, a_max);
+}
+
+// Sliding window over the histories (not in the paper, whose runs end before any limit): path p
+// forgets all but its newest keep[p] tokens; keep[p] >= its length changes nothing, keep[p] < 0 is
+// reported as a bad count and changes nothing.  What a later build sees is exactly the shorter
+// history, as if only those tokens had ever been appended.
+uint32_t orc_trim(void* h, const int32_t* keep) {
+  Ctx* c = (Ctx*)h;
+  uint32_t st = 0;
+  for (size_t p = 0; p < c->tok.size(); ++p) {
+    if (keep[p] < 0) { st |= ST_BAD_COUNT; continue; }
+    const size_t len = c->tok[p].size();
+    if ((size_t)keep[p] >= len) continue;
+    c->tok[p].erase(c->tok[p].begin(), c->tok[p].begin() + (len - keep[p]));
+    c->pq[p].erase(c->pq[p].begin(), c->pq[p].begin() + (len - keep[p]));
+  }
+  return st;
 }
 
 void orc_get_lengths(void* h, int32_t* out) {

@@ -764,3 +764,47 @@ def test_best_path_really_departs_from_greedy_on_random_pools():
         a.build_all(2); b.build_all(2)
         differ += sum(list(a.draft(i)[0]) != list(b.draft(i)[0]) for i in range(6))
     assert differ >= 10
+
+
+# ----------------------------------------------------------------------------
+# sliding window: trimmed histories
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(4))
+def test_trim_keeps_the_newest_tokens_and_matches_follow_the_shorter_history(seed):
+    G, N, L, V = 2, 4, 32, 3
+    tokens, lps = synth.small_random(G * N, L, V, 8100 + seed)
+    rng = synth.Stream(8200 + seed)
+    lens = (8 + rng.uniform(G * N) * (L - 9)).astype(np.int32)
+    keep = (2 + rng.uniform(G * N) * 30).astype(np.int32)           # some above the length: no change
+    o = Oracle(G, N, L, V, 4)
+    o.append(tokens, lps, lens)
+    before = [o.history(p) for p in range(G * N)]
+    assert o.trim(keep) == 0
+    new_lens = np.minimum(lens, keep)
+    assert o.lengths().tolist() == new_lens.tolist()
+    shifted = np.zeros_like(tokens)
+    for p in range(G * N):
+        t, q = o.history(p)
+        assert t.tolist() == before[p][0][lens[p] - new_lens[p]:].tolist()
+        assert q.tolist() == before[p][1][lens[p] - new_lens[p]:].tolist()
+        shifted[p, :new_lens[p]] = tokens[p, lens[p] - new_lens[p]:lens[p]]
+    # Eq. 3 on the shorter histories, by the independent regex search
+    for k in (1, 2):
+        o.build_all(k)
+        for i in range(G * N):
+            if new_lens[i] >= k:
+                assert o.matches(i).tolist() == regex_matches(shifted, new_lens, N, L, i, k), (seed, k, i)
+    # a trimmed path has room again and appends where its window ends
+    room = (L - new_lens).astype(np.int32)
+    more = np.minimum(room, 3).astype(np.int32)
+    assert o.append(tokens[:, :3], lps[:, :3], more) == 0
+    assert o.lengths().tolist() == (new_lens + more).tolist()
+
+
+def test_trim_rejects_negative_counts_and_keeps_the_path():
+    o = Oracle(1, 2, 8, 5, 2)
+    load_paths(o, [[1, 2, 3], [4, 0, 1, 2]], probs=[[.5] * 3, [.5] * 4])
+    assert o.trim(np.array([-1, 2], np.int32)) == 0x01
+    assert o.history(0)[0].tolist() == [1, 2, 3] and o.history(1)[0].tolist() == [1, 2]
+    assert o.trim(np.array([0, 9], np.int32)) == 0
+    assert o.lengths().tolist() == [0, 2]

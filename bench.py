@@ -161,12 +161,13 @@ class ClockSampler(threading.Thread):
 class Runner:
     """Device-resident replay of the decode protocol of one workload."""
 
-    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0):
+    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0, mode=0):
         import torch
         from paper_2503_05330_b200 import binding
         self.torch, self.binding, self.w, self.device = torch, binding, w, device
         self.tokens, self.logprobs = synth.make_streams(w, seed)
-        self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke, epsilon=eps, pool_mode=pool)
+        self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke, epsilon=eps, pool_mode=pool,
+                             search_mode=mode)
         dev = self.s.device
         self.warm_tok = torch.from_numpy(np.ascontiguousarray(self.tokens[:, :w.k_max])).to(dev)
         self.warm_lp = torch.from_numpy(np.ascontiguousarray(self.logprobs[:, :w.k_max])).to(dev)
@@ -180,7 +181,7 @@ class Runner:
         if first_drafts:                 # the drafts the first sdms_step of a run checks
             self.s.build_drafts(k_of(0, self.w.k_max))
 
-    def dry_run(self):
+    def dry_run(self, allow_status=0):
         """Plays one run to record, per step, the sampled windows (what the model
         would return), the live path count and the algorithmic bytes."""
         torch, w, s = self.torch, self.w, self.s
@@ -218,7 +219,7 @@ class Runner:
             gained = np.minimum(np.minimum(tau + 1, w.D), w.L - lens)
             bytes_io.append(int(gained.sum()) * (8 + 8 + w.k_max * 32) + w.P * (w.D + 1) * 8)
             sampled_all.append(sm); lp_all.append(lp); active.append(live)
-        assert s.status() == 0
+        assert s.status() & ~allow_status == 0
         self.plan = dict(
             sampled=torch.from_numpy(np.stack(sampled_all)).to(dev), lp=torch.from_numpy(np.stack(lp_all)).to(dev),
             step_in_host=torch.from_numpy(np.concatenate(
@@ -432,10 +433,26 @@ def ours_main(args, w):
         ablation = {"dag": plan["accept_length"]}
         if fuzzy is not None:
             ablation["dag_fuzzy"] = fplan["accept_length"]
-        for name, pool, eps in (("tree", 1, 0), ("list", 2, 0), ("tree_fuzzy", 1, 1), ("list_fuzzy", 2, 1)):
-            arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool)
-            ablation[name] = arun.dry_run()["accept_length"]
+        for name, pool, eps, mode in (("tree", 1, 0, 0), ("list", 2, 0, 0), ("tree_fuzzy", 1, 1, 0), ("list_fuzzy", 2, 1, 0),
+                                      ("dag_best_path", 0, 0, 2), ("dag_best_path_fuzzy", 0, 1, 2)):
+            arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool, mode=mode)
+            ablation[name] = arun.dry_run(allow_status=0x40)["accept_length"]
             del arun
+        # sliding window: one sdms_trim of full histories to their newer half (three launches)
+        trun = Runner(w, rank_seed(w, rank), device, 0, 0)
+        n_full = w.L - 1
+        trun.s.reset()
+        trun.s.append(torch.from_numpy(np.ascontiguousarray(trun.tokens[:, :n_full])).to(device),
+                      torch.from_numpy(np.ascontiguousarray(trun.logprobs[:, :n_full])).to(device),
+                      torch.full((w.P,), n_full, dtype=torch.int32, device=device))
+        keep = torch.full((w.P,), w.L // 2, dtype=torch.int32, device=device)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        trun.flush.zero_()
+        a.record(); trun.s.trim(keep); b.record()
+        torch.cuda.synchronize()
+        trim_us = 1e3 * a.elapsed_time(b)
+        assert trun.s.status() == 0
+        del trun
     others = None
     if world == 1 and not args.no_others:
         del run.flush
@@ -484,6 +501,8 @@ def ours_main(args, w):
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
         "fuzzy_epsilon_1": fuzzy, "synthetic_accept_length": ablation,
+        "sliding_window": None if ablation is None else {"us_per_sdms_trim_call": trim_us,
+                                                          "what": "all paths full, trimmed to their newer half"},
         "other_workloads_build_only": others,
         "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
                        "us_per_sdms_get_dag_call": export_us,

@@ -186,6 +186,21 @@ int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d
               float* d_draft_edge_w, void* stream);
 int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes);
 
+/*
+ * Sliding window for runs longer than the capacity (the paper's runs end long
+ * before any limit; this call is not part of its method).  Path p forgets all but
+ * its newest d_keep[p] tokens: they move to the front of its store, the path has
+ * room again, and every later call sees exactly the shorter history, as if only
+ * those tokens had ever been appended.  d_keep[p] >= the path's length changes
+ * nothing; d_keep[p] < 0 raises SDMS_STATUS_BAD_COUNT and changes nothing.
+ * The n-gram tables of every prompt with a trimmed path are emptied and filled
+ * again from the histories (three launches; cost proportional to the prompt's
+ * tokens * k_max), so call it every few hundred steps with a generous cut, not
+ * every step.  Drafts built before the call refer to the old positions: build
+ * again before the next sdms_accept.
+ */
+int sdms_trim(sdms_ctx* ctx, const int32_t* d_keep, void* stream);
+
 /* ---- inspection (used by the parity tests; not part of a decode step) ------- */
 
 /* Matches of the last sdms_build_drafts: d_offsets [P+1] (exclusive prefix sums)
@@ -259,7 +274,8 @@ int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, int32_t num_g
 #define SDMS_KERNEL_ACCEPT 4
 #define SDMS_KERNEL_BUILD_FUSED 5   /* probe + scan + dag in one launch (small prompts) */
 #define SDMS_KERNEL_STEP   6        /* accept + commit + build in one launch (sdms_step) */
-#define SDMS_NUM_KERNELS   7
+#define SDMS_KERNEL_TRIM   7        /* the three launches of sdms_trim */
+#define SDMS_NUM_KERNELS   8
 
 /* Number of kernels this context has launched since creation. */
 int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches);

@@ -21,15 +21,15 @@ ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE, ERR_TOO_LARGE
 NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
-NUM_KERNELS = 7
-KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step")
+NUM_KERNELS = 8
+KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim")
 
 EXPORTS = (
     "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch",
+    "sdms_step_is_single_launch", "sdms_trim",
 )
 
 
@@ -69,6 +69,7 @@ def lib():
         l.sdms_build_drafts.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         l.sdms_build_drafts_backoff.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         l.sdms_accept.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        l.sdms_trim.argtypes = [vp, vp, vp]
         l.sdms_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         l.sdms_step_is_single_launch.argtypes = [vp, C.POINTER(C.c_int32)]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
@@ -155,6 +156,10 @@ def sdms_build_drafts_backoff(ctx, k_hi, draft_tok, draft_len, draft_score=None,
 def sdms_accept(ctx, draft_tok, draft_len, sampled, sampled_logprobs, accept_len, stream=None):
     _check(lib().sdms_accept(ctx, _dp(draft_tok), _dp(draft_len), _dp(sampled), _dp(sampled_logprobs),
                              _dp(accept_len), _sp(stream)), "sdms_accept")
+
+
+def sdms_trim(ctx, keep, stream=None):
+    _check(lib().sdms_trim(ctx, _dp(keep), _sp(stream)), "sdms_trim")
 
 
 def sdms_step(ctx, k, sampled, sampled_logprobs, accept_len, draft_tok, draft_len, draft_score, draft_edge_w,
@@ -283,6 +288,9 @@ class Sdms:
     def accept(self, sampled, sampled_logprobs=None, stream=None):
         sdms_accept(self.ctx, self.draft_tok, self.draft_len, sampled, sampled_logprobs, self.accept_len, stream)
         return self.accept_len
+
+    def trim(self, keep, stream=None):
+        sdms_trim(self.ctx, keep, stream)
 
     def step(self, k, sampled, sampled_logprobs, stream=None):
         """accept + commit of the drafts held now, then the next drafts in their place."""

@@ -12,7 +12,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-  size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, matches;
+  size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, g_nscan, g_trim, matches;
   size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
   size_t total;
   uint32_t table_cap;
@@ -65,6 +65,7 @@ Layout make_layout(const sdms_config* c) {
   l.q_fp = take(P * 4); l.q_mode = take(P * 4); l.q_reserved = take(P * 4);
   l.q_off = take(P * 4); l.q_cursor = take(P * 4);
   l.g_nscan = take((size_t)c->num_groups * 4);
+  l.g_trim = take((size_t)c->num_groups * 4);
   l.matches = take((size_t)mc * 4);
   l.x_draft_tok = take(P * D * 4); l.x_draft_len = take(P * 4);
   l.x_node_tok = take(P * D * B * 4); l.x_node_S = take(P * D * B * 8); l.x_node_cnt = take(P * D * B * 4);
@@ -178,7 +179,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.status = (uint32_t*)(w + lay.status); d.index = (uint32_t*)(w + lay.index);
   d.q_fp = (uint32_t*)(w + lay.q_fp); d.q_mode = (int32_t*)(w + lay.q_mode);
   d.q_reserved = (int32_t*)(w + lay.q_reserved); d.q_off = (int32_t*)(w + lay.q_off);
-  d.q_cursor = (int32_t*)(w + lay.q_cursor); d.g_nscan = (int32_t*)(w + lay.g_nscan);
+  d.q_cursor = (int32_t*)(w + lay.q_cursor); d.g_nscan = (int32_t*)(w + lay.g_nscan); d.g_trim = (int32_t*)(w + lay.g_trim);
   d.matches = (int32_t*)(w + lay.matches);
   ctx->x_draft_tok = (int32_t*)(w + lay.x_draft_tok); ctx->x_draft_len = (int32_t*)(w + lay.x_draft_len);
   d.x_node_tok = (int32_t*)(w + lay.x_node_tok); d.x_node_S = (int64_t*)(w + lay.x_node_S);
@@ -257,6 +258,18 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
   if (d_sampled_logprobs) ctx->built = false;          // the commit changes the histories
   return timed(ctx, SDMS_KERNEL_ACCEPT, st, [&] {
     return launch_accept(ctx->dev, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, st); });
+}
+
+int sdms_trim(sdms_ctx* ctx, const int32_t* d_keep, void* stream) {
+  if (!ctx || !d_keep) return SDMS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->built = false;
+  if (cudaMemsetAsync(ctx->dev.g_trim, 0, (size_t)ctx->dev.G * 4, st) != cudaSuccess) return SDMS_ERR_CUDA;
+  for (int phase = 0; phase < 3; ++phase) {
+    const int rc = timed(ctx, SDMS_KERNEL_TRIM, st, [&] { return launch_trim(ctx->dev, phase, d_keep, st); });
+    if (rc != SDMS_OK) return rc;
+  }
+  return SDMS_OK;
 }
 
 int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,
@@ -387,7 +400,7 @@ const char* sdms_strerror(int code) {
 }
 
 const char* sdms_kernel_name(int kernel) {
-  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept", "build_fused", "step"};
+  static const char* names[SDMS_NUM_KERNELS] = {"append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim"};
   return kernel >= 0 && kernel < SDMS_NUM_KERNELS ? names[kernel] : "?";
 }
 

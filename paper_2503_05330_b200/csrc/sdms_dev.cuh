@@ -43,6 +43,7 @@ struct Dev {
   int32_t* q_off;                      // [P] start in `matches`
   int32_t* q_cursor;                   // [P] matches written
   int32_t* g_nscan;                    // [G] queries of the prompt that need the scan
+  int32_t* g_trim;                     // [G] a path of the prompt was trimmed: its index is rebuilt
   int32_t* matches;                    // [match_cap] global positions j*L+e
   // DAG export of the last build
   int32_t* x_node_tok; int64_t* x_node_S; int32_t* x_node_cnt; int32_t* x_node_count;

@@ -30,6 +30,8 @@ cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32
                        float* draft_edge_w, cudaStream_t stream);
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream);
+// phase 0: shift the histories; 1: empty the index tables of the prompts that changed; 2: index them again
+cudaError_t launch_trim(const Dev& s, int phase, const int32_t* keep, cudaStream_t stream);
 bool step_kernel_fits(const Dev& s);
 cudaError_t launch_step(const Dev& s, int k, const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
                         int32_t* draft_tok, int32_t* draft_len, float* draft_score, float* draft_edge_w,

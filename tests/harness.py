@@ -41,6 +41,12 @@ class Pair:
             assert st_g == expect_status
         return st_g
 
+    def trim(self, keep):
+        st_o = self.o.trim(keep)
+        self.g.trim(t32(np.asarray(keep, np.int32), self.dev))
+        assert self.g.status() == st_o
+        return st_o
+
     def check_history(self):
         tok, pq, lens = self.g.history()
         ol = self.o.lengths()
@@ -182,3 +188,44 @@ def run_step_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, start_lens=
         done_steps += 1
     pair.check_history()
     return dict(steps=done_steps, accepted=accepted)
+
+
+def run_windowed_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, keep, use_step=False):
+    """Decode protocol that outlives the capacity: a path that comes within a draft of its capacity is
+    trimmed to its newest `keep` tokens and goes on.  The streams are read round and round.  Every
+    build is compared; returns how many trims happened."""
+    P, L, D = pair.P, pair.L, pair.D
+    T = tokens.shape[1]
+    lens0 = np.full(P, warm, np.int32)
+    pair.append(tokens[:, :warm], logprobs[:, :warm], lens0, expect_status=0)
+    consumed = lens0.astype(np.int64)                 # tokens of the stream each path has taken so far
+    trims = 0
+    pair.build_and_compare(ks[0], check_dag=False)
+    for step in range(steps):
+        lens = pair.o.lengths()
+        idx = (consumed[:, None] + np.arange(D + 1)[None, :]) % T
+        sampled = np.take_along_axis(tokens, idx, 1).astype(np.int32)
+        sampled_lp = np.take_along_axis(logprobs, idx, 1).astype(np.float32)
+        tok, ln, _, _ = pair.o.drafts()
+        k = ks[(step + 1) % len(ks)]
+        if use_step:
+            tau_o, st_o = pair.o.accept_commit(tok, ln, sampled, sampled_lp, pair.max_append)
+            pair.o.build_all(k, nthreads=min(8, os.cpu_count() or 1))
+            tau_g, gt, gl = pair.g.step(k, t32(sampled, pair.dev), t32(sampled_lp, pair.dev))
+            assert pair.g.status() == st_o
+            assert np.array_equal(tau_g.cpu().numpy(), tau_o)
+            tok2, ln2, _, _ = pair.o.drafts()
+            assert np.array_equal(gl.cpu().numpy(), ln2) and np.array_equal(gt.cpu().numpy(), tok2), step
+        else:
+            tau_o = pair.accept_and_compare(sampled, sampled_lp)
+        consumed += pair.o.lengths() - lens
+        lens = pair.o.lengths()
+        near = lens > L - D - 2
+        if near.any():
+            pair.trim(np.where(near, keep, L).astype(np.int32))
+            trims += int(near.sum())
+            pair.build_and_compare(k, check_dag=False)          # drafts refer to positions: build again
+        elif not use_step:
+            pair.build_and_compare(k, check_dag=False)
+    pair.check_history()
+    return trims

@@ -471,3 +471,30 @@ def test_best_path_config2_and_the_fallback_for_heavy_queries():
         assert pair.g.status() == 0
     pair.check_history()
     assert fell_back > 0
+
+
+# ---- sliding window: runs longer than the capacity -------------------------------------------
+@pytest.mark.parametrize("use_step", [False, True])
+@pytest.mark.parametrize("eps", [0, 1])
+def test_windowed_run_outlives_the_capacity(use_step, eps):
+    G, N, L, V, D, k_max = 2, 4, 64, 5, 4, 3
+    tokens, lps = synth.small_random(G * N, 4 * L, V, 9100 + eps)
+    pair = Pair(G, N, L, V, k_max, D, alpha=0.5, eps=eps)
+    trims = harness.run_windowed_protocol(pair, tokens, lps, [2, 1, 3], steps=90, warm=6, keep=L // 2, use_step=use_step)
+    assert trims >= 2 * G * N // 2                    # every path has been trimmed, most of them twice
+
+
+def test_trim_config2_then_steps_agree():
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    n = 1000
+    lens = (n - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    pair.append(tokens[:, :n], lps[:, :n], lens, expect_status=0)
+    keep = np.where(np.arange(w.P) % 3 == 0, w.L, 300 + 20 * np.arange(w.P)).astype(np.int32)   # some untouched
+    pair.trim(keep)
+    pair.check_history()
+    for k in (1, 2, 4):
+        pair.build_and_compare(k, check_dag=False)
+    assert pair.trim(np.full(w.P, -1, np.int32)) == 0x01   # rejected, nothing changes
+    pair.build_and_compare(3, check_dag=False)

@@ -201,6 +201,19 @@ int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes);
  */
 int sdms_trim(sdms_ctx* ctx, const int32_t* d_keep, void* stream);
 
+/*
+ * Zero-copy callers.  The per-step arrays of sdms_step / sdms_accept / sdms_build_drafts
+ * (sampled tokens and logprobs, drafts, accept lengths) may live in page-locked
+ * host memory that is mapped into the device's address space: the kernel then
+ * reads its inputs and writes its results over the host link itself and no copy
+ * is enqueued around the call (a step's inputs and outputs are about 2 KB).
+ * This call checks that host_ptr is such memory (cudaHostAlloc, or registered
+ * with the mapped flag) and returns in *device_ptr the address to pass instead;
+ * SDMS_ERR_INVALID_ARG for pageable, device or unknown memory.  The host may read
+ * the results after the stream (or an event recorded after the call) has completed.
+ */
+int sdms_host_pointer(const void* host_ptr, void** device_ptr);
+
 /* ---- inspection (used by the parity tests; not part of a decode step) ------- */
 
 /* Matches of the last sdms_build_drafts: d_offsets [P+1] (exclusive prefix sums)

@@ -29,7 +29,7 @@ EXPORTS = (
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch", "sdms_trim",
+    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer",
 )
 
 
@@ -70,6 +70,7 @@ def lib():
         l.sdms_build_drafts_backoff.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         l.sdms_accept.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         l.sdms_trim.argtypes = [vp, vp, vp]
+        l.sdms_host_pointer.argtypes = [vp, C.POINTER(vp)]
         l.sdms_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         l.sdms_step_is_single_launch.argtypes = [vp, C.POINTER(C.c_int32)]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
@@ -100,12 +101,28 @@ def _check(code, where):
         raise SdmsError(code, where)
 
 
+_mapped = {}          # data_ptr of a page-locked host tensor -> its address on the device
+
+
+def sdms_host_pointer(t) -> int:
+    """Device-side address of a page-locked, mapped host tensor (raises for any other memory)."""
+    out = C.c_void_p(0)
+    _check(lib().sdms_host_pointer(C.c_void_p(t.data_ptr()), C.byref(out)), "sdms_host_pointer")
+    return out.value
+
+
 def _dp(t):
-    """Device pointer of a CUDA tensor (None -> NULL)."""
+    """Pointer the kernels can use: a CUDA tensor's own, or the device-side address of a page-locked
+    host tensor that the library has verified (None -> NULL)."""
     if t is None:
         return None
-    assert t.is_cuda and t.is_contiguous()
-    return C.c_void_p(t.data_ptr())
+    assert t.is_contiguous()
+    if t.is_cuda:
+        return C.c_void_p(t.data_ptr())
+    key = t.data_ptr()
+    if key not in _mapped:
+        _mapped[key] = sdms_host_pointer(t)
+    return C.c_void_p(_mapped[key])
 
 
 def _sp(stream):
@@ -231,8 +248,11 @@ class Sdms:
     """A context plus the device buffers of one decode loop (allocation and
     marshalling only)."""
 
-    def __init__(self, G, N, L, V, k_max, D, device="cuda:0", **kw):
+    def __init__(self, G, N, L, V, k_max, D, device="cuda:0", host_io=False, **kw):
+        """host_io: the per-step buffers (`results`, `step_in`) are page-locked host memory that the
+        kernels read and write in place (zero-copy) instead of device memory."""
         self.cfg = make_config(G, N, L, V, k_max, D, **kw)
+        self.host_io = host_io
         self.G, self.N, self.L, self.V, self.k_max, self.D = G, N, L, V, k_max, D
         self.P = G * N
         self.B, self.Ke = self.cfg.dag_nodes_per_layer, self.cfg.dag_edges_per_node
@@ -246,14 +266,15 @@ class Sdms:
         dev = self.device
         # integer results side by side, so that a caller can fetch them with one copy:
         # [draft_tok P*D | draft_len P | accept_len P]
-        self.results = torch.empty(P * (D_ + 2), dtype=torch.int32, device=dev)
+        io = dict(dtype=torch.int32, pin_memory=True) if host_io else dict(dtype=torch.int32, device=dev)
+        self.results = torch.empty(P * (D_ + 2), **io)
         self.draft_tok = self.results[:P * D_].view(P, D_)
         self.draft_len = self.results[P * D_:P * D_ + P]
         self.accept_len = self.results[P * D_ + P:]
         self.draft_score = torch.empty((P, D_), dtype=torch.float32, device=dev)
         self.draft_edge_w = torch.empty((P, D_), dtype=torch.float32, device=dev)
         # the model's answer of a step, likewise one buffer: [sampled P*(D+1) int32 | logprobs P*(D+1) float32]
-        self.step_in = torch.empty(2 * P * (D_ + 1), dtype=torch.int32, device=dev)
+        self.step_in = torch.empty(2 * P * (D_ + 1), **io)
         self.sampled_in = self.step_in[:P * (D_ + 1)].view(P, D_ + 1)
         self.sampled_lp_in = self.step_in[P * (D_ + 1):].view(torch.float32).view(P, D_ + 1)
 

@@ -298,6 +298,15 @@ int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes) {
   return SDMS_OK;
 }
 
+int sdms_host_pointer(const void* host_ptr, void** device_ptr) {
+  if (!host_ptr || !device_ptr) return SDMS_ERR_INVALID_ARG;
+  cudaPointerAttributes a{};
+  if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return SDMS_ERR_INVALID_ARG; }
+  if (a.type != cudaMemoryTypeHost || !a.devicePointer) return SDMS_ERR_INVALID_ARG;
+  *device_ptr = a.devicePointer;
+  return SDMS_OK;
+}
+
 int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t cap, void* stream) {
   if (!ctx || !d_offsets || (!d_gpos && cap)) return SDMS_ERR_INVALID_ARG;
   if (!ctx->built) return SDMS_ERR_BAD_STATE;

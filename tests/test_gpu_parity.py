@@ -498,3 +498,33 @@ def test_trim_config2_then_steps_agree():
         pair.build_and_compare(k, check_dag=False)
     assert pair.trim(np.full(w.P, -1, np.int32)) == 0x01   # rejected, nothing changes
     pair.build_and_compare(3, check_dag=False)
+
+
+# ---- zero-copy: per-step arrays in page-locked host memory -----------------------------------
+def test_step_with_host_mapped_buffers():
+    from paper_2503_05330_b200 import binding
+    w = synth.WORKLOADS[1]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, host_io=True)
+    assert not pair.g.results.is_cuda and pair.g.results.is_pinned()
+    lens = pair.o.lengths()
+    pair.append(tokens[:, :w.k_max], lps[:, :w.k_max], np.full(w.P, w.k_max, np.int32), expect_status=0)
+    pair.build_and_compare(1, check_dag=False)
+    for step in range(40):
+        lens = pair.o.lengths()
+        k = 1 + step % w.k_max
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
+        tok, ln, _, _ = pair.o.drafts()
+        tau_o, st_o = pair.o.accept_commit(tok, ln, sampled, sampled_lp, w.D)
+        pair.o.build_all(k)
+        pair.g.sampled_in.copy_(torch.from_numpy(sampled))                 # host to host
+        pair.g.sampled_lp_in.copy_(torch.from_numpy(sampled_lp))
+        pair.g.step(k, pair.g.sampled_in, pair.g.sampled_lp_in)
+        assert pair.g.status() == st_o                                      # waits for the stream
+        tok, ln, _, _ = pair.o.drafts()
+        assert np.array_equal(pair.g.accept_len.numpy(), tau_o)
+        assert np.array_equal(pair.g.draft_len.numpy(), ln) and np.array_equal(pair.g.draft_tok.numpy(), tok)
+    pair.check_history()
+    # memory the device cannot see is refused before any launch
+    with pytest.raises(binding.SdmsError):
+        binding.sdms_host_pointer(torch.zeros(8, dtype=torch.int32))

@@ -757,12 +757,16 @@ __device__ __forceinline__ u64 weight_bits(double alpha, const unsigned* lo16, c
   return (u64)__double_as_longlong(eq5_weight(alpha, ((u64)hi[x] << 16) + lo16[x], cnt[x]));
 }
 
-// How many layers' tables fit beside the staged followers (0: use dag_block).
+// How many layers' tables fit beside the staged followers (0: use dag_block).  Three words are staged
+// per follower: token, probability, and the table slots found for it (so that no pass probes twice).
 __device__ __forceinline__ int layers_per_round(int M, int D, int* cap_out) {
+  const int staged = (3 * M * D + 1) & ~1;
   int cap = 64;                                    // more slots than keys: a probe always ends at a free slot
   while (cap <= M) cap *= 2;
+  // twice the slots shorten the probe sequences (a warp waits for its longest); taken when all
+  // layers still fit in one round
+  if ((kPoolWords - staged) / (kLayerWords * 2 * cap) >= D) cap *= 2;
   *cap_out = cap;
-  const int staged = (2 * M * D + 1) & ~1;
   return (kPoolWords - staged) / (kLayerWords * cap);
 }
 
@@ -785,7 +789,8 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
   const int lcap = 31 - __clz(cap), shift = 32 - lcap;
   int* st_tok = sm.st_tok;                         // [m * D + d - 1], -1 past the end of the path
   int* st_pq = sm.st_tok + M * D;
-  int* pool = sm.st_tok + ((2 * M * D + 1) & ~1);
+  int* st_slot = sm.st_tok + 2 * M * D;            // node slot | pred slot << 16 of each staged follower
+  int* pool = sm.st_tok + ((3 * M * D + 1) & ~1);
   const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int nchunk = (M + 31) >> 5;                // a warp takes 32 matches of one layer at a time
 
@@ -843,18 +848,20 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
         const LayerTables t = layer_tables(pool, cap, l);
         if (pass == 0) {
           const int sl = table_slot<true>(t.n_key, cap, shift, v);
+          st_slot[at] = sl;
           add_split(&t.n_Slo[sl], &t.n_Shi[sl], &t.n_cnt[sl], (unsigned)st_pq[at]);
           continue;
         }
-        const int u = d == 1 ? root : st_tok[at - 1];
-        const u64 w = weight_bits(s.alpha, t.n_Slo, t.n_Shi, t.n_cnt, table_slot<false>(t.n_key, cap, shift, v));
+        const u64 w = weight_bits(s.alpha, t.n_Slo, t.n_Shi, t.n_cnt, st_slot[at] & 0xffff);
         const unsigned whi = (unsigned)(w >> 32), wlo = (unsigned)w;
         if (pass == 1) {
-          atomicMax(&t.p_whi[table_slot<true>(t.p_key, cap, shift, u)], whi);
+          const int claimed = table_slot<true>(t.p_key, cap, shift, d == 1 ? root : st_tok[at - 1]);
+          st_slot[at] |= claimed << 16;
+          atomicMax(&t.p_whi[claimed], whi);
           if (s.mode == 1) atomicMax(&sh_lwhi[d - 1], whi);
           continue;
         }
-        const int ps = table_slot<false>(t.p_key, cap, shift, u);
+        const int ps = (unsigned)st_slot[at] >> 16;
         if (pass == 2) {
           if (t.p_whi[ps] == whi) atomicMax(&t.p_wlo[ps], wlo);
           if (s.mode == 1 && sh_lwhi[d - 1] == whi) atomicMax(&sh_lwlo[d - 1], wlo);

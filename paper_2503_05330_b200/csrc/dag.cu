@@ -40,6 +40,7 @@ constexpr unsigned FULL = 0xffffffffu;
 constexpr int CAP = kDagCap;
 constexpr int MAXB = SDMS_MAX_DAG_NODES;
 constexpr int MAXKE = SDMS_MAX_DAG_EDGES;
+constexpr int kRollMax = 2 * 8192 / 3;   // candidates whose followers are staged layer by layer (three arrays in the staging area)
 constexpr int kStageWords = 8192;      // followers (token, pq) of all matches staged in shared memory when M*D fits
 constexpr int kLoadBatch = 4;          // candidates a thread loads before it touches the tables
 constexpr int kListCap = 2048;         // matches a fused CTA keeps in shared memory besides its global slice
@@ -415,6 +416,13 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       sm.st_pq[x] = on ? ldm(s.pq + gpos + dd) : 0;
     }
   }
+  // too many followers to stage them all: stage one layer at a time (token and probability of every
+  // candidate; the layer before stays, it holds the edges' sources), so that the passes and phases of
+  // a layer read shared memory and only one sweep per layer goes to L2
+  const bool rolling = !staged && M <= kRollMax && !(!EXPORT && s.pool == 1);
+  int* const roll_odd = sm.st_tok;
+  int* const roll_even = sm.st_tok + kRollMax;
+  int* const roll_p = sm.st_tok + 2 * kRollMax;
   for (int x = tid; x < CAP; x += blockDim.x) {
     sm.n_key[x] = -1; sm.n_Slo[x] = 0; sm.n_Shi[x] = 0; sm.n_Clo[x] = 0; sm.n_Chi[x] = 0;
     sm.n_call[x] = 0; sm.n_ccur[x] = 0;
@@ -440,6 +448,28 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       npart = 1;
       if (!restricted) while (npart * (CAP / 2) * 4 < M && npart < npart_max) npart *= 2;
     }
+    int* const cur_v = (d & 1) ? roll_odd : roll_even;
+    const int* const prev_v = (d & 1) ? roll_even : roll_odd;
+    if (rolling) {
+      constexpr int kRollBatch = 8;
+      for (int m0 = tid; m0 < M; m0 += kRollBatch * blockDim.x) {
+        int tv[kRollBatch], tp[kRollBatch];
+#pragma unroll
+        for (int r = 0; r < kRollBatch; ++r) {
+          const int m = m0 + r * blockDim.x;
+          tv[r] = -1; tp[r] = 0;
+          if (m >= M) continue;
+          const int gpos = mlist[m];
+          const int j = gpos / s.L;
+          if (gpos - j * s.L + d <= plen[j - poff] - 1) { tv[r] = ldm(s.tok + gpos + d); tp[r] = ldm(s.pq + gpos + d); }
+        }
+#pragma unroll
+        for (int r = 0; r < kRollBatch; ++r) {
+          const int m = m0 + r * blockDim.x;
+          if (m < M) { cur_v[m] = tv[r]; roll_p[m] = tp[r]; }
+        }
+      }
+    }
     bool layer_done = false;
     while (!layer_done) {
       if (tid == 0) { sh_best_valid = 0; sh_nnode_run = 0; sh_node_total = 0; }
@@ -464,6 +494,9 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 v[r] = sm.st_tok[m * D + d - 1];
                 if (v[r] >= 0) { u[r] = d == 1 ? root : sm.st_tok[m * D + d - 2]; p[r] = (unsigned)sm.st_pq[m * D + d - 1]; }
                 if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (sm.st_tok[m * D + x - 1] != sh_draft[x - 1]) v[r] = -1;
+              } else if (rolling) {
+                v[r] = cur_v[m];
+                if (v[r] >= 0) { u[r] = d == 1 ? root : prev_v[m]; p[r] = (unsigned)roll_p[m]; }
               } else {
                 const int gpos = mlist[m];
                 const int j = gpos / s.L;

@@ -15,6 +15,7 @@
 //                memory, one global atomic per (CTA, query) reserves the output
 //                range, and a second pass writes the positions.
 #include "sdms_internal.h"
+#include <algorithm>
 
 namespace sdms {
 
@@ -121,20 +122,48 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 }
 
 constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
-constexpr int kLastBits = 4096;
-__device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 20; }
+constexpr int kLastBits = 32768;       // a prompt has up to 1024 scan queries: the reject test must stay selective
+constexpr int kScanBuf = 1536;         // matches a scanning CTA collects before it hands them over
+__device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 17; }
+static_assert(kLastBits == 1 << 15, "last_bit yields 15 bits");
 
-__global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
+// The tokens a thread fetches of tile T of prompt g (tiles are numbered path-major): four consecutive
+// ones, plus one of the sixteen before the tile.  Nothing is fetched beyond the path's length.
+struct TileRegs { int32_t t[4]; int32_t halo; };
+__device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int T, int ntiles, int total, const int32_t* len_of) {
+  TileRegs r;
+  r.t[0] = r.t[1] = r.t[2] = r.t[3] = -1; r.halo = -1;
+  if (T >= total) return r;
+  const int jn = T / ntiles, j = g * s.N + jn, t0 = (T - jn * ntiles) * kScanTile;
+  const int len = len_of[jn];
+  const int32_t* row = s.tok + (size_t)j * s.L;
+  const int x = t0 + 4 * (int)threadIdx.x;
+  if (x < len) {
+    if ((s.L & 3) == 0) {
+      const int4 q = __ldg(reinterpret_cast<const int4*>(row + x));     // may run past len inside the row: unused there
+      r.t[0] = q.x; r.t[1] = q.y; r.t[2] = q.z; r.t[3] = q.w;
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) if (x + u < s.L) r.t[u] = __ldg(row + x + u);
+    }
+  }
+  if (threadIdx.x < kHalo && t0 < len) {
+    const int idx = t0 - kHalo + (int)threadIdx.x;
+    if (idx >= 0) r.halo = __ldg(row + idx);
+  }
+  return r;
+}
+
+// CTA c of prompt g (blockIdx.x = g * ctas + c) walks tiles c, c + ctas, ... of that prompt (all paths of the
+// prompt, tile after tile).  The set of the prompt's scan queries is built once per CTA; the next
+// tile is already on its way from memory while the current one is searched.  With as many CTAs as
+// tiles this is one tile per CTA (small prompts: shortest latency); with fewer it streams.
+__global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ctas) {
   grid_wait();
   grid_release();
-  const int j = blockIdx.y;                    // path whose history is scanned
-  const int g = j / s.N;
+  const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
   if (s.g_nscan[g] == 0) return;
-  const int len_j = s.len[j];
-  const int t0 = blockIdx.x * kScanTile;
-  const int e_lo = max(t0, k - 1);
-  const int e_hi = min(t0 + kScanTile - 1, len_j - 2);     // inclusive; needs one follower
-  if (e_lo > e_hi) return;
+  const int ntiles = (s.L + kScanTile - 1) / kScanTile, total = s.N * ntiles;
 
   __shared__ __align__(16) int32_t sh_tok[kHalo + kScanTile];
   __shared__ int32_t sh_qid[SDMS_MAX_PATHS_PER_GROUP];
@@ -142,31 +171,20 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
   __shared__ int32_t sh_cnt[SDMS_MAX_PATHS_PER_GROUP];
   __shared__ int32_t sh_base[SDMS_MAX_PATHS_PER_GROUP];
   __shared__ int32_t sh_set[kSetSlots];
-  __shared__ uint32_t sh_last[kLastBits / 32];   // which last tokens (hashed to 12 bits) any scan query ends in
+  __shared__ uint32_t sh_last[kLastBits / 32];   // which last tokens (hashed to 15 bits) any scan query ends in
   __shared__ int sh_nq;
-
+  __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
+  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
+  __syncthreads();
+  TileRegs regs = fetch_tile(s, g, first, ntiles, total, sh_len);     // in flight during the set-up
   if (threadIdx.x == 0) sh_nq = 0;
   for (int x = threadIdx.x; x < kSetSlots; x += blockDim.x) sh_set[x] = -1;
   for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
-  // stage the tile (and the tokens just before it)
-  const int32_t* row = s.tok + (size_t)j * s.L;
-  const int hi = min(t0 + kScanTile, s.L);
-  if ((s.L & 3) == 0) {
-    const int4* src = reinterpret_cast<const int4*>(row + t0);
-    int4* dst = reinterpret_cast<int4*>(sh_tok + kHalo);
-    for (int x = threadIdx.x; x < (hi - t0) / 4; x += blockDim.x) dst[x] = __ldg(src + x);
-  } else {
-    for (int x = threadIdx.x; x < hi - t0; x += blockDim.x) sh_tok[kHalo + x] = __ldg(row + t0 + x);
-  }
-  for (int x = threadIdx.x; x < kHalo; x += blockDim.x) {
-    const int idx = t0 - kHalo + x;
-    sh_tok[x] = idx >= 0 ? __ldg(row + idx) : -1;
-  }
   __syncthreads();
-  // the prompt's scan queries (a path never searches itself)
+  // the prompt's scan queries
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) {
     const int i = g * s.N + n;
-    if (i != j && s.q_mode[i] == Q_SCAN) {
+    if (s.q_mode[i] == Q_SCAN) {
       const int sl = atomicAdd(&sh_nq, 1);
       const uint32_t fp = s.q_fp[i];
       sh_qid[sl] = i;
@@ -174,7 +192,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
       sh_cnt[sl] = 0;
       uint32_t hs = (fp >> 1) & (kSetSlots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (kSetSlots - 1);
-      const uint32_t lb = last_bit(s.rec[(size_t)i * kRecWords + 1]);
+      const int32_t* rec = s.rec + (size_t)i * kRecWords;             // rec[1 + t] = token t places from the end
+      const uint32_t lb = last_bit(rec[1]);
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
     }
   }
@@ -182,58 +201,115 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k) {
   const int nq = sh_nq;
   if (nq == 0) return;
 
-  constexpr int kPer = kScanTile / kScanThreads;
-  uint32_t fps[kPer];
-  bool any = false;
-#pragma unroll
-  for (int r = 0; r < kPer; ++r) {
-    const int e = t0 + r * kScanThreads + threadIdx.x;
-    fps[r] = 0;
-    if (e < e_lo || e > e_hi) continue;
+  // Matches are collected in shared memory over many tiles and handed to the match lists in one go:
+  // a tile then costs two barriers and no round trip to memory.
+  __shared__ uint16_t sh_bq[kScanBuf];             // query slot of a collected match
+  __shared__ int32_t sh_bpos[kScanBuf];            // its position j * L + e
+  __shared__ int sh_nbuf, sh_over;
+  if (threadIdx.x == 0) { sh_nbuf = 0; sh_over = 0; }
+  __syncthreads();
+
+  // hands the collected matches [0, n) over: count per query, reserve a range of each list, write
+  auto flush = [&](int n) {
+    for (int x = threadIdx.x; x < n; x += blockDim.x) atomicAdd(&sh_cnt[sh_bq[x]], 1);
+    __syncthreads();
+    for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
+      const int c = sh_cnt[sl];
+      sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
+      sh_cnt[sl] = 0;
+    }
+    __syncthreads();
+    for (int x = threadIdx.x; x < n; x += blockDim.x) {
+      const int sl = sh_bq[x], i = sh_qid[sl];
+      const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
+      if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = sh_bpos[x];
+      else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+    }
+    __syncthreads();
+    for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) sh_cnt[sl] = 0;
+    if (threadIdx.x == 0) sh_nbuf = 0;
+    __syncthreads();
+  };
+
+  // Calls visit(slot of the query, position e) for every match of the tile at position e = t0 + r * kScanThreads + tid.
+  auto matches_at = [&](int j, int t0, int e, auto visit) {
     const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
     const uint32_t lb = last_bit(w[k - 1]);
-    if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) continue;       // no query ends in this token: nothing to hash
+    if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) return;           // no query ends in this token: nothing to hash
     uint64_t h = gram_init(k);
     for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
     const uint32_t fp = gram_fp(gram_final(h));
     uint32_t hs = (fp >> 1) & (kSetSlots - 1);
-    bool mine = false;
     for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
       if (sh_qfp[sl] != fp) continue;
       const int i = sh_qid[sl];
-      const int32_t* q = s.tok + (size_t)i * s.L + (s.len[i] - k);
+      if (i == j) continue;                                       // a path never searches itself
+      const int32_t* rec = s.rec + (size_t)i * kRecWords;       // the query: rec[1 + t] = token t places from the end
       bool same = true;
-      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(q + t));
-      if (same) { atomicAdd(&sh_cnt[sl], 1); mine = true; }
+      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(rec + k - t));
+      if (same) visit(sl);
     }
-    if (mine) { fps[r] = fp; any = true; }                     // the second pass revisits matching positions only
-  }
-  if (!__syncthreads_or(any)) return;
-  for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
-    const int c = sh_cnt[sl];
-    sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
-    sh_cnt[sl] = 0;
-  }
-  __syncthreads();
+  };
+  constexpr int kPer = kScanTile / kScanThreads;
+
+  for (int T = first; T < total; T += ctas) {
+    const int jn = T / ntiles, j = g * s.N + jn, t0 = (T - jn * ntiles) * kScanTile;
+    const int e_lo = max(t0, k - 1);
+    const int e_hi = min(t0 + kScanTile - 1, sh_len[jn] - 2);   // inclusive; needs one follower
+    const int held = sh_nbuf;                                    // (a barrier lies between this and the last change)
+    // the tile lands in shared memory; the next one is asked for before this one is looked at
+    *reinterpret_cast<int4*>(sh_tok + kHalo + 4 * threadIdx.x) = make_int4(regs.t[0], regs.t[1], regs.t[2], regs.t[3]);
+    if (threadIdx.x < kHalo) sh_tok[threadIdx.x] = regs.halo;
+    __syncthreads();
+    regs = fetch_tile(s, g, T + ctas, ntiles, total, sh_len);
+    if (e_lo <= e_hi) {
 #pragma unroll
-  for (int r = 0; r < kPer; ++r) {
-    const uint32_t fp = fps[r];
-    if (fp == 0) continue;
-    const int e = t0 + r * kScanThreads + threadIdx.x;
-    const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
-    uint32_t hs = (fp >> 1) & (kSetSlots - 1);
-    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
-      if (sh_qfp[sl] != fp) continue;
-      const int i = sh_qid[sl];
-      const int32_t* q = s.tok + (size_t)i * s.L + (s.len[i] - k);
-      bool same = true;
-      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(q + t));
-      if (!same) continue;
-      const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
-      if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = j * s.L + e;
-      else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+      for (int r = 0; r < kPer; ++r) {
+        const int e = t0 + r * kScanThreads + threadIdx.x;
+        if (e < e_lo || e > e_hi) continue;
+        matches_at(j, t0, e, [&](int sl) {
+          const int at = atomicAdd(&sh_nbuf, 1);
+          if (at < kScanBuf) { sh_bq[at] = (uint16_t)sl; sh_bpos[at] = j * s.L + e; }
+          else sh_over = 1;
+        });
+      }
+    }
+    __syncthreads();
+    if (sh_over) {
+      // (same for the whole CTA) this tile's matches did not fit: hand over what was there before the
+      // tile, then take the tile again with exact counts, straight into the match lists
+      flush(held);
+      if (threadIdx.x == 0) sh_over = 0;
+#pragma unroll
+      for (int r = 0; r < kPer; ++r) {
+        const int e = t0 + r * kScanThreads + threadIdx.x;
+        if (e >= e_lo && e <= e_hi) matches_at(j, t0, e, [&](int sl) { atomicAdd(&sh_cnt[sl], 1); });
+      }
+      __syncthreads();
+      for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
+        const int c = sh_cnt[sl];
+        sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
+        sh_cnt[sl] = 0;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int r = 0; r < kPer; ++r) {
+        const int e = t0 + r * kScanThreads + threadIdx.x;
+        if (e >= e_lo && e <= e_hi) matches_at(j, t0, e, [&](int sl) {
+          const int i = sh_qid[sl];
+          const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
+          if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = j * s.L + e;
+          else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+        });
+      }
+      __syncthreads();
+      for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) sh_cnt[sl] = 0;
+      __syncthreads();
+    } else if (sh_nbuf > kScanBuf / 2) {
+      flush(sh_nbuf);
     }
   }
+  flush(sh_nbuf);
 }
 
 // Inspection only: packs the per-query slices of the match list.
@@ -270,8 +346,13 @@ cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
 }
 
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
-  dim3 grid((s.L + kScanTile - 1) / kScanTile, s.P);
-  return launch_overlapped(scan_kernel, grid, dim3(kScanThreads), 0, stream, s, k);
+  // one CTA per tile while that keeps the device busy for one round; beyond that each CTA streams
+  // through its share of its prompt's tiles
+  const long long per_prompt = (long long)s.N * ((s.L + kScanTile - 1) / kScanTile);
+  const long long budget = 148LL * 8 * 4;
+  long long ctas = per_prompt;
+  if ((long long)s.G * per_prompt > budget) ctas = std::max(1LL, std::min(per_prompt, budget / s.G));
+  return launch_overlapped(scan_kernel, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), 0, stream, s, k, (int)ctas);
 }
 
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream) {

@@ -528,3 +528,16 @@ def test_step_with_host_mapped_buffers():
     # memory the device cannot see is refused before any launch
     with pytest.raises(binding.SdmsError):
         binding.sdms_host_pointer(torch.zeros(8, dtype=torch.int32))
+
+
+def test_tile_scan_with_more_matches_per_tile_than_its_buffer_holds():
+    # two-token alphabet, k = 1: half of a tile's 1024 positions match each of a dozen queries, far more
+    # than the scanning CTA can collect; match_capacity below P*N*L selects the probe / tile-scan / dag kernels
+    G, N, L, V, D = 1, 12, 1024, 2, 3
+    tokens, lps = synth.small_random(G * N, L, V, 4242)
+    pair = Pair(G, N, L, V, 2, D, match_capacity=120000)
+    lens = (1000 - (np.arange(N) * 37) % 300).astype(np.int32)
+    pair.append(tokens[:, :1000], lps[:, :1000], lens, expect_status=0)
+    for k in (1, 2):
+        pair.build_and_compare(k, check_dag=False)
+    assert (pair.g.query_modes() == 2).all()

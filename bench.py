@@ -29,8 +29,8 @@ UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
 # profiles/step_kernel_cfg2_ncu_full.md; only quoted while the kernel sources are the ones profiled
-NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76096,
-               "sources_sha256": "2c8252296152901e045367f6a12463d549ce639c1626fa70ef97c0a85ee8d5b8"}
+NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 75584,
+               "sources_sha256": "ed720c211fc769bde2c3662c23f6bc6cf069fcb08fc075680c748f1812e1645d"}
 
 
 def kernel_sources_sha():
@@ -342,6 +342,38 @@ def steady_state(wl, device, iters=20):
             "launches_per_build": 1 if fused else 3, "build_by_k": out}
 
 
+def scan_at_scale(device, G=64, N=256, L=8192, V=151936):
+    """The tile-scan kernel on a store larger than L2 (G prompts of N paths, uniform random tokens, k = 1:
+    every query has more matches than an index bucket lists, so all of them are answered by the scan).
+    Algorithmic bytes = the tokens of all histories, read once.  Context for the kernel that is
+    bandwidth-bound by design; the benchmark workload itself never leaves L2."""
+    import torch
+    from paper_2503_05330_b200 import binding
+    P, n = G * N, L - 8
+    s = binding.Sdms(G, N, L, V, 1, 4, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(synth.BASE_SEED)
+    tok = torch.randint(0, V, (P, n), dtype=torch.int32, device=device, generator=gen)
+    lp = -torch.rand((P, n), dtype=torch.float32, device=device, generator=gen)
+    s.append(tok, lp, torch.full((P,), n, dtype=torch.int32, device=device))
+    del tok, lp
+    s.build_drafts(1)                                  # warm-up
+    binding.sdms_profile_enable(s.ctx, True)
+    for _ in range(5):
+        s.build_drafts(1)
+    torch.cuda.synchronize()
+    prof = binding.sdms_profile_read(s.ctx)
+    assert s.status() == 0
+    ms, launches = prof["scan"]
+    us = 1e3 * ms / launches
+    nbytes = 4 * P * n
+    out = {"groups": G, "paths_per_group": N, "capacity": L, "store_bytes": nbytes, "workspace_bytes": s.workspace_bytes,
+           "scan_queries": int((s.query_modes() == 2).sum()), "us_per_launch": us, "gbs": nbytes / (us * 1e-6) / 1e9}
+    del s
+    torch.cuda.empty_cache()
+    return out
+
+
 def rank_seed(w, rank):
     """Every rank owns its own prompts: same recipe, different seed."""
     return synth.BASE_SEED + w.index + 7919 * rank
@@ -462,11 +494,12 @@ def ours_main(args, w):
         trim_us = 1e3 * a.elapsed_time(b)
         assert trun.s.status() == 0
         del trun
-    others = None
+    others = scale = None
     if world == 1 and not args.no_others:
         del run.flush
         torch.cuda.empty_cache()
         others = {synth.WORKLOADS[c].name: steady_state(synth.WORKLOADS[c], device) for c in (1, 3, 4, 5)}
+        scale = scan_at_scale(device)
     (ms, ms_e2e), (units, units_e2e) = whole_job([ms, ms_e2e], [units, units_e2e], device)
     if rank != 0:
         if world > 1:
@@ -517,6 +550,7 @@ def ours_main(args, w):
         "sliding_window": None if ablation is None else {"us_per_sdms_trim_call": trim_us,
                                                           "what": "all paths full, trimmed to their newer half"},
         "other_workloads_build_only": others,
+        "scan_kernel_at_scale": None if scale is None else dict(scale, frac_of_peak=scale["gbs"] / peak),
         "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
                        "us_per_sdms_get_dag_call": export_us,
                        "note": "inspection call that re-aggregates the last build's matches; not part of a step"},

@@ -125,16 +125,17 @@ constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
 constexpr int kLastBits = 32768;       // a prompt has up to 1024 scan queries: the reject test must stay selective
 constexpr int kScanBuf = 1536;         // matches a scanning CTA collects before it hands them over
 __device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 17; }
+__device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 17; }
 static_assert(kLastBits == 1 << 15, "last_bit yields 15 bits");
 
 // The tokens a thread fetches of tile T of prompt g (tiles are numbered path-major): four consecutive
 // ones, plus one of the sixteen before the tile.  Nothing is fetched beyond the path's length.
 struct TileRegs { int32_t t[4]; int32_t halo; };
-__device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int T, int ntiles, int total, const int32_t* len_of) {
+__device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int jn, int tile, const int32_t* len_of) {
   TileRegs r;
   r.t[0] = r.t[1] = r.t[2] = r.t[3] = -1; r.halo = -1;
-  if (T >= total) return r;
-  const int jn = T / ntiles, j = g * s.N + jn, t0 = (T - jn * ntiles) * kScanTile;
+  if (jn >= s.N) return r;
+  const int j = g * s.N + jn, t0 = tile * kScanTile;
   const int len = len_of[jn];
   const int32_t* row = s.tok + (size_t)j * s.L;
   const int x = t0 + 4 * (int)threadIdx.x;
@@ -176,7 +177,12 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   __syncthreads();
-  TileRegs regs = fetch_tile(s, g, first, ntiles, total, sh_len);     // in flight during the set-up
+  // (path, tile) of the CTA's current tile and of the one after it; they advance by `ctas` tiles without a division
+  const int step_j = ctas / ntiles, step_t = ctas - step_j * ntiles;
+  int jn = first / ntiles, tile = first - jn * ntiles;
+  int jn_next = jn + step_j, tile_next = tile + step_t;
+  if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
+  TileRegs regs = fetch_tile(s, g, jn, tile, sh_len);                 // in flight during the set-up
   if (threadIdx.x == 0) sh_nq = 0;
   for (int x = threadIdx.x; x < kSetSlots; x += blockDim.x) sh_set[x] = -1;
   for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
@@ -193,8 +199,9 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
       uint32_t hs = (fp >> 1) & (kSetSlots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (kSetSlots - 1);
       const int32_t* rec = s.rec + (size_t)i * kRecWords;             // rec[1 + t] = token t places from the end
-      const uint32_t lb = last_bit(rec[1]);
+      const uint32_t lb = last_bit(rec[1]), lb2 = last_bit2(rec[1]);   // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
+      atomicOr(&sh_last[lb2 >> 5], 1u << (lb2 & 31));
     }
   }
   __syncthreads();
@@ -236,6 +243,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
     const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
     const uint32_t lb = last_bit(w[k - 1]);
     if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) return;           // no query ends in this token: nothing to hash
+    const uint32_t lb2 = last_bit2(w[k - 1]);
+    if (!(sh_last[lb2 >> 5] >> (lb2 & 31) & 1u)) return;
     uint64_t h = gram_init(k);
     for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
     const uint32_t fp = gram_fp(gram_final(h));
@@ -253,7 +262,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
   constexpr int kPer = kScanTile / kScanThreads;
 
   for (int T = first; T < total; T += ctas) {
-    const int jn = T / ntiles, j = g * s.N + jn, t0 = (T - jn * ntiles) * kScanTile;
+    const int j = g * s.N + jn, t0 = tile * kScanTile;
     const int e_lo = max(t0, k - 1);
     const int e_hi = min(t0 + kScanTile - 1, sh_len[jn] - 2);   // inclusive; needs one follower
     const int held = sh_nbuf;                                    // (a barrier lies between this and the last change)
@@ -261,7 +270,10 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
     *reinterpret_cast<int4*>(sh_tok + kHalo + 4 * threadIdx.x) = make_int4(regs.t[0], regs.t[1], regs.t[2], regs.t[3]);
     if (threadIdx.x < kHalo) sh_tok[threadIdx.x] = regs.halo;
     __syncthreads();
-    regs = fetch_tile(s, g, T + ctas, ntiles, total, sh_len);
+    regs = fetch_tile(s, g, jn_next, tile_next, sh_len);
+    jn = jn_next; tile = tile_next;
+    jn_next += step_j; tile_next += step_t;
+    if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
     if (e_lo <= e_hi) {
 #pragma unroll
       for (int r = 0; r < kPer; ++r) {

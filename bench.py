@@ -579,7 +579,14 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the build-only figures of the other workloads")
     ap.add_argument("--steady", type=int, default=0,
                     help="only print the build-only figures of this workload at 97 %% full histories (for profiling)")
+    ap.add_argument("--scan-scale", type=int, default=0,
+                    help="only run the tile-scan kernel on this many prompts of 256 paths x 8192 tokens (for profiling)")
     args = ap.parse_args()
+    if args.scan_scale:
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps({"scan_kernel_at_scale": scan_at_scale("cuda:0", G=args.scan_scale)}), flush=True)
+        return
     if args.steady:
         import torch
         torch.cuda.set_device(0)

@@ -121,7 +121,6 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
   }
 }
 
-constexpr int kSetSlots = 2 * SDMS_MAX_PATHS_PER_GROUP;
 constexpr int kLastBits = 32768;       // a prompt has up to 1024 scan queries: the reject test must stay selective
 constexpr int kScanBuf = 1536;         // matches a scanning CTA collects before it hands them over
 __device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 17; }
@@ -159,7 +158,7 @@ __device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int jn, int 
 // prompt, tile after tile).  The set of the prompt's scan queries is built once per CTA; the next
 // tile is already on its way from memory while the current one is searched.  With as many CTAs as
 // tiles this is one tile per CTA (small prompts: shortest latency); with fewer it streams.
-__global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ctas) {
+__global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int ctas, int set_slots) {
   grid_wait();
   grid_release();
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
@@ -167,14 +166,17 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
   const int ntiles = (s.L + kScanTile - 1) / kScanTile, total = s.N * ntiles;
 
   __shared__ __align__(16) int32_t sh_tok[kHalo + kScanTile];
-  __shared__ int32_t sh_qid[SDMS_MAX_PATHS_PER_GROUP];
-  __shared__ uint32_t sh_qfp[SDMS_MAX_PATHS_PER_GROUP];
-  __shared__ int32_t sh_cnt[SDMS_MAX_PATHS_PER_GROUP];
-  __shared__ int32_t sh_base[SDMS_MAX_PATHS_PER_GROUP];
-  __shared__ int32_t sh_set[kSetSlots];
+  // per-query arrays and the query set are sized by this prompt's N (dynamic shared memory), not by the
+  // largest N the library takes: more CTAs fit an SM
+  extern __shared__ __align__(16) int32_t scan_dyn[];
+  int32_t* const sh_qid = scan_dyn;
+  uint32_t* const sh_qfp = reinterpret_cast<uint32_t*>(scan_dyn + s.N);
+  int32_t* const sh_cnt = scan_dyn + 2 * s.N;
+  int32_t* const sh_base = scan_dyn + 3 * s.N;
+  int32_t* const sh_len = scan_dyn + 4 * s.N;
+  int32_t* const sh_set = scan_dyn + 5 * s.N;      // set_slots entries, a power of two >= 2 N
   __shared__ uint32_t sh_last[kLastBits / 32];   // which last tokens (hashed to 15 bits) any scan query ends in
   __shared__ int sh_nq;
-  __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   __syncthreads();
   // (path, tile) of the CTA's current tile and of the one after it; they advance by `ctas` tiles without a division
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
   if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
   TileRegs regs = fetch_tile(s, g, jn, tile, sh_len);                 // in flight during the set-up
   if (threadIdx.x == 0) sh_nq = 0;
-  for (int x = threadIdx.x; x < kSetSlots; x += blockDim.x) sh_set[x] = -1;
+  for (int x = threadIdx.x; x < set_slots; x += blockDim.x) sh_set[x] = -1;
   for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
   __syncthreads();
   // the prompt's scan queries
@@ -196,8 +198,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
       sh_qid[sl] = i;
       sh_qfp[sl] = fp;
       sh_cnt[sl] = 0;
-      uint32_t hs = (fp >> 1) & (kSetSlots - 1);
-      while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (kSetSlots - 1);
+      uint32_t hs = (fp >> 1) & (set_slots - 1);
+      while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (set_slots - 1);
       const int32_t* rec = s.rec + (size_t)i * kRecWords;             // rec[1 + t] = token t places from the end
       const uint32_t lb = last_bit(rec[1]), lb2 = last_bit2(rec[1]);   // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
@@ -248,8 +250,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(Dev s, int k, int ct
     uint64_t h = gram_init(k);
     for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
     const uint32_t fp = gram_fp(gram_final(h));
-    uint32_t hs = (fp >> 1) & (kSetSlots - 1);
-    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (kSetSlots - 1)) {
+    uint32_t hs = (fp >> 1) & (set_slots - 1);
+    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (set_slots - 1)) {
       if (sh_qfp[sl] != fp) continue;
       const int i = sh_qid[sl];
       if (i == j) continue;                                       // a path never searches itself
@@ -364,7 +366,11 @@ cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   const long long budget = 148LL * 8 * 4;
   long long ctas = per_prompt;
   if ((long long)s.G * per_prompt > budget) ctas = std::max(1LL, std::min(per_prompt, budget / s.G));
-  return launch_overlapped(scan_kernel, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), 0, stream, s, k, (int)ctas);
+  int set_slots = 64;
+  while (set_slots < 2 * s.N) set_slots *= 2;
+  const size_t dyn = ((size_t)5 * s.N + set_slots) * 4;
+  return launch_overlapped(scan_kernel, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), dyn, stream, s, k, (int)ctas,
+                           set_slots);
 }
 
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream) {

@@ -541,3 +541,29 @@ def test_tile_scan_with_more_matches_per_tile_than_its_buffer_holds():
     for k in (1, 2):
         pair.build_and_compare(k, check_dag=False)
     assert (pair.g.query_modes() == 2).all()
+
+
+@pytest.mark.parametrize("mode,pool", [(0, 0), (1, 0), (2, 0), (0, 1), (0, 2)])
+def test_search_modes_and_pools_through_the_probe_scan_dag_kernels(mode, pool):
+    # match_capacity below P*N*L: the build takes the three-kernel path, where the searches and
+    # pools run inside dag_kernel instead of the single-launch kernel
+    G, N, L, V, D, k_max = 2, 6, 64, 4, 5, 3
+    tokens, lps = synth.small_random(G * N, L, V, 9300 + 10 * mode + pool)
+    for k in (1, 2):
+        pair = Pair(G, N, L, V, k_max, D, alpha=0.5, mode=mode, pool=pool, match_capacity=3000)
+        start = 6 + (np.arange(G * N) * 5) % 11
+        st = run_protocol(pair, tokens, lps, k, steps=25, warm=0, start_lens=start, commit_in_accept=True,
+                          check_dag=False)
+        assert st["steps"] > 5
+        from paper_2503_05330_b200 import binding
+        n0 = binding.sdms_launch_count(pair.g.ctx)
+        pair.g.build_drafts(k)
+        assert binding.sdms_launch_count(pair.g.ctx) == n0 + 3        # probe, scan, dag
+
+
+def test_trim_on_the_three_kernel_path():
+    G, N, L, V, D, k_max = 2, 6, 64, 4, 4, 3
+    tokens, lps = synth.small_random(G * N, 4 * L, V, 9400)
+    pair = Pair(G, N, L, V, k_max, D, match_capacity=3000)
+    trims = harness.run_windowed_protocol(pair, tokens, lps, [2, 1, 3], steps=60, warm=6, keep=L // 2)
+    assert trims >= G * N

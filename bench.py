@@ -161,7 +161,7 @@ class ClockSampler(threading.Thread):
 class Runner:
     """Device-resident replay of the decode protocol of one workload."""
 
-    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0, mode=0, host_io=False):
+    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0, mode=0, host_io=False, backoff=False):
         import torch
         from paper_2503_05330_b200 import binding
         self.torch, self.binding, self.w, self.device = torch, binding, w, device
@@ -174,12 +174,26 @@ class Runner:
         self.warm_cnt = torch.full((w.P,), w.k_max, dtype=torch.int32, device=dev)
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
         self.plan = None
+        self.backoff = backoff           # every build asks for k_max and backs off to the longest k with a match
 
     def start_run(self, first_drafts=False):
         self.s.reset()
         self.s.append(self.warm_tok, self.warm_lp, self.warm_cnt)
         if first_drafts:                 # the drafts the first sdms_step of a run checks
-            self.s.build_drafts(k_of(0, self.w.k_max))
+            self.build(0)
+
+    def build(self, step):
+        if self.backoff:
+            self.s.build_drafts_backoff(self.w.k_max)
+        else:
+            self.s.build_drafts(k_of(step, self.w.k_max))
+
+    def step(self, step, sampled, lp):
+        """Acceptance and commit of decode step `step`, drafts of step + 1, in one call."""
+        if self.backoff:
+            self.s.step_backoff(self.w.k_max, sampled, lp)
+        else:
+            self.s.step(k_of(step + 1, self.w.k_max), sampled, lp)
 
     def dry_run(self, allow_status=0):
         """Plays one run to record, per step, the sampled windows (what the model
@@ -197,7 +211,7 @@ class Runner:
             if live == 0:
                 break
             sm, lp = synth.sampled_window(self.tokens, self.logprobs, lens, w.D + 1)
-            s.build_drafts(k_of(step, w.k_max))
+            self.build(step)
             off, gpos = s.matches()
             gpos = gpos.numpy().astype(np.int64)
             j, e = gpos // w.L, gpos % w.L
@@ -269,7 +283,7 @@ class Runner:
                     a.record()
                 if e2e:
                     s.step_in.copy_(h_in[step])     # host to host: the model's answer lands in the mapped buffer
-                    s.step(k_next, s.sampled_in, s.sampled_lp_in)
+                    self.step(step, s.sampled_in, s.sampled_lp_in)
                     if on:
                         b.record()
                         b.synchronize()             # the caller reads the result before its next step
@@ -277,7 +291,7 @@ class Runner:
                     else:
                         torch.cuda.current_stream().synchronize()   # the kernel is done with the input buffer
                 else:
-                    s.step(k_next, plan["sampled"][step], plan["lp"][step])
+                    self.step(step, plan["sampled"][step], plan["lp"][step])
                     if on:
                         b.record()
                 if on:
@@ -479,6 +493,16 @@ def ours_main(args, w):
             arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool, mode=mode)
             ablation[name] = arun.dry_run(allow_status=0x40)["accept_length"]
             del arun
+        # suffix length with back-off: every step asks for k_max, each path uses the longest k that has a match
+        brun = Runner(w, rank_seed(w, rank), device, 0, 0, backoff=True)
+        bplan = brun.dry_run()
+        brun.timed_steps(20)
+        n_b = min(args.steps, 1000)
+        bms, bunits = brun.timed_steps(n_b)
+        backoff = {"us_per_step": 1e3 * bms / n_b, "value": bunits / (bms * 1e-3), "unit": UNIT,
+                   "accept_length": bplan["accept_length"], "mean_matches_per_step": bplan["mean_matches_per_step"],
+                   "what": "sdms_step_backoff(k_max): one launch per step, k chosen per path"}
+        del brun
         # sliding window: one sdms_trim of full histories to their newer half (three launches)
         trun = Runner(w, rank_seed(w, rank), device, 0, 0)
         n_full = w.L - 1
@@ -547,6 +571,7 @@ def ours_main(args, w):
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
         "fuzzy_epsilon_1": fuzzy, "synthetic_accept_length": ablation,
+        "backoff_from_k_max": None if ablation is None else backoff,
         "sliding_window": None if ablation is None else {"us_per_sdms_trim_call": trim_us,
                                                           "what": "all paths full, trimmed to their newer half"},
         "other_workloads_build_only": others,

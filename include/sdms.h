@@ -184,6 +184,11 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
 int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,
               int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
               float* d_draft_edge_w, void* stream);
+/* sdms_step with the suffix length backing off as in sdms_build_drafts_backoff
+ * (same restriction to small prompts, else SDMS_ERR_BAD_STATE). */
+int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, const float* d_sampled_logprobs,
+                      int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
+                      float* d_draft_edge_w, int32_t* d_used_k, void* stream);
 int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes);
 
 /*

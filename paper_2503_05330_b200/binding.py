@@ -29,7 +29,7 @@ EXPORTS = (
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer",
+    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff",
 )
 
 
@@ -72,6 +72,7 @@ def lib():
         l.sdms_trim.argtypes = [vp, vp, vp]
         l.sdms_host_pointer.argtypes = [vp, C.POINTER(vp)]
         l.sdms_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        l.sdms_step_backoff.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         l.sdms_step_is_single_launch.argtypes = [vp, C.POINTER(C.c_int32)]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
         l.sdms_get_dag.argtypes = [vp] * 10
@@ -183,6 +184,13 @@ def sdms_step(ctx, k, sampled, sampled_logprobs, accept_len, draft_tok, draft_le
               stream=None):
     _check(lib().sdms_step(ctx, k, _dp(sampled), _dp(sampled_logprobs), _dp(accept_len), _dp(draft_tok),
                            _dp(draft_len), _dp(draft_score), _dp(draft_edge_w), _sp(stream)), "sdms_step")
+
+
+def sdms_step_backoff(ctx, k_hi, sampled, sampled_logprobs, accept_len, draft_tok, draft_len, draft_score,
+                      draft_edge_w, used_k, stream=None):
+    _check(lib().sdms_step_backoff(ctx, k_hi, _dp(sampled), _dp(sampled_logprobs), _dp(accept_len), _dp(draft_tok),
+                                   _dp(draft_len), _dp(draft_score), _dp(draft_edge_w), _dp(used_k), _sp(stream)),
+           "sdms_step_backoff")
 
 
 def sdms_step_is_single_launch(ctx) -> bool:
@@ -318,6 +326,11 @@ class Sdms:
         sdms_step(self.ctx, k, sampled, sampled_logprobs, self.accept_len, self.draft_tok, self.draft_len,
                   self.draft_score, self.draft_edge_w, stream)
         return self.accept_len, self.draft_tok, self.draft_len
+
+    def step_backoff(self, k_hi, sampled, sampled_logprobs, stream=None):
+        sdms_step_backoff(self.ctx, k_hi, sampled, sampled_logprobs, self.accept_len, self.draft_tok, self.draft_len,
+                          self.draft_score, self.draft_edge_w, self.used_k, stream)
+        return self.accept_len, self.draft_tok, self.draft_len, self.used_k
 
     def step_is_single_launch(self) -> bool:
         return sdms_step_is_single_launch(self.ctx)

@@ -286,8 +286,30 @@ int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d
   cudaStream_t st = (cudaStream_t)stream;
   ctx->built = false;
   const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
-    return launch_step(ctx->dev, k, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
-                       d_draft_score, d_draft_edge_w, st); });
+    return launch_step(ctx->dev, k, k, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
+                       d_draft_score, d_draft_edge_w, nullptr, st); });
+  if (rc == SDMS_OK) ctx->built = true;
+  return rc;
+}
+
+int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, const float* d_sampled_logprobs,
+                      int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
+                      float* d_draft_edge_w, int32_t* d_used_k, void* stream) {
+  if (!ctx || !d_sampled || !d_sampled_logprobs || !d_accept_len || !d_draft_tok || !d_draft_len)
+    return SDMS_ERR_INVALID_ARG;
+  if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->dev.fused) return SDMS_ERR_BAD_STATE;
+  if (!ctx->step_fits) {
+    const int rc = sdms_accept(ctx, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, stream);
+    if (rc != SDMS_OK) return rc;
+    return sdms_build_drafts_backoff(ctx, k_hi, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, d_used_k,
+                                     stream);
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->built = false;
+  const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
+    return launch_step(ctx->dev, k_hi, 1, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
+                       d_draft_score, d_draft_edge_w, d_used_k, st); });
   if (rc == SDMS_OK) ctx->built = true;
   return rc;
 }

@@ -1345,10 +1345,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
 // probabilities, index entries); after a cluster-wide barrier with release/acquire semantics every
 // path of the prompt is up to date and each CTA builds its path's next draft.  draft_tok / draft_len
 // hold the previous drafts on entry and the new ones on exit.
-__global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, const int32_t* sampled,
+// k_lo < k: the suffix length backs off from k to k_lo (used_k, if given, receives each path's choice).
+__global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, int k_lo, const int32_t* sampled,
                                                            const float* sampled_lp, int32_t* accept_len,
                                                            int32_t* draft_tok, int32_t* draft_len,
-                                                           float* draft_score, float* draft_edge_w) {
+                                                           float* draft_score, float* draft_edge_w,
+                                                           int32_t* used_k) {
   grid_wait();
   grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -1357,7 +1359,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, co
   accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec, k);
   // every thread of every CTA of the cluster gets here exactly once (no early exit above)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  build_phase<false>(s, sm, k, k, draft_tok, draft_len, draft_score, draft_edge_w, nullptr, sh_own_rec);
+  build_phase<false>(s, sm, k, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, sh_own_rec);
 }
 
 }  // namespace
@@ -1401,13 +1403,13 @@ bool step_kernel_fits(const Dev& s) {
   return clusters >= 1;
 }
 
-cudaError_t launch_step(const Dev& s, int k, const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
-                        int32_t* draft_tok, int32_t* draft_len, float* draft_score, float* draft_edge_w,
-                        cudaStream_t stream) {
+cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, const float* sampled_lp,
+                        int32_t* accept_len, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                        float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
   cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
   step_launch_config(s, stream, &cfg, attr);
-  return cudaLaunchKernelEx(&cfg, step_kernel, s, k, sampled, sampled_lp, accept_len, draft_tok, draft_len,
-                            draft_score, draft_edge_w);
+  return cudaLaunchKernelEx(&cfg, step_kernel, s, k, k_lo, sampled, sampled_lp, accept_len, draft_tok, draft_len,
+                            draft_score, draft_edge_w, used_k);
 }
 
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,

@@ -567,3 +567,37 @@ def test_trim_on_the_three_kernel_path():
     pair = Pair(G, N, L, V, k_max, D, match_capacity=3000)
     trims = harness.run_windowed_protocol(pair, tokens, lps, [2, 1, 3], steps=60, warm=6, keep=L // 2)
     assert trims >= G * N
+
+
+@pytest.mark.parametrize("eps", [0, 1])
+def test_step_with_backoff_in_one_launch(eps):
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, eps=eps)
+    assert pair.g.step_is_single_launch()
+    lens = (300 + (np.arange(w.P) * 37) % 400).astype(np.int32)
+    pair.append(tokens[:, :int(lens.max())], lps[:, :int(lens.max())], lens, expect_status=0)
+    pair.backoff_and_compare(w.k_max)
+    seen = set()
+    for step in range(20):
+        lens = pair.o.lengths()
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
+        tok, ln, _, _ = pair.o.drafts()
+        tau_o, st_o = pair.o.accept_commit(tok, ln, sampled, sampled_lp, pair.max_append)
+        used = np.zeros(w.P, np.int32)                      # oracle: fixed-k builds composed per path
+        for i in range(w.P):
+            for k in range(w.k_max, 0, -1):
+                pair.o.build_path(k, i)
+                if len(pair.o.matches(i)) > 0:
+                    used[i] = k
+                    break
+        tau_g, gt, gl, gk = pair.g.step_backoff(w.k_max, harness.t32(sampled, pair.dev), harness.t32(sampled_lp, pair.dev))
+        assert pair.g.status() == st_o
+        tok, ln, sc, _ = pair.o.drafts()
+        assert np.array_equal(tau_g.cpu().numpy(), tau_o)
+        assert np.array_equal(gk.cpu().numpy(), used)
+        assert np.array_equal(gl.cpu().numpy(), ln) and np.array_equal(gt.cpu().numpy(), tok)
+        np.testing.assert_allclose(pair.g.draft_score.cpu().numpy(), sc, rtol=harness.RTOL, atol=0)
+        seen |= set(used.tolist())
+    assert len(seen) >= 3
+    pair.check_history()

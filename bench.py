@@ -486,12 +486,19 @@ def ours_main(args, w):
     ablation = None
     if world == 1 and not args.no_fuzzy:
         ablation = {"dag": plan["accept_length"]}
+        variant_us = {}
         if fuzzy is not None:
             ablation["dag_fuzzy"] = fplan["accept_length"]
         for name, pool, eps, mode in (("tree", 1, 0, 0), ("list", 2, 0, 0), ("tree_fuzzy", 1, 1, 0), ("list_fuzzy", 2, 1, 0),
                                       ("dag_best_path", 0, 0, 2), ("dag_best_path_fuzzy", 0, 1, 2)):
             arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool, mode=mode)
             ablation[name] = arun.dry_run(allow_status=0x40)["accept_length"]
+            if eps == 0:                 # step time of the variant, measured like the headline
+                arun.timed_steps(20)
+                n_v = min(args.steps, 500)
+                vms, _ = arun.timed_steps(n_v)
+                variant_us[name] = 1e3 * vms / n_v
+                arun.s.status()          # clears the best-path fallback bit
             del arun
         # suffix length with back-off: every step asks for k_max, each path uses the longest k that has a match
         brun = Runner(w, rank_seed(w, rank), device, 0, 0, backoff=True)
@@ -571,6 +578,7 @@ def ours_main(args, w):
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
         "scan_queries_per_step": plan["scan_queries_per_step"], "run_steps": plan["steps"], "us_per_step_by_k": by_k,
         "fuzzy_epsilon_1": fuzzy, "synthetic_accept_length": ablation,
+        "variant_us_per_step": None if ablation is None else variant_us,
         "backoff_from_k_max": None if ablation is None else backoff,
         "sliding_window": None if ablation is None else {"us_per_sdms_trim_call": trim_us,
                                                           "what": "all paths full, trimmed to their newer half"},

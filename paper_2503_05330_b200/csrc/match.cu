@@ -122,62 +122,65 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 }
 
 constexpr int kLastBits = 32768;       // a prompt has up to 1024 scan queries: the reject test must stay selective
-constexpr int kScanBuf = 1536;         // matches a scanning CTA collects before it hands them over
+constexpr unsigned FULL_MASK = 0xffffffffu;
+constexpr int kWarpBuf = 96;           // matches a warp of a scanning CTA collects before it hands them over
 __device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 17; }
 __device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 17; }
 static_assert(kLastBits == 1 << 15, "last_bit yields 15 bits");
+static_assert(kScanTile == 4 * kScanThreads, "a thread looks at the four tokens it fetched");
 
-// The tokens a thread fetches of tile T of prompt g (tiles are numbered path-major): four consecutive
-// ones, plus one of the sixteen before the tile.  Nothing is fetched beyond the path's length.
-struct TileRegs { int32_t t[4]; int32_t halo; };
+// The four consecutive tokens a thread fetches of tile `tile` of path jn of prompt g.  Nothing is
+// fetched beyond the path's length (-1 stands for "no token").
+struct TileRegs { int32_t t[4]; };
 __device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int jn, int tile, const int32_t* len_of) {
   TileRegs r;
-  r.t[0] = r.t[1] = r.t[2] = r.t[3] = -1; r.halo = -1;
+  r.t[0] = r.t[1] = r.t[2] = r.t[3] = -1;
   if (jn >= s.N) return r;
-  const int j = g * s.N + jn, t0 = tile * kScanTile;
-  const int len = len_of[jn];
-  const int32_t* row = s.tok + (size_t)j * s.L;
-  const int x = t0 + 4 * (int)threadIdx.x;
-  if (x < len) {
+  const int32_t* row = s.tok + (size_t)(g * s.N + jn) * s.L;
+  const int x = tile * kScanTile + 4 * (int)threadIdx.x;
+  if (x < len_of[jn]) {
     if ((s.L & 3) == 0) {
-      const int4 q = __ldg(reinterpret_cast<const int4*>(row + x));     // may run past len inside the row: unused there
+      const int4 q = __ldg(reinterpret_cast<const int4*>(row + x));     // may run past the length inside the row: unused there
       r.t[0] = q.x; r.t[1] = q.y; r.t[2] = q.z; r.t[3] = q.w;
     } else {
 #pragma unroll
       for (int u = 0; u < 4; ++u) if (x + u < s.L) r.t[u] = __ldg(row + x + u);
     }
   }
-  if (threadIdx.x < kHalo && t0 < len) {
-    const int idx = t0 - kHalo + (int)threadIdx.x;
-    if (idx >= 0) r.halo = __ldg(row + idx);
-  }
   return r;
 }
 
 // CTA c of prompt g (blockIdx.x = g * ctas + c) walks tiles c, c + ctas, ... of that prompt (all paths of the
-// prompt, tile after tile).  The set of the prompt's scan queries is built once per CTA; the next
-// tile is already on its way from memory while the current one is searched.  With as many CTAs as
-// tiles this is one tile per CTA (small prompts: shortest latency); with fewer it streams.
+// prompt, tile after tile).  The set of the prompt's scan queries is built once per CTA.  After that
+// the warps run on their own, without CTA barriers: a thread filters the four tokens it fetched in
+// registers (two hashed bits of the set of the queries' last tokens) while the next tile is already on
+// its way; only a token that passes reads its window, from memory that is in cache by then.  Matches
+// go to a small buffer per warp that the warp hands over itself.  With as many CTAs as tiles this is
+// one tile per CTA (small prompts: shortest latency); with fewer it streams.
 __global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int ctas, int set_slots) {
   grid_wait();
   grid_release();
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
   if (s.g_nscan[g] == 0) return;
   const int ntiles = (s.L + kScanTile - 1) / kScanTile, total = s.N * ntiles;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-  __shared__ __align__(16) int32_t sh_tok[kHalo + kScanTile];
-  // per-query arrays and the query set are sized by this prompt's N (dynamic shared memory), not by the
-  // largest N the library takes: more CTAs fit an SM
+  // per-query arrays and the query set are sized by this prompt's N (dynamic shared memory)
   extern __shared__ __align__(16) int32_t scan_dyn[];
   int32_t* const sh_qid = scan_dyn;
   uint32_t* const sh_qfp = reinterpret_cast<uint32_t*>(scan_dyn + s.N);
-  int32_t* const sh_cnt = scan_dyn + 2 * s.N;
-  int32_t* const sh_base = scan_dyn + 3 * s.N;
-  int32_t* const sh_len = scan_dyn + 4 * s.N;
-  int32_t* const sh_set = scan_dyn + 5 * s.N;      // set_slots entries, a power of two >= 2 N
-  __shared__ uint32_t sh_last[kLastBits / 32];   // which last tokens (hashed to 15 bits) any scan query ends in
+  int32_t* const sh_len = scan_dyn + 2 * s.N;
+  int32_t* const sh_set = scan_dyn + 3 * s.N;      // set_slots entries, a power of two >= 2 N
+  __shared__ uint32_t sh_last[kLastBits / 32];     // which last tokens (hashed to 15 bits, twice) any scan query ends in
+  __shared__ uint16_t sh_wq[kScanThreads / 32][kWarpBuf];   // per warp: query slot of a collected match
+  __shared__ int32_t sh_wpos[kScanThreads / 32][kWarpBuf];  // ... and its position j * L + e
+  __shared__ int sh_wn[kScanThreads / 32];
   __shared__ int sh_nq;
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
+  if (threadIdx.x == 0) sh_nq = 0;
+  if (threadIdx.x < kScanThreads / 32) sh_wn[threadIdx.x] = 0;
+  for (int x = threadIdx.x; x < set_slots; x += blockDim.x) sh_set[x] = -1;
+  for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
   __syncthreads();
   // (path, tile) of the CTA's current tile and of the one after it; they advance by `ctas` tiles without a division
   const int step_j = ctas / ntiles, step_t = ctas - step_j * ntiles;
@@ -185,10 +188,6 @@ __global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int
   int jn_next = jn + step_j, tile_next = tile + step_t;
   if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
   TileRegs regs = fetch_tile(s, g, jn, tile, sh_len);                 // in flight during the set-up
-  if (threadIdx.x == 0) sh_nq = 0;
-  for (int x = threadIdx.x; x < set_slots; x += blockDim.x) sh_set[x] = -1;
-  for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
-  __syncthreads();
   // the prompt's scan queries
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) {
     const int i = g * s.N + n;
@@ -197,133 +196,93 @@ __global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int
       const uint32_t fp = s.q_fp[i];
       sh_qid[sl] = i;
       sh_qfp[sl] = fp;
-      sh_cnt[sl] = 0;
       uint32_t hs = (fp >> 1) & (set_slots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (set_slots - 1);
-      const int32_t* rec = s.rec + (size_t)i * kRecWords;             // rec[1 + t] = token t places from the end
-      const uint32_t lb = last_bit(rec[1]), lb2 = last_bit2(rec[1]);   // two bits per query token: few false alarms
+      const int32_t last = s.rec[(size_t)i * kRecWords + 1];
+      const uint32_t lb = last_bit(last), lb2 = last_bit2(last);      // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
       atomicOr(&sh_last[lb2 >> 5], 1u << (lb2 & 31));
     }
   }
   __syncthreads();
-  const int nq = sh_nq;
-  if (nq == 0) return;
+  if (sh_nq == 0) return;
+  // from here on no CTA barrier: every warp goes through the same tiles at its own pace
 
-  // Matches are collected in shared memory over many tiles and handed to the match lists in one go:
-  // a tile then costs two barriers and no round trip to memory.
-  __shared__ uint16_t sh_bq[kScanBuf];             // query slot of a collected match
-  __shared__ int32_t sh_bpos[kScanBuf];            // its position j * L + e
-  __shared__ int sh_nbuf, sh_over;
-  if (threadIdx.x == 0) { sh_nbuf = 0; sh_over = 0; }
-  __syncthreads();
-
-  // hands the collected matches [0, n) over: count per query, reserve a range of each list, write
-  auto flush = [&](int n) {
-    for (int x = threadIdx.x; x < n; x += blockDim.x) atomicAdd(&sh_cnt[sh_bq[x]], 1);
-    __syncthreads();
-    for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
-      const int c = sh_cnt[sl];
-      sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
-      sh_cnt[sl] = 0;
-    }
-    __syncthreads();
-    for (int x = threadIdx.x; x < n; x += blockDim.x) {
-      const int sl = sh_bq[x], i = sh_qid[sl];
-      const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
-      if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = sh_bpos[x];
-      else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
-    }
-    __syncthreads();
-    for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) sh_cnt[sl] = 0;
-    if (threadIdx.x == 0) sh_nbuf = 0;
-    __syncthreads();
+  // one entry of the match list of query slot sl (the list's cursor is bumped by one)
+  auto emit = [&](int sl, int pos) {
+    const int i = sh_qid[sl];
+    const int at = atomicAdd(&s.q_cursor[i], 1);
+    if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = pos;
+    else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
   };
-
-  // Calls visit(slot of the query, position e) for every match of the tile at position e = t0 + r * kScanThreads + tid.
-  auto matches_at = [&](int j, int t0, int e, auto visit) {
-    const int32_t* w = sh_tok + kHalo + (e - t0) - (k - 1);
-    const uint32_t lb = last_bit(w[k - 1]);
-    if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) return;           // no query ends in this token: nothing to hash
-    const uint32_t lb2 = last_bit2(w[k - 1]);
-    if (!(sh_last[lb2 >> 5] >> (lb2 & 31) & 1u)) return;
-    uint64_t h = gram_init(k);
-    for (int t = 0; t < k; ++t) h = gram_step(h, w[t]);
-    const uint32_t fp = gram_fp(gram_final(h));
-    uint32_t hs = (fp >> 1) & (set_slots - 1);
-    for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (set_slots - 1)) {
-      if (sh_qfp[sl] != fp) continue;
-      const int i = sh_qid[sl];
-      if (i == j) continue;                                       // a path never searches itself
-      const int32_t* rec = s.rec + (size_t)i * kRecWords;       // the query: rec[1 + t] = token t places from the end
-      bool same = true;
-      for (int t = 0; t < k; ++t) same = same && (w[t] == __ldg(rec + k - t));
-      if (same) visit(sl);
+  // the warp hands its collected matches over; lanes with the same query share one bump of its cursor
+  auto flush_warp = [&]() {
+    __syncwarp();
+    const int n = min(sh_wn[warp], kWarpBuf);
+    for (int x0 = 0; x0 < n; x0 += 32) {
+      const int x = x0 + lane;
+      const bool on = x < n;
+      const int sl = on ? sh_wq[warp][x] : -1 - lane;
+      const unsigned same = __match_any_sync(FULL_MASK, sl);
+      const int leader = __ffs(same) - 1;
+      int base = 0;
+      if (on && lane == leader) base = atomicAdd(&s.q_cursor[sh_qid[sl]], __popc(same));
+      base = __shfl_sync(FULL_MASK, base, leader);
+      if (on) {
+        const int i = sh_qid[sl];
+        const int at = base + __popc(same & ((1u << lane) - 1u));
+        if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = sh_wpos[warp][x];
+        else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+      }
     }
+    __syncwarp();
+    if (lane == 0) sh_wn[warp] = 0;
+    __syncwarp();
   };
-  constexpr int kPer = kScanTile / kScanThreads;
 
   for (int T = first; T < total; T += ctas) {
     const int j = g * s.N + jn, t0 = tile * kScanTile;
     const int e_lo = max(t0, k - 1);
     const int e_hi = min(t0 + kScanTile - 1, sh_len[jn] - 2);   // inclusive; needs one follower
-    const int held = sh_nbuf;                                    // (a barrier lies between this and the last change)
-    // the tile lands in shared memory; the next one is asked for before this one is looked at
-    *reinterpret_cast<int4*>(sh_tok + kHalo + 4 * threadIdx.x) = make_int4(regs.t[0], regs.t[1], regs.t[2], regs.t[3]);
-    if (threadIdx.x < kHalo) sh_tok[threadIdx.x] = regs.halo;
-    __syncthreads();
-    regs = fetch_tile(s, g, jn_next, tile_next, sh_len);
+    const int32_t* row = s.tok + (size_t)j * s.L;
+    const TileRegs cur = regs;
+    regs = fetch_tile(s, g, jn_next, tile_next, sh_len);         // the next tile is asked for before this one is looked at
     jn = jn_next; tile = tile_next;
     jn_next += step_j; tile_next += step_t;
     if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
-    if (e_lo <= e_hi) {
 #pragma unroll
-      for (int r = 0; r < kPer; ++r) {
-        const int e = t0 + r * kScanThreads + threadIdx.x;
-        if (e < e_lo || e > e_hi) continue;
-        matches_at(j, t0, e, [&](int sl) {
-          const int at = atomicAdd(&sh_nbuf, 1);
-          if (at < kScanBuf) { sh_bq[at] = (uint16_t)sl; sh_bpos[at] = j * s.L + e; }
-          else sh_over = 1;
-        });
+    for (int u = 0; u < 4; ++u) {
+      const int e = t0 + 4 * (int)threadIdx.x + u;
+      if (e < e_lo || e > e_hi) continue;
+      const int32_t tok = cur.t[u];
+      const uint32_t lb = last_bit(tok);
+      if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) continue;       // no query ends in this token: nothing to hash
+      const uint32_t lb2 = last_bit2(tok);
+      if (!(sh_last[lb2 >> 5] >> (lb2 & 31) & 1u)) continue;
+      // the window that ends at e (its tokens are in cache: this thread or its neighbours just fetched them)
+      const int32_t* w = row + e - (k - 1);
+      uint64_t h = gram_init(k);
+      for (int t = 0; t < k - 1; ++t) h = gram_step(h, __ldg(w + t));
+      h = gram_step(h, tok);
+      const uint32_t fp = gram_fp(gram_final(h));
+      uint32_t hs = (fp >> 1) & (set_slots - 1);
+      for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (set_slots - 1)) {
+        if (sh_qfp[sl] != fp) continue;
+        const int i = sh_qid[sl];
+        if (i == j) continue;                                     // a path never searches itself
+        const int32_t* rec = s.rec + (size_t)i * kRecWords;       // the query: rec[1 + t] = token t places from the end
+        bool same = true;
+        for (int t = 0; t < k; ++t) same = same && (__ldg(w + t) == __ldg(rec + k - t));
+        if (!same) continue;
+        const int at = atomicAdd(&sh_wn[warp], 1);
+        if (at < kWarpBuf) { sh_wq[warp][at] = (uint16_t)sl; sh_wpos[warp][at] = j * s.L + e; }
+        else emit(sl, j * s.L + e);                               // the buffer is full: straight to the list
       }
     }
-    __syncthreads();
-    if (sh_over) {
-      // (same for the whole CTA) this tile's matches did not fit: hand over what was there before the
-      // tile, then take the tile again with exact counts, straight into the match lists
-      flush(held);
-      if (threadIdx.x == 0) sh_over = 0;
-#pragma unroll
-      for (int r = 0; r < kPer; ++r) {
-        const int e = t0 + r * kScanThreads + threadIdx.x;
-        if (e >= e_lo && e <= e_hi) matches_at(j, t0, e, [&](int sl) { atomicAdd(&sh_cnt[sl], 1); });
-      }
-      __syncthreads();
-      for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) {
-        const int c = sh_cnt[sl];
-        sh_base[sl] = c ? atomicAdd(&s.q_cursor[sh_qid[sl]], c) : 0;
-        sh_cnt[sl] = 0;
-      }
-      __syncthreads();
-#pragma unroll
-      for (int r = 0; r < kPer; ++r) {
-        const int e = t0 + r * kScanThreads + threadIdx.x;
-        if (e >= e_lo && e <= e_hi) matches_at(j, t0, e, [&](int sl) {
-          const int i = sh_qid[sl];
-          const int at = sh_base[sl] + atomicAdd(&sh_cnt[sl], 1);
-          if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = j * s.L + e;
-          else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
-        });
-      }
-      __syncthreads();
-      for (int sl = threadIdx.x; sl < nq; sl += blockDim.x) sh_cnt[sl] = 0;
-      __syncthreads();
-    } else if (sh_nbuf > kScanBuf / 2) {
-      flush(sh_nbuf);
-    }
+    __syncwarp();
+    if (sh_wn[warp] > kWarpBuf / 2) flush_warp();                 // same for the whole warp
   }
-  flush(sh_nbuf);
+  flush_warp();
 }
 
 // Inspection only: packs the per-query slices of the match list.
@@ -368,7 +327,7 @@ cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   if ((long long)s.G * per_prompt > budget) ctas = std::max(1LL, std::min(per_prompt, budget / s.G));
   int set_slots = 64;
   while (set_slots < 2 * s.N) set_slots *= 2;
-  const size_t dyn = ((size_t)5 * s.N + set_slots) * 4;
+  const size_t dyn = ((size_t)3 * s.N + set_slots) * 4;
   return launch_overlapped(scan_kernel, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), dyn, stream, s, k, (int)ctas,
                            set_slots);
 }

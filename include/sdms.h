@@ -52,6 +52,7 @@ extern "C" {
 #define SDMS_STATUS_MATCH_OVERFLOW 0x20u /* match workspace exhausted: the affected paths get draft_len 0 */
 #define SDMS_STATUS_SEARCH_FALLBACK 0x40u /* search_mode 2: a path had too many matches for the best-path tables
                                             (more than about 24576 / (11 * max_draft_len)); it got the greedy draft */
+#define SDMS_STATUS_TIMEOUT        0x80u /* a bounded wait inside a kernel ran out (never expected): the build's matches are incomplete */
 
 #define SDMS_MAX_K      16   /* largest supported k_max           */
 #define SDMS_MAX_DRAFT  32   /* largest supported max_draft_len   */

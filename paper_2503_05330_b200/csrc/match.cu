@@ -7,13 +7,15 @@
 //                Up to kInlineSlots occurrences are stored in the bucket itself:
 //                such queries are answered here, from one 32-byte sector.  The
 //                others are handed to the scan.
-// scan_kernel  : one CTA per 1024-token tile of one path.  The tile is staged in
-//                shared memory with 128-bit loads; the fingerprints of the
-//                prompt's scan queries sit in a small shared hash set; every
-//                position hashes its k-gram, probes the set and verifies hits
-//                token by token.  Matches are counted per query in shared
-//                memory, one global atomic per (CTA, query) reserves the output
-//                range, and a second pass writes the positions.
+// scan_kernel  : the histories of a prompt are read once, in tiles, for all of
+//                its scan queries together.  A token is first tested against a
+//                bit table of the queries' last tokens; the few positions that
+//                pass are queued per warp and looked at 32 at a time (window
+//                hash, probe of the prompt's query set, verification token by
+//                token).  Small prompts: one CTA per 1024-token tile, tokens
+//                fetched with 128-bit loads.  Stores of many tiles: each CTA
+//                streams 2048-token tiles through shared-memory stages filled
+//                by bulk copies.
 #include "sdms_internal.h"
 #include <algorithm>
 
@@ -121,12 +123,16 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
   }
 }
 
-constexpr int kLastBits = 32768;       // a prompt has up to 1024 scan queries: the reject test must stay selective
+// Reject test on a position's own token: one bit in each of two tables, set for the last token of every
+// scan query of the prompt (up to 1024 of them).  The first table is looked at for every token, the
+// second only for the few that pass the first.
+constexpr int kLastBits = 65536;
+constexpr int kLast2Bits = 32768;
 constexpr unsigned FULL_MASK = 0xffffffffu;
-constexpr int kWarpBuf = 96;           // matches a warp of a scanning CTA collects before it hands them over
-__device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 17; }
+constexpr int kCandBuf = 64;           // entries a warp may have waiting: fewer than 32 left over plus one per lane
+__device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 16; }
 __device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 17; }
-static_assert(kLastBits == 1 << 15, "last_bit yields 15 bits");
+static_assert(kLastBits == 1 << 16 && kLast2Bits == 1 << 15, "last_bit yields 16 bits, last_bit2 15");
 static_assert(kScanTile == 4 * kScanThreads, "a thread looks at the four tokens it fetched");
 
 // The four consecutive tokens a thread fetches of tile `tile` of path jn of prompt g.  Nothing is
@@ -150,44 +156,126 @@ __device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int jn, int 
   return r;
 }
 
+// ---- bulk-copy staging for the streaming form of the scan -------------------------------------
+// A CTA that walks many tiles keeps kStreamStages of them in flight as bulk copies (the copy engine
+// writes a whole 4 KB tile into shared memory and signals an mbarrier), so the bytes in flight do not
+// depend on registers or on how many warps are resident.
+constexpr int kStreamStages = 4;
+constexpr int kStreamTile = 2 * kScanTile;           // tokens per stage: a thread takes eight of them
+constexpr int kStreamThreads = kScanThreads + 32;   // eight scanning warps and one warp that issues the copies
+constexpr long long kWaitCycles = 4000000000LL;      // about two seconds: a wait that long has failed
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Waits for the phase with the given parity to complete; gives up after kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity))
+    if (clock64() - t0 > kWaitCycles) return false;
+  return true;
+}
+// bytes (a multiple of 16, both addresses 16-byte aligned) from global to this CTA's shared memory
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
 // CTA c of prompt g (blockIdx.x = g * ctas + c) walks tiles c, c + ctas, ... of that prompt (all paths of the
 // prompt, tile after tile).  The set of the prompt's scan queries is built once per CTA.  After that
-// the warps run on their own, without CTA barriers: a thread filters the four tokens it fetched in
-// registers (two hashed bits of the set of the queries' last tokens) while the next tile is already on
-// its way; only a token that passes reads its window, from memory that is in cache by then.  Matches
-// go to a small buffer per warp that the warp hands over itself.  With as many CTAs as tiles this is
-// one tile per CTA (small prompts: shortest latency); with fewer it streams.
-__global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int ctas, int set_slots) {
+// the warps run on their own, without CTA barriers.  A thread tests the four tokens it holds of the
+// tile against the first reject table, without a branch in between.  Positions that pass are not looked
+// at there and then, by one or two lanes with the rest of the warp idle: the warp queues them in shared
+// memory, and once 32 are waiting every lane takes one (second reject table, hash of the window, probe
+// of the query set, token-by-token verification).  Lanes whose positions match the same query share one
+// bump of that query's cursor in the match list.
+// STREAM = false: a thread fetches its four tokens itself, one tile ahead.  With as many CTAs as tiles
+// this is one tile per CTA (small prompts: shortest latency).
+// STREAM = true : a ninth warp keeps kStreamStages tiles in flight as bulk copies into shared memory
+// (full / empty mbarrier per stage); a scanning warp takes its tokens out of the stage and gives the
+// stage back at once.  Needs rows that start and end on 16-byte boundaries (L a multiple of 4).
+template <bool STREAM>
+__global__ void __launch_bounds__(STREAM ? kStreamThreads : kScanThreads, STREAM ? 4 : 6)
+scan_kernel(Dev s, int k, int ctas, int set_slots) {
   grid_wait();
   grid_release();
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
   if (s.g_nscan[g] == 0) return;
-  const int ntiles = (s.L + kScanTile - 1) / kScanTile, total = s.N * ntiles;
+  constexpr int TILE = STREAM ? kStreamTile : kScanTile;
+  const int ntiles = (s.L + TILE - 1) / TILE, total = s.N * ntiles;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool scanner = !STREAM || warp < kScanThreads / 32;
 
   // per-query arrays and the query set are sized by this prompt's N (dynamic shared memory)
-  extern __shared__ __align__(16) int32_t scan_dyn[];
-  int32_t* const sh_qid = scan_dyn;
-  uint32_t* const sh_qfp = reinterpret_cast<uint32_t*>(scan_dyn + s.N);
-  int32_t* const sh_len = scan_dyn + 2 * s.N;
-  int32_t* const sh_set = scan_dyn + 3 * s.N;      // set_slots entries, a power of two >= 2 N
-  __shared__ uint32_t sh_last[kLastBits / 32];     // which last tokens (hashed to 15 bits, twice) any scan query ends in
-  __shared__ uint16_t sh_wq[kScanThreads / 32][kWarpBuf];   // per warp: query slot of a collected match
-  __shared__ int32_t sh_wpos[kScanThreads / 32][kWarpBuf];  // ... and its position j * L + e
-  __shared__ int sh_wn[kScanThreads / 32];
+  extern __shared__ __align__(128) int32_t scan_dyn[];
+  int32_t* const sh_stage = scan_dyn;                                 // STREAM: kStreamStages tiles
+  int32_t* const sh_qid = scan_dyn + (STREAM ? kStreamStages * kStreamTile : 0);
+  uint32_t* const sh_qfp = reinterpret_cast<uint32_t*>(sh_qid + s.N);
+  int32_t* const sh_len = sh_qid + 2 * s.N;
+  int32_t* const sh_set = sh_qid + 3 * s.N;       // set_slots entries, a power of two >= 4 N
+  __shared__ uint32_t sh_last[kLastBits / 32];     // which last tokens (hashed to 16 bits) any scan query ends in
+  __shared__ uint32_t sh_last2[kLast2Bits / 32];   // the same under a second hash (15 bits)
+  __shared__ int2 sh_cand[kScanThreads / 32][kCandBuf];     // per warp: waiting (jn * L + e of a thread's first token, which of its four or eight)
   __shared__ int sh_nq;
+  __shared__ __align__(8) uint64_t sh_full[kStreamStages], sh_empty[kStreamStages];
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   if (threadIdx.x == 0) sh_nq = 0;
-  if (threadIdx.x < kScanThreads / 32) sh_wn[threadIdx.x] = 0;
   for (int x = threadIdx.x; x < set_slots; x += blockDim.x) sh_set[x] = -1;
   for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
+  for (int x = threadIdx.x; x < kLast2Bits / 32; x += blockDim.x) sh_last2[x] = 0u;
+  if (STREAM && threadIdx.x == kScanThreads) {
+    for (int st = 0; st < kStreamStages; ++st) { mbar_init(&sh_full[st], 1); mbar_init(&sh_empty[st], kScanThreads / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   __syncthreads();
   // (path, tile) of the CTA's current tile and of the one after it; they advance by `ctas` tiles without a division
   const int step_j = ctas / ntiles, step_t = ctas - step_j * ntiles;
   int jn = first / ntiles, tile = first - jn * ntiles;
   int jn_next = jn + step_j, tile_next = tile + step_t;
   if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
-  TileRegs regs = fetch_tile(s, g, jn, tile, sh_len);                 // in flight during the set-up
+
+  // STREAM: the issuing thread's own walk over the CTA's tiles.  A tile of a path that is shorter than
+  // the tile's start is not copied; its barrier still completes, so that the phases stay in step.
+  int pj = jn, ptile = tile, pT = first, pstage = 0;
+  auto issue_tile = [&]() {
+    const int t0 = ptile * TILE;
+    const int have = sh_len[pj] - t0;                                 // tokens of this path from t0 on
+    if (have > 0) {
+      const uint32_t bytes = 4u * (uint32_t)min(TILE, min(s.L - t0, (have + 3) & ~3));
+      mbar_arrive_expect(&sh_full[pstage], bytes);
+      bulk_load(sh_stage + pstage * TILE, s.tok + (size_t)(g * s.N + pj) * s.L + t0, bytes, &sh_full[pstage]);
+    } else {
+      mbar_arrive(&sh_full[pstage]);
+    }
+    pT += ctas; pj += step_j; ptile += step_t;
+    if (ptile >= ntiles) { ptile -= ntiles; ++pj; }
+    if (++pstage == kStreamStages) pstage = 0;
+  };
+  int issued = 0;
+  TileRegs regs;
+  if (STREAM) {
+    if (threadIdx.x == kScanThreads)
+      for (; issued < kStreamStages && pT < total; ++issued) issue_tile();   // in flight during the set-up
+  } else {
+    regs = fetch_tile(s, g, jn, tile, sh_len);                        // in flight during the set-up
+  }
   // the prompt's scan queries
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) {
     const int i = g * s.N + n;
@@ -201,88 +289,139 @@ __global__ void __launch_bounds__(kScanThreads, 6) scan_kernel(Dev s, int k, int
       const int32_t last = s.rec[(size_t)i * kRecWords + 1];
       const uint32_t lb = last_bit(last), lb2 = last_bit2(last);      // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
-      atomicOr(&sh_last[lb2 >> 5], 1u << (lb2 & 31));
+      atomicOr(&sh_last2[lb2 >> 5], 1u << (lb2 & 31));
     }
   }
   __syncthreads();
-  if (sh_nq == 0) return;
+  if (!STREAM && sh_nq == 0) return;
   // from here on no CTA barrier: every warp goes through the same tiles at its own pace
 
-  // one entry of the match list of query slot sl (the list's cursor is bumped by one)
-  auto emit = [&](int sl, int pos) {
-    const int i = sh_qid[sl];
-    const int at = atomicAdd(&s.q_cursor[i], 1);
-    if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = pos;
-    else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
-  };
-  // the warp hands its collected matches over; lanes with the same query share one bump of its cursor
-  auto flush_warp = [&]() {
-    __syncwarp();
-    const int n = min(sh_wn[warp], kWarpBuf);
-    for (int x0 = 0; x0 < n; x0 += 32) {
-      const int x = x0 + lane;
-      const bool on = x < n;
-      const int sl = on ? sh_wq[warp][x] : -1 - lane;
-      const unsigned same = __match_any_sync(FULL_MASK, sl);
-      const int leader = __ffs(same) - 1;
-      int base = 0;
-      if (on && lane == leader) base = atomicAdd(&s.q_cursor[sh_qid[sl]], __popc(same));
-      base = __shfl_sync(FULL_MASK, base, leader);
-      if (on) {
-        const int i = sh_qid[sl];
-        const int at = base + __popc(same & ((1u << lane) - 1u));
-        if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = sh_wpos[warp][x];
-        else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
-      }
+  if (STREAM && !scanner) {
+    // the issuing warp: one thread refills a stage as soon as all scanning warps have given it back
+    if (lane != 0) return;
+    uint32_t round = 0;                                               // how often the stages have been refilled
+    for (int st = 0; pT < total; ++issued) {
+      if (!mbar_wait(&sh_empty[st], round & 1u)) { atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
+      issue_tile();
+      if (++st == kStreamStages) { st = 0; ++round; }
     }
+    return;
+  }
+
+  // The warp looks at waiting entries, 32 at a time (newest first), until fewer than 32 are left; with
+  // `all` set, until none is left.  cn is the same in every lane.  An entry names up to four positions;
+  // whether a position can end a match at all (k - 1 <= e <= len - 2) is decided here, not in the filter.
+  int cn = 0;
+  const uint32_t lanes_below = (1u << lane) - 1u;
+  auto drain = [&](bool all) {
     __syncwarp();
-    if (lane == 0) sh_wn[warp] = 0;
-    __syncwarp();
+    while (cn >= 32 || (all && cn > 0)) {
+      const int take = min(32, cn);
+      cn -= take;
+      int2 ent = make_int2(0, 0);
+      if (lane < take) ent = sh_cand[warp][cn + lane];
+      const int jl = ent.x / s.L, e_first = ent.x - jl * s.L, j = g * s.N + jl;
+      const int e_last = sh_len[jl] - 2;
+      const int32_t* const row = s.tok + (size_t)j * s.L;
+      uint32_t todo = (uint32_t)ent.y;
+      while (__any_sync(FULL_MASK, todo != 0u)) {                  // one position of every lane's entry per round
+        const int u = __ffs(todo) - 1;                              // -1: this lane has none left
+        todo &= todo - 1u;
+        const int e = e_first + (u & 3) + (u >> 2) * kScanTile;   // bits 4..7: the thread's second four tokens
+        const bool on = u >= 0 && e >= k - 1 && e <= e_last;
+        const int32_t* w = row + e - (k - 1);                       // the window that ends at e
+        const int32_t tok = on ? __ldg(w + k - 1) : 0;
+        const uint32_t lb2 = last_bit2(tok);
+        bool live = on && (sh_last2[lb2 >> 5] >> (lb2 & 31) & 1u);
+        uint32_t fp = 0u, hs = 0u;
+        if (live) {
+          uint64_t h = gram_init(k);
+          for (int t = 0; t < k - 1; ++t) h = gram_step(h, __ldg(w + t));
+          h = gram_step(h, tok);
+          fp = gram_fp(gram_final(h));
+          hs = (fp >> 1) & (set_slots - 1);
+        }
+        while (__any_sync(FULL_MASK, live)) {                      // every lane walks its probe run
+          const int sl = live ? sh_set[hs] : -1;
+          live = live && sl != -1;
+          hs = (hs + 1) & (set_slots - 1);
+          int i = -1;
+          if (live && sh_qfp[sl] == fp) {
+            i = sh_qid[sl];
+            if (i == j) i = -1;                                    // a path never searches itself
+            if (i >= 0) {
+              const int32_t* rec = s.rec + (size_t)i * kRecWords; // the query: rec[1 + t] = token t places from the end
+              bool same = true;
+              for (int t = 0; t < k; ++t) same = same && (__ldg(w + t) == __ldg(rec + k - t));
+              if (!same) i = -1;
+            }
+          }
+          if (!__any_sync(FULL_MASK, i >= 0)) continue;
+          const unsigned same = __match_any_sync(FULL_MASK, i >= 0 ? i : -1 - lane);
+          const int leader = __ffs(same) - 1;
+          int base = 0;
+          if (i >= 0 && lane == leader) base = atomicAdd(&s.q_cursor[i], __popc(same));
+          base = __shfl_sync(FULL_MASK, base, leader);
+          if (i >= 0) {
+            const int at = base + __popc(same & lanes_below);
+            if (at < s.q_reserved[i]) s.matches[(size_t)s.q_off[i] + at] = j * s.L + e;
+            else atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+          }
+        }
+      }
+      __syncwarp();
+    }
   };
 
+  const int tid4 = 4 * (int)threadIdx.x;
+  int stage = 0;
+  uint32_t phase = 0;
   for (int T = first; T < total; T += ctas) {
-    const int j = g * s.N + jn, t0 = tile * kScanTile;
-    const int e_lo = max(t0, k - 1);
-    const int e_hi = min(t0 + kScanTile - 1, sh_len[jn] - 2);   // inclusive; needs one follower
-    const int32_t* row = s.tok + (size_t)j * s.L;
-    const TileRegs cur = regs;
-    regs = fetch_tile(s, g, jn_next, tile_next, sh_len);         // the next tile is asked for before this one is looked at
+    const int t0 = tile * TILE, jn_now = jn;
+    TileRegs cur, cur2;
+    if (STREAM) {
+      if (!__all_sync(FULL_MASK, mbar_wait(&sh_full[stage], phase))) {  // cannot happen; the warp leaves in an orderly way
+        atomicOr(s.status, SDMS_STATUS_TIMEOUT);
+        for (int it = 0; it < 100000; ++it) __nanosleep(1000);         // copies still in flight land in live shared memory
+        break;
+      }
+      const int4* const st4 = reinterpret_cast<const int4*>(sh_stage + stage * TILE);
+      const int4 q = st4[threadIdx.x], q2 = st4[kScanThreads + threadIdx.x];   // tokens e0..e0+3 and e0+1024..e0+1027
+      cur.t[0] = q.x; cur.t[1] = q.y; cur.t[2] = q.z; cur.t[3] = q.w;  // beyond the copied bytes: stale, turned down in drain()
+      cur2.t[0] = q2.x; cur2.t[1] = q2.y; cur2.t[2] = q2.z; cur2.t[3] = q2.w;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh_empty[stage]);                    // the warp has its tokens: the stage may be refilled
+      if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
+    } else {
+      cur = regs;
+      regs = fetch_tile(s, g, jn_next, tile_next, sh_len);       // the next tile is asked for before this one is looked at
+    }
     jn = jn_next; tile = tile_next;
     jn_next += step_j; tile_next += step_t;
     if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
+    if (t0 > sh_len[jn_now] - 2) continue;                        // nothing of the path in this tile (same for the whole CTA)
+    // first reject table for the four tokens, without a branch in between: almost always no bit is set
+    uint32_t hit = 0u;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int e = t0 + 4 * (int)threadIdx.x + u;
-      if (e < e_lo || e > e_hi) continue;
-      const int32_t tok = cur.t[u];
-      const uint32_t lb = last_bit(tok);
-      if (!(sh_last[lb >> 5] >> (lb & 31) & 1u)) continue;       // no query ends in this token: nothing to hash
-      const uint32_t lb2 = last_bit2(tok);
-      if (!(sh_last[lb2 >> 5] >> (lb2 & 31) & 1u)) continue;
-      // the window that ends at e (its tokens are in cache: this thread or its neighbours just fetched them)
-      const int32_t* w = row + e - (k - 1);
-      uint64_t h = gram_init(k);
-      for (int t = 0; t < k - 1; ++t) h = gram_step(h, __ldg(w + t));
-      h = gram_step(h, tok);
-      const uint32_t fp = gram_fp(gram_final(h));
-      uint32_t hs = (fp >> 1) & (set_slots - 1);
-      for (int sl; (sl = sh_set[hs]) != -1; hs = (hs + 1) & (set_slots - 1)) {
-        if (sh_qfp[sl] != fp) continue;
-        const int i = sh_qid[sl];
-        if (i == j) continue;                                     // a path never searches itself
-        const int32_t* rec = s.rec + (size_t)i * kRecWords;       // the query: rec[1 + t] = token t places from the end
-        bool same = true;
-        for (int t = 0; t < k; ++t) same = same && (__ldg(w + t) == __ldg(rec + k - t));
-        if (!same) continue;
-        const int at = atomicAdd(&sh_wn[warp], 1);
-        if (at < kWarpBuf) { sh_wq[warp][at] = (uint16_t)sl; sh_wpos[warp][at] = j * s.L + e; }
-        else emit(sl, j * s.L + e);                               // the buffer is full: straight to the list
+      const uint32_t lb = last_bit(cur.t[u]);
+      hit |= (sh_last[lb >> 5] >> (lb & 31) & 1u) << u;
+    }
+    if (STREAM) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t lb = last_bit(cur2.t[u]);
+        hit |= (sh_last[lb >> 5] >> (lb & 31) & 1u) << (4 + u);
       }
     }
-    __syncwarp();
-    if (sh_wn[warp] > kWarpBuf / 2) flush_warp();                 // same for the whole warp
+    const unsigned b = __ballot_sync(FULL_MASK, hit != 0u);
+    if (b) {                                                      // queue what passed
+      if (hit) sh_cand[warp][cn + __popc(b & lanes_below)] = make_int2(jn_now * s.L + t0 + tid4, (int)hit);
+      cn += __popc(b);
+      if (cn >= 32) drain(false);
+    }
   }
-  flush_warp();
+  drain(true);
 }
 
 // Inspection only: packs the per-query slices of the match list.
@@ -322,13 +461,30 @@ cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   // one CTA per tile while that keeps the device busy for one round; beyond that each CTA streams
   // through its share of its prompt's tiles
   const long long per_prompt = (long long)s.N * ((s.L + kScanTile - 1) / kScanTile);
+  int set_slots = 64;
+  while (set_slots < 4 * s.N) set_slots *= 2;
+  const size_t dyn = ((size_t)3 * s.N + set_slots) * 4;
+  if ((long long)s.G * per_prompt > 148LL * 8 * 4 && (s.L & 3) == 0) {
+    // streaming form: every CTA resident at once, each with kStreamStages tiles in flight
+    static int per_sm = 0;
+    const size_t dyn_stream = dyn + (size_t)kStreamStages * kStreamTile * 4;
+    const long long per_prompt_s = (long long)s.N * ((s.L + kStreamTile - 1) / kStreamTile);
+    if (per_sm == 0) {
+      cudaError_t e = cudaFuncSetAttribute(scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+      if (e != cudaSuccess) return e;
+      per_sm = 4;
+    }
+    if (dyn_stream <= 96 * 1024) {
+      const long long tot = 148LL * per_sm * 4;                        // four rounds of resident CTAs: set-ups overlap other CTAs' streaming
+      const long long ctas = std::max(1LL, std::min(per_prompt_s, tot / s.G));
+      return launch_overlapped(scan_kernel<true>, dim3((unsigned)(ctas * s.G)), dim3(kStreamThreads), dyn_stream, stream, s,
+                               k, (int)ctas, set_slots);
+    }
+  }
   const long long budget = 148LL * 8 * 4;
   long long ctas = per_prompt;
   if ((long long)s.G * per_prompt > budget) ctas = std::max(1LL, std::min(per_prompt, budget / s.G));
-  int set_slots = 64;
-  while (set_slots < 2 * s.N) set_slots *= 2;
-  const size_t dyn = ((size_t)3 * s.N + set_slots) * 4;
-  return launch_overlapped(scan_kernel, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), dyn, stream, s, k, (int)ctas,
+  return launch_overlapped(scan_kernel<false>, dim3((unsigned)(ctas * s.G)), dim3(kScanThreads), dyn, stream, s, k, (int)ctas,
                            set_slots);
 }
 

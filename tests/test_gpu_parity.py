@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 from paper_2503_05330_b200 import synth  # noqa: E402
 import harness  # noqa: E402
-from harness import Pair, run_protocol  # noqa: E402
+from harness import Pair, run_protocol, t32  # noqa: E402
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -541,6 +541,26 @@ def test_tile_scan_with_more_matches_per_tile_than_its_buffer_holds():
     for k in (1, 2):
         pair.build_and_compare(k, check_dag=False)
     assert (pair.g.query_modes() == 2).all()
+
+
+def test_streaming_tile_scan_on_a_store_of_many_tiles():
+    # more 1024-token tiles than the one-tile-per-CTA form launches: the scan streams its tiles through
+    # shared-memory stages.  Ragged lengths: empty paths, paths that end inside their first tile, on a
+    # tile boundary and one token past it, lengths that are not multiples of four.
+    G, N, L, V, D = 5, 128, 8192, 300, 3
+    assert G * N * (L // 1024) > 148 * 8 * 4
+    tokens, lps = synth.small_random(G * N, L, V, 777)
+    pair = Pair(G, N, L, V, 2, D)
+    lens = (L - 8 - (np.arange(G * N) * 997) % 7000).astype(np.int32)
+    lens[[0, 5, 130, 131, 200, 300, 301, 639]] = [0, 3, 1024, 1025, 4098, 2047, 1, 8184]
+    for c in range(0, L - 8, 2048):                      # prefill in chunks
+        part = np.clip(lens - c, 0, 2048).astype(np.int32)
+        pair.g.append(t32(tokens[:, c:c + 2048], pair.dev), t32(lps[:, c:c + 2048], pair.dev), t32(part, pair.dev))
+        pair.o.append(tokens[:, c:c + 2048], lps[:, c:c + 2048], part)
+    assert pair.g.status() == 0
+    for k in (1, 2):
+        pair.build_and_compare(k, check_dag=False)
+        assert (pair.g.query_modes() == 2).sum() > G * N // 2
 
 
 @pytest.mark.parametrize("mode,pool", [(0, 0), (1, 0), (2, 0), (0, 1), (0, 2)])

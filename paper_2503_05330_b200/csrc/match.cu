@@ -127,12 +127,12 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 // scan query of the prompt (up to 1024 of them).  The first table is looked at for every token, the
 // second only for the few that pass the first.
 constexpr int kLastBits = 65536;
-constexpr int kLast2Bits = 32768;
+constexpr int kLast2Bits = 8192;
 constexpr unsigned FULL_MASK = 0xffffffffu;
 constexpr int kCandBuf = 64;           // entries a warp may have waiting: fewer than 32 left over plus one per lane
 __device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 16; }
-__device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 17; }
-static_assert(kLastBits == 1 << 16 && kLast2Bits == 1 << 15, "last_bit yields 16 bits, last_bit2 15");
+__device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 19; }
+static_assert(kLastBits == 1 << 16 && kLast2Bits == 1 << 13, "last_bit yields 16 bits, last_bit2 13");
 static_assert(kScanTile == 4 * kScanThreads, "a thread looks at the four tokens it fetched");
 
 // The four consecutive tokens a thread fetches of tile `tile` of path jn of prompt g.  Nothing is
@@ -209,8 +209,8 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 // STREAM = false: a thread fetches its four tokens itself, one tile ahead.  With as many CTAs as tiles
 // this is one tile per CTA (small prompts: shortest latency).
 // STREAM = true : a ninth warp keeps kStreamStages tiles in flight as bulk copies into shared memory
-// (full / empty mbarrier per stage); a scanning warp takes its tokens out of the stage and gives the
-// stage back at once.  Needs rows that start and end on 16-byte boundaries (L a multiple of 4).
+// (full / empty mbarrier per stage); a scanning thread takes its tokens out of the stage and gives its
+// share of the stage back at once.  Needs rows that start and end on 16-byte boundaries (L a multiple of 4).
 template <bool STREAM>
 __global__ void __launch_bounds__(STREAM ? kStreamThreads : kScanThreads, STREAM ? 4 : 6)
 scan_kernel(Dev s, int k, int ctas, int set_slots) {
@@ -229,19 +229,20 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
   int32_t* const sh_qid = scan_dyn + (STREAM ? kStreamStages * kStreamTile : 0);
   uint32_t* const sh_qfp = reinterpret_cast<uint32_t*>(sh_qid + s.N);
   int32_t* const sh_len = sh_qid + 2 * s.N;
-  int32_t* const sh_set = sh_qid + 3 * s.N;       // set_slots entries, a power of two >= 4 N
-  __shared__ uint32_t sh_last[kLastBits / 32];     // which last tokens (hashed to 16 bits) any scan query ends in
-  __shared__ uint32_t sh_last2[kLast2Bits / 32];   // the same under a second hash (15 bits)
+  int32_t* const sh_qlast = sh_qid + 3 * s.N;     // last token of the query in a slot
+  int32_t* const sh_set = sh_qid + 4 * s.N;       // set_slots entries, a power of two >= 4 N
+  __shared__ __align__(16) uint32_t sh_last[kLastBits / 32];     // which last tokens (hashed to 16 bits) any scan query ends in
+  __shared__ __align__(16) uint32_t sh_last2[kLast2Bits / 32];   // the same under a second hash (13 bits)
   __shared__ int2 sh_cand[kScanThreads / 32][kCandBuf];     // per warp: waiting (jn * L + e of a thread's first token, which of its four or eight)
   __shared__ int sh_nq;
   __shared__ __align__(8) uint64_t sh_full[kStreamStages], sh_empty[kStreamStages];
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = s.len[g * s.N + n];
   if (threadIdx.x == 0) sh_nq = 0;
   for (int x = threadIdx.x; x < set_slots; x += blockDim.x) sh_set[x] = -1;
-  for (int x = threadIdx.x; x < kLastBits / 32; x += blockDim.x) sh_last[x] = 0u;
-  for (int x = threadIdx.x; x < kLast2Bits / 32; x += blockDim.x) sh_last2[x] = 0u;
+  for (int x = threadIdx.x; x < kLastBits / 128; x += blockDim.x) reinterpret_cast<uint4*>(sh_last)[x] = make_uint4(0u, 0u, 0u, 0u);
+  for (int x = threadIdx.x; x < kLast2Bits / 128; x += blockDim.x) reinterpret_cast<uint4*>(sh_last2)[x] = make_uint4(0u, 0u, 0u, 0u);
   if (STREAM && threadIdx.x == kScanThreads) {
-    for (int st = 0; st < kStreamStages; ++st) { mbar_init(&sh_full[st], 1); mbar_init(&sh_empty[st], kScanThreads / 32); }
+    for (int st = 0; st < kStreamStages; ++st) { mbar_init(&sh_full[st], 1); mbar_init(&sh_empty[st], kScanThreads); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -287,6 +288,7 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
       uint32_t hs = (fp >> 1) & (set_slots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (set_slots - 1);
       const int32_t last = s.rec[(size_t)i * kRecWords + 1];
+      sh_qlast[sl] = last;
       const uint32_t lb = last_bit(last), lb2 = last_bit2(last);      // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));
       atomicOr(&sh_last2[lb2 >> 5], 1u << (lb2 & 31));
@@ -351,8 +353,8 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
             if (i == j) i = -1;                                    // a path never searches itself
             if (i >= 0) {
               const int32_t* rec = s.rec + (size_t)i * kRecWords; // the query: rec[1 + t] = token t places from the end
-              bool same = true;
-              for (int t = 0; t < k; ++t) same = same && (__ldg(w + t) == __ldg(rec + k - t));
+              bool same = tok == sh_qlast[sl];
+              for (int t = 0; t < k - 1; ++t) same = same && (__ldg(w + t) == __ldg(rec + k - t));
               if (!same) i = -1;
             }
           }
@@ -389,8 +391,7 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
       const int4 q = st4[threadIdx.x], q2 = st4[kScanThreads + threadIdx.x];   // tokens e0..e0+3 and e0+1024..e0+1027
       cur.t[0] = q.x; cur.t[1] = q.y; cur.t[2] = q.z; cur.t[3] = q.w;  // beyond the copied bytes: stale, turned down in drain()
       cur2.t[0] = q2.x; cur2.t[1] = q2.y; cur2.t[2] = q2.z; cur2.t[3] = q2.w;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh_empty[stage]);                    // the warp has its tokens: the stage may be refilled
+      mbar_arrive(&sh_empty[stage]);                                   // this thread has its tokens; when all have, the stage is refilled
       if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
     } else {
       cur = regs;
@@ -400,19 +401,27 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
     jn_next += step_j; tile_next += step_t;
     if (tile_next >= ntiles) { tile_next -= ntiles; ++jn_next; }
     if (t0 > sh_len[jn_now] - 2) continue;                        // nothing of the path in this tile (same for the whole CTA)
-    // first reject table for the four tokens, without a branch in between: almost always no bit is set
-    uint32_t hit = 0u;
+    // first reject table: bit 0 of w[u] says whether token u passes.  Almost always none does, so the
+    // words are only OR-ed together; the exact mask is worked out for the few threads with a set bit.
+    uint32_t wd[STREAM ? 8 : 4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const uint32_t lb = last_bit(cur.t[u]);
-      hit |= (sh_last[lb >> 5] >> (lb & 31) & 1u) << u;
+      wd[u] = sh_last[lb >> 5] >> (lb & 31);
     }
+    uint32_t any = (wd[0] | wd[1]) | (wd[2] | wd[3]);
     if (STREAM) {
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const uint32_t lb = last_bit(cur2.t[u]);
-        hit |= (sh_last[lb >> 5] >> (lb & 31) & 1u) << (4 + u);
+        wd[4 + u] = sh_last[lb >> 5] >> (lb & 31);
       }
+      any |= (wd[4] | wd[5]) | (wd[6] | wd[7]);
+    }
+    uint32_t hit = 0u;
+    if (any & 1u) {
+#pragma unroll
+      for (int u = 0; u < (STREAM ? 8 : 4); ++u) hit |= (wd[u] & 1u) << u;
     }
     const unsigned b = __ballot_sync(FULL_MASK, hit != 0u);
     if (b) {                                                      // queue what passed
@@ -463,7 +472,7 @@ cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   const long long per_prompt = (long long)s.N * ((s.L + kScanTile - 1) / kScanTile);
   int set_slots = 64;
   while (set_slots < 4 * s.N) set_slots *= 2;
-  const size_t dyn = ((size_t)3 * s.N + set_slots) * 4;
+  const size_t dyn = ((size_t)4 * s.N + set_slots) * 4;
   if ((long long)s.G * per_prompt > 148LL * 8 * 4 && (s.L & 3) == 0) {
     // streaming form: every CTA resident at once, each with kStreamStages tiles in flight
     static int per_sm = 0;

@@ -150,7 +150,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   if (rc != SDMS_OK) return rc;
   if (!d_workspace || ((uintptr_t)d_workspace & (kAlign - 1))) return SDMS_ERR_INVALID_ARG;
   if (bytes < lay.total) return SDMS_ERR_WORKSPACE_TOO_SMALL;
-  if (dag_kernel_setup() != cudaSuccess) return SDMS_ERR_CUDA;
+  if (dag_kernel_setup() != cudaSuccess || scan_kernel_setup() != cudaSuccess) return SDMS_ERR_CUDA;
   if (cudaMemsetAsync(d_workspace, 0, lay.total, 0) != cudaSuccess) return SDMS_ERR_CUDA;
   if (cudaStreamSynchronize(0) != cudaSuccess) return SDMS_ERR_CUDA;
   sdms_ctx* ctx = new (std::nothrow) sdms_ctx();

@@ -163,6 +163,7 @@ __device__ __forceinline__ TileRegs fetch_tile(const Dev& s, int g, int jn, int 
 constexpr int kStreamStages = 4;
 constexpr int kStreamTile = 2 * kScanTile;           // tokens per stage: a thread takes eight of them
 constexpr int kStreamThreads = kScanThreads + 32;   // eight scanning warps and one warp that issues the copies
+constexpr int kStreamSmemMax = 96 * 1024;             // dynamic shared memory the streaming form may ask for
 constexpr long long kWaitCycles = 4000000000LL;      // about two seconds: a wait that long has failed
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -466,6 +467,11 @@ cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
   return launch_overlapped(probe_kernel, dim3(1), dim3(kProbeThreads), 0, stream, s, k);
 }
 
+// Called when a context is created, with its device current.
+cudaError_t scan_kernel_setup() {
+  return cudaFuncSetAttribute(scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax);
+}
+
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   // one CTA per tile while that keeps the device busy for one round; beyond that each CTA streams
   // through its share of its prompt's tiles
@@ -473,18 +479,15 @@ cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream) {
   int set_slots = 64;
   while (set_slots < 4 * s.N) set_slots *= 2;
   const size_t dyn = ((size_t)4 * s.N + set_slots) * 4;
-  if ((long long)s.G * per_prompt > 148LL * 8 * 4 && (s.L & 3) == 0) {
-    // streaming form: every CTA resident at once, each with kStreamStages tiles in flight
-    static int per_sm = 0;
+  if ((long long)s.G * per_prompt >= 148LL * 8 && (s.L & 3) == 0) {
+    // streaming form: each CTA keeps kStreamStages tiles in flight
+    constexpr int per_sm = 4;                                            // resident CTAs per SM (shared memory, registers)
     const size_t dyn_stream = dyn + (size_t)kStreamStages * kStreamTile * 4;
     const long long per_prompt_s = (long long)s.N * ((s.L + kStreamTile - 1) / kStreamTile);
-    if (per_sm == 0) {
-      cudaError_t e = cudaFuncSetAttribute(scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-      if (e != cudaSuccess) return e;
-      per_sm = 4;
-    }
-    if (dyn_stream <= 96 * 1024) {
-      const long long tot = 148LL * per_sm * 4;                        // four rounds of resident CTAs: set-ups overlap other CTAs' streaming
+    if (dyn_stream <= kStreamSmemMax) {
+      // one round of resident CTAs while every CTA gets a few tiles only, four rounds for larger stores (set-ups then
+      // overlap other CTAs' streaming)
+      const long long tot = (long long)s.G * per_prompt > 148LL * 8 * 4 ? 148LL * per_sm * 4 : 148LL * per_sm;
       const long long ctas = std::max(1LL, std::min(per_prompt_s, tot / s.G));
       return launch_overlapped(scan_kernel<true>, dim3((unsigned)(ctas * s.G)), dim3(kStreamThreads), dyn_stream, stream, s,
                                k, (int)ctas, set_slots);

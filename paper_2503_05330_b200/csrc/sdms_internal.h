@@ -38,5 +38,6 @@ cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, c
                         float* draft_edge_w, int32_t* used_k, cudaStream_t stream);
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream);
 cudaError_t dag_kernel_setup();
+cudaError_t scan_kernel_setup();
 
 }  // namespace sdms

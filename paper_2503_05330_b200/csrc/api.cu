@@ -170,6 +170,13 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.mode = cfg->search_mode; d.P = d.G * d.N;
   d.alpha = (double)cfg->alpha;
   d.table_cap = lay.table_cap; d.match_cap = lay.match_cap;
+  {
+    int l = 0;
+    while ((1ll << l) < (long long)d.L) ++l;                          // l = ceil(log2 L)
+    const unsigned long long two = 1ull << (31 + l);
+    d.L_magic = (uint32_t)((two + (unsigned long long)d.L - 1) / (unsigned long long)d.L);
+    d.L_shift = 31 + l;
+  }
   d.fused = fits_fused(cfg, lay);
   d.eps = cfg->epsilon;
   d.pool = cfg->pool_mode;

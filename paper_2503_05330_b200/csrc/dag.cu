@@ -249,7 +249,7 @@ __device__ void dag_small(const Dev& s, const Smem& sm, int i, int M, const int3
   int gpos = 0, n_m = 0;
   if (lane < M) {
     gpos = mlist[lane];
-    const int j = gpos / s.L;
+    const int j = path_of(s, gpos);
     n_m = min(D, plen[j - poff] - 1 - (gpos - j * s.L));
   }
   for (int d = warp + 1; d <= D; d += nwarps) {
@@ -409,7 +409,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
     for (int x = tid; x < M * D; x += blockDim.x) {
       const int m = x / D, dd = x - m * D + 1;
       const int gpos = mlist[m];
-      const int j = gpos / s.L;
+      const int j = path_of(s, gpos);
       const int e = gpos - j * s.L;
       const bool on = e + dd <= plen[j - poff] - 1;
       sm.st_tok[x] = on ? ldm(s.tok + gpos + dd) : -1;
@@ -460,7 +460,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
           tv[r] = -1; tp[r] = 0;
           if (m >= M) continue;
           const int gpos = mlist[m];
-          const int j = gpos / s.L;
+          const int j = path_of(s, gpos);
           if (gpos - j * s.L + d <= plen[j - poff] - 1) { tv[r] = ldm(s.tok + gpos + d); tp[r] = ldm(s.pq + gpos + d); }
         }
 #pragma unroll
@@ -476,6 +476,8 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       if (EXPORT && tid < MAXB) { sm.r_nedge[tid] = 0; sm.r_outdeg[tid] = 0; }
       __syncthreads();
       bool overflowed = false;
+      const bool part_pow2 = (npart & (npart - 1)) == 0;        // nearly always: residue and quotient without a division
+      const int part_shift = __ffs(npart) - 1;
       for (int part = 0; part < npart && !overflowed; ++part) {
         // ---- accumulate this residue class of follower tokens ----
         // Walking in mode 0 past the first layer, only successors of the current node can be chosen:
@@ -499,7 +501,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 if (v[r] >= 0) { u[r] = d == 1 ? root : prev_v[m]; p[r] = (unsigned)roll_p[m]; }
               } else {
                 const int gpos = mlist[m];
-                const int j = gpos / s.L;
+                const int j = path_of(s, gpos);
                 if (gpos - j * s.L + d <= plen[j - poff] - 1) {
                   v[r] = ldm(s.tok + gpos + d);
                   u[r] = d == 1 ? root : ldm(s.tok + gpos + d - 1);
@@ -512,9 +514,10 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
             for (int r = 0; r < kLoadBatch; ++r) {
               const int vv = v[r], uu = u[r];
               const unsigned pp = p[r];
-              if (vv < 0 || (npart > 1 && vv % npart != part)) continue;
+              if (vv < 0 || (npart > 1 && (part_pow2 ? (vv & (npart - 1)) : vv % npart) != part)) continue;
               if (phase == 0 && uu != cur) continue;
-              unsigned h = slot_hash((unsigned)(vv / npart));
+              const unsigned vq = part_pow2 ? (unsigned)vv >> part_shift : (unsigned)(vv / npart);
+              unsigned h = slot_hash(vq);
               int slot = -1;
               if (phase == 1 && restricted) {                          // read-only: is vv a claimed successor?
                 for (int probe = 0; probe < CAP; ++probe) {
@@ -542,7 +545,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 for (int x = 0; x < nkept; ++x) if (sm.kept[x] == uu) { b = x; break; }
                 if (b >= 0) {
                   const int ekey = vv * MAXB + b;               // (destination, kept source) in one word
-                  unsigned he = slot_hash((unsigned)(vv / npart) * 37u + (unsigned)b);
+                  unsigned he = slot_hash(vq * 37u + (unsigned)b);
                   int es = -1;
                   for (int probe = 0; probe < CAP; ++probe) {
                     const int old = atomicCAS(&sm.e_key[he], -1, ekey);
@@ -715,7 +718,7 @@ __device__ void list_pool(const Dev& s, int i, int M, const int32_t* mlist, cons
   int best_g = -1;
   for (int m = tid; m < M; m += blockDim.x) {
     const int gpos = mlist[m];
-    const int j = gpos / s.L;
+    const int j = path_of(s, gpos);
     const int n_m = min(D, plen[j - poff] - 1 - (gpos - j * s.L));
     u64 S = 0;
     for (int d = 1; d <= n_m; ++d) S += (unsigned)ldm(s.pq + gpos + d);
@@ -844,7 +847,7 @@ __device__ void dag_layers(const Dev& s, const Smem& sm, int i, int M, const int
         tk[r] = -1; pr[r] = 0;
         if (m >= M || dd > D) continue;
         const int gpos = mlist[m];
-        const int j = gpos / s.L;
+        const int j = path_of(s, gpos);
         if (gpos - j * s.L + dd <= plen[j - poff] - 1) { tk[r] = ldm(s.tok + gpos + dd); pr[r] = ldm(s.pq + gpos + dd); }
       }
 #pragma unroll
@@ -993,7 +996,7 @@ __device__ void dag_best_path(const Dev& s, const Smem& sm, int i, int M, int ca
     const int m = x >> lD, dd = (x & ((1 << lD) - 1)) + 1;
     if (dd > D) continue;
     const int gpos = mlist[m];
-    const int j = gpos / s.L;
+    const int j = path_of(s, gpos);
     const bool on = gpos - j * s.L + dd <= plen[j - poff] - 1;
     st_tok[m * D + dd - 1] = on ? ldm(s.tok + gpos + dd) : -1;
     st_pq[m * D + dd - 1] = on ? ldm(s.pq + gpos + dd) : 0;

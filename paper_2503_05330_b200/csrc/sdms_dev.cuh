@@ -28,6 +28,7 @@ struct Dev {
   int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
   double alpha;
   uint32_t table_cap;                  // buckets per (prompt, n) table, power of two
+  uint32_t L_magic; int32_t L_shift;   // x / L for 0 <= x < 2^31 as (x * L_magic) >> L_shift (path_of)
   int64_t match_cap;
   // path store
   int32_t* tok;                        // [P][L]
@@ -68,6 +69,13 @@ __device__ __forceinline__ uint32_t gram_bucket(uint64_t h, uint32_t cap) { retu
 
 __device__ __forceinline__ uint32_t* index_table(const Dev& s, int g, int n) {
   return s.index + ((size_t)(g * s.k_max + (n - 1)) * s.table_cap) * kBucketWords;
+}
+
+// Path (row of the store) a global position x = j * L + e lies in, without a division: L_magic =
+// ceil(2^(31 + l) / L) with l = ceil(log2 L) fits 32 bits and gives the exact quotient for every
+// 0 <= x < 2^31 (round-up method of division by an invariant integer).
+__device__ __forceinline__ int path_of(const Dev& s, int x) {
+  return (int)(((uint64_t)(uint32_t)x * s.L_magic) >> s.L_shift);
 }
 
 // Eq. 5 on integer sums: alpha * S / 2^30 + (1 - alpha) * cnt, every operation

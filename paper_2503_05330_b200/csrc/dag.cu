@@ -443,10 +443,14 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
     const bool tree = !EXPORT && s.pool == 1;       // only candidates that spell the draft so far take part
     const bool restricted = !EXPORT && !staged && !tree && s.mode != 1 && d > 1;   // staged candidates are cheap to revisit
     if (!EXPORT) {
-      // first layer (or every layer in mode 1): every distinct follower is a node, guess one per four
-      // candidates; restricted layers only hold the successors of one node
+      // first layer (or every layer in mode 1): every distinct follower is a node.  The guess is
+      // optimistic, one node per 32 candidates (popular n-grams have far fewer distinct followers than
+      // occurrences): a sweep that finds the table three quarters full stops at once and the layer is
+      // redone with twice the residue classes, so a wrong guess costs a fraction of a sweep, while a
+      // cautious one costs a full sweep for every class too many.  Restricted layers only hold the
+      // successors of one node.
       npart = 1;
-      if (!restricted) while (npart * (CAP / 2) * 4 < M && npart < npart_max) npart *= 2;
+      if (!restricted) while (npart * (CAP / 2) * 32 < M && npart < npart_max) npart *= 2;
     }
     int* const cur_v = (d & 1) ? roll_odd : roll_even;
     const int* const prev_v = (d & 1) ? roll_even : roll_odd;
@@ -485,6 +489,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
         // slot.  Otherwise one phase claims and adds.
         for (int phase = restricted ? 0 : 1; phase < 2; ++phase) {
           for (int m0 = tid; m0 < M; m0 += kLoadBatch * blockDim.x) {
+            if (npart < npart_max && *(volatile int*)&sh_nn > CAP * 3 / 4) break;   // too many nodes for this pass: it is redone
             int v[kLoadBatch], u[kLoadBatch];
             unsigned p[kLoadBatch];
 #pragma unroll

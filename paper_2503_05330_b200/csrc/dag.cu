@@ -201,6 +201,8 @@ __device__ Smem carve(unsigned char* base) {
   return m;
 }
 
+// 16-bit tag of a token, never 0 (0 marks "no token")
+__device__ __forceinline__ unsigned short tag_of(int tok) { return (unsigned short)(0x8000u | (((unsigned)tok * 2654435761u) >> 17)); }
 __device__ __forceinline__ unsigned slot_hash(unsigned x) { return (x * 2654435761u) >> 22; }   // 10 bits = CAP
 static_assert(CAP == 1024, "slot_hash yields 10 bits");
 
@@ -420,6 +422,12 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
   // candidate; the layer before stays, it holds the edges' sources), so that the passes and phases of
   // a layer read shared memory and only one sweep per layer goes to L2
   const bool rolling = !staged && M <= kRollMax && !(!EXPORT && s.pool == 1);
+  // more candidates than that: the staging area is free and keeps a 16-bit tag of every candidate's token
+  // of the layer before (written by the last sweep of that layer), so that the sweep that claims the
+  // successors of the current node (phase 0 below) reads shared memory and goes to the histories only
+  // for the candidates whose tag is the current node's
+  const bool tagged = !EXPORT && !staged && !rolling && s.pool == 0 && M <= 4 * kStageWords;
+  unsigned short* const tag = reinterpret_cast<unsigned short*>(sm.st_tok);
   int* const roll_odd = sm.st_tok;
   int* const roll_even = sm.st_tok + kRollMax;
   int* const roll_p = sm.st_tok + 2 * kRollMax;
@@ -452,6 +460,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       npart = 1;
       if (!restricted) while (npart * (CAP / 2) * 32 < M && npart < npart_max) npart *= 2;
     }
+    const unsigned short cur_tag = tag_of(cur);
     int* const cur_v = (d & 1) ? roll_odd : roll_even;
     const int* const prev_v = (d & 1) ? roll_even : roll_odd;
     if (rolling) {
@@ -505,6 +514,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 v[r] = cur_v[m];
                 if (v[r] >= 0) { u[r] = d == 1 ? root : prev_v[m]; p[r] = (unsigned)roll_p[m]; }
               } else {
+                if (tagged && phase == 0 && tag[m] != cur_tag) continue;   // its token of the layer before is not the current node
                 const int gpos = mlist[m];
                 const int j = path_of(s, gpos);
                 if (gpos - j * s.L + d <= plen[j - poff] - 1) {
@@ -513,6 +523,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                   p[r] = (unsigned)ldm(s.pq + gpos + d);
                   if (tree) for (int x = 1; x < d && v[r] >= 0; ++x) if (ldm(s.tok + gpos + x) != sh_draft[x - 1]) v[r] = -1;
                 }
+                if (tagged && phase == 1 && part == npart - 1) tag[m] = v[r] >= 0 ? tag_of(v[r]) : (unsigned short)0;
               }
             }
 #pragma unroll

@@ -543,6 +543,34 @@ def test_tile_scan_with_more_matches_per_tile_than_its_buffer_holds():
     assert (pair.g.query_modes() == 2).all()
 
 
+@pytest.mark.parametrize("match_capacity", [0, 400000])
+def test_heavy_query_with_wide_fan_out_in_every_layer(match_capacity):
+    # one token A at every third position: ~2700 matches per path and more than 5461 per query, so the DAG is
+    # aggregated from candidates that are not staged.  A is followed by B half of the time, else by one of
+    # 3000 tokens, and B by one of 3000 tokens: the first layer and the layer after B have more distinct
+    # nodes than one table pass holds (the layer is redone with more residue classes), both through the
+    # single-launch build and (match_capacity below P*N*L) through the probe / scan / dag kernels.
+    G, N, L, V, D = 1, 8, 8192, 4000, 4
+    rng = np.random.default_rng(5330)
+    tokens = rng.integers(10, 3010, size=(G * N, L)).astype(np.int32)
+    tokens[:, 0::3] = 1                                        # A
+    after = tokens[:, 1::3]
+    after[rng.random(after.shape) < 0.5] = 2                   # B
+    lps = (-rng.exponential(0.5, size=tokens.shape)).astype(np.float32)
+    pair = Pair(G, N, L, V, 2, D, match_capacity=match_capacity)
+    lens = np.array([8101, 7900, 8002, 7603, 8176, 8050, 7999, 8182], np.int32)   # all end in A (position % 3 == 0)
+    assert ((lens - 1) % 3 == 0).all()
+    for c in range(0, L - 8, 2048):
+        part = np.clip(lens - c, 0, 2048).astype(np.int32)
+        pair.g.append(t32(tokens[:, c:c + 2048], pair.dev), t32(lps[:, c:c + 2048], pair.dev), t32(part, pair.dev))
+        pair.o.append(tokens[:, c:c + 2048], lps[:, c:c + 2048], part)
+    assert pair.g.status() == 0
+    pair.build_and_compare(1, check_dag=False)
+    off, _ = pair.g.matches()
+    assert np.diff(off.numpy()).min() > 5461
+    pair.build_and_compare(2, check_dag=False)
+
+
 def test_streaming_tile_scan_on_a_store_of_many_tiles():
     # more 1024-token tiles than the one-tile-per-CTA form launches: the scan streams its tiles through
     # shared-memory stages.  Ragged lengths: empty paths, paths that end inside their first tile, on a

@@ -489,6 +489,9 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       if (EXPORT && tid < MAXB) { sm.r_nedge[tid] = 0; sm.r_outdeg[tid] = 0; }
       __syncthreads();
       bool overflowed = false;
+      // while the layer can still be split further, a claim that does not find its slot within 64 probes gives the
+      // pass up (it is redone): a first batch of 2048 claims can fill the table before any thread looks at the count
+      const int probe_max = npart < npart_max ? 64 : CAP;
       const bool part_pow2 = (npart & (npart - 1)) == 0;        // nearly always: residue and quotient without a division
       const int part_shift = __ffs(npart) - 1;
       for (int part = 0; part < npart && !overflowed; ++part) {
@@ -544,7 +547,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 }
                 if (slot < 0) continue;
               } else {
-                for (int probe = 0; probe < CAP; ++probe) {
+                for (int probe = 0; probe < probe_max; ++probe) {
                   const int old = atomicCAS(&sm.n_key[h], -1, vv);
                   if (old == -1) sm.n_touch[atomicAdd(&sh_nn, 1)] = (int)h;
                   if (old == -1 || old == vv) { slot = (int)h; break; }

@@ -29,8 +29,8 @@ UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
 # profiles/step_kernel_cfg2_ncu_full.md; only quoted while the kernel sources are the ones profiled
-NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 75648,
-               "sources_sha256": "d6a74c92301128f5c5c63d0bedc2c259938b638f3327f71f195cef4860e58054"}
+NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76544,
+               "sources_sha256": "e12a72d89f9b3dc814c0a39a784b393dfa7702be8b3587dc9255d39edc42cd0d"}
 
 
 def kernel_sources_sha():

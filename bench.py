@@ -27,8 +27,8 @@ from paper_2503_05330_b200 import synth  # noqa: E402
 METRIC = "draft-construction paths*steps/sec at N=16 (and us/step)"
 UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
-# profiles/step_kernel_cfg2_ncu_full.md; only quoted while the kernel sources are the ones profiled
+# DRAM bytes per launch of the dominant kernel from its last ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum); only quoted while the kernel sources are the ones profiled
 NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76544,
                "sources_sha256": "e12a72d89f9b3dc814c0a39a784b393dfa7702be8b3587dc9255d39edc42cd0d"}
 
@@ -50,9 +50,66 @@ def k_of(step, k_max):
     return 1 + (h ^ (h >> 13)) % k_max
 
 
+def timed_step_plan(K, S):
+    """Which steps of which decode run are timed: K timed steps spread evenly over ceil(K / S) whole
+    runs of S steps each (warm start .. histories full), so that a small K still sees short and long
+    histories and every k alike.  The steps in between run untimed because the state has to evolve.
+    Both arms of the benchmark time exactly these steps."""
+    runs = -(-K // S)
+    plan = []
+    for r in range(runs):
+        quota = K // runs + (1 if r < K % runs else 0)
+        plan.append(set(int((x + 0.5) * S / quota) for x in range(quota)) if quota < S else set(range(S)))
+    return plan
+
+
 # ----------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands, on the host cores
 # ----------------------------------------------------------------------------
+def oracle_decode_run(w, tokens, logprobs, timed, threads=1):
+    """One whole decode run on the oracle.  A step is what the CUDA arm times as one sdms_step call:
+    acceptance check and commit of the drafts of decode step t, then the drafts of step t + 1.  Only the
+    steps in `timed` are clocked (None: none, the run only counts its steps).
+    Returns (paths*steps, seconds, timed steps, steps in the run)."""
+    from oracle import Oracle
+    o = Oracle(w.G, w.N, w.L, w.V, w.D)
+    lens = np.full(w.P, w.k_max, np.int32)
+    o.append(tokens[:, :w.k_max], logprobs[:, :w.k_max], lens)
+    o.build_all(k_of(0, w.k_max), nthreads=threads)
+    units, secs, done, step = 0, 0.0, 0, 0
+    for step in range(w.steps):
+        lens = o.lengths()
+        active = int((lens < w.L).sum())
+        if active == 0:
+            break
+        sampled, sampled_lp = synth.sampled_window(tokens, logprobs, lens, w.D + 1)
+        tok, ln, _, _ = o.drafts()
+        on = timed is not None and step in timed
+        t0 = time.perf_counter()
+        o.accept_commit(tok, ln, sampled, sampled_lp, w.D)
+        o.build_all(k_of(step + 1, w.k_max), nthreads=threads)
+        if on:
+            secs += time.perf_counter() - t0
+            units += active
+            done += 1
+    else:
+        step = w.steps
+    return units, secs, done, step
+
+
+def oracle_timed_steps(w, tokens, logprobs, K, threads=1, budget_s=None):
+    """Times the same K steps as Runner.timed_steps (timed_step_plan over whole runs)."""
+    S = oracle_decode_run(w, tokens, logprobs, None, threads)[3]
+    units, secs, done = 0, 0.0, 0
+    t_all = time.perf_counter()
+    for timed in timed_step_plan(K, S):
+        u, t, d, _ = oracle_decode_run(w, tokens, logprobs, timed, threads)
+        units += u; secs += t; done += d
+        if budget_s is not None and time.perf_counter() - t_all > budget_s:
+            break
+    return units, secs, done, S
+
+
 def oracle_run(w, tokens, logprobs, max_steps, budget_s, threads=1):
     """Decode protocol on the oracle; returns (paths*steps, seconds, steps, restarts)."""
     from oracle import Oracle
@@ -88,8 +145,8 @@ def reference_main(args, w):
     if rank != 0:
         return
     tokens, logprobs = synth.make_streams(w)
-    oracle_run(w, tokens, logprobs, args.warmup, 30.0)
-    units, secs, steps, runs = oracle_run(w, tokens, logprobs, args.steps, 120.0)
+    oracle_timed_steps(w, tokens, logprobs, max(args.warmup, 1))
+    units, secs, steps, S = oracle_timed_steps(w, tokens, logprobs, args.steps, budget_s=150.0)
     value = units / secs
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -97,7 +154,8 @@ def reference_main(args, w):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32/int64 (f64 weights)",
         "data": "synthetic", "config": workload_config(w),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{steps} decode steps of {w.name} ({runs} run(s) from the warm start)"},
+                         "sample": f"the same {steps} steps the CUDA arm times: spread evenly over whole decode runs of "
+                                   f"{S} steps of {w.name}, the steps in between run untimed"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -252,45 +310,50 @@ class Runner:
         """Times exactly K steps (CUDA events around each step on the launch
         stream), restarting the run when it ends.  A step is one sdms_step call: acceptance check
         and commit of the drafts of decode step t, then the drafts of step t + 1.
-        Returns (ms, paths*steps)."""
+        Returns (ms, paths*steps).  With e2e the step goes through host buffers and is also timed on
+        the host clock, from the moment the model's answer is handed over in host memory to the moment
+        the results have been read on the host (self.last_host_ms)."""
         torch, w, s, plan = self.torch, self.w, self.s, self.plan
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         units = 0
         done = 0
         ks = []
+        host_s = 0.0
         if e2e:
             # zero-copy: the step's inputs are written into page-locked host memory that the kernel reads
             # in place, and the kernel writes drafts and accept lengths into page-locked host memory
             assert s.host_io
-            h_in = plan["step_in_host"]                                        # [steps][sampled | logprobs]
+            h_in = plan["step_in_host"].numpy()                                # [steps][sampled | logprobs]
+            step_in = s.step_in.numpy()                                        # the mapped input buffer, as the host sees it
+            results = s.results.numpy()
             seen = 0
-        # K timed steps spread evenly over whole runs (warm start .. histories full), so that a
-        # small K still sees short and long histories and every k alike; the steps in between run
-        # untimed because the state has to evolve
+            stream = torch.cuda.current_stream()
         S = plan["steps"]
-        runs = -(-K // S)
-        for r in range(runs):
-            quota = K // runs + (1 if r < K % runs else 0)
-            timed = set(int((x + 0.5) * S / quota) for x in range(quota)) if quota < S else set(range(S))
+        for timed in timed_step_plan(K, S):
             self.start_run(first_drafts=True)
             for step in range(S):
                 on = step in timed
                 k_next = k_of(step + 1, w.k_max)
                 if on and flush:
                     self.flush.zero_()
-                if on:
-                    a, b = ev[done]
-                    a.record()
                 if e2e:
-                    s.step_in.copy_(h_in[step])     # host to host: the model's answer lands in the mapped buffer
+                    if on:
+                        torch.cuda.synchronize()    # the flush is over: the host clock sees this step only
+                        a, b = ev[done]
+                        t0 = time.perf_counter()
+                        a.record()
+                    np.copyto(step_in, h_in[step])  # host to host: the model's answer lands in the mapped buffer
                     self.step(step, s.sampled_in, s.sampled_lp_in)
                     if on:
                         b.record()
-                        b.synchronize()             # the caller reads the result before its next step
-                        seen += int(s.accept_len[0]) + int(s.draft_len[-1])    # read on the host, no copy
-                    else:
-                        torch.cuda.current_stream().synchronize()   # the kernel is done with the input buffer
+                    stream.synchronize()            # the caller reads the result before its next step
+                    if on:
+                        seen += int(results[-1]) + int(results[w.P * w.D])     # an accept length and a draft length, read in place
+                        host_s += time.perf_counter() - t0
                 else:
+                    if on:
+                        a, b = ev[done]
+                        a.record()
                     self.step(step, plan["sampled"][step], plan["lp"][step])
                     if on:
                         b.record()
@@ -301,6 +364,7 @@ class Runner:
         assert done == K
         torch.cuda.synchronize()
         per_step = [a.elapsed_time(b) for a, b in ev]
+        self.last_host_ms = 1e3 * host_s
         self.last_by_k = {}
         for kk in range(1, w.k_max + 1):
             t = [per_step[x] for x in range(K) if ks[x] == kk]
@@ -309,10 +373,11 @@ class Runner:
         return sum(per_step), units
 
 
-def steady_state(wl, device, iters=20):
-    """Build latency of another workload at 97 % full histories: per k the median time of
-    sdms_build_drafts (CUDA events on the launch stream, L2 flushed before every call), the
-    matches it found and the kernel's own byte count per call.  Context for the headline."""
+def steady_state(wl, device, iters=20, peak=None):
+    """Build latency of a workload at 97 % full histories (a full path builds no draft): per k the
+    median, 10th and 90th percentile of the time of sdms_build_drafts (CUDA events on the launch
+    stream, L2 flushed before every call), the matches it found, the kernel's own byte count per call
+    and, for prompts scanned by every query CTA, the bytes of a scan shared by the whole prompt."""
     import torch
     from paper_2503_05330_b200 import binding
     tokens, logprobs = synth.make_streams(wl)
@@ -334,7 +399,8 @@ def steady_state(wl, device, iters=20):
             a.record(); s.build_drafts(k); b.record()
             evs.append((a, b))
         torch.cuda.synchronize()
-        us = 1e3 * float(np.median([a.elapsed_time(b) for a, b in evs]))
+        t_us = 1e3 * np.array([a.elapsed_time(b) for a, b in evs])
+        us = float(np.median(t_us))
         binding.sdms_profile_enable(s.ctx, True)                 # per-kernel split (events between the launches)
         for _ in range(5):
             flush.zero_()
@@ -348,12 +414,17 @@ def steady_state(wl, device, iters=20):
         fused = wl.N * wl.L <= 131072
         scan_bytes = int(4 * (glen - lens)[modes == 2].sum()) if fused else (4 * int(lens.sum()) if (modes == 2).any() else 0)
         nbytes = scan_bytes + int((modes > 0).sum()) * (32 + 4 * k) + int(m.sum()) * (4 + 8 * wl.D) + wl.P * (12 * wl.D + 4)
-        out[str(k)] = {"us": us, "paths_per_s": wl.P / (us * 1e-6), "matches": int(m.sum()), "max_matches": int(m.max()),
+        shared_scan = 4 * int(lens.reshape(wl.G, wl.N)[(modes == 2).reshape(wl.G, wl.N).any(1)].sum())   # scan model: once per prompt
+        out[str(k)] = {"us": us, "p10_us": float(np.percentile(t_us, 10)), "p90_us": float(np.percentile(t_us, 90)),
+                       "launches_timed": iters, "paths_per_s": wl.P / (us * 1e-6), "matches": int(m.sum()),
+                       "max_matches": int(m.max()),
                        "scanned_queries": int((modes == 2).sum()), "bytes": nbytes, "gbs": nbytes / (us * 1e-6) / 1e9,
+                       "frac_of_peak": None if peak is None else nbytes / (us * 1e-6) / 1e9 / peak,
+                       "scan_bytes_moved": scan_bytes, "scan_bytes_shared_pass": shared_scan,
                        "kernel_us": split}
     assert s.status() == 0
     return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
-            "launches_per_build": 1 if fused else 3, "build_by_k": out}
+            "launches_per_build": 1 if fused else 3, "workspace_bytes": s.workspace_bytes, "build_by_k": out}
 
 
 def scan_at_scale(device, G=64, N=256, L=8192, V=151936):
@@ -383,6 +454,49 @@ def scan_at_scale(device, G=64, N=256, L=8192, V=151936):
     nbytes = 4 * P * n
     out = {"groups": G, "paths_per_group": N, "capacity": L, "store_bytes": nbytes, "workspace_bytes": s.workspace_bytes,
            "scan_queries": int((s.query_modes() == 2).sum()), "us_per_launch": us, "gbs": nbytes / (us * 1e-6) / 1e9}
+    del s
+    torch.cuda.empty_cache()
+    return out
+
+
+def gather_at_scale(device, G=64, N=256, L=8192, V=16384, D=16):
+    """Follower gather + DAG aggregation + search (dag_kernel) on a store larger than L2: G prompts of N
+    paths, uniform random tokens over a vocabulary small enough that a k = 1 query finds a hundred-odd
+    matches (N * L / V), spread at random over the prompt's histories, so that every match costs a fresh
+    read of its D followers (token and probability) from HBM and no single query dominates.
+    Algorithmic bytes = 8 per follower (token and probability of each of the n_m followers of every match)
+    plus the match list and the outputs."""
+    import torch
+    from paper_2503_05330_b200 import binding
+    P, n = G * N, L - 8
+    s = binding.Sdms(G, N, L, V, 1, D, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(synth.BASE_SEED + 1)
+    tok = torch.randint(0, V, (P, n), dtype=torch.int32, device=device, generator=gen)
+    lp = -torch.rand((P, n), dtype=torch.float32, device=device, generator=gen)
+    s.append(tok, lp, torch.full((P,), n, dtype=torch.int32, device=device))
+    del tok, lp
+    s.build_drafts(1)                                  # warm-up
+    binding.sdms_profile_enable(s.ctx, True)
+    for _ in range(5):
+        s.build_drafts(1)
+    torch.cuda.synchronize()
+    prof = binding.sdms_profile_read(s.ctx)
+    assert s.status() == 0
+    off, gpos = s.matches()
+    gpos = gpos.numpy().astype(np.int64)
+    n_m = np.minimum(D, n - 1 - gpos % L)
+    m = np.diff(off.numpy())
+    out = {"groups": G, "paths_per_group": N, "capacity": L, "vocab": V, "max_draft_len": D,
+           "store_bytes": 8 * P * n, "workspace_bytes": s.workspace_bytes,
+           "matches": int(m.sum()), "mean_matches_per_query": float(m.mean()), "max_matches_per_query": int(m.max())}
+    nbytes = int(8 * n_m.sum() + 4 * len(gpos) + P * (12 * D + 4))
+    for name in ("dag", "dag_heavy"):
+        if name in prof and prof[name][1]:
+            ms, launches = prof[name]
+            out[name + "_us_per_launch"] = 1e3 * ms / launches
+    us = sum(out[k] for k in out if k.endswith("_us_per_launch"))
+    out.update(algorithmic_bytes=nbytes, us_per_build_gather_side=us, gbs=nbytes / (us * 1e-6) / 1e9)
     del s
     torch.cuda.empty_cache()
     return out
@@ -446,6 +560,7 @@ def ours_main(args, w):
     hrun.plan = plan
     hrun.timed_steps(3, e2e=True)
     ms_e2e, units_e2e = hrun.timed_steps(args.steps, e2e=True)
+    host_ms_e2e = hrun.last_host_ms
     del hrun
 
     # per-kernel times over a further pass of the same steps
@@ -525,23 +640,25 @@ def ours_main(args, w):
         trim_us = 1e3 * a.elapsed_time(b)
         assert trun.s.status() == 0
         del trun
-    others = scale = None
-    if world == 1 and not args.no_others:
-        del run.flush
-        torch.cuda.empty_cache()
-        others = {synth.WORKLOADS[c].name: steady_state(synth.WORKLOADS[c], device) for c in (1, 3, 4, 5)}
-        scale = scan_at_scale(device)
-    (ms, ms_e2e), (units, units_e2e) = whole_job([ms, ms_e2e], [units, units_e2e], device)
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
     peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_file):
         peak, peak_src = float(json.load(open(peaks_file))["hbm_gbs"]), "measured copy bandwidth (burst)"
     else:
         peak, peak_src = 6650.0, "fallback"
+    others = scale = gscale = steady2 = None
+    if world == 1 and not args.no_others:
+        del run.flush
+        torch.cuda.empty_cache()
+        steady2 = steady_state(w, device, iters=200, peak=peak)
+        others = {synth.WORKLOADS[c].name: steady_state(synth.WORKLOADS[c], device, peak=peak) for c in (1, 3, 4, 5)}
+        scale = scan_at_scale(device)
+        gscale = gather_at_scale(device)
+    (ms, ms_e2e, host_ms_e2e), (units, units_e2e, _) = whole_job([ms, ms_e2e, host_ms_e2e], [units, units_e2e, 0.0], device)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     per_kernel = {}
     for name, (kms, n) in prof.items():
         if n:
@@ -560,19 +677,28 @@ def ours_main(args, w):
                                "prompt for each scanned query, followers of every match, outputs",
                 "useful_bytes_per_launch_index_model": plan["useful_bytes_build"],
                 "note": "the whole store of this workload is 128 KiB: a step is bound by launch and "
-                        "dependent-access latency, not by bandwidth"}
+                        "dependent-access latency, not by bandwidth",
+                # the figures the bandwidth clause is judged on: kernels on stores larger than L2, and the
+                # build of every configuration at 97 % full histories
+                "match_at_scale": None if scale is None else dict(scale, frac=scale["gbs"] / peak),
+                "gather_at_scale": None if gscale is None else dict(gscale, frac=gscale["gbs"] / peak),
+                "steady_state_full_history": steady2,
+                "by_config": others}
 
     line = {
         "metric": METRIC, "value": units / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "us_per_step": 1e3 * ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32/int64 (f64 weights)", "data": "synthetic", "config": workload_config(w),
-        "e2e": {"value": units_e2e / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": 1e3 * ms_e2e / args.steps,
+        "e2e": {"value": units_e2e / (host_ms_e2e * 1e-3), "unit": UNIT, "us_per_step": 1e3 * host_ms_e2e / args.steps,
+                "clock": "host (perf_counter): from the model's answer being handed over in host memory, through the "
+                         "C-ABI call, to the results having been read on the host; the L2 flush is waited for before",
+                "device_us": 1e3 * ms_e2e / args.steps,
                 "h2d_bytes_per_step": w.P * (w.D + 1) * 8 + w.P * (w.D + 1) * 4,
                 "d2h_bytes_per_step": w.P * (w.D + 2) * 4,
                 "how": "zero-copy: sampled tokens, logprobs and the previous drafts are read by the step kernel from "
                        "page-locked host memory, drafts and accept lengths written to it; the host reads them after "
-                       "the step's event"},
+                       "the stream has drained"},
         "gpu_launches": launches, "single_launch_step": run.s.step_is_single_launch(), "clocks": clocks, "roofline": roofline, "kernels": per_kernel,
         "warm_l2_us_per_step": 1e3 * ms_warm / args.steps,
         "wall_s_timed_region": wall, "mean_matches_per_step": plan["mean_matches_per_step"],
@@ -582,17 +708,23 @@ def ours_main(args, w):
         "backoff_from_k_max": None if ablation is None else backoff,
         "sliding_window": None if ablation is None else {"us_per_sdms_trim_call": trim_us,
                                                           "what": "all paths full, trimmed to their newer half"},
-        "other_workloads_build_only": others,
-        "scan_kernel_at_scale": None if scale is None else dict(scale, frac_of_peak=scale["gbs"] / peak),
         "dag_export": {"nodes_per_layer": args.dag_nodes, "edges_per_node": args.dag_edges,
                        "us_per_sdms_get_dag_call": export_us,
                        "note": "inspection call that re-aggregates the last build's matches; not part of a step"},
     }
     if world == 1 and not args.no_cpu_baseline:
-        units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 10 ** 9, 10.0)
-        line["cpu_baseline"] = {"value": units_c / secs_c, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "us_per_step": 1e6 * secs_c / steps_c,
-                                "sample": f"{steps_c} decode steps of {w.name} ({runs_c} run(s) from the warm start)"}
+        # the oracle as it stands: single-threaded, and with its thread fan-out over query paths on all host cores
+        cores = os.cpu_count() or 1
+        legs = {}
+        for threads in sorted({1, cores}):
+            units_c, secs_c, steps_c, runs_c = oracle_run(w, run.tokens, run.logprobs, 10 ** 9, 8.0, threads=threads)
+            legs[threads] = {"value": units_c / secs_c, "us_per_step": 1e6 * secs_c / steps_c, "steps": steps_c, "runs": runs_c}
+        best = max(legs, key=lambda t: legs[t]["value"])
+        line["cpu_baseline"] = {"value": legs[best]["value"], "unit": UNIT, "cores": best, "kind": "oracle",
+                                "us_per_step": legs[best]["us_per_step"], "host_cores": cores,
+                                "by_threads": {str(t): legs[t] for t in legs},
+                                "sample": f"{legs[best]['steps']} decode steps of {w.name} ({legs[best]['runs']} whole run(s) from "
+                                          f"the warm start, every step timed); the faster of 1 thread and {cores} threads"}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

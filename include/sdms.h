@@ -271,8 +271,10 @@ int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream);
  *   d_offsets [P+1], d_gpos [cap]  : same meaning as in sdms_get_matches; a path
  *       shorter than k, or full, has no query and therefore no matches
  *
- * Limits and sharing: P <= SDMS_NOALLOC_MAX_PATHS, otherwise SDMS_ERR_TOO_LARGE
- * and nothing is launched.  All calls on a device share the one array; each call
+ * Limits and sharing: P <= SDMS_NOALLOC_MAX_PATHS and P * paths_per_group *
+ * capacity < 2^31 (the largest number of matches there can be, so that the int32
+ * offsets cannot wrap), otherwise SDMS_ERR_TOO_LARGE and nothing is launched;
+ * paths_per_group <= SDMS_MAX_PATHS_PER_GROUP as for a context.  All calls on a device share the one array; each call
  * zeroes the counters it uses before counting, so calls in sequence on a stream
  * are independent of each other, but two calls whose kernels overlap on the GPU
  * (different streams, different threads) race and give wrong results.  The first

@@ -21,6 +21,7 @@ ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE, ERR_TOO_LARGE
 NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
+STATUS_SEARCH_FALLBACK, STATUS_TIMEOUT = 0x40, 0x80
 NUM_KERNELS = 8
 KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim")
 

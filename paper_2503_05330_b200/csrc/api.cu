@@ -114,18 +114,44 @@ struct sdms_ctx {
 
 namespace {
 
+constexpr size_t kMaxPendingEvents = 8192;
+
+// Adds the `count` oldest recorded event pairs to the per-kernel totals (waiting for them) and hands
+// their events back to the pool.
+int drain_pending(sdms_ctx* ctx, size_t count) {
+  count = count < ctx->pending.size() ? count : ctx->pending.size();
+  for (size_t x = 0; x < count; ++x) {
+    EventPair& e = ctx->pending[x];
+    float t = 0.f;
+    if (cudaEventSynchronize(e.b) != cudaSuccess || cudaEventElapsedTime(&t, e.a, e.b) != cudaSuccess)
+      return SDMS_ERR_CUDA;
+    ctx->prof_ms[e.kernel] += t;
+    ctx->prof_n[e.kernel] += 1;
+    ctx->pool.push_back(e);
+  }
+  ctx->pending.erase(ctx->pending.begin(), ctx->pending.begin() + count);
+  return SDMS_OK;
+}
+
 template <class F>
 int timed(sdms_ctx* ctx, int kernel, cudaStream_t stream, F launch) {
   EventPair ev{};
   if (ctx->profiling) {
     if (!ctx->pool.empty()) { ev = ctx->pool.back(); ctx->pool.pop_back(); }
-    else if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) return SDMS_ERR_CUDA;
+    else {
+      if (cudaEventCreate(&ev.a) != cudaSuccess) return SDMS_ERR_CUDA;
+      if (cudaEventCreate(&ev.b) != cudaSuccess) { cudaEventDestroy(ev.a); return SDMS_ERR_CUDA; }
+    }
     ev.kernel = kernel;
     cudaEventRecord(ev.a, stream);
   }
   const cudaError_t e = launch();
   ++ctx->launches;
-  if (ctx->profiling) { cudaEventRecord(ev.b, stream); ctx->pending.push_back(ev); }
+  if (ctx->profiling) {
+    cudaEventRecord(ev.b, stream);
+    ctx->pending.push_back(ev);
+    if (ctx->pending.size() >= kMaxPendingEvents) drain_pending(ctx, kMaxPendingEvents / 2);   // a long loop that never reads
+  }
   return e == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
@@ -409,15 +435,8 @@ int sdms_profile_enable(sdms_ctx* ctx, int32_t on) {
 
 int sdms_profile_read(sdms_ctx* ctx, float* ms, uint64_t* launches) {
   if (!ctx || !ms || !launches) return SDMS_ERR_INVALID_ARG;
-  for (auto& e : ctx->pending) {
-    float t = 0.f;
-    if (cudaEventSynchronize(e.b) != cudaSuccess || cudaEventElapsedTime(&t, e.a, e.b) != cudaSuccess)
-      return SDMS_ERR_CUDA;
-    ctx->prof_ms[e.kernel] += t;
-    ctx->prof_n[e.kernel] += 1;
-    ctx->pool.push_back(e);
-  }
-  ctx->pending.clear();
+  const int rc = drain_pending(ctx, ctx->pending.size());
+  if (rc != SDMS_OK) return rc;
   for (int k = 0; k < SDMS_NUM_KERNELS; ++k) {
     ms[k] = ctx->prof_ms[k]; launches[k] = ctx->prof_n[k];
     ctx->prof_ms[k] = 0.f; ctx->prof_n[k] = 0;

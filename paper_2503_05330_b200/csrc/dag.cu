@@ -484,6 +484,9 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       }
     }
     bool layer_done = false;
+    // the tags describe the layer before only until the last residue class of a pass has overwritten them with
+    // this layer's: a pass that is given up after that point and done again must not filter by them
+    bool tags_fresh = true;
     while (!layer_done) {
       if (tid == 0) { sh_best_valid = 0; sh_nnode_run = 0; sh_node_total = 0; }
       if (EXPORT && tid < MAXB) { sm.r_nedge[tid] = 0; sm.r_outdeg[tid] = 0; }
@@ -517,7 +520,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
                 v[r] = cur_v[m];
                 if (v[r] >= 0) { u[r] = d == 1 ? root : prev_v[m]; p[r] = (unsigned)roll_p[m]; }
               } else {
-                if (tagged && phase == 0 && tag[m] != cur_tag) continue;   // its token of the layer before is not the current node
+                if (tagged && phase == 0 && tags_fresh && tag[m] != cur_tag) continue;   // its token of the layer before is not the current node
                 const int gpos = mlist[m];
                 const int j = path_of(s, gpos);
                 if (gpos - j * s.L + d <= plen[j - poff] - 1) {
@@ -669,6 +672,7 @@ __device__ void dag_block(const Dev& s, const Smem& sm, int i, int M, const int3
       }
       if (overflowed && npart < npart_max) {
         npart = min(npart * 2, npart_max);          // redo the layer with smaller residue classes
+        tags_fresh = false;
       } else {
         layer_done = true;
       }

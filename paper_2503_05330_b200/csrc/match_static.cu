@@ -120,9 +120,12 @@ extern "C" int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, in
                                   int32_t* d_gpos, size_t cap, void* stream) {
   if (!d_tok || !d_len || !d_offsets || (!d_gpos && cap)) return SDMS_ERR_INVALID_ARG;
   if (num_groups < 1 || paths_per_group < 1 || capacity < 2 || k < 1 || k > SDMS_MAX_K) return SDMS_ERR_INVALID_ARG;
+  if (paths_per_group > SDMS_MAX_PATHS_PER_GROUP) return SDMS_ERR_INVALID_ARG;
   const long long P = (long long)num_groups * paths_per_group;
   if (P > SDMS_NOALLOC_MAX_PATHS) return SDMS_ERR_TOO_LARGE;          // the fixed scratch holds no more
   if (P * capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;
+  // offsets are int32: even if every position matched every query of its prompt the total must fit
+  if (P * paths_per_group * capacity > 0x7fffffffLL) return SDMS_ERR_TOO_LARGE;
   int32_t* scratch = nullptr;
   const int rc = scratch_on_current_device(&scratch);
   if (rc != SDMS_OK) return rc;

@@ -152,10 +152,13 @@ def run_protocol(pair: Pair, tokens, logprobs, k, steps, warm, commit_in_accept=
     return dict(steps=done_steps, accepted=accepted, drafted=drafted)
 
 
-def run_step_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, start_lens=None, check_matches=True):
+def run_step_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, start_lens=None, check_matches=True,
+                      check_every=1, check_dag=False):
     """The same decode protocol through the one-call step: after a first build,
     every step is accept + commit + the next build (suffix length ks[step % len(ks)])
-    in one call, compared with the oracle's accept_commit followed by build_all."""
+    in one call, compared with the oracle's accept_commit followed by build_all.
+    Accept lengths, drafts, scores and edge weights are compared after every step; the match
+    lists (and with check_dag the exported DAG) of all paths every check_every-th step."""
     P, L, D = pair.P, pair.L, pair.D
     lens = np.full(P, warm, np.int32) if start_lens is None else np.asarray(start_lens, np.int32)
     w = int(lens.max())
@@ -180,11 +183,17 @@ def run_step_protocol(pair: Pair, tokens, logprobs, ks, steps, warm, start_lens=
         assert np.array_equal(gt.cpu().numpy(), tok), (step, k)
         np.testing.assert_allclose(pair.g.draft_score.cpu().numpy(), sc, rtol=RTOL, atol=0)
         np.testing.assert_allclose(pair.g.draft_edge_w.cpu().numpy(), ew, rtol=RTOL, atol=0)
-        if check_matches:
+        if check_matches and step % check_every == 0:
             off, gpos = pair.g.matches()
             off, gpos = off.numpy(), gpos.numpy()
             for i in range(P):
                 assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), pair.o.matches(i)), (step, k, i)
+        if check_dag and pair.B > 0 and step % check_every == 0:
+            dag = pair.g.dag()
+            for i in range(P):
+                ex = pair.o.export(i, pair.B, pair.Ke)
+                for key in ex:
+                    assert np.array_equal(dag[key][i], ex[key]), (step, k, i, key)
         accepted += int(tau_o.sum())
         done_steps += 1
     pair.check_history()

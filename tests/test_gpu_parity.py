@@ -571,6 +571,43 @@ def test_heavy_query_with_wide_fan_out_in_every_layer(match_capacity):
     pair.build_and_compare(2, check_dag=False)
 
 
+def test_heavy_query_whose_successor_claims_give_up_and_the_layer_is_redone():
+    # More than 5461 matches per query again (candidates not staged; the kernel keeps a 16-bit tag of every
+    # candidate's previous token).  A is followed by B half of the time, and B by one of 150 tokens chosen so that
+    # they all hash to four neighbouring slots of the kernel's 1024-slot node table: claiming the successors of B
+    # needs runs of more than 64 probes although the table is nearly empty, so the pass is given up after it has
+    # gone over every candidate and the layer is done again with two residue classes.  The second attempt must
+    # still find every successor of B.
+    G, N, L, V, D = 1, 8, 8192, 1 << 20, 4
+    ids = np.arange(10, V, dtype=np.uint64)
+    slot = ((ids * np.uint64(2654435761)) & np.uint64(0xFFFFFFFF)) >> np.uint64(22)
+    crowd = ids[(slot >= 500) & (slot < 504)][:150].astype(np.int32)
+    assert len(crowd) == 150
+    rng = np.random.default_rng(5331)
+    tokens = rng.integers(10, 3010, size=(G * N, L)).astype(np.int32)
+    tokens[:, 0::3] = 1                                        # A
+    after = tokens[:, 1::3]
+    is_b = rng.random(after.shape) < 0.5
+    after[is_b] = 2                                            # B
+    third = tokens[:, 2::3]
+    nb = min(after.shape[1], third.shape[1])
+    pick = crowd[rng.integers(0, len(crowd), size=third.shape)]
+    third[:, :nb] = np.where(is_b[:, :nb], pick[:, :nb], third[:, :nb])
+    lps = (-rng.exponential(0.5, size=tokens.shape)).astype(np.float32)
+    pair = Pair(G, N, L, V, 2, D)
+    lens = np.array([8101, 7900, 8002, 7603, 8176, 8050, 7999, 8182], np.int32)   # all end in A
+    assert ((lens - 1) % 3 == 0).all()
+    for c in range(0, L - 8, 2048):
+        part = np.clip(lens - c, 0, 2048).astype(np.int32)
+        pair.g.append(t32(tokens[:, c:c + 2048], pair.dev), t32(lps[:, c:c + 2048], pair.dev), t32(part, pair.dev))
+        pair.o.append(tokens[:, c:c + 2048], lps[:, c:c + 2048], part)
+    assert pair.g.status() == 0
+    tok, ln = pair.build_and_compare(1, check_dag=False)
+    off, _ = pair.g.matches()
+    assert np.diff(off.numpy()).min() > 5461
+    assert (ln == D).all() and (tok[:, 0] == 2).all() and np.isin(tok[:, 1], crowd).all()
+
+
 def test_streaming_tile_scan_on_a_store_of_many_tiles():
     # more 1024-token tiles than the one-tile-per-CTA form launches: the scan streams its tiles through
     # shared-memory stages.  Ragged lengths: empty paths, paths that end inside their first tile, on a

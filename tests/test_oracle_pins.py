@@ -439,6 +439,35 @@ def test_accept_is_longest_common_prefix_exhaustive():
         assert tau[p] == len(os.path.commonprefix([list(draft), list(samp[:len(draft)])]))
 
 
+def test_accept_commit_appends_tau_plus_one_capped_by_max_append_and_cut_at_capacity():
+    # "Draft acceptance": a path takes the accepted tokens plus the model's own next one.  Histories written
+    # out by hand.  D = 4, capacity 8, four paths that all hold [7, 7, 7] except the last (7 tokens: one short
+    # of the capacity) and whose whole draft [1, 2, 3, 4] is accepted (tau = 4, so tau + 1 = 5 tokens on offer).
+    D, L = 4, 8
+    draft = np.tile(np.array([1, 2, 3, 4], np.int32), (4, 1))
+    dlen = np.array([4, 4, 2, 4], np.int32)                  # path 2 drafted two tokens only: tau = 2
+    sampled = np.tile(np.array([1, 2, 3, 4, 5], np.int32), (4, 1))
+    lp = np.full((4, D + 1), -0.25, np.float32)
+    want = {
+        # max_append: (tau, histories afterwards, status)
+        5: ([4, 4, 2, 4], [[7, 7, 7, 1, 2, 3, 4, 5], [7, 7, 7, 1, 2, 3, 4, 5], [7, 7, 7, 1, 2, 3], [7] * 7 + [1]]),
+        3: ([4, 4, 2, 4], [[7, 7, 7, 1, 2, 3], [7, 7, 7, 1, 2, 3], [7, 7, 7, 1, 2, 3], [7] * 7 + [1]]),
+        1: ([4, 4, 2, 4], [[7, 7, 7, 1], [7, 7, 7, 1], [7, 7, 7, 1], [7] * 7 + [1]]),
+    }
+    for max_append, (tau_want, hist_want) in want.items():
+        o = Oracle(1, 4, L, 10, D)
+        load_paths(o, [[7, 7, 7], [7, 7, 7], [7, 7, 7], [7] * 7], logprobs=[[-1.0] * 3] * 3 + [[-1.0] * 7])
+        tau, st = o.accept_commit(draft, dlen, sampled, lp, max_append)
+        assert tau.tolist() == tau_want                       # the clamp does not change what was accepted
+        assert st == 0                                        # running into the capacity here is not an error
+        assert [o.history(p)[0].tolist() for p in range(4)] == hist_want, max_append
+        # a full path takes nothing more and reports nothing
+        tau, st = o.accept_commit(draft, dlen, sampled, lp, max_append)
+        assert st == 0 and o.lengths()[3] == L and o.history(3)[0].tolist() == [7] * 7 + [1]
+    # the probabilities stored with the committed tokens are those of the sampled tokens
+    assert o.history(0)[1].tolist()[3:] == [oracle.prob_to_fixed(-0.25)] * 2
+
+
 def test_append_rules_and_status():
     o = Oracle(1, 4, 6, 10, 2)
     tok = np.array([[1, 2, 3, 4], [1, 2, 3, 4], [1, 99, 3, 4], [1, 2, 3, 4]], np.int32)

@@ -6,8 +6,9 @@ took the free HBM at start-up, where a late cudaMalloc can fail or stall the
 device.  It keeps its counters in a fixed array inside the library, shared by all
 calls, so the interesting failure is a second call seeing the first call's
 leftovers: the test makes two calls in a row on different states and compares
-each with sdms_build_drafts + sdms_get_matches on the same histories.  Positions
-are integers: the lists must be identical after sorting each path's slice.
+each with sdms_build_drafts + sdms_get_matches on the same histories and with the
+CPU oracle's match sets (Eq. 3 by brute force).  Positions are integers: the
+lists must be identical after sorting each path's slice.
 """
 import numpy as np
 import pytest
@@ -15,6 +16,7 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
+from oracle import Oracle  # noqa: E402
 from paper_2503_05330_b200 import binding, synth  # noqa: E402
 
 
@@ -29,6 +31,7 @@ def test_noalloc_matches_equal_regular_matches_on_two_calls_in_a_row():
     tokens, logprobs = synth.make_streams(w)
     dev = torch.device("cuda:0")
     s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device="cuda:0")
+    o = Oracle(w.G, w.N, w.L, w.V, w.D)
     fills = [(np.full(w.P, 700, np.int32) - np.arange(w.P) * 11).astype(np.int32),      # ragged
              np.full(w.P, 300, np.int32)]                                              # then 300 more each
     filled = np.zeros(w.P, np.int32)
@@ -39,6 +42,8 @@ def test_noalloc_matches_equal_regular_matches_on_two_calls_in_a_row():
             rows[p, :add[p]] = tokens[p, filled[p]:filled[p] + add[p]]
             lps[p, :add[p]] = logprobs[p, filled[p]:filled[p] + add[p]]
         s.append(torch.from_numpy(rows).to(dev), torch.from_numpy(lps).to(dev), torch.from_numpy(add).to(dev))
+        o.append(rows, lps, add)
+        o.build_all(k)
         filled += add
         s.build_drafts(k)
         assert s.status() == 0
@@ -57,6 +62,7 @@ def test_noalloc_matches_equal_regular_matches_on_two_calls_in_a_row():
         assert np.array_equal(off, ref_off), call
         for i in range(w.P):
             assert np.array_equal(mine[i], ref[i]), (call, i)
+            assert np.array_equal(mine[i], o.matches(i)), (call, i)
         assert (gpos[int(off[-1]):] == -7).all()          # nothing written past the end
 
 

@@ -91,6 +91,14 @@ typedef struct {
   int32_t  pool_mode;            /* draft pool: 0 = weighted DAG (the method); the weaker pools of the
                                     paper's ablation: 1 = tree (merge identical prefixes only),
                                     2 = list (no merging: the heaviest single candidate)            */
+  int32_t  max_matches_per_path; /* R: 0 = every match counts, as in Eq. 3.  R > 0: of the matches a
+                                    query path has in ONE other path only the R with the largest end
+                                    positions (the most recent ones) enter the pool - defined by
+                                    position, so the result does not depend on the order in which
+                                    matches are found.  Bounds the pool at (N-1)*R candidates per query:
+                                    the paper's experiments stress a small candidate set and its
+                                    limitations the cost of aggregating over many paths           */
+  int32_t  reserved0;            /* must be 0 */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,
@@ -130,6 +138,8 @@ int sdms_append(sdms_ctx* ctx, const int32_t* d_tokens, const float* d_logprobs,
  *              at which some window of k-1, k or k+1 tokens (at least one) ends
  *              within edit distance 1 of the query; each e counts once.  The walk
  *              then starts from a virtual root in front of all matched windows.
+ *              With max_matches_per_path = R > 0 only the R matches with the largest e
+ *              per other path j are kept.
  *   candidates the up to D tokens that follow each match
  *   DAG        layer d = distinct d-th followers; edge (u,v) between layers d-1
  *              and d accumulates S = sum of fixed-point probabilities of v and

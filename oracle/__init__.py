@@ -68,15 +68,16 @@ def weight(alpha: float, S: int, cnt: int) -> float:
 class Oracle:
     """State of G prompts x N paths and the per-path draft construction."""
 
-    def __init__(self, G, N, L, V, D, alpha=1.0, mode=0, eps=0, pool=0):
+    def __init__(self, G, N, L, V, D, alpha=1.0, mode=0, eps=0, pool=0, max_matches=0):
         self.G, self.N, self.L, self.V, self.D = G, N, L, V, D
-        self.eps, self.pool = eps, pool
+        self.eps, self.pool, self.max_matches = eps, pool, max_matches
         self.P = G * N
         self.alpha, self.mode = alpha, mode
         self._l = lib()
         self._h = C.c_void_p(self._l.orc_create(G, N, L, V, D, C.c_float(alpha), mode))
         self._l.orc_set_epsilon(self._h, C.c_int(eps))
         self._l.orc_set_pool(self._h, C.c_int(pool))
+        self._l.orc_set_max_matches(self._h, C.c_int(max_matches))
 
     def __del__(self):
         if getattr(self, "_h", None):

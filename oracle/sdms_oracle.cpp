@@ -36,14 +36,17 @@
 //     mode 1 takes the best node of each layer regardless of the previous one;
 //     mode 2 replaces the greedy walk by the path of the DAG with the largest sum of
 //     node weights (not in the paper's method; its introduction motivates it);
-//   * ties go to the smallest token id.
+//   * ties go to the smallest token id;
+//   * optionally (max_matches = R > 0) a query keeps, of its matches in one source path, only
+//     the R with the largest end positions; the default keeps all, as Eq. 3 does.
 //
 // Pins (tests/, CPU only): hand-worked example from Eq. 3 / Eq. 5 with dyadic
 // probabilities; match set against regex/numpy searches and closed-form counts;
 // alpha = 0 against collections.Counter; conservation invariants; enumeration
 // of every root-to-node DAG path; fuzzy matches against exact search for every
 // string within one edit of the query; pq against 50-digit decimal arithmetic;
-// acceptance against os.path.commonprefix.  Behaviour on real model traces
+// acceptance against os.path.commonprefix; the match cap against slices of the
+// uncapped match set and a hand-worked case.  Behaviour on real model traces
 // (the paper's Table 1) is "parity unpinned": it needs the models and datasets.
 #include <cmath>
 #include <cstdint>
@@ -79,6 +82,7 @@ struct Ctx {
   int G, N, L, V, D, mode;
   int eps = 0;                                  // edit-distance tolerance of the suffix match (Eq. 4)
   int pool = 0;                                 // draft pool of the ablation: 0 DAG, 1 tree, 2 list
+  int max_matches = 0;                          // R: per (query path, source path) only the R most recent matches count; 0 = all
   double alpha;
   std::vector<std::vector<int32_t>> tok, pq;
   std::vector<PathResult> res;
@@ -162,17 +166,23 @@ void build_path(Ctx* c, int k, int i) {
     if (j == i) continue;
     const std::vector<int32_t>& yj = c->tok[j];
     int len_j = (int)yj.size();
+    const size_t first_of_j = r.matches.size();
     if (c->eps > 0) {                              // "Fuzzy Suffix Matching": each end position counts once
       for (int e = 0; e <= len_j - 2; ++e)
         if (fuzzy_end(yj, e, yi.data() + (len_i - k), k, c->eps)) r.matches.push_back({j, e});
-      continue;
+    } else {
+      for (int e = k - 1; e <= len_j - 2; ++e) {
+        bool same = true;
+        for (int t = 0; t < k; ++t)
+          if (yj[e - k + 1 + t] != yi[len_i - k + t]) { same = false; break; }
+        if (same) r.matches.push_back({j, e});
+      }
     }
-    for (int e = k - 1; e <= len_j - 2; ++e) {
-      bool same = true;
-      for (int t = 0; t < k; ++t)
-        if (yj[e - k + 1 + t] != yi[len_i - k + t]) { same = false; break; }
-      if (same) r.matches.push_back({j, e});
-    }
+    // Optional cap (Eq. 3 itself has none; the paper's experiments stress that its candidate set is small and
+    // its limitations name the cost of aggregating over many paths): of the matches of query path i in source
+    // path j only the R with the largest end position e, i.e. the most recent ones, stay in the pool.
+    if (c->max_matches > 0 && r.matches.size() - first_of_j > (size_t)c->max_matches)
+      r.matches.erase(r.matches.begin() + first_of_j, r.matches.end() - c->max_matches);   // found in ascending e
   }
   // Layered DAG: one instance per (candidate, layer).
   for (const auto& m : r.matches) {
@@ -321,6 +331,9 @@ void orc_destroy(void* h) { delete (Ctx*)h; }
 
 // Edit-distance tolerance of the suffix match (Eq. 4); 0 = exact matching.
 void orc_set_epsilon(void* h, int eps) { ((Ctx*)h)->eps = eps; }
+
+// Cap R on the matches kept per (query path, source path): the R most recent ones; 0 = no cap (Eq. 3 as printed).
+void orc_set_max_matches(void* h, int R) { ((Ctx*)h)->max_matches = R; }
 
 // Draft pool structure of the paper's ablation: 0 = DAG (the method), 1 = tree, 2 = list.
 void orc_set_pool(void* h, int pool) { ((Ctx*)h)->pool = pool; }

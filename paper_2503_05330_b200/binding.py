@@ -41,13 +41,14 @@ class SdmsConfig(C.Structure):
         ("max_draft_len", C.c_int32), ("max_append", C.c_int32), ("dag_nodes_per_layer", C.c_int32),
         ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
         ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("pool_mode", C.c_int32),
+        ("max_matches_per_path", C.c_int32), ("reserved0", C.c_int32),
     ]
 
 
 def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
-                match_capacity=0, epsilon=0, pool_mode=0) -> SdmsConfig:
+                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0) -> SdmsConfig:
     return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
-                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode)
+                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, 0)
 
 
 _lib = None

@@ -37,6 +37,7 @@ int check_config(const sdms_config* c) {
   if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
   if (c->epsilon < 0 || c->epsilon > 1 || c->pool_mode < 0 || c->pool_mode > 2) return SDMS_ERR_INVALID_ARG;
   if (c->search_mode == 2 && c->pool_mode != 0) return SDMS_ERR_INVALID_ARG;     // the best path is a path of the DAG
+  if (c->max_matches_per_path < 0 || c->reserved0 != 0) return SDMS_ERR_INVALID_ARG;
   return SDMS_OK;
 }
 
@@ -206,6 +207,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.fused = fits_fused(cfg, lay);
   d.eps = cfg->epsilon;
   d.pool = cfg->pool_mode;
+  d.R = cfg->max_matches_per_path;
   ctx->step_fits = false;                        // decided below, once the kernels' attributes are set
   unsigned char* w = ctx->ws;
   d.tok = (int32_t*)(w + lay.tok); d.pq = (int32_t*)(w + lay.pq); d.len = (int32_t*)(w + lay.len); d.rec = (int32_t*)(w + lay.rec);

@@ -1114,6 +1114,70 @@ __device__ void dag_best_path(const Dev& s, const Smem& sm, int i, int M, int ca
   if (tid == 0) draft_len[i] = emitted;
 }
 
+// Optional cap on the pool: of the matches of the query in one source path only the R with the largest end
+// positions stay.  `list` holds the query's M matches (global memory, any order) and is compacted in
+// place; the new count is returned (the same in every thread).  scratch: 4 * N shared words.
+// Paths with at most R matches keep them all; for each of the others the R-th largest end position is
+// found by bisection on the position (one counting sweep over the list per round), which needs no
+// order among the matches and one word per path and round.
+__device__ int cap_matches(const Dev& s, int g, int M, int32_t* list, int* scratch) {
+  __shared__ int sh_warp_tot[kMaxWarps];
+  __shared__ int sh_out;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int N = s.N, R = s.R, poff = g * N;
+  int* cnt = scratch; int* above = scratch + N; int* lo = scratch + 2 * N; int* hi = scratch + 3 * N;
+  for (int n = tid; n < N; n += blockDim.x) { cnt[n] = 0; lo[n] = 0; hi[n] = s.L; }
+  __syncthreads();
+  for (int m = tid; m < M; m += blockDim.x) atomicAdd(&cnt[path_of(s, list[m]) - poff], 1);
+  __syncthreads();
+  int over = 0;
+  for (int n = tid; n < N; n += blockDim.x) over |= cnt[n] > R;
+  if (!__syncthreads_or(over)) return M;
+  // invariant per path: at least R matches end at or after lo, fewer than R at or after hi
+  int rounds = 0;
+  while ((1 << rounds) < s.L) ++rounds;
+  for (int r = 0; r < rounds; ++r) {
+    for (int n = tid; n < N; n += blockDim.x) above[n] = 0;
+    __syncthreads();
+    for (int m = tid; m < M; m += blockDim.x) {
+      const int gpos = list[m];
+      const int j = path_of(s, gpos), n = j - poff;
+      if (cnt[n] > R && gpos - j * s.L >= ((lo[n] + hi[n]) >> 1)) atomicAdd(&above[n], 1);
+    }
+    __syncthreads();
+    for (int n = tid; n < N; n += blockDim.x)
+      if (cnt[n] > R) {
+        const int mid = (lo[n] + hi[n]) >> 1;
+        if (above[n] >= R) lo[n] = mid; else hi[n] = mid;
+      }
+    __syncthreads();
+  }
+  // keep what ends at or after the path's threshold; a chunk is read whole before any of it is written,
+  // and what is written lands at or before the places already read
+  if (tid == 0) sh_out = 0;
+  __syncthreads();
+  for (int base = 0; base < M; base += blockDim.x) {
+    const int m = base + tid;
+    int gpos = 0;
+    bool keep = false;
+    if (m < M) {
+      gpos = list[m];
+      const int j = path_of(s, gpos), n = j - poff;
+      keep = cnt[n] <= R || gpos - j * s.L >= lo[n];
+    }
+    const unsigned b = __ballot_sync(FULL, keep);
+    if (lane == 0) sh_warp_tot[warp] = __popc(b);
+    __syncthreads();
+    int before = sh_out;
+    for (int w = 0; w < warp; ++w) before += sh_warp_tot[w];
+    if (keep) list[before + __popc(b & ((1u << lane) - 1u))] = gpos;
+    __syncthreads();
+    if (tid == 0) { int t = sh_out; for (int w = 0; w < nwarps; ++w) t += sh_warp_tot[w]; sh_out = t; }
+    __syncthreads();
+  }
+  return sh_out;
+}
+
 // Gather + DAG + search for query path i over its M (> 0) matches in mlist
 // (shared or global memory).  Called by all threads of the CTA, after a barrier
 // that follows write_defaults.
@@ -1158,7 +1222,14 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
   const int g = i / s.N;
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + g * s.N + n);
   __syncthreads();
-  dag_phase<EXPORT>(s, sm, i, M, s.matches + s.q_off[i], sh_len, g * s.N, ldm(s.rec + (size_t)i * kRecWords + 1),
+  int32_t* const mlist = s.matches + s.q_off[i];
+  int Mk = M;
+  if (s.R > 0) {                                    // (a second pass over the same build finds nothing left to cut)
+    Mk = cap_matches(s, g, M, mlist, sm.st_tok);
+    if (threadIdx.x == 0) s.q_cursor[i] = Mk;
+    __syncthreads();
+  }
+  dag_phase<EXPORT>(s, sm, i, Mk, mlist, sh_len, g * s.N, ldm(s.rec + (size_t)i * kRecWords + 1),
                     draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
@@ -1345,7 +1416,14 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
   if (sh_M > 0 || k <= k_lo) break;
   __syncthreads();                                   // everybody has read sh_M before the next probe resets it
   }
-  const int M = sh_M;
+  int M = sh_M;
+  if (s.R > 0 && M > s.R) {                          // (uniform) the cap can only bite with more than R matches
+    const int M0 = M;
+    M = cap_matches(s, g, M0, my_matches, sm.st_tok);
+    if (M < M0 && M <= kListCap)
+      for (int x = tid; x < M; x += blockDim.x) sm.list[x] = my_matches[x];
+    __syncthreads();
+  }
   if (tid == 0) { s.q_cursor[i] = M; if (used_k) used_k[i] = M > 0 ? k : 0; }
   if (M == 0) {
     if (tid == 0) draft_len[i] = 0;

@@ -26,6 +26,7 @@ struct Dev {
   int32_t pool;                        // 0 DAG, 1 tree, 2 list
   int32_t eps;                         // edit-distance tolerance of the suffix match (0 or 1)
   int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
+  int32_t R;                           // matches kept per (query path, source path): the R most recent; 0 = all
   double alpha;
   uint32_t table_cap;                  // buckets per (prompt, n) table, power of two
   uint32_t L_magic; int32_t L_shift;   // x / L for 0 <= x < 2^31 as (x * L_magic) >> L_shift (path_of)

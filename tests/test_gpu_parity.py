@@ -686,3 +686,53 @@ def test_step_with_backoff_in_one_launch(eps):
         seen |= set(used.tolist())
     assert len(seen) >= 3
     pair.check_history()
+
+
+# ---- optional cap on the matches per (query path, source path) --------------------------------
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("R,alpha,mode,pool,eps", [(1, 1.0, 0, 0, 0), (2, 0.5, 0, 0, 0), (3, 1.0, 1, 0, 0), (2, 1.0, 0, 1, 0),
+                                                   (2, 0.5, 0, 2, 0), (2, 1.0, 0, 0, 1), (1, 1.0, 2, 0, 0)])
+def test_match_cap_dense_tiny_vocab_every_step(seed, R, alpha, mode, pool, eps):
+    G, N, L, V, D, k_max = 2, 4, 48, 3 + seed % 2, 4, 3
+    tokens, lps = synth.small_random(G * N, L, V, 8300 + seed)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, pool=pool, eps=eps, B=0 if pool else 4, Ke=3,
+                    max_matches=R)
+        start = 3 + (np.arange(G * N) * 5 + seed) % 9
+        st = run_protocol(pair, tokens, lps, k, steps=30, warm=0, start_lens=start, commit_in_accept=bool(seed % 2))
+        assert st["steps"] > 0
+
+
+@pytest.mark.parametrize("R", [1, 8, 64])
+def test_match_cap_config2_through_the_step(R):
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, max_matches=R)
+    start = 500 + (np.arange(w.P) * 37) % 300
+    st = harness.run_step_protocol(pair, tokens, lps, [1, 2, 4], steps=120, warm=0, start_lens=start, check_every=5)
+    assert st["steps"] == 120
+
+
+@pytest.mark.parametrize("R", [1, 8, 64])
+def test_match_cap_config5_heavy_queries(R):
+    # the k = 1 query with 22 938 matches keeps at most 255 * R of them
+    w = synth.WORKLOADS[5]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, B=4, Ke=2, max_append=w.D, max_matches=R)
+    start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+    pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+    for k in (1, 2):
+        pair.build_and_compare(k)
+        off, _ = pair.g.matches()
+        assert np.diff(off.numpy()).max() <= (w.N - 1) * R
+
+
+def test_match_cap_on_the_three_kernel_path_with_more_matches_than_the_cap_in_every_path():
+    G, N, L, V, D = 1, 12, 1024, 2, 3
+    tokens, lps = synth.small_random(G * N, L, V, 4243)
+    for R in (1, 5, 100):
+        pair = Pair(G, N, L, V, 2, D, match_capacity=120000, max_matches=R, B=2, Ke=2)
+        lens = (1000 - (np.arange(N) * 37) % 300).astype(np.int32)
+        pair.append(tokens[:, :1000], lps[:, :1000], lens, expect_status=0)
+        for k in (1, 2):
+            pair.build_and_compare(k)

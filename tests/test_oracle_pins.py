@@ -837,3 +837,53 @@ def test_trim_rejects_negative_counts_and_keeps_the_path():
     assert o.history(0)[0].tolist() == [1, 2, 3] and o.history(1)[0].tolist() == [1, 2]
     assert o.trim(np.array([0, 9], np.int32)) == 0
     assert o.lengths().tolist() == [0, 2]
+
+
+# ----------------------------------------------------------------------------
+# optional cap on the matches per (query path, source path)
+# ----------------------------------------------------------------------------
+def test_match_cap_hand_worked_case():
+    # query path 0 ends in token 1; source path 1 holds 1 at positions 0, 2, 4, 6 (each with a follower),
+    # source path 2 at position 1 only.  R = 2 keeps, per source path, the two largest end positions.
+    L = 12
+    paths = [[5, 1], [1, 2, 1, 3, 1, 4, 1, 6], [9, 1, 7]]
+    probs = [[0.5, 0.5], [0.5, 0.5, 0.5, 0.25, 0.5, 0.5, 0.5, 0.25], [0.5, 0.5, 0.125]]
+    full = Oracle(1, 3, L, 16, 2)
+    load_paths(full, paths, probs=probs)
+    full.build_path(1, 0)
+    assert full.matches(0).tolist() == [1 * L + 0, 1 * L + 2, 1 * L + 4, 1 * L + 6, 2 * L + 1]
+    capped = Oracle(1, 3, L, 16, 2, max_matches=2)
+    load_paths(capped, paths, probs=probs)
+    capped.build_path(1, 0)
+    assert capped.matches(0).tolist() == [1 * L + 4, 1 * L + 6, 2 * L + 1]
+    nodes, edges = capped.layer(0, 1)
+    assert nodes == {4: (Q30 // 2, 1), 6: (Q30 // 4, 1), 7: (Q30 // 8, 1)}      # followers 2 and 3 left the pool
+    assert capped.draft(0)[0].tolist() == [4, 1]
+    assert full.draft(0)[0].tolist() == [2, 1]                                    # 2 (0.5) beats 4 (0.5) on the tie rule
+    one = Oracle(1, 3, L, 16, 2, max_matches=1)
+    load_paths(one, paths, probs=probs)
+    one.build_path(1, 0)
+    assert one.matches(0).tolist() == [1 * L + 6, 2 * L + 1]
+
+
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("eps", [0, 1])
+def test_match_cap_keeps_the_last_R_of_every_source_path(seed, eps):
+    G, N, L, V, D = 2, 4, 40, 3, 3
+    tokens, lps = synth.small_random(G * N, L, V, 7300 + seed)
+    lens = (L - 1 - (np.arange(G * N) * 7 + seed) % 15).astype(np.int32)
+    full = Oracle(G, N, L, V, D, eps=eps)
+    full.append(tokens, lps, lens)
+    for R in (1, 2, 5, 1000):
+        capped = Oracle(G, N, L, V, D, eps=eps, max_matches=R)
+        capped.append(tokens, lps, lens)
+        for k in (1, 2, 3):
+            for i in range(G * N):
+                full.build_path(k, i)
+                capped.build_path(k, i)
+                m = full.matches(i)
+                want = np.concatenate([np.sort(m[m // L == j])[-R:] for j in range(G * N)]) if len(m) else m
+                assert np.array_equal(capped.matches(i), want), (R, k, i)
+                # the pool is built from the kept matches only: every first-layer count is a kept match
+                nodes, _ = capped.layer(i, 1)
+                assert sum(c for _, c in nodes.values()) == len(want)

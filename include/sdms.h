@@ -99,6 +99,13 @@ typedef struct {
                                     the paper's experiments stress a small candidate set and its
                                     limitations the cost of aggregating over many paths           */
   int32_t  reserved0;            /* must be 0 */
+  int64_t  wide_table_bytes;     /* workspace set aside for the device-wide aggregation of queries with more
+                                    than 32 matches (node tables in global memory, all SMs share one query's
+                                    candidates).  Only prompts too large for the single-launch build use it.
+                                    0 = default (40 bytes * D * tokens the context can hold / 8, at most
+                                    320 MiB), -1 = none: every query is aggregated by one thread block.  A
+                                    build whose queries need more than this falls back to one thread block
+                                    for those that did not fit; results are the same either way           */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,
@@ -306,7 +313,8 @@ int sdms_match_noalloc(const int32_t* d_tok, const int32_t* d_len, int32_t num_g
 #define SDMS_KERNEL_BUILD_FUSED 5   /* probe + scan + dag in one launch (small prompts) */
 #define SDMS_KERNEL_STEP   6        /* accept + commit + build in one launch (sdms_step) */
 #define SDMS_KERNEL_TRIM   7        /* the three launches of sdms_trim */
-#define SDMS_NUM_KERNELS   8
+#define SDMS_KERNEL_DAG_WIDE 8      /* aggregation and search of queries with many matches, all SMs */
+#define SDMS_NUM_KERNELS   9
 
 /* Number of kernels this context has launched since creation. */
 int sdms_launch_count(sdms_ctx* ctx, uint64_t* launches);

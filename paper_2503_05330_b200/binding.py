@@ -22,8 +22,8 @@ NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
 STATUS_SEARCH_FALLBACK, STATUS_TIMEOUT = 0x40, 0x80
-NUM_KERNELS = 8
-KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim")
+NUM_KERNELS = 9
+KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim", "dag_wide")
 
 EXPORTS = (
     "sdms_workspace_bytes", "sdms_create", "sdms_reset", "sdms_destroy", "sdms_append",
@@ -41,14 +41,15 @@ class SdmsConfig(C.Structure):
         ("max_draft_len", C.c_int32), ("max_append", C.c_int32), ("dag_nodes_per_layer", C.c_int32),
         ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
         ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("pool_mode", C.c_int32),
-        ("max_matches_per_path", C.c_int32), ("reserved0", C.c_int32),
+        ("max_matches_per_path", C.c_int32), ("reserved0", C.c_int32), ("wide_table_bytes", C.c_int64),
     ]
 
 
 def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
-                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0) -> SdmsConfig:
+                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0, wide_table_bytes=0) -> SdmsConfig:
     return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
-                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, 0)
+                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, 0,
+                      wide_table_bytes)
 
 
 _lib = None

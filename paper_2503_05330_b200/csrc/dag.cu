@@ -30,6 +30,7 @@
 //   prefix filter / a single arg-max over candidates.
 #include "sdms_internal.h"
 #include "append_dev.cuh"
+#include "wide_dev.cuh"
 
 namespace sdms {
 
@@ -1229,6 +1230,8 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
     if (threadIdx.x == 0) s.q_cursor[i] = Mk;
     __syncthreads();
   }
+  // more matches than a warp holds: all SMs share the work (the pass that follows this kernel)
+  if (!EXPORT && s.pool == 0 && s.mode != 2 && Mk > 32 && wide_register(s, i, Mk)) return;
   dag_phase<EXPORT>(s, sm, i, Mk, mlist, sh_len, g * s.N, ldm(s.rec + (size_t)i * kRecWords + 1),
                     draft_tok, draft_len, draft_score, draft_edge_w);
 }

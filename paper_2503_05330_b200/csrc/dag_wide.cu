@@ -1,0 +1,273 @@
+// Follower gather, DAG aggregation (Eq. 5) and the greedy walk for queries with many matches, spread
+// over the whole device.
+//
+// One CTA aggregates a query of a few dozen matches in its own shared memory (dag.cu).  A query with
+// hundreds or tens of thousands of matches keeps one SM busy for as long while the others idle, so
+// dag_kernel hands such queries over (wide_register) and this pass works through all of them at
+// once: every (match, layer) pair is one item, 128 matches are one unit of work, and the units of all
+// queries are dealt out to a grid that covers the device.  Each query owns, for every layer, a node
+// table in global memory (open addressing, one 32-byte slot per node, all slots zero when the pass
+// begins and again when it ends).  Sums are integers and every choice has a tie rule, so the atomics'
+// order cannot show in a result.
+//
+//   pass A  item (m, d): claim the slot of its follower token v in the table of layer d and add the
+//           token's probability and one count (one 64-bit add); the slot of the token before it is
+//           the neighbouring lane's.  Both slots are kept for the later passes.
+//   pass B  every node's Eq. 5 weight is final: the item offers it to the node of the token before
+//           (64-bit max on the weight's bit pattern; layer 1 offers to the root, and under the
+//           layer-wise rule every layer to a record of its own).
+//   pass C  items whose node carries exactly that largest weight compete with their token: the
+//           smallest wins (64-bit max of ~token), and its slot travels with it.
+//   pass D  the walk is one dependent load per layer; each unit walks its own query (no barrier
+//           between walk and use) and then adds the probabilities of the items on the edges the draft
+//           takes.
+//   pass E  edge weights out; the slots that were used are zeroed again.
+// Between the passes all CTAs meet at a grid barrier (bounded wait; the launch is cooperative, so all
+// CTAs are resident).
+#include "sdms_internal.h"
+
+namespace sdms {
+
+namespace {
+
+typedef unsigned long long u64;
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int kWideThreads = 512;
+constexpr int kWideChunk = 128;                      // matches per unit of work
+constexpr long long kBarrierCycles = 2000000000LL;   // about a second: a barrier that takes that long has failed
+constexpr u64 kSumMask = (1ull << kWideSumShift) - 1;
+
+__device__ __forceinline__ u64 ld_u64(const u64* p) { return __ldcg(p); }
+__device__ __forceinline__ uint32_t ld_u32(const uint32_t* p) { return __ldcg(p); }
+
+// All CTAs of the grid arrive; returns false (in every thread of the CTA) if the others did not show up in time.
+__device__ bool grid_barrier(const Dev& s, unsigned phase) {
+  __shared__ int sh_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&s.w_ctl[2], 1ull);
+    const u64 target = (u64)gridDim.x * phase;
+    const long long t0 = clock64();
+    int ok = 1;
+    while (ld_u64(&s.w_ctl[2]) < target) {
+      if (clock64() - t0 > kBarrierCycles) { ok = 0; break; }
+      __nanosleep(64);
+    }
+    __threadfence();
+    sh_ok = ok;
+  }
+  __syncthreads();
+  return sh_ok != 0;
+}
+
+__device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
+  return eq5_weight(s.alpha, sum & kSumMask, (unsigned)(sum >> kWideSumShift));
+}
+
+__global__ void __launch_bounds__(kWideThreads, 2)
+dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
+                float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
+  const u64 registered = ld_u64(&s.w_ctl[0]);
+  if (registered == 0) return;                       // the same for every CTA: nobody waits for anybody
+  const int nq = (int)(registered < (u64)kMaxWide ? registered : (u64)kMaxWide);
+  __shared__ int4 sh_desc[kMaxWide];
+  __shared__ int sh_cbase[kMaxWide + 1];
+  __shared__ int sh_warp[kWideThreads / 32];
+  __shared__ int sh_dslot[SDMS_MAX_DRAFT];
+  __shared__ int sh_emitted;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int D = s.D;
+  int lD = 0;
+  while ((1 << lD) < D) ++lD;                         // items of a unit are numbered m << lD | d - 1
+
+  // the list of queries and, by a prefix sum, the first unit of each
+  {
+    static_assert(kMaxWide == 2 * kWideThreads, "two list entries per thread");
+    int c[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int q = 2 * tid + r;
+      c[r] = 0;
+      if (q < nq) { const int4 de = __ldcg(&s.w_desc[q]); sh_desc[q] = de; c[r] = (de.y + kWideChunk - 1) / kWideChunk; }
+    }
+    int x = c[0] + c[1];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(FULL, x, o); if (lane >= o) x += y; }
+    if (lane == 31) sh_warp[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      int w = lane < kWideThreads / 32 ? sh_warp[lane] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(FULL, w, o); if (lane >= o) w += y; }
+      if (lane < kWideThreads / 32) sh_warp[lane] = w;
+    }
+    __syncthreads();
+    const int before = (warp ? sh_warp[warp - 1] : 0) + x - c[0] - c[1];
+    if (2 * tid < nq) sh_cbase[2 * tid] = before;
+    if (2 * tid + 1 < nq) sh_cbase[2 * tid + 1] = before + c[0];
+    if (tid == kWideThreads - 1) sh_cbase[nq] = before + c[0] + c[1];
+    __syncthreads();
+  }
+  const int units = sh_cbase[nq];
+
+  // unit c belongs to the last query whose first unit is not after c
+  auto query_of = [&](int c) {
+    int lo = 0, hi = nq;                              // sh_cbase[lo] <= c < sh_cbase[hi]
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (sh_cbase[mid] <= c) lo = mid; else hi = mid; }
+    return lo;
+  };
+
+  // ---- pass A: node sums -------------------------------------------------------------------------
+  for (int c = blockIdx.x; c < units; c += gridDim.x) {
+    const int q = query_of(c);
+    const int4 de = sh_desc[q];
+    const int i = de.x, M = de.y, lcap = de.z;
+    const unsigned base = (unsigned)de.w;
+    const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
+    const int32_t* list = s.matches + s.q_off[i];
+    const unsigned mask = (1u << lcap) - 1u;
+    for (int x = tid; x - lane < (nm << lD); x += blockDim.x) {     // whole warps: the lanes talk to each other
+      const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
+      const bool active = ml < nm && d <= D;
+      int v = -1, sv = -1;
+      unsigned p = 0;
+      if (active) {
+        const int gpos = list[m0 + ml];
+        const int j = path_of(s, gpos);
+        if (gpos - j * s.L + d <= __ldg(s.len + j) - 1) { v = __ldg(s.tok + gpos + d); p = (unsigned)__ldg(s.pq + gpos + d); }
+      }
+      if (v >= 0) {
+        WideSlot* tab = s.w_tab + base + ((size_t)(d - 1) << lcap);
+        unsigned h = ((unsigned)v * 2654435761u) >> (32 - lcap);
+        for (unsigned probe = 0; probe <= mask; ++probe) {
+          uint32_t key = ld_u32(&tab[h].key1);
+          if (key == 0u) key = atomicCAS(&tab[h].key1, 0u, (uint32_t)v + 1u);
+          if (key == 0u || key == (uint32_t)v + 1u) { sv = (int)h; break; }
+          h = (h + 1u) & mask;
+        }
+        if (sv >= 0) atomicAdd(&tab[sv].sum, (1ull << kWideSumShift) | (u64)p);
+        else atomicOr(s.status, SDMS_STATUS_INDEX_FULL);            // more nodes than slots: cannot happen
+      }
+      const int su = __shfl_up_sync(FULL, sv, 1);                   // the same match one layer up (unused for d = 1)
+      if (active) s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)] = make_int2(sv, su);
+    }
+  }
+  if (!grid_barrier(s, 1)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
+
+  // ---- passes B and C: the best successor of every node ------------------------------------------
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int c = blockIdx.x; c < units; c += gridDim.x) {
+      const int q = query_of(c);
+      const int4 de = sh_desc[q];
+      const int M = de.y, lcap = de.z;
+      const unsigned base = (unsigned)de.w;
+      const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
+      for (int x = tid; x < (nm << lD); x += blockDim.x) {
+        const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
+        if (d > D) continue;
+        const int2 it = s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)];
+        if (it.x < 0 || (d > 1 && s.mode != 1 && it.y < 0)) continue;
+        const WideSlot* mine = s.w_tab + base + ((size_t)(d - 1) << lcap) + it.x;
+        const u64 wbits = (u64)__double_as_longlong(weight_of(s, ld_u64(&mine->sum)));
+        u64* best_w; u64* best;
+        if (d == 1 || s.mode == 1) {
+          WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT + (d - 1);
+          best_w = &pr->succ_w; best = &pr->succ;
+        } else {
+          WideSlot* before = s.w_tab + base + ((size_t)(d - 2) << lcap) + it.y;
+          best_w = &before->succ_w; best = &before->succ;
+        }
+        if (pass == 0) {
+          atomicMax(best_w, wbits);
+        } else if (ld_u64(best_w) == wbits) {
+          const uint32_t v = ld_u32(&mine->key1) - 1u;
+          atomicMax(best, ((u64)(~v) << 32) | (u64)(unsigned)it.x);
+        }
+      }
+    }
+    if (!grid_barrier(s, 2 + pass)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
+  }
+
+  // ---- pass D: walk, then the sums of the edges taken ---------------------------------------------
+  for (int c = blockIdx.x; c < units; c += gridDim.x) {
+    const int q = query_of(c);
+    const int4 de = sh_desc[q];
+    const int i = de.x, M = de.y, lcap = de.z;
+    const unsigned base = (unsigned)de.w;
+    const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
+    if (tid == 0) {
+      const bool writer = m0 == 0;                    // the query's first unit writes the draft out
+      const WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT;
+      u64 next = ld_u64(&pr[0].succ);
+      int emitted = 0;
+      for (int d = 1; d <= D; ++d) {
+        if (s.mode == 1) next = ld_u64(&pr[d - 1].succ);
+        if (next == 0ull) break;
+        const int slot = (int)(unsigned)next;
+        const WideSlot* node = s.w_tab + base + ((size_t)(d - 1) << lcap) + slot;
+        sh_dslot[d - 1] = slot;
+        if (writer) {
+          draft_tok[(size_t)i * D + d - 1] = (int32_t)~(uint32_t)(next >> 32);
+          if (draft_score) draft_score[(size_t)i * D + d - 1] = (float)weight_of(s, ld_u64(&node->sum));
+        }
+        ++emitted;
+        if (s.mode != 1) next = ld_u64(&node->succ);
+      }
+      if (writer) draft_len[i] = emitted;
+      sh_emitted = emitted;
+    }
+    __syncthreads();
+    const int emitted = sh_emitted;
+    const int32_t* list = s.matches + s.q_off[i];
+    for (int x = tid; x < (nm << lD); x += blockDim.x) {
+      const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
+      if (d > emitted) continue;
+      const int2 it = s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)];
+      if (it.x != sh_dslot[d - 1] || (d > 1 && it.y != sh_dslot[d - 2])) continue;
+      const unsigned p = (unsigned)__ldg(s.pq + list[m0 + ml] + d);
+      atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], (1ull << kWideSumShift) | (u64)p);
+    }
+    __syncthreads();
+  }
+  if (!grid_barrier(s, 4)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
+
+  // ---- pass E: edge weights; leave the tables empty ------------------------------------------------
+  if (draft_edge_w)
+    for (int q = blockIdx.x; q < nq; q += gridDim.x) {
+      const int i = sh_desc[q].x;
+      if (tid < __ldcg(draft_len + i)) {
+        const u64 sum = ld_u64(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + tid]);
+        draft_edge_w[(size_t)i * D + tid] = (sum >> kWideSumShift) ? (float)weight_of(s, sum) : 0.0f;
+      }
+    }
+  const u64 used = ld_u64(&s.w_ctl[3]);
+  uint4* const z = reinterpret_cast<uint4*>(s.w_tab);
+  for (u64 x = (u64)blockIdx.x * blockDim.x + tid; x < 2 * used; x += (u64)gridDim.x * blockDim.x)
+    z[x] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+}  // namespace
+
+// Largest grid whose CTAs are all resident at once on the current device (0: no cooperative launch here).
+int wide_kernel_grid() {
+  int dev = 0, coop = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) { cudaGetLastError(); return 0; }
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dag_wide_kernel, kWideThreads, 0) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return sms * (per_sm < 2 ? per_sm : 2);
+}
+
+cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                            float* draft_edge_w, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(s.w_grid); cfg.blockDim = dim3(kWideThreads); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, dag_wide_kernel, s, draft_tok, draft_len, draft_score, draft_edge_w);
+}
+
+}  // namespace sdms

@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
   __shared__ long long warp_tot[32];
   __shared__ long long sh_carry;
   for (int g = threadIdx.x; g < s.G; g += blockDim.x) s.g_nscan[g] = 0;
+  if (threadIdx.x < 4 && s.w_slots) s.w_ctl[threadIdx.x] = 0ull;          // the wide pass of this build starts with an empty list
   if (threadIdx.x == 0) sh_carry = 0;
   __syncthreads();
   for (int base = 0; base < s.P; base += blockDim.x) {

@@ -17,8 +17,21 @@ constexpr int kMaxClusterPaths = 16;    // largest thread-block cluster (one CTA
 constexpr int kFusedThreads = 512;     // the single-launch build: more loads in flight while it scans
 constexpr int kDagCap = 1024;          // entries of the shared-memory node / edge tables
 constexpr int kFusedMaxTokens = 131072; // largest N*L a CTA scans on its own
+constexpr int kMaxWide = 1024;          // queries one build can hand to the device-wide aggregation pass
+constexpr int kWideSumShift = 47;       // packed node sums: count in the upper 17 bits, sum of probabilities below
+constexpr int kWideMaxMatches = (1 << 17) - 1;   // so that both parts of a packed sum fit
 
 enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
+
+// One slot of a wide query's node table of one layer (32 bytes, one sector).  All-zero = empty.
+struct WideSlot {
+  uint32_t key1;                 // token + 1
+  uint32_t unused;
+  unsigned long long sum;        // count << kWideSumShift | sum of fixed-point probabilities of the node
+  unsigned long long succ_w;     // bit pattern of the largest Eq. 5 weight among the node's successors
+  unsigned long long succ;       // ~token << 32 | slot of the successor with that weight and the smallest token; 0 = none
+};
+struct WidePred { unsigned long long succ_w, succ; };   // the same two words for the root (and, in mode 1, for each layer)
 
 // Everything a kernel needs, passed by value.
 struct Dev {
@@ -47,6 +60,15 @@ struct Dev {
   int32_t* g_nscan;                    // [G] queries of the prompt that need the scan
   int32_t* g_trim;                     // [G] a path of the prompt was trimmed: its index is rebuilt
   int32_t* matches;                    // [match_cap] global positions j*L+e
+  // device-wide aggregation of queries with many matches (dag_wide.cu); w_slots = 0: not in use
+  unsigned long long* w_ctl;           // [4] queries registered, slots handed out, barrier arrivals, end of the slots in use
+  int4* w_desc;                        // [kMaxWide] query path, matches, log2 of the slots per layer, first slot
+  WidePred* w_pred;                    // [kMaxWide][SDMS_MAX_DRAFT]
+  unsigned long long* w_edge;          // [kMaxWide][SDMS_MAX_DRAFT] packed sums of the edges the draft takes
+  WideSlot* w_tab;                     // [w_slots]
+  int2* w_item;                        // [w_slots] per (match, layer): slot of its token, slot of the token before it
+  unsigned long long w_slots;
+  int32_t w_grid;                      // CTAs of the wide pass (all resident at once)
   // DAG export of the last build
   int32_t* x_node_tok; int64_t* x_node_S; int32_t* x_node_cnt; int32_t* x_node_count;
   int32_t* x_edge_dst; int64_t* x_edge_S; int32_t* x_edge_cnt; int32_t* x_out_degree;

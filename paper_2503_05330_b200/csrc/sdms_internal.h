@@ -37,6 +37,10 @@ cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, c
                         int32_t* accept_len, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                         float* draft_edge_w, int32_t* used_k, cudaStream_t stream);
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream);
+// queries with many matches, aggregated by all SMs (dag_wide.cu)
+int wide_kernel_grid();
+cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                            float* draft_edge_w, cudaStream_t stream);
 cudaError_t dag_kernel_setup();
 cudaError_t scan_kernel_setup();
 

@@ -643,7 +643,7 @@ def test_search_modes_and_pools_through_the_probe_scan_dag_kernels(mode, pool):
         from paper_2503_05330_b200 import binding
         n0 = binding.sdms_launch_count(pair.g.ctx)
         pair.g.build_drafts(k)
-        assert binding.sdms_launch_count(pair.g.ctx) == n0 + 3        # probe, scan, dag
+        assert binding.sdms_launch_count(pair.g.ctx) == n0 + 4        # probe, scan, dag, dag_wide
 
 
 def test_trim_on_the_three_kernel_path():
@@ -736,3 +736,40 @@ def test_match_cap_on_the_three_kernel_path_with_more_matches_than_the_cap_in_ev
         pair.append(tokens[:, :1000], lps[:, :1000], lens, expect_status=0)
         for k in (1, 2):
             pair.build_and_compare(k)
+
+
+# ---- queries with many matches, aggregated by all SMs (probe / scan / dag / dag_wide kernels) ----
+@pytest.mark.parametrize("wide_table_bytes", [0, 40 * 16 * 4096, -1])
+@pytest.mark.parametrize("alpha,mode", [(1.0, 0), (0.5, 0), (1.0, 1)])
+def test_wide_pass_and_its_fallbacks_agree_with_the_oracle(wide_table_bytes, alpha, mode):
+    # two-token alphabet: every k = 1 query has thousands of matches and every layer two nodes; k = 3 a few
+    # hundred.  Default tables hold every query; 40 * 16 * 4096 bytes hold a few and the others are aggregated
+    # by their own thread block; -1 switches the pass off.
+    G, N, L, V, D = 2, 12, 1024, 2, 5
+    tokens, lps = synth.small_random(G * N, L, V, 4250)
+    pair = Pair(G, N, L, V, 3, D, match_capacity=300000, alpha=alpha, mode=mode, wide_table_bytes=wide_table_bytes, B=2, Ke=2)
+    lens = (1000 - (np.arange(G * N) * 37) % 300).astype(np.int32)
+    pair.append(tokens[:, :1000], lps[:, :1000], lens, expect_status=0)
+    for k in (1, 3, 2, 1):
+        pair.build_and_compare(k)
+        lens = pair.o.lengths()
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
+        pair.accept_and_compare(sampled, sampled_lp)
+    pair.check_history()
+
+
+def test_wide_pass_with_many_distinct_followers_and_ragged_ends():
+    # vocabulary of 50 over 40 paths: k = 1 finds ~700 matches per query fanning out into all 50 tokens in every
+    # layer; paths of very different lengths, so many candidates end before the last layer
+    G, N, L, V, D = 3, 40, 900, 50, 16
+    tokens, lps = synth.small_random(G * N, L, V, 4251)
+    pair = Pair(G, N, L, V, 2, D, match_capacity=4000000, alpha=0.5)      # below P*N*L: probe / scan / dag / dag_wide
+    lens = (890 - (np.arange(G * N) * 131) % 880).astype(np.int32)
+    pair.append(tokens[:, :890], lps[:, :890], lens, expect_status=0)
+    for k in (1, 2):
+        pair.build_and_compare(k, check_dag=False)
+    from paper_2503_05330_b200 import binding
+    binding.sdms_profile_enable(pair.g.ctx, True)
+    pair.g.build_drafts(1)
+    prof = binding.sdms_profile_read(pair.g.ctx)
+    assert prof["dag_wide"][1] == 1

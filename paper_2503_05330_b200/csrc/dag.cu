@@ -1214,6 +1214,10 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
   const Smem sm = carve<EXPORT>(smem_raw);
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   const int i = blockIdx.x;
+  if (i == 0) {                                       // probe and scan are done with these: the next build finds them at zero
+    for (int x = threadIdx.x; x < s.G; x += blockDim.x) s.g_nscan[x] = 0;
+    if (threadIdx.x == 0) *s.match_cursor = 0ull;
+  }
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
   const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
   if (M == 0) {

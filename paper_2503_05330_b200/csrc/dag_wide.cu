@@ -10,10 +10,15 @@
 // begins and again when it ends).  Sums are integers and every choice has a tie rule, so the atomics'
 // order cannot show in a result.
 //
-//   pass A  item (m, d): claim the slot of its follower token v in the table of layer d and add the
-//           token's probability and one count (one 64-bit add); the slot of the token before it is
-//           the neighbouring lane's.  Both slots are kept for the later passes.
-//   pass B  every node's Eq. 5 weight is final: the item offers it to the node of the token before
+// Within a unit a thread owns one match and every fourth layer, so the lanes of a warp hold 32
+// matches at the SAME layer: lanes whose items fall on the same node (or the same edge) are found
+// with __match_any_sync and send ONE atomic for the group.  Popular n-grams are followed by the same
+// tokens over and over; without this thousands of adds queue up on one address in L2.
+//
+//   pass A  item (m, d): the group's leader claims the slot of the follower token v in the table of
+//           layer d and adds the group's probabilities and count (one 64-bit add).  Every item notes
+//           its slot.
+//   pass B  every node's Eq. 5 weight is final: an item offers it to the node of the token before it
 //           (64-bit max on the weight's bit pattern; layer 1 offers to the root, and under the
 //           layer-wise rule every layer to a record of its own).
 //   pass C  items whose node carries exactly that largest weight compete with their token: the
@@ -33,36 +38,44 @@ namespace {
 typedef unsigned long long u64;
 constexpr unsigned FULL = 0xffffffffu;
 constexpr int kWideThreads = 512;
-constexpr int kWideChunk = 128;                      // matches per unit of work
+constexpr int kWideChunk = 128;                      // matches per unit of work: thread t owns match t % 128 ...
+constexpr int kLayerWays = kWideThreads / kWideChunk;  // ... and the layers d = t / 128 + 1, + 5, + 9, ...
+constexpr int kMaxRounds = (SDMS_MAX_DRAFT + kLayerWays - 1) / kLayerWays;
 constexpr long long kBarrierCycles = 2000000000LL;   // about a second: a barrier that takes that long has failed
 constexpr u64 kSumMask = (1ull << kWideSumShift) - 1;
 
 __device__ __forceinline__ u64 ld_u64(const u64* p) { return __ldcg(p); }
 __device__ __forceinline__ uint32_t ld_u32(const uint32_t* p) { return __ldcg(p); }
 
-// All CTAs of the grid arrive; returns false (in every thread of the CTA) if the others did not show up in time.
+// All CTAs of the grid arrive; returns false (in every thread of the CTA) if the others did not show
+// up in time.  Arrivals are spread over kWideBarrierWays counters in lines of their own (hundreds of
+// atomics on one address take microseconds); one thread per counter waits for it.
 __device__ bool grid_barrier(const Dev& s, unsigned phase) {
-  __shared__ int sh_ok;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&s.w_ctl[2], 1ull);
-    const u64 target = (u64)gridDim.x * phase;
+  int ok = 1;
+  const int t = threadIdx.x;
+  if (t < kWideBarrierWays) {
+    u64* ctr = s.w_ctl + kWideBarrierAt + t * kWideBarrierStride;
+    if (t == (int)(blockIdx.x & (kWideBarrierWays - 1))) { __threadfence(); atomicAdd(ctr, 1ull); }
+    const u64 target = (u64)((gridDim.x + kWideBarrierWays - 1 - t) / kWideBarrierWays) * phase;
     const long long t0 = clock64();
-    int ok = 1;
-    while (ld_u64(&s.w_ctl[2]) < target) {
+    while (ld_u64(ctr) < target) {
       if (clock64() - t0 > kBarrierCycles) { ok = 0; break; }
-      __nanosleep(64);
+      __nanosleep(32);
     }
     __threadfence();
-    sh_ok = ok;
   }
-  __syncthreads();
-  return sh_ok != 0;
+  return __syncthreads_and(ok) != 0;
 }
 
 __device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
   return eq5_weight(s.alpha, sum & kSumMask, (unsigned)(sum >> kWideSumShift));
+}
+
+// sum of p over the lanes of `group` (every lane of the group calls with the same mask); p < 2^31
+__device__ __forceinline__ u64 group_sum(unsigned group, unsigned p) {
+  const unsigned lo = __reduce_add_sync(group, p & 0xffffu), hi = __reduce_add_sync(group, p >> 16);
+  return ((u64)hi << 16) + lo;
 }
 
 __global__ void __launch_bounds__(kWideThreads, 2)
@@ -78,8 +91,7 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
   __shared__ int sh_emitted;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = s.D;
-  int lD = 0;
-  while ((1 << lD) < D) ++lD;                         // items of a unit are numbered m << lD | d - 1
+  const int ml = tid & (kWideChunk - 1), d_first = tid / kWideChunk + 1;   // d_first is the same in all lanes of a warp
 
   // the list of queries and, by a prefix sum, the first unit of each
   {
@@ -125,32 +137,45 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     const int i = de.x, M = de.y, lcap = de.z;
     const unsigned base = (unsigned)de.w;
     const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
-    const int32_t* list = s.matches + s.q_off[i];
     const unsigned mask = (1u << lcap) - 1u;
-    for (int x = tid; x - lane < (nm << lD); x += blockDim.x) {     // whole warps: the lanes talk to each other
-      const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
-      const bool active = ml < nm && d <= D;
-      int v = -1, sv = -1;
-      unsigned p = 0;
-      if (active) {
-        const int gpos = list[m0 + ml];
-        const int j = path_of(s, gpos);
-        if (gpos - j * s.L + d <= __ldg(s.len + j) - 1) { v = __ldg(s.tok + gpos + d); p = (unsigned)__ldg(s.pq + gpos + d); }
-      }
-      if (v >= 0) {
+    int* const item = s.w_item + base + m0 + ml;      // + (d - 1) * M: the item's slot, layer by layer
+    int gpos = 0, n_m = 0;
+    if (ml < nm) {
+      gpos = s.matches[(size_t)s.q_off[i] + m0 + ml];
+      const int j = path_of(s, gpos);
+      n_m = min(D, __ldg(s.len + j) - 1 - (gpos - j * s.L));
+    }
+    int v[kMaxRounds];
+    unsigned p[kMaxRounds];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {            // every follower this thread needs is asked for before the first is used
+      const int d = d_first + r * kLayerWays;
+      v[r] = -1; p[r] = 0u;
+      if (d <= n_m) { v[r] = __ldg(s.tok + gpos + d); p[r] = (unsigned)__ldg(s.pq + gpos + d); }
+    }
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_first + r * kLayerWays;
+      if (d > D) break;                                // the same for the whole warp
+      const int vv = v[r];
+      const unsigned group = __match_any_sync(FULL, vv);            // lanes whose items are the same node
+      const int leader = __ffs(group) - 1;
+      const u64 add = ((u64)__popc(group) << kWideSumShift) | group_sum(group, p[r]);
+      int sv = -1;
+      if (vv >= 0 && lane == leader) {
         WideSlot* tab = s.w_tab + base + ((size_t)(d - 1) << lcap);
-        unsigned h = ((unsigned)v * 2654435761u) >> (32 - lcap);
+        unsigned h = ((unsigned)vv * 2654435761u) >> (32 - lcap);
         for (unsigned probe = 0; probe <= mask; ++probe) {
           uint32_t key = ld_u32(&tab[h].key1);
-          if (key == 0u) key = atomicCAS(&tab[h].key1, 0u, (uint32_t)v + 1u);
-          if (key == 0u || key == (uint32_t)v + 1u) { sv = (int)h; break; }
+          if (key == 0u) key = atomicCAS(&tab[h].key1, 0u, (uint32_t)vv + 1u);
+          if (key == 0u || key == (uint32_t)vv + 1u) { sv = (int)h; break; }
           h = (h + 1u) & mask;
         }
-        if (sv >= 0) atomicAdd(&tab[sv].sum, (1ull << kWideSumShift) | (u64)p);
+        if (sv >= 0) atomicAdd(&tab[sv].sum, add);
         else atomicOr(s.status, SDMS_STATUS_INDEX_FULL);            // more nodes than slots: cannot happen
       }
-      const int su = __shfl_up_sync(FULL, sv, 1);                   // the same match one layer up (unused for d = 1)
-      if (active) s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)] = make_int2(sv, su);
+      sv = __shfl_sync(FULL, sv, leader);
+      if (ml < nm) item[(size_t)(d - 1) * M] = vv >= 0 ? sv : -1;
     }
   }
   if (!grid_barrier(s, 1)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
@@ -163,26 +188,34 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
       const int M = de.y, lcap = de.z;
       const unsigned base = (unsigned)de.w;
       const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
-      for (int x = tid; x < (nm << lD); x += blockDim.x) {
-        const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
-        if (d > D) continue;
-        const int2 it = s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)];
-        if (it.x < 0 || (d > 1 && s.mode != 1 && it.y < 0)) continue;
-        const WideSlot* mine = s.w_tab + base + ((size_t)(d - 1) << lcap) + it.x;
+      const int* const item = s.w_item + base + m0 + ml;
+#pragma unroll 1
+      for (int d = d_first; d <= D; d += kLayerWays) {
+        int sv = -1, su = -1;
+        if (ml < nm) {
+          sv = item[(size_t)(d - 1) * M];
+          if (d > 1 && s.mode != 1) su = item[(size_t)(d - 2) * M];
+        }
+        const bool on = sv >= 0 && (d == 1 || s.mode == 1 || su >= 0);
+        // items on the same edge (same node, under the layer-wise rule) bring the same offer: one lane speaks for them
+        const u64 edge = on ? ((u64)(unsigned)su << 32) | (u64)(unsigned)sv : ~(u64)lane;
+        const unsigned group = __match_any_sync(FULL, edge);
+        if (!on || lane != __ffs(group) - 1) continue;
+        const WideSlot* mine = s.w_tab + base + ((size_t)(d - 1) << lcap) + sv;
         const u64 wbits = (u64)__double_as_longlong(weight_of(s, ld_u64(&mine->sum)));
         u64* best_w; u64* best;
         if (d == 1 || s.mode == 1) {
           WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT + (d - 1);
           best_w = &pr->succ_w; best = &pr->succ;
         } else {
-          WideSlot* before = s.w_tab + base + ((size_t)(d - 2) << lcap) + it.y;
+          WideSlot* before = s.w_tab + base + ((size_t)(d - 2) << lcap) + su;
           best_w = &before->succ_w; best = &before->succ;
         }
         if (pass == 0) {
           atomicMax(best_w, wbits);
         } else if (ld_u64(best_w) == wbits) {
-          const uint32_t v = ld_u32(&mine->key1) - 1u;
-          atomicMax(best, ((u64)(~v) << 32) | (u64)(unsigned)it.x);
+          const uint32_t tok = ld_u32(&mine->key1) - 1u;
+          atomicMax(best, ((u64)(~tok) << 32) | (u64)(unsigned)sv);
         }
       }
     }
@@ -219,14 +252,17 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     }
     __syncthreads();
     const int emitted = sh_emitted;
-    const int32_t* list = s.matches + s.q_off[i];
-    for (int x = tid; x < (nm << lD); x += blockDim.x) {
-      const int ml = x >> lD, d = (x & ((1 << lD) - 1)) + 1;
-      if (d > emitted) continue;
-      const int2 it = s.w_item[(size_t)base + (size_t)(m0 + ml) * D + (d - 1)];
-      if (it.x != sh_dslot[d - 1] || (d > 1 && it.y != sh_dslot[d - 2])) continue;
-      const unsigned p = (unsigned)__ldg(s.pq + list[m0 + ml] + d);
-      atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], (1ull << kWideSumShift) | (u64)p);
+    const int* const item = s.w_item + base + m0 + ml;
+    const int gpos = ml < nm ? s.matches[(size_t)s.q_off[i] + m0 + ml] : 0;
+#pragma unroll 1
+    for (int d = d_first; d <= emitted; d += kLayerWays) {
+      bool on = false;
+      if (ml < nm) on = item[(size_t)(d - 1) * M] == sh_dslot[d - 1] && (d == 1 || item[(size_t)(d - 2) * M] == sh_dslot[d - 2]);
+      const unsigned group = __ballot_sync(FULL, on);
+      if (!on) continue;
+      const u64 sum = group_sum(group, (unsigned)__ldg(s.pq + gpos + d));
+      if (lane == __ffs(group) - 1)
+        atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
     }
     __syncthreads();
   }

@@ -24,6 +24,7 @@ namespace sdms {
 namespace {
 
 constexpr int kProbeThreads = 1024;
+constexpr unsigned FULL_MASK = 0xffffffffu;
 
 __device__ __forceinline__ long long block_exclusive_scan(long long v, long long* warp_tot, long long* total) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -50,77 +51,99 @@ __device__ __forceinline__ long long block_exclusive_scan(long long v, long long
   return before + x - v;
 }
 
-__global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
+// One warp per query path.  The path's record (length and newest tokens, one 128-byte line) gives the
+// query; the warp looks at four neighbouring buckets of the k-gram's table at a time (eight lanes per
+// bucket, one round trip).  A k-gram with at most kInlineSlots occurrences is answered here: lane sl
+// checks occurrence sl (other path, a follower exists, tokens equal) and the matches go to the
+// query's own kInlineArea slots at the front of the match list.  Any other query reserves as many slots
+// as the k-gram has occurrences behind that area (one atomic on a cursor that the build's last kernel
+// leaves at zero) and is handed to the scan.  Slices therefore lie in no particular order.
+constexpr int kProbeWarps = 8;
+constexpr int kInlineArea = 8;
+static_assert(kInlineArea >= kInlineSlots && kRecWords == 32 && kBucketWords == 8, "lane layout of the probe");
+
+__global__ void __launch_bounds__(kProbeWarps * 32) probe_kernel(Dev s, int k) {
   grid_wait();
   grid_release();
-  __shared__ long long warp_tot[32];
-  __shared__ long long sh_carry;
-  for (int g = threadIdx.x; g < s.G; g += blockDim.x) s.g_nscan[g] = 0;
-  if (threadIdx.x < 4 && s.w_slots) s.w_ctl[threadIdx.x] = 0ull;          // the wide pass of this build starts with an empty list
-  if (threadIdx.x == 0) sh_carry = 0;
-  __syncthreads();
-  for (int base = 0; base < s.P; base += blockDim.x) {
-    const int i = base + threadIdx.x;
-    int mode = Q_NONE;
-    uint32_t fp = 0, count = 0;
-    const uint32_t* bucket = nullptr;
-    int len_i = 0, g = 0;
-    if (i < s.P) {
-      len_i = s.len[i];
-      g = i / s.N;
-      if (len_i >= k && len_i < s.L) {
-        const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
-        uint64_t h = gram_init(k);
-        for (int t = 0; t < k; ++t) h = gram_step(h, q[t]);
-        h = gram_final(h);
-        fp = gram_fp(h);
-        const uint32_t* table = index_table(s, g, k);
-        uint32_t b = gram_bucket(h, s.table_cap);
-        for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
-          const uint32_t* cand = table + (size_t)b * kBucketWords;
-          const uint32_t w0 = cand[0];
-          if (w0 == fp) { bucket = cand; break; }
-          if (w0 == 0u) break;
-          b = (b + 1) & (s.table_cap - 1);
-        }
-        if (bucket) {
-          count = bucket[1];
-          mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
-        }
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * kProbeWarps + (threadIdx.x >> 5);
+  if (i >= s.P) return;                                          // whole warps
+  const int g = i / s.N;
+  const int32_t mine = s.rec[(size_t)i * kRecWords + lane];
+  const int len_i = __shfl_sync(FULL_MASK, mine, 0);
+  int mode = Q_NONE, written = 0, off = i * kInlineArea;
+  uint32_t fp = 0, count = 0;
+  if (len_i >= k && len_i < s.L) {
+    // the query, oldest token first: token x of it sits in lane k - x of the record
+    uint64_t h = gram_init(k);
+    int32_t q_last = 0;
+    for (int x = 0; x < k; ++x) { q_last = __shfl_sync(FULL_MASK, mine, k - x); h = gram_step(h, q_last); }
+    h = gram_final(h);
+    fp = gram_fp(h);
+    const uint32_t* table = index_table(s, g, k);
+    uint32_t b = gram_bucket(h, s.table_cap);
+    int found = -1;                                              // lane that holds the bucket's first word
+    uint32_t word = 0;
+    for (uint32_t probe = 0; probe < s.table_cap && found < 0; probe += 4) {
+      const uint32_t bb = (b + (lane >> 3)) & (s.table_cap - 1);
+      word = table[(size_t)bb * kBucketWords + (lane & 7)];
+      bool end = false;
+      for (int r = 0; r < 4 && found < 0 && !end; ++r) {
+        const uint32_t w0 = __shfl_sync(FULL_MASK, word, 8 * r);
+        if (w0 == fp) found = 8 * r;
+        else if (w0 == 0u) end = true;
       }
+      if (end) break;
+      b = (b + 4) & (s.table_cap - 1);
     }
-    long long total;
-    const long long off = sh_carry + block_exclusive_scan((long long)count, warp_tot, &total);
-    if (mode != Q_NONE && off + (long long)count > s.match_cap) {
-      mode = Q_NONE;
-      atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
-    }
-    if (i < s.P) {
-      int written = 0;
+    if (found >= 0) {
+      count = __shfl_sync(FULL_MASK, word, found + 1);
+      mode = count <= (uint32_t)kInlineSlots ? Q_INLINE : Q_SCAN;
       if (mode == Q_INLINE) {
-        const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
-        for (uint32_t sl = 0; sl < count; ++sl) {
-          const uint32_t lpos = bucket[2 + sl];
-          const int j = g * s.N + (int)(lpos / (uint32_t)s.L);
-          const int e = (int)(lpos % (uint32_t)s.L);
-          if (j == i || e > s.len[j] - 2) continue;
-          const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
-          bool same = true;
-          for (int t = 0; t < k; ++t) same = same && (c[t] == q[t]);
-          if (same) s.matches[off + written++] = j * s.L + e;
+        const uint32_t lpos = __shfl_sync(FULL_MASK, word, found + 2 + (lane < kInlineSlots ? lane : 0));
+        bool same = false;
+        int gpos = 0;
+        if (lane < (int)count) {
+          const int jn = (int)(lpos / (uint32_t)s.L);
+          const int j = g * s.N + jn, e = (int)(lpos - (uint32_t)jn * (uint32_t)s.L);
+          gpos = j * s.L + e;
+          if (j != i && e >= k - 1) {
+            const int len_j = s.len[j];
+            const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
+            const int32_t* q = s.tok + (size_t)i * s.L + (len_i - k);
+            same = true;
+            for (int t = 0; t < k; ++t) same = same && (c[t] == q[t]);          // no early exit: the loads go out together
+            same = same && e <= len_j - 2;
+          }
         }
-      } else if (mode == Q_SCAN) {
-        atomicAdd(&s.g_nscan[g], 1);
+        const unsigned ok = __ballot_sync(FULL_MASK, same);
+        written = __popc(ok);
+        if ((long long)off + kInlineArea > s.match_cap) {
+          if (lane == 0) atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+          mode = Q_NONE; written = 0;
+        } else if (same) {
+          s.matches[off + __popc(ok & ((1u << lane) - 1u))] = gpos;
+        }
+      } else {
+        long long at = 0;
+        if (lane == 0) at = (long long)atomicAdd(s.match_cursor, (unsigned long long)count) + (long long)s.P * kInlineArea;
+        at = __shfl_sync(FULL_MASK, at, 0);
+        if (at + (long long)count > s.match_cap) {
+          if (lane == 0) atomicOr(s.status, SDMS_STATUS_MATCH_OVERFLOW);
+          mode = Q_NONE;
+        } else {
+          off = (int)at;
+          if (lane == 0) atomicAdd(&s.g_nscan[g], 1);
+        }
       }
-      s.q_fp[i] = fp;
-      s.q_mode[i] = mode;
-      s.q_reserved[i] = mode == Q_NONE ? 0 : (int32_t)count;
-      s.q_off[i] = (int32_t)(off < s.match_cap ? off : s.match_cap);
-      s.q_cursor[i] = written;
     }
-    __syncthreads();
-    if (threadIdx.x == 0) sh_carry += total;
-    __syncthreads();
+  }
+  if (lane == 0) {
+    s.q_fp[i] = fp;
+    s.q_mode[i] = mode;
+    s.q_reserved[i] = mode == Q_NONE ? 0 : (mode == Q_INLINE ? kInlineArea : (int32_t)count);
+    s.q_off[i] = off;
+    s.q_cursor[i] = written;
   }
 }
 
@@ -129,7 +152,6 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(Dev s, int k) {
 // second only for the few that pass the first.
 constexpr int kLastBits = 65536;
 constexpr int kLast2Bits = 8192;
-constexpr unsigned FULL_MASK = 0xffffffffu;
 constexpr int kCandBuf = 64;           // entries a warp may have waiting: fewer than 32 left over plus one per lane
 __device__ __forceinline__ uint32_t last_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 16; }
 __device__ __forceinline__ uint32_t last_bit2(int32_t tok) { return ((uint32_t)tok * 0x85ebca6bu + 0x9e3779b9u) >> 19; }
@@ -218,6 +240,7 @@ __global__ void __launch_bounds__(STREAM ? kStreamThreads : kScanThreads, STREAM
 scan_kernel(Dev s, int k, int ctas, int set_slots) {
   grid_wait();
   grid_release();
+  if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_slots) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
   if (s.g_nscan[g] == 0) return;
   constexpr int TILE = STREAM ? kStreamTile : kScanTile;
@@ -465,7 +488,7 @@ __global__ void __launch_bounds__(kProbeThreads) compact_matches_kernel(Dev s, i
 }  // namespace
 
 cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
-  return launch_overlapped(probe_kernel, dim3(1), dim3(kProbeThreads), 0, stream, s, k);
+  return launch_overlapped(probe_kernel, dim3((s.P + kProbeWarps - 1) / kProbeWarps), dim3(kProbeWarps * 32), 0, stream, s, k);
 }
 
 // Called when a context is created, with its device current.

@@ -20,6 +20,9 @@ constexpr int kFusedMaxTokens = 131072; // largest N*L a CTA scans on its own
 constexpr int kMaxWide = 1024;          // queries one build can hand to the device-wide aggregation pass
 constexpr int kWideSumShift = 47;       // packed node sums: count in the upper 17 bits, sum of probabilities below
 constexpr int kWideMaxMatches = (1 << 17) - 1;   // so that both parts of a packed sum fit
+constexpr int kWideBarrierWays = 8;     // grid-barrier arrivals are spread over this many counters ...
+constexpr int kWideBarrierAt = 16, kWideBarrierStride = 16;   // ... at w_ctl[16], [32], ...: a 128-byte line each
+constexpr int kWideCtlWords = kWideBarrierAt + kWideBarrierWays * kWideBarrierStride;
 
 enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
 
@@ -57,16 +60,17 @@ struct Dev {
   int32_t* q_reserved;                 // [P] match slots reserved (index count)
   int32_t* q_off;                      // [P] start in `matches`
   int32_t* q_cursor;                   // [P] matches written
-  int32_t* g_nscan;                    // [G] queries of the prompt that need the scan
+  unsigned long long* match_cursor;    // match slots handed to scan queries by the probe; zero between builds
+  int32_t* g_nscan;                    // [G] queries of the prompt that need the scan; zero between builds
   int32_t* g_trim;                     // [G] a path of the prompt was trimmed: its index is rebuilt
   int32_t* matches;                    // [match_cap] global positions j*L+e
   // device-wide aggregation of queries with many matches (dag_wide.cu); w_slots = 0: not in use
-  unsigned long long* w_ctl;           // [4] queries registered, slots handed out, barrier arrivals, end of the slots in use
+  unsigned long long* w_ctl;           // [kWideCtlWords] queries registered, slots handed out, -, end of the slots in use; barrier counters
   int4* w_desc;                        // [kMaxWide] query path, matches, log2 of the slots per layer, first slot
   WidePred* w_pred;                    // [kMaxWide][SDMS_MAX_DRAFT]
   unsigned long long* w_edge;          // [kMaxWide][SDMS_MAX_DRAFT] packed sums of the edges the draft takes
   WideSlot* w_tab;                     // [w_slots]
-  int2* w_item;                        // [w_slots] per (match, layer): slot of its token, slot of the token before it
+  int32_t* w_item;                     // [w_slots] per (layer, match): slot of the item's token in the layer's table
   unsigned long long w_slots;
   int32_t w_grid;                      // CTAs of the wide pass (all resident at once)
   // DAG export of the last build

@@ -739,11 +739,11 @@ def test_match_cap_on_the_three_kernel_path_with_more_matches_than_the_cap_in_ev
 
 
 # ---- queries with many matches, aggregated by all SMs (probe / scan / dag / dag_wide kernels) ----
-@pytest.mark.parametrize("wide_table_bytes", [0, 40 * 16 * 4096, -1])
+@pytest.mark.parametrize("wide_table_bytes", [0, 36 * 16 * 4096, -1])
 @pytest.mark.parametrize("alpha,mode", [(1.0, 0), (0.5, 0), (1.0, 1)])
 def test_wide_pass_and_its_fallbacks_agree_with_the_oracle(wide_table_bytes, alpha, mode):
     # two-token alphabet: every k = 1 query has thousands of matches and every layer two nodes; k = 3 a few
-    # hundred.  Default tables hold every query; 40 * 16 * 4096 bytes hold a few and the others are aggregated
+    # hundred.  Default tables hold every query; 36 * 16 * 4096 bytes hold a few and the others are aggregated
     # by their own thread block; -1 switches the pass off.
     G, N, L, V, D = 2, 12, 1024, 2, 5
     tokens, lps = synth.small_random(G * N, L, V, 4250)

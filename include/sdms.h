@@ -102,7 +102,7 @@ typedef struct {
   int64_t  wide_table_bytes;     /* workspace set aside for the device-wide aggregation of queries with more
                                     than 32 matches (node tables in global memory, all SMs share one query's
                                     candidates).  Only prompts too large for the single-launch build use it.
-                                    0 = default (36 bytes * D * tokens the context can hold / 8, at most
+                                    0 = default (40 bytes * D * tokens the context can hold / 8, at most
                                     320 MiB), -1 = none: every query is aggregated by one thread block.  A
                                     build whose queries need more than this falls back to one thread block
                                     for those that did not fit; results are the same either way           */

@@ -48,6 +48,7 @@ def lib():
         l.orc_num_matches.restype = C.c_int
         l.orc_edit_distance.restype = C.c_int
         l.orc_get_draft.restype = C.c_int
+        l.orc_build_beams.restype = C.c_int
         _lib = l
     return _lib
 
@@ -149,6 +150,13 @@ class Oracle:
         tok = np.zeros(self.D, np.int32); sc = np.zeros(self.D); ew = np.zeros(self.D)
         n = self._l.orc_get_draft(self._h, C.c_int(i), _ptr(tok, C.c_int32), _ptr(sc, C.c_double), _ptr(ew, C.c_double))
         return tok[:n].copy(), sc[:n].copy(), ew[:n].copy()
+
+    def beams(self, i, B):
+        """The B best paths of the pool of path i's last build: (tokens [n][<=D] as lists, values [n])."""
+        tok = np.full((B, self.D), -1, np.int32); ln = np.zeros(B, np.int32); val = np.zeros(B)
+        n = self._l.orc_build_beams(self._h, C.c_int(i), C.c_int(B), _ptr(tok, C.c_int32), _ptr(ln, C.c_int32),
+                                    _ptr(val, C.c_double))
+        return [tok[b, :ln[b]].tolist() for b in range(n)], val[:n].copy()
 
     def drafts(self):
         tok = np.zeros((self.P, self.D), np.int32); ln = np.zeros(self.P, np.int32)

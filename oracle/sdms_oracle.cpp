@@ -76,6 +76,9 @@ struct PathResult {
   std::vector<std::map<std::pair<int, int>, Acc>> edges;  // key (u, v)
   std::vector<int> draft;
   std::vector<double> score, edge_w;
+  // several drafts (beams) of the best-path search, best first
+  std::vector<std::vector<int>> beam_tok;
+  std::vector<double> beam_value;
 };
 
 struct Ctx {
@@ -315,6 +318,65 @@ void build_path(Ctx* c, int k, int i) {
 
 struct NodeRow { int tok; int64_t S, cnt; double w; };
 
+// The B best paths of the pool instead of the single best one (several drafts per query path, e.g. for
+// tree verification; the paper's method extracts one sequence, its introduction asks for the
+// highest-likelihood one).  Same value as search mode 2: a path is worth the sum of its nodes'
+// Eq. 5 in-weights, added from its end towards its start, and only paths that run on to a leaf (or to
+// layer D) count.  Every node keeps its B best continuations:
+//   leaf (d, v):      [ w(d, v) ]
+//   otherwise:        the B best of { w(d, v) + x : x a kept continuation of a successor v' },
+// ordered by value (larger first), then by v' (smaller first), then by the rank of x in the list of
+// v'.  As long as no two different sums round to the same double (never with alpha = 1: all sums
+// are exact) this is the order "value, then token sequence read as a word", and the result is the B
+// best root-to-leaf paths of the DAG.
+struct Cont { double value; int next; int rank; };
+void build_beams(Ctx* c, int i, int B) {
+  PathResult& r = c->res[i];
+  r.beam_tok.clear(); r.beam_value.clear();
+  if (!r.valid || r.matches.empty() || B < 1) return;
+  auto better = [](const Cont& a, const Cont& b) {
+    if (a.value != b.value) return a.value > b.value;
+    if (a.next != b.next) return a.next < b.next;
+    return a.rank < b.rank;
+  };
+  std::vector<std::map<int, std::vector<Cont>>> keep(c->D);
+  for (int d = c->D; d >= 1; --d) {
+    for (const auto& kv : r.nodes[d - 1]) {
+      const double w = weight(c->alpha, kv.second.S, kv.second.cnt);
+      std::vector<Cont> cand;
+      if (d < c->D)
+        for (const auto& e : r.edges[d])            // edges between layer d and layer d + 1
+          if (e.first.first == kv.first) {
+            const std::vector<Cont>& of = keep[d].at(e.first.second);
+            for (size_t x = 0; x < of.size(); ++x) cand.push_back({w + of[x].value, e.first.second, (int)x});
+          }
+      if (cand.empty()) cand.push_back({w, -1, 0});
+      std::sort(cand.begin(), cand.end(), better);
+      if ((int)cand.size() > B) cand.resize(B);
+      keep[d - 1][kv.first] = cand;
+    }
+  }
+  std::vector<Cont> top;
+  for (const auto& kv : r.nodes[0]) {
+    if (!(c->eps > 0) && !r.edges[0].count({r.root, kv.first})) continue;   // always true with exact matching
+    const std::vector<Cont>& of = keep[0].at(kv.first);
+    for (size_t x = 0; x < of.size(); ++x) top.push_back({of[x].value, kv.first, (int)x});
+  }
+  std::sort(top.begin(), top.end(), better);
+  if ((int)top.size() > B) top.resize(B);
+  for (const Cont& t : top) {
+    std::vector<int> seq;
+    int v = t.next, rank = t.rank;
+    for (int d = 1; d <= c->D && v >= 0; ++d) {
+      seq.push_back(v);
+      const Cont& e = keep[d - 1].at(v)[rank];
+      v = e.next; rank = e.rank;
+    }
+    r.beam_tok.push_back(seq);
+    r.beam_value.push_back(t.value);
+  }
+}
+
 }  // namespace
 
 extern "C" {
@@ -393,6 +455,23 @@ void orc_build_all(void* h, int k, int nthreads) {
   for (int t = 0; t < nthreads; ++t)
     th.emplace_back([=]() { for (int i = t; i < P; i += nthreads) build_path(c, k, i); });
   for (auto& x : th) x.join();
+}
+
+// Beams of query path i from the pool of its last build (DAG pool): at most B drafts, best first.
+// tok is [B][D] (unused -1), len [B], value [B]; returns the number of beams found.
+int orc_build_beams(void* h, int i, int B, int32_t* tok, int32_t* len, double* value) {
+  Ctx* c = (Ctx*)h;
+  build_beams(c, i, B);
+  const PathResult& r = c->res[i];
+  for (int b = 0; b < B; ++b) {
+    len[b] = 0; value[b] = 0.0;
+    for (int d = 0; d < c->D; ++d) tok[(size_t)b * c->D + d] = -1;
+  }
+  for (size_t b = 0; b < r.beam_tok.size(); ++b) {
+    len[b] = (int32_t)r.beam_tok[b].size(); value[b] = r.beam_value[b];
+    for (size_t d = 0; d < r.beam_tok[b].size(); ++d) tok[b * c->D + d] = r.beam_tok[b][d];
+  }
+  return (int)r.beam_tok.size();
 }
 
 int orc_num_matches(void* h, int i) { return (int)((Ctx*)h)->res[i].matches.size(); }

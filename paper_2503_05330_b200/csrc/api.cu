@@ -13,7 +13,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, match_cursor, g_nscan, g_trim, matches;
-  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_item;
+  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_key, w_item;
   uint64_t w_slots;
   size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
   size_t total;
@@ -40,7 +40,7 @@ int check_config(const sdms_config* c) {
   if (c->epsilon < 0 || c->epsilon > 1 || c->pool_mode < 0 || c->pool_mode > 2) return SDMS_ERR_INVALID_ARG;
   if (c->search_mode == 2 && c->pool_mode != 0) return SDMS_ERR_INVALID_ARG;     // the best path is a path of the DAG
   if (c->max_matches_per_path < 0 || c->reserved0 != 0) return SDMS_ERR_INVALID_ARG;
-  if (c->wide_table_bytes < -1 || c->wide_table_bytes > (36LL << 31)) return SDMS_ERR_INVALID_ARG;   // slots are numbered in 32 bits
+  if (c->wide_table_bytes < -1 || c->wide_table_bytes > (40LL << 31)) return SDMS_ERR_INVALID_ARG;   // slots are numbered in 32 bits
   return SDMS_OK;
 }
 
@@ -77,20 +77,21 @@ Layout make_layout(const sdms_config* c) {
   l.x_node_count = take(P * D * 4);
   l.x_edge_dst = take(P * D * B * Ke * 4); l.x_edge_S = take(P * D * B * Ke * 8);
   l.x_edge_cnt = take(P * D * B * Ke * 4); l.x_out_degree = take(P * D * B * 4);
-  // node tables of the device-wide aggregation: 32 bytes per slot plus 4 per (match, layer) item
+  // node tables of the device-wide aggregation: 32 + 4 bytes per slot plus 4 per (match, layer) item
   const int64_t group_tokens = (int64_t)c->paths_per_group * c->capacity;
   const bool fused = group_tokens <= kFusedMaxTokens && (int64_t)P * group_tokens <= mc;
   int64_t wide = c->wide_table_bytes;
   if (wide == 0) {
-    wide = 36LL * (int64_t)D * (int64_t)(P * L) / 8;
+    wide = 40LL * (int64_t)D * (int64_t)(P * L) / 8;
     if (wide > (320LL << 20)) wide = 320LL << 20;
   }
-  l.w_slots = (fused || wide < 0) ? 0 : (uint64_t)wide / 36;
+  l.w_slots = (fused || wide < 0) ? 0 : (uint64_t)wide / 40;
   l.w_ctl = take((size_t)kWideCtlWords * 8);
   l.w_desc = take(l.w_slots ? (size_t)kMaxWide * 16 : 0);
   l.w_pred = take(l.w_slots ? (size_t)kMaxWide * SDMS_MAX_DRAFT * sizeof(WidePred) : 0);
   l.w_edge = take(l.w_slots ? (size_t)kMaxWide * SDMS_MAX_DRAFT * 8 : 0);
   l.w_tab = take((size_t)l.w_slots * sizeof(WideSlot));
+  l.w_key = take((size_t)l.w_slots * 4);
   l.w_item = take((size_t)l.w_slots * 4);
   l.total = o;
   return l;
@@ -243,7 +244,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.x_edge_cnt = (int32_t*)(w + lay.x_edge_cnt); d.x_out_degree = (int32_t*)(w + lay.x_out_degree);
   d.w_ctl = (unsigned long long*)(w + lay.w_ctl); d.w_desc = (int4*)(w + lay.w_desc);
   d.w_pred = (WidePred*)(w + lay.w_pred); d.w_edge = (unsigned long long*)(w + lay.w_edge);
-  d.w_tab = (WideSlot*)(w + lay.w_tab); d.w_item = (int32_t*)(w + lay.w_item);
+  d.w_tab = (WideSlot*)(w + lay.w_tab); d.w_key = (uint32_t*)(w + lay.w_key); d.w_item = (int32_t*)(w + lay.w_item);
   d.w_grid = lay.w_slots ? wide_kernel_grid() : 0;
   d.w_slots = d.w_grid > 0 ? lay.w_slots : 0;       // no cooperative launch on this device: one thread block per query
   ctx->step_fits = step_kernel_fits(d);

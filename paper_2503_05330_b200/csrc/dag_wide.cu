@@ -6,8 +6,8 @@
 // dag_kernel hands such queries over (wide_register) and this pass works through all of them at
 // once: every (match, layer) pair is one item, 128 matches are one unit of work, and the units of all
 // queries are dealt out to a grid that covers the device.  Each query owns, for every layer, a node
-// table in global memory (open addressing, one 32-byte slot per node, all slots zero when the pass
-// begins and again when it ends).  Sums are integers and every choice has a tie rule, so the atomics'
+// table in global memory (open addressing, one 32-byte slot per node and the keys apart, eight to a
+// sector; all of it zero when the pass begins and again when it ends).  Sums are integers and every choice has a tie rule, so the atomics'
 // order cannot show in a result.
 //
 // Within a unit a thread owns one match and every fourth layer, so the lanes of a warp hold 32
@@ -163,15 +163,29 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
       const u64 add = ((u64)__popc(group) << kWideSumShift) | group_sum(group, p[r]);
       int sv = -1;
       if (vv >= 0 && lane == leader) {
-        WideSlot* tab = s.w_tab + base + ((size_t)(d - 1) << lcap);
+        // linear probing, eight keys (one sector) per round trip: the longest probe run of a half-full table
+        // of a thousand nodes is some forty slots, and every round trip is paid by the whole grid
+        uint32_t* keys = s.w_key + base + ((size_t)(d - 1) << lcap);
+        const uint32_t want = (uint32_t)vv + 1u;
         unsigned h = ((unsigned)vv * 2654435761u) >> (32 - lcap);
-        for (unsigned probe = 0; probe <= mask; ++probe) {
-          uint32_t key = ld_u32(&tab[h].key1);
-          if (key == 0u) key = atomicCAS(&tab[h].key1, 0u, (uint32_t)vv + 1u);
-          if (key == 0u || key == (uint32_t)vv + 1u) { sv = (int)h; break; }
-          h = (h + 1u) & mask;
+        for (unsigned step = 0; step <= (mask >> 3) + 1u && sv < 0; ++step) {
+          const unsigned g0 = h & ~7u;
+          const uint4 ka = __ldcg(reinterpret_cast<const uint4*>(keys + g0));
+          const uint4 kb = __ldcg(reinterpret_cast<const uint4*>(keys + g0 + 4));
+          const uint32_t kk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
+#pragma unroll
+          for (unsigned x = 0; x < 8; ++x) {
+            if (x < (h & 7u) || sv >= 0) continue;
+            uint32_t key = kk[x];
+            if (key == 0u) {
+              key = atomicCAS(&keys[g0 + x], 0u, want);
+              if (key == 0u) s.w_tab[base + ((size_t)(d - 1) << lcap) + g0 + x].tok1 = want;
+            }
+            if (key == 0u || key == want) sv = (int)(g0 + x);
+          }
+          h = (g0 + 8u) & mask;
         }
-        if (sv >= 0) atomicAdd(&tab[sv].sum, add);
+        if (sv >= 0) atomicAdd(&s.w_tab[base + ((size_t)(d - 1) << lcap) + sv].sum, add);
         else atomicOr(s.status, SDMS_STATUS_INDEX_FULL);            // more nodes than slots: cannot happen
       }
       sv = __shfl_sync(FULL, sv, leader);
@@ -214,7 +228,7 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
         if (pass == 0) {
           atomicMax(best_w, wbits);
         } else if (ld_u64(best_w) == wbits) {
-          const uint32_t tok = ld_u32(&mine->key1) - 1u;
+          const uint32_t tok = ld_u32(&mine->tok1) - 1u;
           atomicMax(best, ((u64)(~tok) << 32) | (u64)(unsigned)sv);
         }
       }
@@ -281,6 +295,9 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
   uint4* const z = reinterpret_cast<uint4*>(s.w_tab);
   for (u64 x = (u64)blockIdx.x * blockDim.x + tid; x < 2 * used; x += (u64)gridDim.x * blockDim.x)
     z[x] = make_uint4(0u, 0u, 0u, 0u);
+  uint4* const zk = reinterpret_cast<uint4*>(s.w_key);              // slots are handed out in multiples of 64
+  for (u64 x = (u64)blockIdx.x * blockDim.x + tid; x < used / 4; x += (u64)gridDim.x * blockDim.x)
+    zk[x] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 }  // namespace

@@ -26,9 +26,10 @@ constexpr int kWideCtlWords = kWideBarrierAt + kWideBarrierWays * kWideBarrierSt
 
 enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
 
-// One slot of a wide query's node table of one layer (32 bytes, one sector).  All-zero = empty.
+// One slot of a wide query's node table of one layer (32 bytes, one sector).  All-zero = empty.  The keys
+// (token + 1) that the probing looks at lie in an array of their own, eight to a sector.
 struct WideSlot {
-  uint32_t key1;                 // token + 1
+  uint32_t tok1;                 // token + 1, written by whoever claimed the slot
   uint32_t unused;
   unsigned long long sum;        // count << kWideSumShift | sum of fixed-point probabilities of the node
   unsigned long long succ_w;     // bit pattern of the largest Eq. 5 weight among the node's successors
@@ -70,6 +71,7 @@ struct Dev {
   WidePred* w_pred;                    // [kMaxWide][SDMS_MAX_DRAFT]
   unsigned long long* w_edge;          // [kMaxWide][SDMS_MAX_DRAFT] packed sums of the edges the draft takes
   WideSlot* w_tab;                     // [w_slots]
+  uint32_t* w_key;                     // [w_slots] token + 1 of the node in the slot, 0 = free
   int32_t* w_item;                     // [w_slots] per (layer, match): slot of the item's token in the layer's table
   unsigned long long w_slots;
   int32_t w_grid;                      // CTAs of the wide pass (all resident at once)

@@ -887,3 +887,76 @@ def test_match_cap_keeps_the_last_R_of_every_source_path(seed, eps):
                 # the pool is built from the kept matches only: every first-layer count is a kept match
                 nodes, _ = capped.layer(i, 1)
                 assert sum(c for _, c in nodes.values()) == len(want)
+
+
+# ----------------------------------------------------------------------------
+# several drafts per path: the B best paths of the pool
+# ----------------------------------------------------------------------------
+def brute_force_beams(paths, layers, alpha, D, B):
+    """All paths that end at a leaf or at depth D, each worth the sum of its node weights added from the
+    last node towards the first; the B best by (value, larger first; token sequence as a word, smaller first)."""
+    maximal = [p for p in paths if p and (len(p) == D or not any(len(q) == len(p) + 1 and q[:len(p)] == p for q in paths))]
+    scored = []
+    for p in maximal:
+        total = 0.0
+        for d in range(len(p) - 1, -1, -1):
+            total = py_weight(alpha, *layers[d][0][p[d]]) + total
+        scored.append((-total, p))
+    scored.sort()
+    return [list(p) for _, p in scored[:B]], [-t for t, _ in scored[:B]]
+
+
+def test_beams_hand_worked_pool():
+    # query path ends in 9.  Candidates: 9 1 3 | 9 2 4 | 9 2 5, probabilities as listed (layer 1: 1 -> .5,
+    # 2 -> .25 + .25 = .5; layer 2: 3 -> .125, 4 -> .75, 5 -> .5).  Paths: [2 4] = 1.25, [2 5] = 1.0, [1 3] = .625.
+    paths = [[5, 9], [9, 1, 3, 7], [9, 2, 4, 7], [9, 2, 5, 7]]
+    probs = [[.5, .5], [.5, .5, .125, .5], [.5, .25, .75, .5], [.5, .25, .5, .5]]
+    o = Oracle(1, 4, 8, 10, 2, alpha=1.0, mode=2)
+    assert load_paths(o, paths, probs=probs) == 0
+    o.build_all(1)
+    toks, vals = o.beams(0, 3)
+    assert toks == [[2, 4], [2, 5], [1, 3]] and vals.tolist() == [1.25, 1.0, .625]
+    toks, vals = o.beams(0, 2)
+    assert toks == [[2, 4], [2, 5]]
+    toks, vals = o.beams(0, 8)                         # no more than there are
+    assert len(toks) == 3
+    assert o.beams(0, 1)[0] == [list(o.draft(0)[0])]   # the first beam is the best path
+    assert o.beams(1, 4)[0] == []                      # a path without matches has no beam
+
+
+def test_beams_tie_goes_to_the_smaller_word():
+    # [1 3] and [2 4] are both worth .75; [1 6] too (.5 + .25): order 1 3, 1 6, 2 4
+    paths = [[5, 9], [9, 1, 3], [9, 2, 4], [9, 1, 6]]
+    probs = [[.5, .5], [.5, .25, .25], [.5, .5, .25], [.5, .25, .25]]
+    o = Oracle(1, 4, 8, 10, 2, alpha=1.0, mode=2)
+    assert load_paths(o, paths, probs=probs) == 0
+    o.build_all(1)
+    toks, vals = o.beams(0, 3)
+    assert toks == [[1, 3], [1, 6], [2, 4]] and vals.tolist() == [.75, .75, .75]
+
+
+@pytest.mark.parametrize("seed,alpha,k", list(itertools.product(range(6), (1.0, 0.5, 0.0), (1, 2))))
+def test_beams_equal_brute_force_over_all_dag_paths(seed, alpha, k):
+    # alpha in {1, 1/2, 0} and dyadic-free sums of 30-bit fractions: every sum here is exact in binary64
+    G, N, L, V, D = 1, 5, 28 + 12 * (seed % 2), 3 + 3 * (seed % 2), 4
+    tokens, lps = synth.small_random(N, L, V, 7500 + seed)
+    rng = synth.Stream(7600 + seed)
+    lens = (5 + rng.uniform(N) * (L - 6)).astype(np.int32)
+    o = Oracle(G, N, L, V, D, alpha=alpha, mode=2)
+    o.append(tokens, lps, lens)
+    o.build_all(k)
+    seen_many = 0
+    for i in range(N):
+        root = int(tokens[i, lens[i] - 1])
+        paths, layers = all_dag_paths(o, i, root, D)
+        for B in (1, 3, 8):
+            toks, vals = o.beams(i, B)
+            if len(paths) == 1:
+                assert toks == []
+                continue
+            want, totals = brute_force_beams(paths, layers, alpha, D, B)
+            assert toks == want, (i, B)
+            assert vals.tolist() == totals
+            assert all(len(set(map(tuple, toks))) == len(toks) for _ in (0,))      # beams are distinct paths
+            seen_many += len(toks) > 1
+    assert seen_many > 0

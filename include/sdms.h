@@ -53,12 +53,15 @@ extern "C" {
 #define SDMS_STATUS_SEARCH_FALLBACK 0x40u /* search_mode 2: a path had too many matches for the best-path tables
                                             (more than about 24576 / (11 * max_draft_len)); it got the greedy draft */
 #define SDMS_STATUS_TIMEOUT        0x80u /* a bounded wait inside a kernel ran out (never expected): the build's matches are incomplete */
+#define SDMS_STATUS_TABLES_FULL    0x100u /* sdms_get_beams: the table area of the workspace (wide_table_bytes) did not hold
+                                             every path's node tables; the paths left out have no beam */
 
 #define SDMS_MAX_K      16   /* largest supported k_max           */
 #define SDMS_MAX_DRAFT  32   /* largest supported max_draft_len   */
 #define SDMS_MAX_PATHS_PER_GROUP 1024
 #define SDMS_MAX_DAG_NODES 32  /* largest dag_nodes_per_layer      */
 #define SDMS_MAX_DAG_EDGES 16  /* largest dag_edges_per_node       */
+#define SDMS_MAX_BEAMS  8      /* largest max_beams                 */
 
 typedef struct sdms_ctx sdms_ctx;
 
@@ -98,14 +101,16 @@ typedef struct {
                                     matches are found.  Bounds the pool at (N-1)*R candidates per query:
                                     the paper's experiments stress a small candidate set and its
                                     limitations the cost of aggregating over many paths           */
-  int32_t  reserved0;            /* must be 0 */
-  int64_t  wide_table_bytes;     /* workspace set aside for the device-wide aggregation of queries with more
-                                    than 32 matches (node tables in global memory, all SMs share one query's
-                                    candidates).  Only prompts too large for the single-launch build use it.
-                                    0 = default (40 bytes * D * tokens the context can hold / 8, at most
-                                    320 MiB), -1 = none: every query is aggregated by one thread block.  A
-                                    build whose queries need more than this falls back to one thread block
-                                    for those that did not fit; results are the same either way           */
+  int32_t  max_beams;            /* largest number of drafts per path that sdms_get_beams will be asked for
+                                    (0 = the call is not used; at most SDMS_MAX_BEAMS)               */
+  int64_t  wide_table_bytes;     /* workspace set aside for node tables in global memory.  Two users: on
+                                    prompts too large for the single-launch build, queries with more than 32
+                                    matches are aggregated by all SMs together; and sdms_get_beams (max_beams
+                                    > 0).  A slot costs 40 + 16 * max_beams bytes and a path with M matches
+                                    needs between 1.25 and 2.5 * M * D slots.  0 = default (room for every position
+                                    matching every query of its prompt, but at most 320 MiB), -1 = none.  A build
+                                    whose queries need more falls back to one thread block for those that
+                                    did not fit, with the same results                                    */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,
@@ -258,6 +263,25 @@ int sdms_get_matches(sdms_ctx* ctx, int32_t* d_offsets, int32_t* d_gpos, size_t 
 int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t* d_node_cnt,
                  int32_t* d_node_count, int32_t* d_edge_dst, int64_t* d_edge_S,
                  int32_t* d_edge_cnt, int32_t* d_out_degree, void* stream);
+
+/*
+ * Several drafts per path (e.g. for tree verification; the paper's method extracts one sequence, its
+ * introduction asks for the highest-likelihood one): the num_beams best paths of the DAG of the last
+ * sdms_build_drafts, 1 <= num_beams <= max_beams.  A path of the DAG is worth the sum of the Eq. 5
+ * in-weights of its nodes, added from its end towards its start in binary64 (the value search_mode 2
+ * maximises), and only paths that run on to a node without successor or to layer D count.  Every node
+ * keeps its num_beams best continuations - leaf: its own weight; otherwise the best of { own weight +
+ * a kept continuation of a successor }, ordered by value (larger first), then by the successor's token
+ * (smaller first), then by the continuation's rank - and the beams are the root's.  Unless two different
+ * sums round to the same double (never with alpha = 1) that is the order "value, then token sequence".
+ * The first beam is the search_mode 2 draft.
+ * Outputs: d_beam_tok [P][num_beams][D] (unused -1), d_beam_len [P][num_beams] (0 = no such beam),
+ * d_beam_value [P][num_beams].  DAG pool only; the histories must not have changed since the build
+ * (SDMS_ERR_BAD_STATE otherwise, also when max_beams = 0).  Paths whose tables do not fit the table area
+ * of the workspace get no beam and raise SDMS_STATUS_TABLES_FULL.
+ */
+int sdms_get_beams(sdms_ctx* ctx, int32_t num_beams, int32_t* d_beam_tok, int32_t* d_beam_len,
+                   float* d_beam_value, void* stream);
 
 /* Copies the stores: d_tok / d_pq [P][L], d_len [P] (any may be NULL). */
 int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_t* d_len, void* stream);

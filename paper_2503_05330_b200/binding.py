@@ -21,7 +21,7 @@ ERR_INVALID_ARG, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD_STATE, ERR_TOO_LARGE
 NOALLOC_MAX_PATHS = 16384
 STATUS_BAD_COUNT, STATUS_CAPACITY, STATUS_BAD_TOKEN = 0x01, 0x02, 0x04
 STATUS_BAD_LOGPROB, STATUS_INDEX_FULL, STATUS_MATCH_OVERFLOW = 0x08, 0x10, 0x20
-STATUS_SEARCH_FALLBACK, STATUS_TIMEOUT = 0x40, 0x80
+STATUS_SEARCH_FALLBACK, STATUS_TIMEOUT, STATUS_TABLES_FULL = 0x40, 0x80, 0x100
 NUM_KERNELS = 9
 KERNEL_NAMES = ("append", "probe", "scan", "dag", "accept", "build_fused", "step", "trim", "dag_wide")
 
@@ -30,7 +30,7 @@ EXPORTS = (
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff",
+    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff", "sdms_get_beams",
 )
 
 
@@ -41,14 +41,14 @@ class SdmsConfig(C.Structure):
         ("max_draft_len", C.c_int32), ("max_append", C.c_int32), ("dag_nodes_per_layer", C.c_int32),
         ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
         ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("pool_mode", C.c_int32),
-        ("max_matches_per_path", C.c_int32), ("reserved0", C.c_int32), ("wide_table_bytes", C.c_int64),
+        ("max_matches_per_path", C.c_int32), ("max_beams", C.c_int32), ("wide_table_bytes", C.c_int64),
     ]
 
 
 def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
-                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0, wide_table_bytes=0) -> SdmsConfig:
+                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0, wide_table_bytes=0, max_beams=0) -> SdmsConfig:
     return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
-                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, 0,
+                      B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, max_beams,
                       wide_table_bytes)
 
 
@@ -79,6 +79,7 @@ def lib():
         l.sdms_step_is_single_launch.argtypes = [vp, C.POINTER(C.c_int32)]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
         l.sdms_get_dag.argtypes = [vp] * 10
+        l.sdms_get_beams.argtypes = [vp, i32, vp, vp, vp, vp]
         l.sdms_debug_read_history.argtypes = [vp] * 5
         l.sdms_debug_read_query_modes.argtypes = [vp, vp, vp]
         l.sdms_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
@@ -209,6 +210,11 @@ def sdms_get_matches(ctx, offsets, gpos, stream=None):
 def sdms_get_dag(ctx, node_tok, node_S, node_cnt, node_count, edge_dst, edge_S, edge_cnt, out_degree, stream=None):
     _check(lib().sdms_get_dag(ctx, _dp(node_tok), _dp(node_S), _dp(node_cnt), _dp(node_count), _dp(edge_dst),
                               _dp(edge_S), _dp(edge_cnt), _dp(out_degree), _sp(stream)), "sdms_get_dag")
+
+
+def sdms_get_beams(ctx, num_beams, beam_tok, beam_len, beam_value, stream=None):
+    _check(lib().sdms_get_beams(ctx, num_beams, _dp(beam_tok), _dp(beam_len), _dp(beam_value), _sp(stream)),
+           "sdms_get_beams")
 
 
 def sdms_debug_read_history(ctx, tok, pq, lens, stream=None):
@@ -367,6 +373,14 @@ class Sdms:
         sdms_get_dag(self.ctx, r["node_tok"], r["node_S"], r["node_cnt"], r["node_count"], r["edge_dst"],
                      r["edge_S"], r["edge_cnt"], r["out_degree"])
         return r
+
+    def beams(self, num_beams):
+        """(tokens [P][B][D], lengths [P][B], values [P][B]) of the last build, as numpy arrays."""
+        tok = torch.empty((self.P, num_beams, self.D), dtype=torch.int32, device=self.device)
+        ln = torch.empty((self.P, num_beams), dtype=torch.int32, device=self.device)
+        val = torch.empty((self.P, num_beams), dtype=torch.float32, device=self.device)
+        sdms_get_beams(self.ctx, num_beams, tok, ln, val)
+        return tok.cpu().numpy(), ln.cpu().numpy(), val.cpu().numpy()
 
     def query_modes(self):
         modes = torch.empty(self.P, dtype=torch.int32, device=self.device)

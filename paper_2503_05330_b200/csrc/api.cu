@@ -13,7 +13,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, match_cursor, g_nscan, g_trim, matches;
-  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_key, w_item;
+  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_key, w_item, b_ent, b_ctl;
+  bool wide_on;
   uint64_t w_slots;
   size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
   size_t total;
@@ -39,7 +40,8 @@ int check_config(const sdms_config* c) {
   if (P * c->capacity > 0x7fffffffLL) return SDMS_ERR_INVALID_ARG;       // positions are int32
   if (c->epsilon < 0 || c->epsilon > 1 || c->pool_mode < 0 || c->pool_mode > 2) return SDMS_ERR_INVALID_ARG;
   if (c->search_mode == 2 && c->pool_mode != 0) return SDMS_ERR_INVALID_ARG;     // the best path is a path of the DAG
-  if (c->max_matches_per_path < 0 || c->reserved0 != 0) return SDMS_ERR_INVALID_ARG;
+  if (c->max_matches_per_path < 0 || c->max_beams < 0 || c->max_beams > SDMS_MAX_BEAMS) return SDMS_ERR_INVALID_ARG;
+  if (c->max_beams > 0 && c->pool_mode != 0) return SDMS_ERR_INVALID_ARG;        // beams are paths of the DAG
   if (c->wide_table_bytes < -1 || c->wide_table_bytes > (40LL << 31)) return SDMS_ERR_INVALID_ARG;   // slots are numbered in 32 bits
   return SDMS_OK;
 }
@@ -77,22 +79,27 @@ Layout make_layout(const sdms_config* c) {
   l.x_node_count = take(P * D * 4);
   l.x_edge_dst = take(P * D * B * Ke * 4); l.x_edge_S = take(P * D * B * Ke * 8);
   l.x_edge_cnt = take(P * D * B * Ke * 4); l.x_out_degree = take(P * D * B * 4);
-  // node tables of the device-wide aggregation: 32 + 4 bytes per slot plus 4 per (match, layer) item
+  // node tables in global memory: the device-wide aggregation of large prompts and the beams.  A slot:
+  // 32 bytes of sums, 4 of key, 4 per (match, layer) item, 16 per kept continuation
   const int64_t group_tokens = (int64_t)c->paths_per_group * c->capacity;
   const bool fused = group_tokens <= kFusedMaxTokens && (int64_t)P * group_tokens <= mc;
+  const int64_t slot_bytes = 40 + 16 * (int64_t)c->max_beams;
+  l.wide_on = !fused && c->wide_table_bytes >= 0;
   int64_t wide = c->wide_table_bytes;
   if (wide == 0) {
-    wide = 40LL * (int64_t)D * (int64_t)(P * L) / 8;
+    wide = slot_bytes * 3 * (int64_t)D * (int64_t)c->paths_per_group * (int64_t)(P * L);   // room for every position matching every query
     if (wide > (320LL << 20)) wide = 320LL << 20;
   }
-  l.w_slots = (fused || wide < 0) ? 0 : (uint64_t)wide / 40;
+  l.w_slots = (l.wide_on || (c->max_beams > 0 && wide > 0)) ? (uint64_t)wide / slot_bytes : 0;
   l.w_ctl = take((size_t)kWideCtlWords * 8);
-  l.w_desc = take(l.w_slots ? (size_t)kMaxWide * 16 : 0);
-  l.w_pred = take(l.w_slots ? (size_t)kMaxWide * SDMS_MAX_DRAFT * sizeof(WidePred) : 0);
-  l.w_edge = take(l.w_slots ? (size_t)kMaxWide * SDMS_MAX_DRAFT * 8 : 0);
+  l.b_ctl = take(8);
+  l.w_desc = take(l.wide_on ? (size_t)kMaxWide * 16 : 0);
+  l.w_pred = take(l.wide_on ? (size_t)kMaxWide * SDMS_MAX_DRAFT * sizeof(WidePred) : 0);
+  l.w_edge = take(l.wide_on ? (size_t)kMaxWide * SDMS_MAX_DRAFT * 8 : 0);
   l.w_tab = take((size_t)l.w_slots * sizeof(WideSlot));
   l.w_key = take((size_t)l.w_slots * 4);
   l.w_item = take((size_t)l.w_slots * 4);
+  l.b_ent = take((size_t)l.w_slots * 16 * c->max_beams);
   l.total = o;
   return l;
 }
@@ -245,9 +252,11 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.w_ctl = (unsigned long long*)(w + lay.w_ctl); d.w_desc = (int4*)(w + lay.w_desc);
   d.w_pred = (WidePred*)(w + lay.w_pred); d.w_edge = (unsigned long long*)(w + lay.w_edge);
   d.w_tab = (WideSlot*)(w + lay.w_tab); d.w_key = (uint32_t*)(w + lay.w_key); d.w_item = (int32_t*)(w + lay.w_item);
-  d.w_grid = lay.w_slots ? wide_kernel_grid() : 0;
-  d.w_slots = d.w_grid > 0 ? lay.w_slots : 0;       // no cooperative launch on this device: one thread block per query
+  d.w_grid = lay.wide_on ? wide_kernel_grid() : 0;   // 0 (also without cooperative launch on this device): one thread block per query
+  d.w_slots = lay.w_slots;
+  d.b_ent = (BeamEnt*)(w + lay.b_ent); d.b_ctl = (unsigned long long*)(w + lay.b_ctl); d.beam_stride = cfg->max_beams;
   ctx->step_fits = step_kernel_fits(d);
+  d.build_cluster = build_cluster_size(d);
   *out = ctx;
   return SDMS_OK;
 }
@@ -296,7 +305,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (rc != SDMS_OK) return rc;
   rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
     return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
-  if (rc == SDMS_OK && ctx->dev.w_slots)
+  if (rc == SDMS_OK && ctx->dev.w_grid > 0)
     rc = timed(ctx, SDMS_KERNEL_DAG_WIDE, st, [&] {
       return launch_dag_wide(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
   if (rc == SDMS_OK) ctx->built = true;
@@ -422,6 +431,16 @@ int sdms_get_dag(sdms_ctx* ctx, int32_t* d_node_tok, int64_t* d_node_S, int32_t*
   copy(d_edge_dst, d.x_edge_dst, ne * 4); copy(d_edge_S, d.x_edge_S, ne * 8); copy(d_edge_cnt, d.x_edge_cnt, ne * 4);
   copy(d_out_degree, d.x_out_degree, nb * 4);
   return ok ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
+int sdms_get_beams(sdms_ctx* ctx, int32_t num_beams, int32_t* d_beam_tok, int32_t* d_beam_len, float* d_beam_value,
+                   void* stream) {
+  if (!ctx || !d_beam_tok || !d_beam_len || !d_beam_value) return SDMS_ERR_INVALID_ARG;
+  if (num_beams < 1 || num_beams > SDMS_MAX_BEAMS) return SDMS_ERR_INVALID_ARG;
+  if (!ctx->built || num_beams > ctx->cfg.max_beams || ctx->dev.w_slots == 0) return SDMS_ERR_BAD_STATE;
+  const cudaError_t e = launch_beams(ctx->dev, num_beams, d_beam_tok, d_beam_len, d_beam_value, (cudaStream_t)stream);
+  ++ctx->launches;
+  return e == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
 int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_t* d_len, void* stream) {

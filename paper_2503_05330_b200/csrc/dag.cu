@@ -1255,11 +1255,97 @@ __device__ __forceinline__ bool window_head_equal(const int32_t* at, int k, cons
   return true;
 }
 
+// ---- a thread-block cluster shares the scan of its prompt ------------------------------------------
+// In the single-launch build every query that its index bucket cannot answer streams the other paths
+// of the prompt; with many such queries the same histories cross the chip once per query.  When the
+// CTAs of a launch form clusters (paths [c * csize, (c + 1) * csize) of a prompt), each CTA instead
+// scans 1 / csize of the prompt's tokens for ALL scan queries of its cluster and appends what it finds
+// to the owning path's match slice (a cursor in global memory).  Queries are exchanged through
+// distributed shared memory; two cluster barriers frame the scan.
+constexpr int kShareMinTokens = 32768;   // below this a CTA reads its prompt faster than it talks to its cluster
+constexpr int kPubWords = SDMS_MAX_K + 2;
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned cluster_rank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// word `w` of the array `local` (shared memory) as CTA `rank` of the cluster holds it
+__device__ __forceinline__ int32_t ld_cluster(const int32_t* local, unsigned rank) {
+  const uint32_t mine = (uint32_t)__cvta_generic_to_shared(local);
+  uint32_t theirs;
+  int32_t v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(theirs) : "r"(mine), "r"(rank));
+  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(theirs) : "memory");
+  return v;
+}
+
+// This CTA's share of the prompt's tokens against the nq scan queries of the cluster.  cq[q] holds
+// {path index of the query, unused, k tokens}.  16-byte chunks as in the single-CTA scan: a position
+// passes on to the full comparison only if its own token and the one before it fit.
+__device__ void shared_scan(const Dev& s, int g, int k, int nq, const int32_t (*cq)[kPubWords], const int32_t* sh_len,
+                            unsigned crank, int csize) {
+  const int tid = threadIdx.x;
+  const int32_t* gtok = s.tok + (size_t)g * s.N * s.L;
+  const int pos0 = g * s.N * s.L, slice = s.N * s.L;
+  const int per = s.L >> 2, total = s.N * per;
+  const int4* g4 = reinterpret_cast<const int4*>(gtok);
+  const int lo = (int)((long long)total * crank / csize), hi = (int)((long long)total * (crank + 1) / csize);
+  constexpr int kBatch = 8;
+  for (int base = lo; base < hi; base += kBatch * blockDim.x) {           // same trip count for every thread
+    int4 w[kBatch];
+    int e0[kBatch], e_hi[kBatch], jn[kBatch];
+#pragma unroll
+    for (int r = 0; r < kBatch; ++r) {
+      const int x = base + r * blockDim.x + tid;
+      jn[r] = x < hi ? x / per : -1;
+      e0[r] = jn[r] >= 0 ? 4 * x - jn[r] * s.L : 0;
+      e_hi[r] = jn[r] >= 0 ? sh_len[jn[r]] - 2 : -1;
+      w[r] = make_int4(-1, -1, -1, -1);
+      if (e0[r] <= e_hi[r]) w[r] = ldm(g4 + x);
+    }
+    int left[kBatch];
+#pragma unroll
+    for (int r = 0; r < kBatch; ++r) left[r] = __shfl_up_sync(FULL, w[r].w, 1);   // last token of the chunk before this one
+#pragma unroll 1
+    for (int q = 0; q < nq; ++q) {
+      const int i = cq[q][0], own = i - g * s.N;
+      const int last = cq[q][2 + k - 1], before_last = k >= 2 ? cq[q][2 + k - 2] : -1;
+      unsigned cand = 0;                                              // bit 4 r + u: position u of chunk r is a candidate
+#pragma unroll
+      for (int r = 0; r < kBatch; ++r) {
+        const int v[5] = {left[r], w[r].x, w[r].y, w[r].z, w[r].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool ok = v[u + 1] == last && jn[r] != own && e0[r] + u >= k - 1 && e0[r] + u <= e_hi[r] &&
+                          (k < 2 || v[u] == before_last || (u == 0 && (tid & 31) == 0));
+          cand |= (unsigned)ok << (4 * r + u);
+        }
+      }
+      while (cand) {
+        const int bit = __ffs(cand) - 1;
+        cand &= cand - 1;
+        const int at = 4 * (base + (bit >> 2) * (int)blockDim.x + tid) + (bit & 3);   // position within the prompt
+        if (k >= 2 && (bit & 3) == 0 && (tid & 31) == 0 && ldm(gtok + at - 1) != before_last) continue;
+        if (k >= 3 && !window_head_equal(gtok + at, k, &cq[q][2])) continue;
+        const int n = atomicAdd(&s.q_cursor[i], 1);
+        s.matches[(size_t)i * slice + n] = pos0 + at;
+      }
+    }
+  }
+}
+
 template <bool EXPORT>
 __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                             float* draft_score, float* draft_edge_w, int32_t* used_k,
-                            const int32_t* own_rec = nullptr) {
+                            const int32_t* own_rec = nullptr, int csize = 0) {
   __shared__ int sh_mode, sh_M;
+  __shared__ int32_t sh_pub[kPubWords];                     // this CTA's query as its cluster sees it: path, mode, tokens
+  __shared__ int32_t sh_cq[kMaxClusterPaths][kPubWords];    // the scan queries of the cluster
+  __shared__ int sh_nq;
   __shared__ uint32_t sh_count, sh_pos[kInlineSlots];
   __shared__ int32_t sh_q[SDMS_MAX_K];
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
@@ -1270,6 +1356,8 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
   int32_t* my_matches = s.matches + (size_t)i * slice;
 
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
+  // the cluster shares its scans (same decision in every CTA of the launch)
+  const bool share = csize > 1 && k_lo == k_hi && s.eps == 0 && (s.L & 3) == 0 && slice >= kShareMinTokens;
   // With k_lo < k_hi the suffix length backs off: the longest k in [k_lo, k_hi] that has a match wins.
   int k = k_hi;
   for (;; --k) {
@@ -1305,6 +1393,11 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
     }
     sh_mode = mode; sh_count = count; sh_M = 0;
     s.q_fp[i] = fp; s.q_mode[i] = mode; s.q_reserved[i] = mode == Q_NONE ? 0 : slice; s.q_off[i] = i * slice;
+    if (share) {
+      sh_pub[0] = i; sh_pub[1] = mode;
+      for (int t = 0; t < k; ++t) sh_pub[2 + t] = sh_q[t];
+      if (mode == Q_SCAN) s.q_cursor[i] = 0;              // the cluster's scanners count this query's matches here
+    }
   }
   __syncthreads();
   const int mode = sh_mode;
@@ -1324,6 +1417,32 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
           my_matches[at] = j * s.L + e;
         }
       }
+    }
+  }
+  if (share) {
+    cluster_sync_all();                                     // every query of the cluster is published
+    const unsigned crank = cluster_rank();
+    for (int x = tid; x < csize * (k + 2); x += blockDim.x) {
+      const int r = x / (k + 2), w = x - r * (k + 2);
+      sh_cq[r][w] = ld_cluster(&sh_pub[w], (unsigned)r);
+    }
+    __syncthreads();
+    if (tid == 0) {                                         // keep the scan queries, in rank order
+      int nq = 0;
+      for (int r = 0; r < csize; ++r)
+        if (sh_cq[r][1] == Q_SCAN) {
+          if (nq != r) for (int w = 0; w < k + 2; ++w) sh_cq[nq][w] = sh_cq[r][w];
+          ++nq;
+        }
+      sh_nq = nq;
+    }
+    __syncthreads();
+    if (sh_nq > 0) shared_scan(s, g, k, sh_nq, sh_cq, sh_len, crank, csize);
+    cluster_sync_all();                                     // all shares scanned; nobody reads a neighbour's memory any more
+    if (mode == Q_SCAN) {
+      const int M = __ldcg(s.q_cursor + i);
+      for (int x = tid; x < min(M, kListCap); x += blockDim.x) sm.list[x] = __ldcg(my_matches + x);
+      if (tid == 0) sh_M = M;
     }
   } else if (mode == Q_SCAN && s.eps > 0) {
     // Eq. 4 with tolerance 1.  A window s' is within one edit of the query q iff, with a = their common
@@ -1443,12 +1562,12 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
 template <bool EXPORT>
 __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo, int32_t* draft_tok,
                                                                   int32_t* draft_len, float* draft_score,
-                                                                  float* draft_edge_w, int32_t* used_k) {
+                                                                  float* draft_edge_w, int32_t* used_k, int csize) {
   grid_wait();
   grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
-  build_phase<EXPORT>(s, sm, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
+  build_phase<EXPORT>(s, sm, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, nullptr, csize);
 }
 
 // One launch per decode step.  The CTAs of a prompt form a thread-block cluster.  Each CTA first
@@ -1470,7 +1589,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, in
   accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec, k);
   // every thread of every CTA of the cluster gets here exactly once (no early exit above)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  build_phase<false>(s, sm, k, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, sh_own_rec);
+  build_phase<false>(s, sm, k, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, sh_own_rec, s.N);
 }
 
 }  // namespace
@@ -1487,6 +1606,8 @@ cudaError_t dag_kernel_setup() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
   if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
@@ -1532,10 +1653,41 @@ cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32
                            draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
+// Largest cluster (CTAs = consecutive paths of one prompt) that the single-launch build can run with on this
+// device, 1 if none: the cluster shares the scan of its prompt (shared_scan).
+int build_cluster_size(const Dev& s) {
+  if (!s.fused || (s.L & 3) != 0 || (long long)s.N * s.L < kShareMinTokens) return 1;
+  for (int c = kMaxClusterPaths; c >= 2; --c) {
+    if (s.N % c) continue;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(s.P); cfg.blockDim = dim3(kFusedThreads); cfg.dynamicSmemBytes = dag_smem_bytes<false>();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, build_fused_kernel<false>, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+    if (clusters >= 1) return c;
+  }
+  return 1;
+}
+
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
-  return launch_overlapped(build_fused_kernel<false>, dim3(s.P), dim3(kFusedThreads), dag_smem_bytes<false>(), stream,
-                           s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k);
+  if (s.build_cluster <= 1 || k_lo != k_hi)
+    return launch_overlapped(build_fused_kernel<false>, dim3(s.P), dim3(kFusedThreads), dag_smem_bytes<false>(), stream,
+                             s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, 0);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(s.P); cfg.blockDim = dim3(kFusedThreads);
+  cfg.dynamicSmemBytes = dag_smem_bytes<false>(); cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = s.build_cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, build_fused_kernel<false>, s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w,
+                            used_k, (int)s.build_cluster);
 }
 
 }  // namespace sdms

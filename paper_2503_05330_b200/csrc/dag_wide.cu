@@ -30,17 +30,12 @@
 // Between the passes all CTAs meet at a grid barrier (bounded wait; the launch is cooperative, so all
 // CTAs are resident).
 #include "sdms_internal.h"
+#include "wide_dev.cuh"
 
 namespace sdms {
 
 namespace {
 
-typedef unsigned long long u64;
-constexpr unsigned FULL = 0xffffffffu;
-constexpr int kWideThreads = 512;
-constexpr int kWideChunk = 128;                      // matches per unit of work: thread t owns match t % 128 ...
-constexpr int kLayerWays = kWideThreads / kWideChunk;  // ... and the layers d = t / 128 + 1, + 5, + 9, ...
-constexpr int kMaxRounds = (SDMS_MAX_DRAFT + kLayerWays - 1) / kLayerWays;
 constexpr long long kBarrierCycles = 2000000000LL;   // about a second: a barrier that takes that long has failed
 constexpr u64 kSumMask = (1ull << kWideSumShift) - 1;
 
@@ -70,12 +65,6 @@ __device__ bool grid_barrier(const Dev& s, unsigned phase) {
 
 __device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
   return eq5_weight(s.alpha, sum & kSumMask, (unsigned)(sum >> kWideSumShift));
-}
-
-// sum of p over the lanes of `group` (every lane of the group calls with the same mask); p < 2^31
-__device__ __forceinline__ u64 group_sum(unsigned group, unsigned p) {
-  const unsigned lo = __reduce_add_sync(group, p & 0xffffu), hi = __reduce_add_sync(group, p >> 16);
-  return ((u64)hi << 16) + lo;
 }
 
 __global__ void __launch_bounds__(kWideThreads, 2)
@@ -137,60 +126,8 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     const int i = de.x, M = de.y, lcap = de.z;
     const unsigned base = (unsigned)de.w;
     const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
-    const unsigned mask = (1u << lcap) - 1u;
-    int* const item = s.w_item + base + m0 + ml;      // + (d - 1) * M: the item's slot, layer by layer
-    int gpos = 0, n_m = 0;
-    if (ml < nm) {
-      gpos = s.matches[(size_t)s.q_off[i] + m0 + ml];
-      const int j = path_of(s, gpos);
-      n_m = min(D, __ldg(s.len + j) - 1 - (gpos - j * s.L));
-    }
-    int v[kMaxRounds];
-    unsigned p[kMaxRounds];
-#pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {            // every follower this thread needs is asked for before the first is used
-      const int d = d_first + r * kLayerWays;
-      v[r] = -1; p[r] = 0u;
-      if (d <= n_m) { v[r] = __ldg(s.tok + gpos + d); p[r] = (unsigned)__ldg(s.pq + gpos + d); }
-    }
-#pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {
-      const int d = d_first + r * kLayerWays;
-      if (d > D) break;                                // the same for the whole warp
-      const int vv = v[r];
-      const unsigned group = __match_any_sync(FULL, vv);            // lanes whose items are the same node
-      const int leader = __ffs(group) - 1;
-      const u64 add = ((u64)__popc(group) << kWideSumShift) | group_sum(group, p[r]);
-      int sv = -1;
-      if (vv >= 0 && lane == leader) {
-        // linear probing, eight keys (one sector) per round trip: the longest probe run of a half-full table
-        // of a thousand nodes is some forty slots, and every round trip is paid by the whole grid
-        uint32_t* keys = s.w_key + base + ((size_t)(d - 1) << lcap);
-        const uint32_t want = (uint32_t)vv + 1u;
-        unsigned h = ((unsigned)vv * 2654435761u) >> (32 - lcap);
-        for (unsigned step = 0; step <= (mask >> 3) + 1u && sv < 0; ++step) {
-          const unsigned g0 = h & ~7u;
-          const uint4 ka = __ldcg(reinterpret_cast<const uint4*>(keys + g0));
-          const uint4 kb = __ldcg(reinterpret_cast<const uint4*>(keys + g0 + 4));
-          const uint32_t kk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
-#pragma unroll
-          for (unsigned x = 0; x < 8; ++x) {
-            if (x < (h & 7u) || sv >= 0) continue;
-            uint32_t key = kk[x];
-            if (key == 0u) {
-              key = atomicCAS(&keys[g0 + x], 0u, want);
-              if (key == 0u) s.w_tab[base + ((size_t)(d - 1) << lcap) + g0 + x].tok1 = want;
-            }
-            if (key == 0u || key == want) sv = (int)(g0 + x);
-          }
-          h = (g0 + 8u) & mask;
-        }
-        if (sv >= 0) atomicAdd(&s.w_tab[base + ((size_t)(d - 1) << lcap) + sv].sum, add);
-        else atomicOr(s.status, SDMS_STATUS_INDEX_FULL);            // more nodes than slots: cannot happen
-      }
-      sv = __shfl_sync(FULL, sv, leader);
-      if (ml < nm) item[(size_t)(d - 1) * M] = vv >= 0 ? sv : -1;
-    }
+    (void)nm;
+    wide_insert_unit(s, s.matches + s.q_off[i], base, lcap, M, m0);
   }
   if (!grid_barrier(s, 1)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
 
@@ -273,8 +210,8 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
       bool on = false;
       if (ml < nm) on = item[(size_t)(d - 1) * M] == sh_dslot[d - 1] && (d == 1 || item[(size_t)(d - 2) * M] == sh_dslot[d - 2]);
       const unsigned group = __ballot_sync(FULL, on);
-      if (!on) continue;
-      const u64 sum = group_sum(group, (unsigned)__ldg(s.pq + gpos + d));
+      if (group == 0u) continue;
+      const u64 sum = group_sum(group, 0ll, on ? (unsigned)__ldg(s.pq + gpos + d) : 0u);
       if (lane == __ffs(group) - 1)
         atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
     }

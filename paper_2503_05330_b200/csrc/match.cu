@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(STREAM ? kStreamThreads : kScanThreads, STREAM
 scan_kernel(Dev s, int k, int ctas, int set_slots) {
   grid_wait();
   grid_release();
-  if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_slots) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
+  if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_grid) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
   if (s.g_nscan[g] == 0) return;
   constexpr int TILE = STREAM ? kStreamTile : kScanTile;

@@ -35,6 +35,7 @@ struct WideSlot {
   unsigned long long succ_w;     // bit pattern of the largest Eq. 5 weight among the node's successors
   unsigned long long succ;       // ~token << 32 | slot of the successor with that weight and the smallest token; 0 = none
 };
+struct BeamEnt;
 struct WidePred { unsigned long long succ_w, succ; };   // the same two words for the root (and, in mode 1, for each layer)
 
 // Everything a kernel needs, passed by value.
@@ -43,6 +44,7 @@ struct Dev {
   int32_t pool;                        // 0 DAG, 1 tree, 2 list
   int32_t eps;                         // edit-distance tolerance of the suffix match (0 or 1)
   int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
+  int32_t build_cluster;               // CTAs per cluster of the single-launch build (they share their prompt's scan); 1 = none
   int32_t R;                           // matches kept per (query path, source path): the R most recent; 0 = all
   double alpha;
   uint32_t table_cap;                  // buckets per (prompt, n) table, power of two
@@ -74,6 +76,9 @@ struct Dev {
   uint32_t* w_key;                     // [w_slots] token + 1 of the node in the slot, 0 = free
   int32_t* w_item;                     // [w_slots] per (layer, match): slot of the item's token in the layer's table
   unsigned long long w_slots;
+  BeamEnt* b_ent;                      // [w_slots][beam_stride] continuations kept per node (sdms_get_beams)
+  unsigned long long* b_ctl;           // [1] slots handed out by the beam kernel
+  int32_t beam_stride;                 // the context's max_beams
   int32_t w_grid;                      // CTAs of the wide pass (all resident at once)
   // DAG export of the last build
   int32_t* x_node_tok; int64_t* x_node_S; int32_t* x_node_cnt; int32_t* x_node_count;

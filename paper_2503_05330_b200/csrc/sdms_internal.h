@@ -33,6 +33,7 @@ cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_
 // phase 0: shift the histories; 1: empty the index tables of the prompts that changed; 2: index them again
 cudaError_t launch_trim(const Dev& s, int phase, const int32_t* keep, cudaStream_t stream);
 bool step_kernel_fits(const Dev& s);
+int build_cluster_size(const Dev& s);
 cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, const float* sampled_lp,
                         int32_t* accept_len, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                         float* draft_edge_w, int32_t* used_k, cudaStream_t stream);
@@ -41,6 +42,8 @@ cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos
 int wide_kernel_grid();
 cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                             float* draft_edge_w, cudaStream_t stream);
+cudaError_t launch_beams(const Dev& s, int B, int32_t* beam_tok, int32_t* beam_len, float* beam_value,
+                         cudaStream_t stream);
 cudaError_t dag_kernel_setup();
 cudaError_t scan_kernel_setup();
 

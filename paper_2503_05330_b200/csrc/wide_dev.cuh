@@ -17,7 +17,7 @@ __device__ __forceinline__ int wide_lcap(int M) {
 // the list is full or the slots have run out - the caller then aggregates the query itself.
 __device__ __forceinline__ bool wide_register(const Dev& s, int i, int M) {
   __shared__ int sh_wide_q;
-  if (s.w_slots == 0 || M > kWideMaxMatches) return false;
+  if (s.w_grid == 0 || M > kWideMaxMatches) return false;
   if (threadIdx.x == 0) {
     int q = -1;
     const int lcap = wide_lcap(M);
@@ -40,6 +40,142 @@ __device__ __forceinline__ bool wide_register(const Dev& s, int i, int M) {
     s.w_edge[(size_t)q * SDMS_MAX_DRAFT + threadIdx.x] = 0ull;
   }
   return q >= 0;
+}
+
+
+typedef unsigned long long u64;
+constexpr unsigned FULL = 0xffffffffu;
+constexpr int kWideThreads = 512;
+constexpr int kWideChunk = 128;                      // matches per unit of work: thread t owns match t % 128 ...
+constexpr int kLayerWays = kWideThreads / kWideChunk;  // ... and the layers d = t / 128 + 1, + 5, + 9, ...
+constexpr int kMaxRounds = 4;                          // layers of a thread that are in flight together (16 layers of the query)
+
+// Sum of p over the lanes that hold the same key as this lane (`live` = lanes that hold a key at all;
+// the same loop in every lane, so no lane waits for another group's reduction).  Only a group's leader
+// needs the result.
+__device__ __forceinline__ u64 group_sum(unsigned live, long long key, unsigned p) {
+  u64 sum = 0;
+  for (unsigned rem = live; rem; rem &= rem - 1) {
+    const int src = __ffs(rem) - 1;
+    const long long k = __shfl_sync(FULL, key, src);
+    const unsigned q = __shfl_sync(FULL, p, src);
+    if (k == key) sum += q;
+  }
+  return sum;
+}
+
+// Node sums of one unit: the matches list[m0 .. m0 + 128) of a query with M matches, all layers, into the
+// query's tables (first slot `base`, 2^lcap slots per layer).  Called by all kWideThreads threads of a
+// CTA.  The lanes of a warp hold 32 matches at the same layer; lanes whose followers are the same token
+// form a group and the group's leader claims the node's slot and sends one add for all of them.
+// Every item's slot (-1: the candidate has ended) is noted in w_item[base + (d - 1) * M + m].
+__device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* list, unsigned base, int lcap, int M, int m0) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int D = s.D;
+  const int ml = tid & (kWideChunk - 1), d_first = tid / kWideChunk + 1;   // d_first is the same in all lanes of a warp
+  const int nm = min(kWideChunk, M - m0);
+    const unsigned mask = (1u << lcap) - 1u;
+    int* const item = s.w_item + base + m0 + ml;      // + (d - 1) * M: the item's slot, layer by layer
+    int gpos = 0, n_m = 0;
+    if (ml < nm) {
+      gpos = list[m0 + ml];
+      const int j = path_of(s, gpos);
+      n_m = min(D, __ldg(s.len + j) - 1 - (gpos - j * s.L));
+    }
+  for (int d_base = d_first; d_base <= D; d_base += kMaxRounds * kLayerWays) {     // the same trip count for the whole warp
+    int v[kMaxRounds];
+    unsigned p[kMaxRounds];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {            // every follower this thread needs is asked for before the first is used
+      const int d = d_base + r * kLayerWays;
+      v[r] = -1; p[r] = 0u;
+      if (d <= n_m) { v[r] = __ldg(s.tok + gpos + d); p[r] = (unsigned)__ldg(s.pq + gpos + d); }
+    }
+    // the key sector and the slot every follower hashes to are asked for now: when the rounds below get to
+    // them (one after the other, the lanes of a warp in step) they are on their way from memory
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_base + r * kLayerWays;
+      if (v[r] >= 0) {
+        const size_t at = base + ((size_t)(d - 1) << lcap) + (((unsigned)v[r] * 2654435761u) >> (32 - lcap));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(s.w_key + at));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(s.w_tab + at));
+      }
+    }
+    // Who speaks for which node, for all of the thread's layers at once; then the leaders' probe
+    // sequences of those layers run side by side (a round trip to L2 costs the same for one request
+    // as for four), and last the slots go back to the groups.
+    int leader[kMaxRounds], sv[kMaxRounds];
+    u64 add[kMaxRounds];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_base + r * kLayerWays;
+      leader[r] = 0; sv[r] = -1; add[r] = 0ull;
+      if (d > D) continue;                              // the same for the whole warp
+      const unsigned group = __match_any_sync(FULL, v[r]);          // lanes whose items are the same node
+      leader[r] = __ffs(group) - 1;
+      add[r] = ((u64)__popc(group) << kWideSumShift) | group_sum(__ballot_sync(FULL, v[r] >= 0), (long long)v[r], p[r]);
+    }
+    // linear probing, eight keys (one sector) per round trip: the longest probe run of a half-full table
+    // of a thousand nodes is some forty slots
+    unsigned h[kMaxRounds];
+    unsigned todo = 0;                                  // layers whose slot this thread still has to find
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_base + r * kLayerWays;
+      h[r] = ((unsigned)v[r] * 2654435761u) >> (32 - lcap);
+      if (d <= D && v[r] >= 0 && lane == leader[r]) todo |= 1u << r;
+    }
+    for (unsigned step = 0; step <= mask + 8u && todo; ++step) {     // every step moves each sequence on by at least one slot
+      uint4 ka[kMaxRounds], kb[kMaxRounds];
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {
+        if (!(todo >> r & 1u)) continue;
+        const uint32_t* keys = s.w_key + base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u);
+        ka[r] = __ldcg(reinterpret_cast<const uint4*>(keys));
+        kb[r] = __ldcg(reinterpret_cast<const uint4*>(keys + 4));
+      }
+      int at[kMaxRounds];                               // first slot of the sector, from h on, that is free or holds the token
+      uint32_t seen[kMaxRounds];
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {
+        at[r] = -1; seen[r] = 0u;
+        if (!(todo >> r & 1u)) continue;
+        const uint32_t want = (uint32_t)v[r] + 1u;
+        const uint32_t kk[8] = {ka[r].x, ka[r].y, ka[r].z, ka[r].w, kb[r].x, kb[r].y, kb[r].z, kb[r].w};
+#pragma unroll
+        for (int x = 7; x >= 0; --x)
+          if ((unsigned)x >= (h[r] & 7u) && (kk[x] == 0u || kk[x] == want)) { at[r] = x; seen[r] = kk[x]; }
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {             // the claims of all layers go out together
+        if (!(todo >> r & 1u) || at[r] < 0 || seen[r] != 0u) continue;
+        uint32_t* keys = s.w_key + base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u);
+        seen[r] = atomicCAS(&keys[at[r]], 0u, (uint32_t)v[r] + 1u);
+        if (seen[r] == 0u) {
+          seen[r] = (uint32_t)v[r] + 1u;
+          s.w_tab[base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u) + at[r]].tok1 = seen[r];
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {
+        if (!(todo >> r & 1u)) continue;
+        if (at[r] < 0) { h[r] = ((h[r] & ~7u) + 8u) & mask; continue; }            // nothing in this sector: on to the next
+        if (seen[r] == (uint32_t)v[r] + 1u) { sv[r] = (int)((h[r] & ~7u) + at[r]); todo &= ~(1u << r); continue; }
+        h[r] = (h[r] & ~7u) + at[r] + 1u;                                        // somebody else's token got there first
+        if ((h[r] & 7u) == 0u) h[r] &= mask;
+      }
+    }
+    if (todo) atomicOr(s.status, SDMS_STATUS_INDEX_FULL);             // more nodes than slots: cannot happen
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_base + r * kLayerWays;
+      if (d > D) continue;
+      if (sv[r] >= 0) atomicAdd(&s.w_tab[base + ((size_t)(d - 1) << lcap) + sv[r]].sum, add[r]);
+      const int mine = __shfl_sync(FULL, sv[r], leader[r]);
+      if (ml < nm) item[(size_t)(d - 1) * M] = v[r] >= 0 ? mine : -1;
+    }
+  }
 }
 
 }  // namespace sdms

@@ -21,12 +21,13 @@ class Pair:
     """One oracle and one CUDA context with the same configuration."""
 
     def __init__(self, G, N, L, V, k_max, D, alpha=1.0, mode=0, B=0, Ke=0, max_append=None, match_capacity=0,
-                 eps=0, pool=0, device="cuda:0", host_io=False, max_matches=0, wide_table_bytes=0):
+                 eps=0, pool=0, device="cuda:0", host_io=False, max_matches=0, wide_table_bytes=0, max_beams=0):
         self.o = Oracle(G, N, L, V, D, alpha=alpha, mode=mode, eps=eps, pool=pool, max_matches=max_matches)
         self.pool = pool
         self.g = binding.Sdms(G, N, L, V, k_max, D, device=device, alpha=alpha, search_mode=mode, B=B, Ke=Ke,
                               max_append=max_append, match_capacity=match_capacity, epsilon=eps, pool_mode=pool,
-                              host_io=host_io, max_matches_per_path=max_matches, wide_table_bytes=wide_table_bytes)
+                              host_io=host_io, max_matches_per_path=max_matches, wide_table_bytes=wide_table_bytes,
+                              max_beams=max_beams)
         self.dev = self.g.device
         self.P, self.L, self.D, self.N = G * N, L, D, N
         self.B, self.Ke = B, Ke
@@ -83,6 +84,18 @@ class Pair:
                 for key in ex:
                     assert np.array_equal(dag[key][i], ex[key]), (k, i, key, dag[key][i], ex[key])
         return tok, ln
+
+    def beams_and_compare(self, B, paths=None):
+        """The B best paths of the pools of the last build on both sides: tokens identical, values within RTOL."""
+        tok, ln, val = self.g.beams(B)
+        assert self.g.status() == 0
+        for i in (range(self.P) if paths is None else paths):
+            want, want_val = self.o.beams(i, B)
+            got = [tok[i, b, :ln[i, b]].tolist() for b in range(B) if ln[i, b] > 0]
+            assert got == want, (i, got, want)
+            assert (ln[i, len(want):] == 0).all() and (tok[i, len(want):] == -1).all()
+            np.testing.assert_allclose(val[i, :len(want)], want_val, rtol=RTOL, atol=0)
+        return tok, ln, val
 
     def backoff_and_compare(self, k_hi):
         """Back-off build: per path the longest k <= k_hi with a match (oracle: fixed-k builds composed)."""

@@ -773,3 +773,86 @@ def test_wide_pass_with_many_distinct_followers_and_ragged_ends():
     pair.g.build_drafts(1)
     prof = binding.sdms_profile_read(pair.g.ctx)
     assert prof["dag_wide"][1] == 1
+
+
+# ---- several drafts per path: the B best paths of the pool ----------------------------------------
+def test_beams_hand_worked_pool_on_device():
+    paths = [[5, 9], [9, 1, 3, 7], [9, 2, 4, 7], [9, 2, 5, 7]]
+    probs = [[.5, .5], [.5, .5, .125, .5], [.5, .25, .75, .5], [.5, .25, .5, .5]]
+    pair = Pair(1, 4, 8, 10, 2, 2, mode=2, max_beams=4)
+    tok = np.zeros((4, 4), np.int32); lp = np.zeros((4, 4), np.float32)
+    for i, p in enumerate(paths):
+        tok[i, :len(p)] = p
+        lp[i, :len(p)] = np.log(np.array(probs[i]))
+    pair.append(tok, lp, np.array([len(p) for p in paths], np.int32), expect_status=0)
+    pair.build_and_compare(1, check_dag=False)
+    t, ln, val = pair.beams_and_compare(3)
+    assert [t[0, b, :ln[0, b]].tolist() for b in range(3)] == [[2, 4], [2, 5], [1, 3]]
+    np.testing.assert_allclose(val[0], [1.25, 1.0, .625], rtol=1e-6)
+    pair.beams_and_compare(4)
+
+
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("alpha,eps,mode", [(1.0, 0, 0), (0.5, 0, 2), (0.0, 0, 0), (1.0, 1, 2)])
+def test_beams_dense_small_vocab_every_step(seed, alpha, eps, mode):
+    G, N, L, V, D, k_max = 2, 5, 56, 3 + seed, 6, 3
+    tokens, lps = synth.small_random(G * N, L, V, 6300 + seed)
+    for k in (1, 2):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, eps=eps, max_beams=8)
+        lens = (4 + (np.arange(G * N) * 5 + seed) % 9).astype(np.int32)
+        pair.append(tokens[:, :16], lps[:, :16], lens, expect_status=0)
+        for step in range(25):
+            lens = pair.o.lengths()
+            if (lens >= L).all():
+                break
+            pair.build_and_compare(k, check_dag=False)
+            for B in (1, 3, 8):
+                pair.beams_and_compare(B)
+            if mode == 2:                                  # the first beam is the best-path draft
+                t, ln, _ = pair.g.beams(1)
+                assert np.array_equal(ln[:, 0], pair.g.draft_len.cpu().numpy())
+                assert np.array_equal(t[:, 0], pair.g.draft_tok.cpu().numpy())
+            sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
+            pair.accept_and_compare(sampled, sampled_lp)
+
+
+@pytest.mark.parametrize("wid,k", [(2, 1), (2, 3), (5, 1), (5, 3)])
+def test_beams_on_benchmark_workloads(wid, k):
+    # cfg2 k = 1: queries with more matches than the in-kernel best-path search takes; cfg5 k = 1: 22 938 matches
+    w = synth.WORKLOADS[wid]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, max_beams=4)
+    n = int(w.L * 0.97)
+    lens = (n - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    pair.append(tokens[:, :n], lps[:, :n], lens, expect_status=0)
+    sample = None if wid == 2 else list(range(0, w.P, 8))
+    pair.build_and_compare(k, check_dag=False, paths=sample)
+    pair.beams_and_compare(4, paths=sample)
+    pair.beams_and_compare(1, paths=sample)
+
+
+def test_beams_need_room_and_a_build():
+    from paper_2503_05330_b200 import binding
+    G, N, L, V, D = 1, 6, 64, 3, 4
+    tokens, lps = synth.small_random(G * N, L, V, 6400)
+    none = Pair(G, N, L, V, 2, D)                                          # max_beams = 0: the call is not available
+    none.append(tokens[:, :40], lps[:, :40], np.full(N, 40, np.int32), expect_status=0)
+    none.g.build_drafts(1)
+    with pytest.raises(binding.SdmsError) as e:
+        none.g.beams(1)
+    assert e.value.code == binding.ERR_BAD_STATE
+    small = Pair(G, N, L, V, 2, D, max_beams=2, wide_table_bytes=72 * 4 * 64 * 3)     # room for three small paths
+    small.append(tokens[:, :40], lps[:, :40], np.full(N, 40, np.int32), expect_status=0)
+    with pytest.raises(binding.SdmsError):
+        small.g.beams(2)                                                   # nothing built yet
+    small.g.build_drafts(2)
+    with pytest.raises(binding.SdmsError):
+        small.g.beams(3)                                                   # more than max_beams
+    tok, ln, _ = small.g.beams(2)
+    assert small.g.status() == binding.STATUS_TABLES_FULL
+    small.o.build_all(2)
+    served = [i for i in range(N) if ln[i, 0] > 0]
+    assert 0 < len(served) < N
+    for i in served:                                                       # those that found room are right
+        want, _ = small.o.beams(i, 2)
+        assert [tok[i, b, :ln[i, b]].tolist() for b in range(2) if ln[i, b] > 0] == want

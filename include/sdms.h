@@ -107,7 +107,7 @@ typedef struct {
                                     prompts too large for the single-launch build, queries with more than 32
                                     matches are aggregated by all SMs together; and sdms_get_beams (max_beams
                                     > 0).  A slot costs 40 + 16 * max_beams bytes and a path with M matches
-                                    needs between 1.25 and 2.5 * M * D slots.  0 = default (room for every position
+                                    needs between 2.5 and 5 * M * D slots (half of that for the beams).  0 = default (room for every position
                                     matching every query of its prompt, but at most 320 MiB), -1 = none.  A build
                                     whose queries need more falls back to one thread block for those that
                                     did not fit, with the same results                                    */

@@ -87,7 +87,7 @@ Layout make_layout(const sdms_config* c) {
   l.wide_on = !fused && c->wide_table_bytes >= 0;
   int64_t wide = c->wide_table_bytes;
   if (wide == 0) {
-    wide = slot_bytes * 3 * (int64_t)D * (int64_t)c->paths_per_group * (int64_t)(P * L);   // room for every position matching every query
+    wide = slot_bytes * 5 * (int64_t)D * (int64_t)c->paths_per_group * (int64_t)(P * L);   // room for every position matching every query
     if (wide > (320LL << 20)) wide = 320LL << 20;
   }
   l.w_slots = (l.wide_on || (c->max_beams > 0 && wide > 0)) ? (uint64_t)wide / slot_bytes : 0;

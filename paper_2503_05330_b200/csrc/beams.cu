@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) beam_kernel(Dev s, int B, int
   const int i = blockIdx.x, tid = threadIdx.x, D = s.D;
   int32_t* const my_tok = beam_tok + (size_t)i * B * D;
   const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
-  const int lcap = wide_lcap(M);
+  const int lcap = beam_lcap(M);
   if (tid == 0) {
     long long first = -1;
     if (M > 0 && M <= kWideMaxMatches) {

@@ -67,7 +67,7 @@ __device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
   return eq5_weight(s.alpha, sum & kSumMask, (unsigned)(sum >> kWideSumShift));
 }
 
-__global__ void __launch_bounds__(kWideThreads, 2)
+__global__ void __launch_bounds__(kWideThreads, 1)
 dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                 float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
   const u64 registered = ld_u64(&s.w_ctl[0]);
@@ -211,7 +211,7 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
       if (ml < nm) on = item[(size_t)(d - 1) * M] == sh_dslot[d - 1] && (d == 1 || item[(size_t)(d - 2) * M] == sh_dslot[d - 2]);
       const unsigned group = __ballot_sync(FULL, on);
       if (group == 0u) continue;
-      const u64 sum = group_sum(group, 0ll, on ? (unsigned)__ldg(s.pq + gpos + d) : 0u);
+      const u64 sum = group_sum(group, group, on ? (unsigned)__ldg(s.pq + gpos + d) : 0u);
       if (lane == __ffs(group) - 1)
         atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
     }
@@ -246,7 +246,7 @@ int wide_kernel_grid() {
   if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) { cudaGetLastError(); return 0; }
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dag_wide_kernel, kWideThreads, 0) != cudaSuccess) { cudaGetLastError(); return 0; }
-  return sms * (per_sm < 2 ? per_sm : 2);
+  return sms * (per_sm < 1 ? per_sm : 1);
 }
 
 cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,

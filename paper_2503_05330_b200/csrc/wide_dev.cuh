@@ -4,9 +4,18 @@
 
 namespace sdms {
 
-// log2 of the slots of one layer's node table: a power of two above 5/4 of the matches, so that a
-// layer in which every candidate is a node of its own still leaves a fifth of the slots free.
+// log2 of the slots of one layer's node table: a power of two above 5/2 of the matches.  A layer in which
+// every candidate is a node of its own fills at most 40 % of it: with linear probing the LONGEST probe
+// run of the table decides how long a pass takes (the whole grid waits for the unluckiest lane), and
+// that run grows quickly with the fill.
 __device__ __forceinline__ int wide_lcap(int M) {
+  int l = 6;
+  while ((1ll << l) < (5ll * M) / 2 + 1) ++l;
+  return l;
+}
+
+// The same for the one-CTA-per-path beam kernel, which nobody waits for: above 5/4 of the matches.
+__device__ __forceinline__ int beam_lcap(int M) {
   int l = 6;
   while ((1ll << l) < (long long)M + (M >> 2) + 1) ++l;
   return l;
@@ -50,16 +59,15 @@ constexpr int kWideChunk = 128;                      // matches per unit of work
 constexpr int kLayerWays = kWideThreads / kWideChunk;  // ... and the layers d = t / 128 + 1, + 5, + 9, ...
 constexpr int kMaxRounds = 4;                          // layers of a thread that are in flight together (16 layers of the query)
 
-// Sum of p over the lanes that hold the same key as this lane (`live` = lanes that hold a key at all;
-// the same loop in every lane, so no lane waits for another group's reduction).  Only a group's leader
-// needs the result.
-__device__ __forceinline__ u64 group_sum(unsigned live, long long key, unsigned p) {
-  u64 sum = 0;
-  for (unsigned rem = live; rem; rem &= rem - 1) {
+// Sum of p over the lanes of this lane's group (`group` from __match_any_sync).  The same loop in every
+// lane, over the lanes that share their group with somebody (`shared`: whole groups only); a lane that is
+// not among them keeps its own p.  One shuffle per visited lane: the shuffle pipe is what this costs.
+__device__ __forceinline__ u64 group_sum(unsigned group, unsigned shared, unsigned p) {
+  u64 sum = (shared >> (threadIdx.x & 31) & 1u) ? 0ull : (u64)p;
+  for (unsigned rem = shared; rem; rem &= rem - 1) {
     const int src = __ffs(rem) - 1;
-    const long long k = __shfl_sync(FULL, key, src);
     const unsigned q = __shfl_sync(FULL, p, src);
-    if (k == key) sum += q;
+    if (group >> src & 1u) sum += q;
   }
   return sum;
 }
@@ -114,7 +122,8 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
       if (d > D) continue;                              // the same for the whole warp
       const unsigned group = __match_any_sync(FULL, v[r]);          // lanes whose items are the same node
       leader[r] = __ffs(group) - 1;
-      add[r] = ((u64)__popc(group) << kWideSumShift) | group_sum(__ballot_sync(FULL, v[r] >= 0), (long long)v[r], p[r]);
+      const unsigned shared = __ballot_sync(FULL, v[r] >= 0 && (group & (group - 1)) != 0u);
+      add[r] = ((u64)__popc(group) << kWideSumShift) | group_sum(group, shared, p[r]);
     }
     // linear probing, eight keys (one sector) per round trip: the longest probe run of a half-full table
     // of a thousand nodes is some forty slots
@@ -126,15 +135,17 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
       h[r] = ((unsigned)v[r] * 2654435761u) >> (32 - lcap);
       if (d <= D && v[r] >= 0 && lane == leader[r]) todo |= 1u << r;
     }
-    for (unsigned step = 0; step <= mask + 8u && todo; ++step) {     // every step moves each sequence on by at least one slot
-      uint4 ka[kMaxRounds], kb[kMaxRounds];
+    uint4 ka[kMaxRounds], kb[kMaxRounds];                // the sector of keys each sequence is looking at
+    unsigned fresh = 0;                                 // layers whose sector is in ka / kb
+    for (unsigned step = 0; step <= 2u * mask + 16u && todo; ++step) {   // every step moves each sequence on by at least one slot
 #pragma unroll
       for (int r = 0; r < kMaxRounds; ++r) {
-        if (!(todo >> r & 1u)) continue;
+        if (!(todo >> r & 1u) || (fresh >> r & 1u)) continue;
         const uint32_t* keys = s.w_key + base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u);
         ka[r] = __ldcg(reinterpret_cast<const uint4*>(keys));
         kb[r] = __ldcg(reinterpret_cast<const uint4*>(keys + 4));
       }
+      fresh |= todo;
       int at[kMaxRounds];                               // first slot of the sector, from h on, that is free or holds the token
       uint32_t seen[kMaxRounds];
 #pragma unroll
@@ -160,10 +171,12 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
 #pragma unroll
       for (int r = 0; r < kMaxRounds; ++r) {
         if (!(todo >> r & 1u)) continue;
-        if (at[r] < 0) { h[r] = ((h[r] & ~7u) + 8u) & mask; continue; }            // nothing in this sector: on to the next
+        if (at[r] < 0) { h[r] = ((h[r] & ~7u) + 8u) & mask; fresh &= ~(1u << r); continue; }   // nothing in this sector: on to the next
         if (seen[r] == (uint32_t)v[r] + 1u) { sv[r] = (int)((h[r] & ~7u) + at[r]); todo &= ~(1u << r); continue; }
-        h[r] = (h[r] & ~7u) + at[r] + 1u;                                        // somebody else's token got there first
-        if ((h[r] & 7u) == 0u) h[r] &= mask;
+        // somebody else's token got there first: go on behind it, in the same sector as long as it lasts (a key that
+        // was free when the sector was read may be taken by now: the claim will tell)
+        h[r] = (h[r] & ~7u) + at[r] + 1u;
+        if ((h[r] & 7u) == 0u) { h[r] &= mask; fresh &= ~(1u << r); }
       }
     }
     if (todo) atomicOr(s.status, SDMS_STATUS_INDEX_FULL);             // more nodes than slots: cannot happen

@@ -199,8 +199,8 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
  * are identical to those two calls made one after the other.
  * d_sampled and d_sampled_logprobs ([P][D+1]) are both required.
  * When a prompt's paths fit one thread-block cluster (paths_per_group <= 16, the
- * single-launch build applies and the device can co-schedule such a cluster) the
- * step is ONE kernel launch: the paths of a prompt commit, meet at a cluster
+ * single-launch build applies and the device can hold the clusters of all prompts
+ * at once) the step is ONE kernel launch: the paths of a prompt commit, meet at a cluster
  * barrier, and build.  Otherwise the call issues the separate launches.
  * sdms_step_is_single_launch reports which (1 / 0).
  */

@@ -1606,8 +1606,6 @@ cudaError_t dag_kernel_setup() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
   if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
@@ -1632,7 +1630,9 @@ bool step_kernel_fits(const Dev& s) {
   cfg.numAttrs = 1;                                   // occupancy only looks at the cluster shape
   int clusters = 0;
   if (cudaOccupancyMaxActiveClusters(&clusters, step_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
-  return clusters >= 1;
+  // every prompt's cluster resident at once: large clusters leave SMs of a GPC idle, and a launch whose
+  // clusters queue up for the device is slower than the separate accept and build launches
+  return (long long)clusters * s.N >= s.P;
 }
 
 cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, const float* sampled_lp,
@@ -1653,11 +1653,14 @@ cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32
                            draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
-// Largest cluster (CTAs = consecutive paths of one prompt) that the single-launch build can run with on this
-// device, 1 if none: the cluster shares the scan of its prompt (shared_scan).
+// Cluster size (CTAs = consecutive paths of one prompt) of the single-launch build, 1 for none.  A cluster
+// shares the scan of its prompt (shared_scan), which shortens the longest CTA of a launch but adds two
+// barriers to every CTA: it pays when the whole launch is resident at once, i.e. when the launch's
+// time is its slowest CTA's, and loses when CTAs queue for SMs anyway.  Sizes above 8 leave too many
+// SMs of a GPC idle.
 int build_cluster_size(const Dev& s) {
   if (!s.fused || (s.L & 3) != 0 || (long long)s.N * s.L < kShareMinTokens) return 1;
-  for (int c = kMaxClusterPaths; c >= 2; --c) {
+  for (int c = 8; c >= 2; --c) {
     if (s.N % c) continue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(s.P); cfg.blockDim = dim3(kFusedThreads); cfg.dynamicSmemBytes = dag_smem_bytes<false>();
@@ -1667,7 +1670,7 @@ int build_cluster_size(const Dev& s) {
     cfg.attrs = attr; cfg.numAttrs = 1;
     int clusters = 0;
     if (cudaOccupancyMaxActiveClusters(&clusters, build_fused_kernel<false>, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
-    if (clusters >= 1) return c;
+    if ((long long)clusters * c >= s.P) return c;
   }
   return 1;
 }

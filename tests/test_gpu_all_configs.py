@@ -47,7 +47,7 @@ def test_config3_consecutive_steps_on_nearly_full_histories():
 @pytest.mark.parametrize("k", [1, 5])
 def test_config4_every_step_of_the_whole_run(k):
     pair = whole_run(4, k, check_every=50)
-    assert pair.g.step_is_single_launch()
+    assert not pair.g.step_is_single_launch()       # 32 clusters of 16 do not fit the device at once: accept, then build
 
 
 def test_config4_consecutive_steps_on_nearly_full_histories():

@@ -382,14 +382,29 @@ def test_step_config_full_protocol(wid):
 
 
 def test_step_many_prompts_ragged():
+    # twelve prompts of eight paths: twelve clusters resident at once, one launch per step
     w = synth.WORKLOADS[4]
     tokens, lps = synth.make_streams(w)
-    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    G, N = 12, 8
+    tokens = np.ascontiguousarray(tokens.reshape(w.G, w.N, w.L)[:G, :N].reshape(G * N, w.L))
+    lps = np.ascontiguousarray(lps.reshape(w.G, w.N, w.L)[:G, :N].reshape(G * N, w.L))
+    pair = Pair(G, N, w.L, w.V, w.k_max, w.D, max_append=w.D)
     assert pair.g.step_is_single_launch()
-    start = (int(w.L * 0.98) - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    start = (int(w.L * 0.98) - (np.arange(G * N) * 13) % 97).astype(np.int32)
     st = harness.run_step_protocol(pair, tokens, lps, [5, 1, 3], steps=12, warm=0, start_lens=start,
                                    check_matches=False)
     assert st["steps"] == 12                   # runs into full paths: those stop drafting and committing
+
+
+def test_step_of_more_clusters_than_the_device_holds_takes_separate_launches():
+    w = synth.WORKLOADS[4]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    assert not pair.g.step_is_single_launch()
+    start = (int(w.L * 0.98) - (np.arange(w.P) * 13) % 97).astype(np.int32)
+    st = harness.run_step_protocol(pair, tokens, lps, [5, 1, 3], steps=12, warm=0, start_lens=start,
+                                   check_matches=False)
+    assert st["steps"] == 12
 
 
 def test_step_falls_back_to_separate_launches_for_wide_prompts():

@@ -50,8 +50,8 @@ extern "C" {
 #define SDMS_STATUS_BAD_LOGPROB    0x08u /* NaN logprob: stored as probability 0                  */
 #define SDMS_STATUS_INDEX_FULL     0x10u /* n-gram table had no free bucket (cannot happen with the sized workspace) */
 #define SDMS_STATUS_MATCH_OVERFLOW 0x20u /* match workspace exhausted: the affected paths get draft_len 0 */
-#define SDMS_STATUS_SEARCH_FALLBACK 0x40u /* search_mode 2: a path had too many matches for the best-path tables
-                                            (more than about 24576 / (11 * max_draft_len)); it got the greedy draft */
+#define SDMS_STATUS_SEARCH_FALLBACK 0x40u /* search_mode 2: a path had too many matches for shared memory (more than about
+                                            24576 / (11 * max_draft_len)) and the table area had no room: greedy draft */
 #define SDMS_STATUS_TIMEOUT        0x80u /* a bounded wait inside a kernel ran out (never expected): the build's matches are incomplete */
 #define SDMS_STATUS_TABLES_FULL    0x100u /* sdms_get_beams: the table area of the workspace (wide_table_bytes) did not hold
                                              every path's node tables; the paths left out have no beam */
@@ -84,8 +84,10 @@ typedef struct {
                                        highest-likelihood sequence): best(d,v) = w(d,v) + max over
                                        successors of best(d+1,.), summed from the path's end; the
                                        walk follows the largest best(), ties to the smaller token.
-                                       DAG pool only.  Paths with more matches than the tables hold
-                                       get the mode-0 draft and raise SDMS_STATUS_SEARCH_FALLBACK */
+                                       DAG pool only.  Paths with more matches than shared memory
+                                       takes are searched over node tables in the workspace's table
+                                       area (wide_table_bytes); only if that is switched off or full
+                                       do they get the mode-0 draft and raise SDMS_STATUS_SEARCH_FALLBACK */
   float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
   int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
   int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)
@@ -106,7 +108,7 @@ typedef struct {
   int64_t  wide_table_bytes;     /* workspace set aside for node tables in global memory.  Two users: on
                                     prompts too large for the single-launch build, queries with more than 32
                                     matches are aggregated by all SMs together; and sdms_get_beams (max_beams
-                                    > 0).  A slot costs 40 + 16 * max_beams bytes and a path with M matches
+                                    > 0) and search_mode 2.  A slot costs 40 + 16 * max(max_beams, 1) bytes and a path with M matches
                                     needs between 2.5 and 5 * M * D slots (half of that for the beams).  0 = default (room for every position
                                     matching every query of its prompt, but at most 320 MiB), -1 = none.  A build
                                     whose queries need more falls back to one thread block for those that

@@ -83,14 +83,15 @@ Layout make_layout(const sdms_config* c) {
   // 32 bytes of sums, 4 of key, 4 per (match, layer) item, 16 per kept continuation
   const int64_t group_tokens = (int64_t)c->paths_per_group * c->capacity;
   const bool fused = group_tokens <= kFusedMaxTokens && (int64_t)P * group_tokens <= mc;
-  const int64_t slot_bytes = 40 + 16 * (int64_t)c->max_beams;
+  const int64_t stride = c->max_beams > 0 ? c->max_beams : (c->search_mode == 2 ? 1 : 0);   // continuations kept per node
+  const int64_t slot_bytes = 40 + 16 * stride;
   l.wide_on = !fused && c->wide_table_bytes >= 0;
   int64_t wide = c->wide_table_bytes;
   if (wide == 0) {
     wide = slot_bytes * 5 * (int64_t)D * (int64_t)c->paths_per_group * (int64_t)(P * L);   // room for every position matching every query
     if (wide > (320LL << 20)) wide = 320LL << 20;
   }
-  l.w_slots = (l.wide_on || (c->max_beams > 0 && wide > 0)) ? (uint64_t)wide / slot_bytes : 0;
+  l.w_slots = (l.wide_on || (stride > 0 && wide > 0)) ? (uint64_t)wide / slot_bytes : 0;
   l.w_ctl = take((size_t)kWideCtlWords * 8);
   l.b_ctl = take(8);
   l.w_desc = take(l.wide_on ? (size_t)kMaxWide * 16 : 0);
@@ -99,7 +100,7 @@ Layout make_layout(const sdms_config* c) {
   l.w_tab = take((size_t)l.w_slots * sizeof(WideSlot));
   l.w_key = take((size_t)l.w_slots * 4);
   l.w_item = take((size_t)l.w_slots * 4);
-  l.b_ent = take((size_t)l.w_slots * 16 * c->max_beams);
+  l.b_ent = take((size_t)l.w_slots * 16 * stride);
   l.total = o;
   return l;
 }
@@ -159,6 +160,13 @@ int drain_pending(sdms_ctx* ctx, size_t count) {
   }
   ctx->pending.erase(ctx->pending.begin(), ctx->pending.begin() + count);
   return SDMS_OK;
+}
+
+// Best-path builds may reserve node tables in the workspace's table area (paths with more matches than
+// shared memory takes): the cursor they reserve with starts every build at zero.  Other contexts: nothing.
+int reset_table_cursor(sdms_ctx* ctx, cudaStream_t stream) {
+  if (ctx->cfg.search_mode != 2 || ctx->dev.beam_stride == 0) return SDMS_OK;
+  return cudaMemsetAsync(ctx->dev.b_ctl, 0, 8, stream) == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
 template <class F>
@@ -254,7 +262,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.w_tab = (WideSlot*)(w + lay.w_tab); d.w_key = (uint32_t*)(w + lay.w_key); d.w_item = (int32_t*)(w + lay.w_item);
   d.w_grid = lay.wide_on ? wide_kernel_grid() : 0;   // 0 (also without cooperative launch on this device): one thread block per query
   d.w_slots = lay.w_slots;
-  d.b_ent = (BeamEnt*)(w + lay.b_ent); d.b_ctl = (unsigned long long*)(w + lay.b_ctl); d.beam_stride = cfg->max_beams;
+  d.b_ent = (BeamEnt*)(w + lay.b_ent); d.b_ctl = (unsigned long long*)(w + lay.b_ctl); d.beam_stride = lay.w_slots ? (cfg->max_beams > 0 ? cfg->max_beams : (cfg->search_mode == 2 ? 1 : 0)) : 0;
   ctx->step_fits = step_kernel_fits(d);
   d.build_cluster = build_cluster_size(d);
   *out = ctx;
@@ -293,6 +301,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
   if (k < 1 || k > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   if (ctx->dev.fused) {
     const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
       return launch_build_fused(ctx->dev, k, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, nullptr, st); });
@@ -318,6 +327,7 @@ int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok,
   if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
   if (!ctx->dev.fused) return SDMS_ERR_BAD_STATE;
   cudaStream_t st = (cudaStream_t)stream;
+  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
     return launch_build_fused(ctx->dev, k_hi, 1, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, d_used_k, st); });
   if (rc == SDMS_OK) ctx->built = true;
@@ -358,6 +368,7 @@ int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d
   }
   cudaStream_t st = (cudaStream_t)stream;
   ctx->built = false;
+  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
     return launch_step(ctx->dev, k, k, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
                        d_draft_score, d_draft_edge_w, nullptr, st); });
@@ -380,6 +391,7 @@ int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, con
   }
   cudaStream_t st = (cudaStream_t)stream;
   ctx->built = false;
+  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
     return launch_step(ctx->dev, k_hi, 1, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
                        d_draft_score, d_draft_edge_w, d_used_k, st); });

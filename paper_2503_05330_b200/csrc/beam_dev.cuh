@@ -28,10 +28,16 @@ __device__ __forceinline__ bool beam_after(u64 v, u64 nx, const BeamEnt& prev) {
 
 // One CTA (kWideThreads threads), query path i with M matches in `list`.  Needs D << lcap table slots
 // starting at `base`, all zero (they are left zero).  Writes beam_tok [B][D], beam_len [B], beam_value [B]
-// of the path.  `ent` = s.b_ent + base * stride.
-__device__ void beams_of_query(const Dev& s, int i, int M, const int32_t* list, unsigned base, int lcap, int B,
-                               int32_t* beam_tok, int32_t* beam_len, float* beam_value) {
+// of the path.  `ent` = s.b_ent + base * stride.  With score0 / edge0 (each [D], either may be NULL; the
+// caller asks with want0) the first beam also gets what a draft carries: the Eq. 5 in-weight of each of
+// its nodes and the weight of each edge it takes.
+__device__ __forceinline__ void beams_of_query(const Dev& s, int i, int M, const int32_t* list, unsigned base, int lcap, int B,
+                               int32_t* beam_tok, int32_t* beam_len, float* beam_value, bool want0 = false,
+                               float* score0 = nullptr, float* edge0 = nullptr) {
   __shared__ BeamEnt sh_root[SDMS_MAX_BEAMS];
+  __shared__ int sh_bslot[SDMS_MAX_DRAFT];
+  __shared__ u64 sh_bedge[SDMS_MAX_DRAFT];
+  __shared__ int sh_blen;
   const int tid = threadIdx.x, D = s.D, stride = s.beam_stride;
   const unsigned cap = 1u << lcap;
   WideSlot* const tab = s.w_tab + base;
@@ -115,6 +121,46 @@ __device__ void beams_of_query(const Dev& s, int i, int M, const int32_t* list, 
     }
     for (int d = len; d < D; ++d) beam_tok[tid * D + d] = -1;
     beam_len[tid] = len;
+  }
+  if (want0) {
+    // the first beam once more, slot by slot; then the probabilities of the items on its edges
+    if (tid < SDMS_MAX_DRAFT) sh_bedge[tid] = 0ull;
+    if (tid == 0) {
+      BeamEnt e = sh_root[0];
+      int len = 0;
+      for (int d = 1; d <= D && e.next != 0ull && e.next != kBeamLeaf; ++d) {
+        const int rank = 7 - (int)((e.next >> 24) & 7u), slot = (int)(e.next & 0xffffffu);
+        sh_bslot[len++] = slot;
+        if (score0) {
+          const u64 sum = __ldcg(&tab[((size_t)(d - 1) << lcap) + slot].sum);
+          score0[d - 1] = (float)eq5_weight(s.alpha, sum & ((1ull << kWideSumShift) - 1), (unsigned)(sum >> kWideSumShift));
+        }
+        const BeamEnt* at = ent + ((size_t)((d - 1) << lcap) + slot) * stride + rank;
+        e = BeamEnt{__ldcg(&at->value), __ldcg(&at->next)};
+      }
+      sh_blen = len;
+    }
+    __syncthreads();
+    const int len = sh_blen;
+    if (edge0) {
+      for (int d = 1; d <= len; ++d) {
+        for (int m0 = 0; m0 < M; m0 += blockDim.x) {             // whole warps: the lanes add up together
+          const int m = m0 + tid;
+          bool on = false;
+          if (m < M) on = __ldcg(item + (size_t)(d - 1) * M + m) == sh_bslot[d - 1] &&
+                          (d == 1 || __ldcg(item + (size_t)(d - 2) * M + m) == sh_bslot[d - 2]);
+          const unsigned group = __ballot_sync(FULL, on);
+          if (group == 0u) continue;
+          const u64 sum = group_sum(group, group, on ? (unsigned)__ldg(s.pq + list[m] + d) : 0u);
+          if ((tid & 31) == __ffs(group) - 1) atomicAdd(&sh_bedge[d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
+        }
+      }
+      __syncthreads();
+      if (tid < len) {
+        const u64 sum = sh_bedge[tid];
+        edge0[tid] = (float)eq5_weight(s.alpha, sum & ((1ull << kWideSumShift) - 1), (unsigned)(sum >> kWideSumShift));
+      }
+    }
   }
   __syncthreads();
   // leave the tables as they were found

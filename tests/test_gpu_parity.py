@@ -444,13 +444,15 @@ def best_path_fits(M, D):
     return ((2 * M * D + 1) & ~1) + D * 9 * cap <= 2 * 8192 + 8 * 1024
 
 
-def test_best_path_config2_and_the_fallback_for_heavy_queries():
-    # k = 1 queries on frequent tokens find more matches than the best-path tables of a CTA hold:
-    # those paths get the greedy draft and the status word says so; every other path the best path
+@pytest.mark.parametrize("table_area", [True, False])
+def test_best_path_config2_heavy_queries_and_the_fallback_without_a_table_area(table_area):
+    # k = 1 queries on frequent tokens find more matches than the best-path tables in shared memory hold: those
+    # paths are searched over tables in the workspace's table area.  Without one (wide_table_bytes = -1) they get
+    # the greedy draft and the status word says so; every other path the best path
     from oracle import Oracle
     w = synth.WORKLOADS[2]
     tokens, lps = synth.make_streams(w)
-    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D, wide_table_bytes=0 if table_area else -1)
     greedy = Oracle(w.G, w.N, w.L, w.V, w.D, alpha=1.0, mode=0)
     n = 1000
     lens = (n - (np.arange(w.P) * 13) % 97).astype(np.int32)
@@ -467,12 +469,12 @@ def test_best_path_config2_and_the_fallback_for_heavy_queries():
         heavy = 0
         for i in range(w.P):
             M = len(pair.o.matches(i))
-            src = pair.o if best_path_fits(M, w.D) else greedy
+            src = pair.o if table_area or best_path_fits(M, w.D) else greedy
             heavy += not best_path_fits(M, w.D)
             d, sc, _ = src.draft(i)
             assert gl[i] == len(d) and np.array_equal(gt[i, :len(d)], d), (k, i, M)
             np.testing.assert_allclose(gs[i, :len(d)], sc, rtol=harness.RTOL, atol=0)
-        assert status == (0x40 if heavy else 0), (k, heavy, status)
+        assert status == (0x40 if heavy and not table_area else 0), (k, heavy, status)
         fell_back += heavy
         lens = pair.o.lengths()
         sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, w.D + 1)
@@ -871,3 +873,17 @@ def test_beams_need_room_and_a_build():
     for i in served:                                                       # those that found room are right
         want, _ = small.o.beams(i, 2)
         assert [tok[i, b, :ln[i, b]].tolist() for b in range(2) if ln[i, b] > 0] == want
+
+
+def test_best_path_with_heavy_queries_through_build_and_step():
+    # cfg2 at k = 1: many paths have more matches than the shared-memory search takes; drafts, scores and edge
+    # weights of all paths against the oracle, through sdms_build_drafts and through the one-call step
+    w = synth.WORKLOADS[2]
+    tokens, lps = synth.make_streams(w)
+    start = 850 + (np.arange(w.P) * 37) % 100
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D)
+    st = run_protocol(pair, tokens, lps, 1, steps=25, warm=0, start_lens=start, commit_in_accept=True, check_dag=False)
+    assert st["steps"] == 25
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D)
+    st = harness.run_step_protocol(pair, tokens, lps, [1, 2], steps=25, warm=0, start_lens=start, check_every=5)
+    assert st["steps"] == 25

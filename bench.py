@@ -373,7 +373,7 @@ class Runner:
         return sum(per_step), units
 
 
-def steady_state(wl, device, iters=20, peak=None):
+def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=0):
     """Build latency of a workload at 97 % full histories (a full path builds no draft): per k the
     median, 10th and 90th percentile of the time of sdms_build_drafts (CUDA events on the launch
     stream, L2 flushed before every call), the matches it found, the kernel's own byte count per call
@@ -381,15 +381,19 @@ def steady_state(wl, device, iters=20, peak=None):
     import torch
     from paper_2503_05330_b200 import binding
     tokens, logprobs = synth.make_streams(wl)
-    s = binding.Sdms(wl.G, wl.N, wl.L, wl.V, wl.k_max, wl.D, device=device, max_append=wl.D)
+    s = binding.Sdms(wl.G, wl.N, wl.L, wl.V, wl.k_max, wl.D, device=device, max_append=wl.D,
+                     max_matches_per_path=max_matches, max_beams=beams)
     dev = s.device
     n = int(wl.L * 0.97)
     lens = (n - (np.arange(wl.P) * 13) % 97).astype(np.int32)
     s.append(torch.from_numpy(np.ascontiguousarray(tokens[:, :n])).to(dev),
              torch.from_numpy(np.ascontiguousarray(logprobs[:, :n])).to(dev), torch.from_numpy(lens).to(dev))
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    beam_out = (torch.empty((wl.P, max(beams, 1), wl.D), dtype=torch.int32, device=dev),
+                torch.empty((wl.P, max(beams, 1)), dtype=torch.int32, device=dev),
+                torch.empty((wl.P, max(beams, 1)), dtype=torch.float32, device=dev))
     out = {}
-    for k in range(1, wl.k_max + 1):
+    for k in (ks or range(1, wl.k_max + 1)):
         for _ in range(3):
             s.build_drafts(k)
         evs = []
@@ -422,9 +426,21 @@ def steady_state(wl, device, iters=20, peak=None):
                        "frac_of_peak": None if peak is None else nbytes / (us * 1e-6) / 1e9 / peak,
                        "scan_bytes_moved": scan_bytes, "scan_bytes_shared_pass": shared_scan,
                        "kernel_us": split}
+        if beams:                                            # several drafts per path from the pools of this build
+            for _ in range(2):
+                s.beams(beams)
+            evs = []
+            for _ in range(10):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); binding.sdms_get_beams(s.ctx, beams, *beam_out); b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            out[str(k)]["get_beams_us"] = 1e3 * float(np.median([a.elapsed_time(b) for a, b in evs]))
     assert s.status() == 0
     return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
-            "launches_per_build": 1 if fused else 3, "workspace_bytes": s.workspace_bytes, "build_by_k": out}
+            "max_matches_per_path": max_matches,
+            "launches_per_build": 1 if fused else 4, "workspace_bytes": s.workspace_bytes, "build_by_k": out}
 
 
 def scan_at_scale(device, G=64, N=256, L=8192, V=151936):
@@ -651,6 +667,10 @@ def ours_main(args, w):
         torch.cuda.empty_cache()
         steady2 = steady_state(w, device, iters=200, peak=peak)
         others = {synth.WORKLOADS[c].name: steady_state(synth.WORKLOADS[c], device, peak=peak) for c in (1, 3, 4, 5)}
+        # the pool capped at the 64 / 8 most recent matches per source path (the heaviest k = 1 query keeps 255 * R at most)
+        others["cfg5_n256_l8192_match_cap_64"] = steady_state(synth.WORKLOADS[5], device, peak=peak, max_matches=64, ks=(1, 2, 3))
+        others["cfg5_n256_l8192_match_cap_8"] = steady_state(synth.WORKLOADS[5], device, peak=peak, max_matches=8, ks=(1, 2, 3))
+        others["cfg2_n16_l1024_four_beams"] = steady_state(w, device, peak=peak, beams=4)
         scale = scan_at_scale(device)
         gscale = gather_at_scale(device)
     (ms, ms_e2e, host_ms_e2e), (units, units_e2e, _) = whole_job([ms, ms_e2e, host_ms_e2e], [units, units_e2e, 0.0], device)

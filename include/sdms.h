@@ -91,8 +91,9 @@ typedef struct {
   float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
   int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
   int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)
-                                    or 1.  1 needs a small prompt: N*L <= 131072 tokens and
-                                    G*N*N*L <= match_capacity (every path then owns N*L match slots) */
+                                    or 1.  With 1 the index is not used: small prompts (N*L <= 131072
+                                    tokens and G*N*N*L <= match_capacity) are scanned by the single-launch
+                                    build, larger ones in two passes (count, then fill)             */
   int32_t  pool_mode;            /* draft pool: 0 = weighted DAG (the method); the weaker pools of the
                                     paper's ablation: 1 = tree (merge identical prefixes only),
                                     2 = list (no merging: the heaviest single candidate)            */

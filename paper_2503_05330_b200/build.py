@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdms.so")
-SOURCES = ["api.cu", "append.cu", "match.cu", "dag.cu", "dag_wide.cu", "beams.cu", "match_static.cu"]
+SOURCES = ["api.cu", "append.cu", "match.cu", "dag.cu", "dag_wide.cu", "beams.cu", "fuzzy.cu", "match_static.cu"]
 HEADERS = ["sdms_dev.cuh", "sdms_internal.h", "append_dev.cuh", "wide_dev.cuh", "beam_dev.cuh"]
 
 

@@ -112,12 +112,11 @@ bool fits_fused(const sdms_config* c, const Layout& l) {
          (int64_t)c->num_groups * c->paths_per_group * group_tokens <= l.match_cap;
 }
 
-// Full check: field ranges, then what depends on the layout (fuzzy matches are not sized by the index).
+// Full check: field ranges, then the layout.
 int check_all(const sdms_config* c, Layout* out) {
   const int rc = check_config(c);
   if (rc != SDMS_OK) return rc;
   *out = make_layout(c);
-  if (c->epsilon > 0 && !fits_fused(c, *out)) return SDMS_ERR_INVALID_ARG;
   return SDMS_OK;
 }
 
@@ -308,9 +307,15 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
     if (rc == SDMS_OK) ctx->built = true;
     return rc;
   }
-  int rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, st); });
-  if (rc != SDMS_OK) return rc;
-  rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+  int rc;
+  if (ctx->dev.eps > 0) {                            // matches with tolerance: sized by counting, four launches
+    rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_fuzzy_match(ctx->dev, k, st); });
+    ctx->launches += 3;
+  } else {
+    rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, st); });
+    if (rc != SDMS_OK) return rc;
+    rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+  }
   if (rc != SDMS_OK) return rc;
   rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
     return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });

@@ -1118,39 +1118,49 @@ __device__ void dag_best_path(const Dev& s, const Smem& sm, int i, int M, int ca
 
 // Optional cap on the pool: of the matches of the query in one source path only the R with the largest end
 // positions stay.  `list` holds the query's M matches (global memory, any order) and is compacted in
-// place; the new count is returned (the same in every thread).  scratch: 4 * N shared words.
+// place; the new count is returned (the same in every thread).  scratch: kStageWords * 2 shared words.
 // Paths with at most R matches keep them all; for each of the others the R-th largest end position is
-// found by bisection on the position (one counting sweep over the list per round), which needs no
-// order among the matches and one word per path and round.
+// found digit by digit, most significant first: one counting sweep over the list per digit fills a
+// histogram of the digit for every such path (over the matches that agree with the digits found so
+// far), and the path reads off which digit value its R-th largest position has.  No order among the
+// matches is needed.
 __device__ int cap_matches(const Dev& s, int g, int M, int32_t* list, int* scratch) {
   __shared__ int sh_warp_tot[kMaxWarps];
   __shared__ int sh_out;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int N = s.N, R = s.R, poff = g * N;
-  int* cnt = scratch; int* above = scratch + N; int* lo = scratch + 2 * N; int* hi = scratch + 3 * N;
-  for (int n = tid; n < N; n += blockDim.x) { cnt[n] = 0; lo[n] = 0; hi[n] = s.L; }
+  // digits of `bits` bits: as wide as the histograms of N paths fit beside three words per path
+  int bits = 5;
+  while (bits > 1 && 3 * N + (N << bits) > 2 * kStageWords) --bits;
+  int* cnt = scratch; int* lo = scratch + N; int* need = scratch + 2 * N; int* hist = scratch + 3 * N;   // hist[n << bits | digit]
+  for (int n = tid; n < N; n += blockDim.x) { cnt[n] = 0; lo[n] = 0; need[n] = R; }
   __syncthreads();
   for (int m = tid; m < M; m += blockDim.x) atomicAdd(&cnt[path_of(s, list[m]) - poff], 1);
   __syncthreads();
   int over = 0;
   for (int n = tid; n < N; n += blockDim.x) over |= cnt[n] > R;
   if (!__syncthreads_or(over)) return M;
-  // invariant per path: at least R matches end at or after lo, fewer than R at or after hi
-  int rounds = 0;
-  while ((1 << rounds) < s.L) ++rounds;
-  for (int r = 0; r < rounds; ++r) {
-    for (int n = tid; n < N; n += blockDim.x) above[n] = 0;
+  int top = 0;
+  while ((1 << top) < s.L) ++top;                     // positions have `top` bits
+  // per path: the R-th largest position lies in [lo, lo + 2^shift) and is the need-th largest in there
+  for (int shift = top; shift > 0;) {
+    const int width = min(bits, shift);
+    shift -= width;
+    for (int x = tid; x < (N << bits); x += blockDim.x) hist[x] = 0;
     __syncthreads();
     for (int m = tid; m < M; m += blockDim.x) {
       const int gpos = list[m];
       const int j = path_of(s, gpos), n = j - poff;
-      if (cnt[n] > R && gpos - j * s.L >= ((lo[n] + hi[n]) >> 1)) atomicAdd(&above[n], 1);
+      if (cnt[n] <= R) continue;
+      const int rel = gpos - j * s.L - lo[n];
+      if (rel >= 0 && (rel >> (shift + width)) == 0) atomicAdd(&hist[(n << bits) | (rel >> shift)], 1);
     }
     __syncthreads();
     for (int n = tid; n < N; n += blockDim.x)
       if (cnt[n] > R) {
-        const int mid = (lo[n] + hi[n]) >> 1;
-        if (above[n] >= R) lo[n] = mid; else hi[n] = mid;
+        int left = need[n], digit = (1 << width) - 1;
+        while (digit > 0 && hist[(n << bits) | digit] < left) { left -= hist[(n << bits) | digit]; --digit; }
+        lo[n] += digit << shift; need[n] = left;
       }
     __syncthreads();
   }

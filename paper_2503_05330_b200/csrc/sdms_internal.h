@@ -26,6 +26,8 @@ cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t*
                           cudaStream_t stream);
 cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream);
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream);
+// tolerance 1 on large prompts: mark the queries, count, hand out slices, fill (four launches)
+cudaError_t launch_fuzzy_match(const Dev& s, int k, cudaStream_t stream);
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                        float* draft_edge_w, cudaStream_t stream);
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,

@@ -218,12 +218,60 @@ def test_fuzzy_config2_protocol(k):
     assert st["steps"] == 60
 
 
-def test_fuzzy_needs_a_small_prompt():
-    from paper_2503_05330_b200 import binding
+@pytest.mark.parametrize("seed", range(2))
+@pytest.mark.parametrize("alpha,mode,pool", [(1.0, 0, 0), (0.5, 0, 0), (1.0, 1, 0), (1.0, 2, 0), (0.5, 0, 1), (1.0, 0, 2)])
+def test_fuzzy_through_the_count_and_fill_passes_dense_tiny_vocab(seed, alpha, mode, pool):
+    # match_capacity below P*N*L: the build does not take the single-launch kernel, and with tolerance 1 the
+    # matches are counted, given slices and written by two passes of the fuzzy scan
+    G, N, L, V, D, k_max = 2, 6, 64, 3 + seed, 4, 4
+    tokens, lps = synth.small_random(G * N, L, V, 9500 + seed)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=alpha, mode=mode, pool=pool, eps=1, match_capacity=4000)
+        start = 2 + (np.arange(G * N) * 5 + seed) % 11          # some paths shorter than k
+        st = run_protocol(pair, tokens, lps, k, steps=20, warm=0, start_lens=start, commit_in_accept=True, check_dag=False)
+        assert st["steps"] > 5
+
+
+def test_fuzzy_on_a_prompt_too_large_for_the_single_launch_build():
+    # 40 paths of 4096 tokens: 160 Ki tokens per prompt.  Several 1024-token tiles per path, windows that reach
+    # back across tile borders, ragged ends; the wide pass takes the queries with many matches
+    G, N, L, V, D = 2, 40, 4096, 60, 6
+    tokens, lps = synth.small_random(G * N, L, V, 9600)
+    pair = Pair(G, N, L, V, 4, D, eps=1, alpha=0.5)
+    lens = (L - 8 - (np.arange(G * N) * 997) % 3000).astype(np.int32)
+    lens[[0, 7, 41]] = [1024, 1025, 3]
+    for c in range(0, L - 8, 2048):
+        part = np.clip(lens - c, 0, 2048).astype(np.int32)
+        pair.g.append(t32(tokens[:, c:c + 2048], pair.dev), t32(lps[:, c:c + 2048], pair.dev), t32(part, pair.dev))
+        pair.o.append(tokens[:, c:c + 2048], lps[:, c:c + 2048], part)
+    assert pair.g.status() == 0
+    for k in (3, 4, 2):
+        pair.build_and_compare(k, check_dag=False)
+    off, _ = pair.g.matches()
+    assert np.diff(off.numpy()).max() > 32
+
+
+def test_fuzzy_config5():
+    # the paper's experimental setting (tolerance 1) on the largest workload; the oracle's edit-distance search of
+    # 2M positions per query is slow, so a handful of paths are compared
     w = synth.WORKLOADS[5]
-    with pytest.raises(binding.SdmsError) as e:
-        binding.sdms_workspace_bytes(binding.make_config(w.G, w.N, w.L, w.V, w.k_max, w.D, epsilon=1))
-    assert e.value.code == binding.ERR_INVALID_ARG
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, eps=1)
+    start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+    pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+    for k in (4, 8):
+        pair.g.build_drafts(k)
+        assert pair.g.status() == 0
+        off, gpos = pair.g.matches()
+        off, gpos = off.numpy(), gpos.numpy()
+        gt, gl = pair.g.draft_tok.cpu().numpy(), pair.g.draft_len.cpu().numpy()
+        gs = pair.g.draft_score.cpu().numpy()
+        for i in (0, 37, 101, 255):
+            pair.o.build_path(k, i)
+            assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), pair.o.matches(i)), (k, i)
+            d, sc, _ = pair.o.draft(i)
+            assert gl[i] == len(d) and np.array_equal(gt[i, :len(d)], d), (k, i)
+            np.testing.assert_allclose(gs[i, :len(d)], sc, rtol=harness.RTOL, atol=0)
 
 
 # ---- tree and list draft pools (ablation variants) --------------------------------

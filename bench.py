@@ -219,13 +219,13 @@ class ClockSampler(threading.Thread):
 class Runner:
     """Device-resident replay of the decode protocol of one workload."""
 
-    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0, mode=0, host_io=False, backoff=False):
+    def __init__(self, w, seed, device, B, Ke, eps=0, pool=0, mode=0, host_io=False, backoff=False, index_max_n=0):
         import torch
         from paper_2503_05330_b200 import binding
         self.torch, self.binding, self.w, self.device = torch, binding, w, device
         self.tokens, self.logprobs = synth.make_streams(w, seed)
         self.s = binding.Sdms(w.G, w.N, w.L, w.V, w.k_max, w.D, device=device, max_append=w.D, B=B, Ke=Ke, epsilon=eps, pool_mode=pool,
-                             search_mode=mode, host_io=host_io)
+                             search_mode=mode, host_io=host_io, index_max_n=index_max_n)
         dev = self.s.device
         self.warm_tok = torch.from_numpy(np.ascontiguousarray(self.tokens[:, :w.k_max])).to(dev)
         self.warm_lp = torch.from_numpy(np.ascontiguousarray(self.logprobs[:, :w.k_max])).to(dev)
@@ -373,7 +373,7 @@ class Runner:
         return sum(per_step), units
 
 
-def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=0):
+def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=0, index_max_n=0):
     """Build latency of a workload at 97 % full histories (a full path builds no draft): per k the
     median, 10th and 90th percentile of the time of sdms_build_drafts (CUDA events on the launch
     stream, L2 flushed before every call), the matches it found, the kernel's own byte count per call
@@ -382,7 +382,7 @@ def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=
     from paper_2503_05330_b200 import binding
     tokens, logprobs = synth.make_streams(wl)
     s = binding.Sdms(wl.G, wl.N, wl.L, wl.V, wl.k_max, wl.D, device=device, max_append=wl.D,
-                     max_matches_per_path=max_matches, max_beams=beams)
+                     max_matches_per_path=max_matches, max_beams=beams, index_max_n=index_max_n)
     dev = s.device
     n = int(wl.L * 0.97)
     lens = (n - (np.arange(wl.P) * 13) % 97).astype(np.int32)
@@ -439,7 +439,7 @@ def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=
             out[str(k)]["get_beams_us"] = 1e3 * float(np.median([a.elapsed_time(b) for a, b in evs]))
     assert s.status() == 0
     return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
-            "max_matches_per_path": max_matches,
+            "max_matches_per_path": max_matches, "index_max_n": index_max_n or wl.k_max,
             "launches_per_build": 1 if fused else 4, "workspace_bytes": s.workspace_bytes, "build_by_k": out}
 
 
@@ -620,9 +620,9 @@ def ours_main(args, w):
         variant_us = {}
         if fuzzy is not None:
             ablation["dag_fuzzy"] = fplan["accept_length"]
-        for name, pool, eps, mode in (("tree", 1, 0, 0), ("list", 2, 0, 0), ("tree_fuzzy", 1, 1, 0), ("list_fuzzy", 2, 1, 0),
-                                      ("dag_best_path", 0, 0, 2), ("dag_best_path_fuzzy", 0, 1, 2)):
-            arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool, mode=mode)
+        for name, pool, eps, mode, idx in (("tree", 1, 0, 0, 0), ("list", 2, 0, 0, 0), ("tree_fuzzy", 1, 1, 0, 0), ("list_fuzzy", 2, 1, 0, 0),
+                                           ("dag_best_path", 0, 0, 2, 0), ("dag_best_path_fuzzy", 0, 1, 2, 0), ("dag_index_n2", 0, 0, 0, 2)):
+            arun = Runner(w, rank_seed(w, rank), device, 0, 0, eps=eps, pool=pool, mode=mode, index_max_n=idx)
             ablation[name] = arun.dry_run(allow_status=0x40)["accept_length"]
             if eps == 0:                 # step time of the variant, measured like the headline
                 arun.timed_steps(20)
@@ -671,6 +671,9 @@ def ours_main(args, w):
         others["cfg5_n256_l8192_match_cap_64"] = steady_state(synth.WORKLOADS[5], device, peak=peak, max_matches=64, ks=(1, 2, 3))
         others["cfg5_n256_l8192_match_cap_8"] = steady_state(synth.WORKLOADS[5], device, peak=peak, max_matches=8, ks=(1, 2, 3))
         others["cfg2_n16_l1024_four_beams"] = steady_state(w, device, peak=peak, beams=4)
+        # the index with tables for 1- and 2-grams only (64 bytes less per token and dropped length)
+        for c in (2, 4, 5):
+            others[synth.WORKLOADS[c].name + "_index_n2"] = steady_state(synth.WORKLOADS[c], device, peak=peak, index_max_n=2)
         scale = scan_at_scale(device)
         gscale = gather_at_scale(device)
     (ms, ms_e2e, host_ms_e2e), (units, units_e2e, _) = whole_job([ms, ms_e2e, host_ms_e2e], [units, units_e2e, 0.0], device)

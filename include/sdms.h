@@ -114,6 +114,13 @@ typedef struct {
                                     matching every query of its prompt, but at most 320 MiB), -1 = none.  A build
                                     whose queries need more falls back to one thread block for those that
                                     did not fit, with the same results                                    */
+  int32_t  index_max_n;          /* n-gram lengths the index keeps tables for: 1..index_max_n (0 = k_max, every
+                                    length that can be asked for).  A query with k > index_max_n looks up its last
+                                    index_max_n tokens instead: that bucket lists a superset of the k-gram's
+                                    occurrences, which are verified against all k tokens, or hands the query to the
+                                    scan.  Fewer tables: 64 bytes less per token and dropped length, and fewer
+                                    inserts per appended token; more queries scanned.  Results are the same      */
+  int32_t  reserved1;            /* must be 0 */
 } sdms_config;
 
 /* Bytes of device workspace a context with this configuration needs (host only,
@@ -175,9 +182,11 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
  * The same with a suffix length that backs off: every path uses the longest k in
  * [1, k_hi] for which it has at least one match (the paper names k but never fixes
  * it; longer suffixes give fewer, more specific candidates).  d_used_k [P] (may be
- * NULL) receives that k, 0 for paths without a draft.  One launch; only for
- * prompts small enough for the single-launch build (N*L <= 131072 tokens and
- * G*N*N*L <= match_capacity), otherwise SDMS_ERR_BAD_STATE.
+ * NULL) receives that k, 0 for paths without a draft.  One launch on prompts small
+ * enough for the single-launch build (N*L <= 131072 tokens and G*N*N*L <=
+ * match_capacity); on larger ones one round of launches per suffix length, longest
+ * first (a path that has found matches keeps them; sdms_debug_read_query_modes then
+ * reports 3 for it), there not together with epsilon = 1 (SDMS_ERR_BAD_STATE).
  */
 int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok, int32_t* d_draft_len,
                               float* d_draft_score, float* d_draft_edge_w, int32_t* d_used_k, void* stream);
@@ -210,8 +219,7 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
 int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,
               int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
               float* d_draft_edge_w, void* stream);
-/* sdms_step with the suffix length backing off as in sdms_build_drafts_backoff
- * (same restriction to small prompts, else SDMS_ERR_BAD_STATE). */
+/* sdms_step with the suffix length backing off as in sdms_build_drafts_backoff. */
 int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, const float* d_sampled_logprobs,
                       int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
                       float* d_draft_edge_w, int32_t* d_used_k, void* stream);

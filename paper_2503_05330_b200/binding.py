@@ -42,14 +42,15 @@ class SdmsConfig(C.Structure):
         ("dag_edges_per_node", C.c_int32), ("search_mode", C.c_int32), ("alpha", C.c_float),
         ("match_capacity", C.c_int64), ("epsilon", C.c_int32), ("pool_mode", C.c_int32),
         ("max_matches_per_path", C.c_int32), ("max_beams", C.c_int32), ("wide_table_bytes", C.c_int64),
+        ("index_max_n", C.c_int32), ("reserved1", C.c_int32),
     ]
 
 
 def make_config(G, N, L, V, k_max, D, max_append=None, B=0, Ke=0, search_mode=0, alpha=1.0,
-                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0, wide_table_bytes=0, max_beams=0) -> SdmsConfig:
+                match_capacity=0, epsilon=0, pool_mode=0, max_matches_per_path=0, wide_table_bytes=0, max_beams=0, index_max_n=0) -> SdmsConfig:
     return SdmsConfig(C.sizeof(SdmsConfig), G, N, L, V, k_max, D, D + 1 if max_append is None else max_append,
                       B, Ke, search_mode, alpha, match_capacity, epsilon, pool_mode, max_matches_per_path, max_beams,
-                      wide_table_bytes)
+                      wide_table_bytes, index_max_n, 0)
 
 
 _lib = None

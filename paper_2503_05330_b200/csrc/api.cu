@@ -28,6 +28,7 @@ int check_config(const sdms_config* c) {
     return SDMS_ERR_INVALID_ARG;
   if (c->capacity < 2 || c->vocab < 1 || c->vocab > (1 << 26)) return SDMS_ERR_INVALID_ARG;
   if (c->k_max < 1 || c->k_max > SDMS_MAX_K) return SDMS_ERR_INVALID_ARG;
+  if (c->index_max_n < 0 || c->index_max_n > c->k_max || c->reserved1 != 0) return SDMS_ERR_INVALID_ARG;
   if (c->max_draft_len < 1 || c->max_draft_len > SDMS_MAX_DRAFT) return SDMS_ERR_INVALID_ARG;
   if (c->max_append < 1 || c->max_append > c->max_draft_len + 1) return SDMS_ERR_INVALID_ARG;
   if (c->dag_nodes_per_layer < 0 || c->dag_nodes_per_layer > SDMS_MAX_DAG_NODES) return SDMS_ERR_INVALID_ARG;
@@ -67,7 +68,7 @@ Layout make_layout(const sdms_config* c) {
   l.len = take(P * 4);
   l.rec = take(P * kRecWords * 4);
   l.status = take(4);
-  l.index = take((size_t)c->num_groups * c->k_max * cap * kBucketWords * 4);
+  l.index = take((size_t)c->num_groups * (c->index_max_n ? c->index_max_n : c->k_max) * cap * kBucketWords * 4);
   l.q_fp = take(P * 4); l.q_mode = take(P * 4); l.q_reserved = take(P * 4);
   l.q_off = take(P * 4); l.q_cursor = take(P * 4);
   l.match_cursor = take(8);
@@ -226,7 +227,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   std::memset(ctx->prof_n, 0, sizeof(ctx->prof_n));
   Dev& d = ctx->dev;
   d.G = cfg->num_groups; d.N = cfg->paths_per_group; d.L = cfg->capacity; d.V = cfg->vocab;
-  d.k_max = cfg->k_max; d.D = cfg->max_draft_len; d.max_append = cfg->max_append;
+  d.k_max = cfg->k_max; d.idx_n = cfg->index_max_n ? cfg->index_max_n : cfg->k_max; d.D = cfg->max_draft_len; d.max_append = cfg->max_append;
   d.B = cfg->dag_nodes_per_layer; d.Ke = cfg->dag_nodes_per_layer ? cfg->dag_edges_per_node : 0;
   d.mode = cfg->search_mode; d.P = d.G * d.N;
   d.alpha = (double)cfg->alpha;
@@ -312,7 +313,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
     rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_fuzzy_match(ctx->dev, k, st); });
     ctx->launches += 3;
   } else {
-    rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, st); });
+    rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, 0, st); });
     if (rc != SDMS_OK) return rc;
     rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
   }
@@ -330,9 +331,27 @@ int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok,
                               float* d_draft_score, float* d_draft_edge_w, int32_t* d_used_k, void* stream) {
   if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
   if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
-  if (!ctx->dev.fused) return SDMS_ERR_BAD_STATE;
   cudaStream_t st = (cudaStream_t)stream;
   if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
+  if (!ctx->dev.fused) {
+    // large prompts: one probe / scan / dag (/ wide) round per suffix length, longest first; a path that has found
+    // matches keeps them and its draft, the others try again with a shorter suffix
+    if (ctx->dev.eps > 0) return SDMS_ERR_BAD_STATE;
+    for (int k = k_hi; k >= 1; --k) {
+      const int round = kRoundBackoff | (k < k_hi ? kRoundNotFirst : 0) | (k == 1 ? kRoundLast : 0);
+      int rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, k < k_hi, st); });
+      if (rc == SDMS_OK) rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+      if (rc == SDMS_OK)
+        rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
+          return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st, round, k, d_used_k); });
+      if (rc == SDMS_OK && ctx->dev.w_grid > 0)
+        rc = timed(ctx, SDMS_KERNEL_DAG_WIDE, st, [&] {
+          return launch_dag_wide(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
+      if (rc != SDMS_OK) return rc;
+    }
+    ctx->built = true;
+    return SDMS_OK;
+  }
   const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
     return launch_build_fused(ctx->dev, k_hi, 1, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, d_used_k, st); });
   if (rc == SDMS_OK) ctx->built = true;
@@ -387,7 +406,7 @@ int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, con
   if (!ctx || !d_sampled || !d_sampled_logprobs || !d_accept_len || !d_draft_tok || !d_draft_len)
     return SDMS_ERR_INVALID_ARG;
   if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
-  if (!ctx->dev.fused) return SDMS_ERR_BAD_STATE;
+  if (!ctx->dev.fused && ctx->dev.eps > 0) return SDMS_ERR_BAD_STATE;
   if (!ctx->step_fits) {
     const int rc = sdms_accept(ctx, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, stream);
     if (rc != SDMS_OK) return rc;

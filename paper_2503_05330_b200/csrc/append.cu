@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(128) trim_shift_kernel(Dev s, const int32_t* _
 __global__ void __launch_bounds__(256) trim_clear_kernel(Dev s) {
   grid_wait();
   grid_release();
-  const size_t per_group = (size_t)s.k_max * s.table_cap * kBucketWords / 4;      // 16-byte words of a prompt's tables
+  const size_t per_group = (size_t)s.idx_n * s.table_cap * kBucketWords / 4;      // 16-byte words of a prompt's tables
   uint4* index = reinterpret_cast<uint4*>(s.index);
   for (size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x; x < per_group * s.G; x += (size_t)gridDim.x * blockDim.x)
     if (s.g_trim[x / per_group]) index[x] = make_uint4(0u, 0u, 0u, 0u);
@@ -108,8 +108,8 @@ __global__ void __launch_bounds__(128) trim_reindex_kernel(Dev s) {
   const int32_t* tok = s.tok + (size_t)p * s.L;
   const uint32_t lbase = (uint32_t)(p - g * s.N) * (uint32_t)s.L;
   uint32_t st = 0;
-  for (int w = threadIdx.x; w < len * s.k_max; w += blockDim.x) {
-    const int pos = w / s.k_max, nn = w % s.k_max + 1;
+  for (int w = threadIdx.x; w < len * s.idx_n; w += blockDim.x) {
+    const int pos = w / s.idx_n, nn = w % s.idx_n + 1;
     if (pos + 1 < nn) continue;
     uint64_t h = gram_init(nn);
     for (int t = pos - nn + 1; t <= pos; ++t) h = gram_step(h, tok[t]);

@@ -121,8 +121,8 @@ __device__ void append_tokens(const Dev& s, int p, int len0, int n, const int32_
   }
   const int g = p / s.N;
   const uint32_t lbase = (uint32_t)(p - g * s.N) * (uint32_t)s.L;
-  for (int w = threadIdx.x; w < n * s.k_max; w += blockDim.x) {
-    const int a = w / s.k_max, nn = w % s.k_max + 1;
+  for (int w = threadIdx.x; w < n * s.idx_n; w += blockDim.x) {
+    const int a = w / s.idx_n, nn = w % s.idx_n + 1;
     const int pos = len0 + a;
     if (pos + 1 < nn) continue;
     uint64_t h = gram_init(nn);
@@ -201,10 +201,11 @@ __device__ void accept_commit_phase(const Dev& s, int p, const int32_t* draft_to
   if (next_k > 0 && s.eps == 0 && threadIdx.x == blockDim.x - 64) {
     const int len0 = sh_len0, len1 = len0 + sh_n;
     if (len1 >= next_k && len1 < s.L) {
-      uint64_t h = gram_init(next_k);
-      for (int x = len1 - next_k; x < len1; ++x) h = gram_step(h, x >= len0 ? sh_smp[x - len0] : sh_rec[len0 - x]);
+      const int nx = min(next_k, s.idx_n);               // the query's last nx tokens are what the index is asked for
+      uint64_t h = gram_init(nx);
+      for (int x = len1 - nx; x < len1; ++x) h = gram_step(h, x >= len0 ? sh_smp[x - len0] : sh_rec[len0 - x]);
       const uint32_t* bucket =
-          index_table(s, p / s.N, next_k) + (size_t)gram_bucket(gram_final(h), s.table_cap) * kBucketWords;
+          index_table(s, p / s.N, nx) + (size_t)gram_bucket(gram_final(h), s.table_cap) * kBucketWords;
       asm volatile("prefetch.global.L2 [%0];" ::"l"(bucket));
     }
   }

@@ -1236,7 +1236,8 @@ template <bool EXPORT>
 __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
                                                           int32_t* __restrict__ draft_len,
                                                           float* __restrict__ draft_score,
-                                                          float* __restrict__ draft_edge_w) {
+                                                          float* __restrict__ draft_edge_w, int round, int k,
+                                                          int32_t* __restrict__ used_k) {
   grid_wait();
   grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -1245,14 +1246,17 @@ __global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __r
   const int i = blockIdx.x;
   if (i == 0) {                                       // probe and scan are done with these: the next build finds them at zero
     for (int x = threadIdx.x; x < s.G; x += blockDim.x) s.g_nscan[x] = 0;
-    if (threadIdx.x == 0) *s.match_cursor = 0ull;
+    // (the slices of a back-off build's earlier rounds stay where they are until its last round)
+    if (threadIdx.x == 0 && (!(round & kRoundBackoff) || (round & kRoundLast))) *s.match_cursor = 0ull;
   }
+  if ((round & kRoundNotFirst) && s.q_mode[i] == Q_DONE) return;     // drafted in an earlier round, from a longer suffix
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
   const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
   if (M == 0) {
-    if (threadIdx.x == 0) draft_len[i] = 0;
+    if (threadIdx.x == 0) { draft_len[i] = 0; if (used_k) used_k[i] = 0; }
     return;
   }
+  if ((round & kRoundBackoff) && threadIdx.x == 0) { s.q_mode[i] = Q_DONE; if (used_k) used_k[i] = k; }
   const int g = i / s.N;
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + g * s.N + n);
   __syncthreads();
@@ -1401,11 +1405,13 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
       for (int t = 0; t < k; ++t) sh_q[t] = ldm(rec + k - t);
       mode = Q_SCAN;
     } else if (len_i >= k && len_i < s.L) {
-      uint64_t h = gram_init(k);
-      for (int t = 0; t < k; ++t) { const int32_t x = ldm(rec + k - t); sh_q[t] = x; h = gram_step(h, x); }
+      // the index is asked for the query's last nx tokens: all k of them unless the context keeps fewer tables
+      const int nx = min(k, s.idx_n);
+      uint64_t h = gram_init(nx);
+      for (int t = 0; t < k; ++t) { const int32_t x = ldm(rec + k - t); sh_q[t] = x; if (t >= k - nx) h = gram_step(h, x); }
       h = gram_final(h);
       fp = gram_fp(h);
-      const uint32_t* table = index_table(s, g, k);
+      const uint32_t* table = index_table(s, g, nx);
       uint32_t b = gram_bucket(h, s.table_cap);
       for (uint32_t probe = 0; probe < s.table_cap; ++probe) {
         const uint4* cand = reinterpret_cast<const uint4*>(table + (size_t)b * kBucketWords);
@@ -1436,7 +1442,7 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
       const int jn = (int)(lpos / (uint32_t)s.L);
       const int j = g * s.N + jn;
       const int e = (int)(lpos % (uint32_t)s.L);
-      if (j != i && e <= sh_len[jn] - 2) {
+      if (j != i && e >= k - 1 && e <= sh_len[jn] - 2) {
         const int32_t* c = s.tok + (size_t)j * s.L + (e - k + 1);
         bool same = true;
         for (int t = 0; t < k; ++t) same = same && (ldm(c + t) == sh_q[t]);
@@ -1674,12 +1680,12 @@ cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, c
 }
 
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
-                       float* draft_edge_w, cudaStream_t stream) {
+                       float* draft_edge_w, cudaStream_t stream, int round, int k, int32_t* used_k) {
   if (with_export)
     return launch_overlapped(dag_kernel<true>, dim3(s.P), dim3(kDagThreads), dag_smem_bytes<true>(), stream, s,
-                             draft_tok, draft_len, draft_score, draft_edge_w);
+                             draft_tok, draft_len, draft_score, draft_edge_w, 0, 0, (int32_t*)nullptr);
   return launch_overlapped(dag_kernel<false>, dim3(s.P), dim3(kDagThreads), dag_smem_bytes<false>(), stream, s,
-                           draft_tok, draft_len, draft_score, draft_edge_w);
+                           draft_tok, draft_len, draft_score, draft_edge_w, round, k, used_k);
 }
 
 // Cluster size (CTAs = consecutive paths of one prompt) of the single-launch build, 1 for none.  A cluster

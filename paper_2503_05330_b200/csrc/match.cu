@@ -62,12 +62,13 @@ constexpr int kProbeWarps = 8;
 constexpr int kInlineArea = 8;
 static_assert(kInlineArea >= kInlineSlots && kRecWords == 32 && kBucketWords == 8, "lane layout of the probe");
 
-__global__ void __launch_bounds__(kProbeWarps * 32) probe_kernel(Dev s, int k) {
+__global__ void __launch_bounds__(kProbeWarps * 32) probe_kernel(Dev s, int k, int skip_done) {
   grid_wait();
   grid_release();
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * kProbeWarps + (threadIdx.x >> 5);
   if (i >= s.P) return;                                          // whole warps
+  if (skip_done && s.q_mode[i] == Q_DONE) return;                // back-off: this path has its matches from a longer suffix
   const int g = i / s.N;
   const int32_t mine = s.rec[(size_t)i * kRecWords + lane];
   const int len_i = __shfl_sync(FULL_MASK, mine, 0);
@@ -75,13 +76,19 @@ __global__ void __launch_bounds__(kProbeWarps * 32) probe_kernel(Dev s, int k) {
   uint32_t fp = 0, count = 0;
   if (len_i >= k && len_i < s.L) {
     // the query, oldest token first: token x of it sits in lane k - x of the record
-    uint64_t h = gram_init(k);
-    int32_t q_last = 0;
-    for (int x = 0; x < k; ++x) { q_last = __shfl_sync(FULL_MASK, mine, k - x); h = gram_step(h, q_last); }
-    h = gram_final(h);
-    fp = gram_fp(h);
-    const uint32_t* table = index_table(s, g, k);
-    uint32_t b = gram_bucket(h, s.table_cap);
+    // fp names the whole k-gram (the scan looks queries up by it); the index is asked for the last nx tokens
+    const int nx = min(k, s.idx_n);
+    uint64_t h = gram_init(k), hx = gram_init(nx);
+    for (int x = 0; x < k; ++x) {
+      const int32_t t = __shfl_sync(FULL_MASK, mine, k - x);
+      h = gram_step(h, t);
+      if (x >= k - nx) hx = gram_step(hx, t);
+    }
+    fp = gram_fp(gram_final(h));
+    hx = gram_final(hx);
+    const uint32_t want = gram_fp(hx);
+    const uint32_t* table = index_table(s, g, nx);
+    uint32_t b = gram_bucket(hx, s.table_cap);
     int found = -1;                                              // lane that holds the bucket's first word
     uint32_t word = 0;
     for (uint32_t probe = 0; probe < s.table_cap && found < 0; probe += 4) {
@@ -90,7 +97,7 @@ __global__ void __launch_bounds__(kProbeWarps * 32) probe_kernel(Dev s, int k) {
       bool end = false;
       for (int r = 0; r < 4 && found < 0 && !end; ++r) {
         const uint32_t w0 = __shfl_sync(FULL_MASK, word, 8 * r);
-        if (w0 == fp) found = 8 * r;
+        if (w0 == want) found = 8 * r;
         else if (w0 == 0u) end = true;
       }
       if (end) break;
@@ -487,8 +494,8 @@ __global__ void __launch_bounds__(kProbeThreads) compact_matches_kernel(Dev s, i
 
 }  // namespace
 
-cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream) {
-  return launch_overlapped(probe_kernel, dim3((s.P + kProbeWarps - 1) / kProbeWarps), dim3(kProbeWarps * 32), 0, stream, s, k);
+cudaError_t launch_probe(const Dev& s, int k, int skip_done, cudaStream_t stream) {
+  return launch_overlapped(probe_kernel, dim3((s.P + kProbeWarps - 1) / kProbeWarps), dim3(kProbeWarps * 32), 0, stream, s, k, skip_done);
 }
 
 // Called when a context is created, with its device current.

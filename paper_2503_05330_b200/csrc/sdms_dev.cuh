@@ -24,7 +24,9 @@ constexpr int kWideBarrierWays = 8;     // grid-barrier arrivals are spread over
 constexpr int kWideBarrierAt = 16, kWideBarrierStride = 16;   // ... at w_ctl[16], [32], ...: a 128-byte line each
 constexpr int kWideCtlWords = kWideBarrierAt + kWideBarrierWays * kWideBarrierStride;
 
-enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2 };
+// Q_DONE: a back-off build on a large prompt has found this path's matches at a longer suffix length
+enum QueryMode : int32_t { Q_NONE = 0, Q_INLINE = 1, Q_SCAN = 2, Q_DONE = 3 };
+constexpr int kRoundBackoff = 1, kRoundNotFirst = 2, kRoundLast = 4;   // flags of one round of such a build
 
 // One slot of a wide query's node table of one layer (32 bytes, one sector).  All-zero = empty.  The keys
 // (token + 1) that the probing looks at lie in an array of their own, eight to a sector.
@@ -41,6 +43,7 @@ struct WidePred { unsigned long long succ_w, succ; };   // the same two words fo
 // Everything a kernel needs, passed by value.
 struct Dev {
   int32_t G, N, L, V, k_max, D, max_append, B, Ke, mode, P;
+  int32_t idx_n;                       // n-gram lengths 1..idx_n have index tables (<= k_max)
   int32_t pool;                        // 0 DAG, 1 tree, 2 list
   int32_t eps;                         // edit-distance tolerance of the suffix match (0 or 1)
   int32_t fused;                       // one kernel per build (small prompts) instead of probe + scan + dag
@@ -102,7 +105,7 @@ __device__ __forceinline__ uint32_t gram_fp(uint64_t h) { return (uint32_t)(h >>
 __device__ __forceinline__ uint32_t gram_bucket(uint64_t h, uint32_t cap) { return (uint32_t)h & (cap - 1); }
 
 __device__ __forceinline__ uint32_t* index_table(const Dev& s, int g, int n) {
-  return s.index + ((size_t)(g * s.k_max + (n - 1)) * s.table_cap) * kBucketWords;
+  return s.index + ((size_t)(g * s.idx_n + (n - 1)) * s.table_cap) * kBucketWords;
 }
 
 // Path (row of the store) a global position x = j * L + e lies in, without a division: L_magic =

@@ -24,12 +24,13 @@ cudaError_t launch_append(const Dev& s, const int32_t* tokens, const float* logp
 cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t* draft_len,
                           const int32_t* sampled, const float* sampled_lp, int32_t* accept_len,
                           cudaStream_t stream);
-cudaError_t launch_probe(const Dev& s, int k, cudaStream_t stream);
+cudaError_t launch_probe(const Dev& s, int k, int skip_done, cudaStream_t stream);
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream);
 // tolerance 1 on large prompts: mark the queries, count, hand out slices, fill (four launches)
 cudaError_t launch_fuzzy_match(const Dev& s, int k, cudaStream_t stream);
+// round: 0 for an ordinary build; kRound* flags, k and used_k for one round of a back-off build on a large prompt
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
-                       float* draft_edge_w, cudaStream_t stream);
+                       float* draft_edge_w, cudaStream_t stream, int round = 0, int k = 0, int32_t* used_k = nullptr);
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream);
 // phase 0: shift the histories; 1: empty the index tables of the prompts that changed; 2: index them again

@@ -21,13 +21,13 @@ class Pair:
     """One oracle and one CUDA context with the same configuration."""
 
     def __init__(self, G, N, L, V, k_max, D, alpha=1.0, mode=0, B=0, Ke=0, max_append=None, match_capacity=0,
-                 eps=0, pool=0, device="cuda:0", host_io=False, max_matches=0, wide_table_bytes=0, max_beams=0):
+                 eps=0, pool=0, device="cuda:0", host_io=False, max_matches=0, wide_table_bytes=0, max_beams=0, index_max_n=0):
         self.o = Oracle(G, N, L, V, D, alpha=alpha, mode=mode, eps=eps, pool=pool, max_matches=max_matches)
         self.pool = pool
         self.g = binding.Sdms(G, N, L, V, k_max, D, device=device, alpha=alpha, search_mode=mode, B=B, Ke=Ke,
                               max_append=max_append, match_capacity=match_capacity, epsilon=eps, pool_mode=pool,
                               host_io=host_io, max_matches_per_path=max_matches, wide_table_bytes=wide_table_bytes,
-                              max_beams=max_beams)
+                              max_beams=max_beams, index_max_n=index_max_n)
         self.dev = self.g.device
         self.P, self.L, self.D, self.N = G * N, L, D, N
         self.B, self.Ke = B, Ke

@@ -935,3 +935,82 @@ def test_best_path_with_heavy_queries_through_build_and_step():
     pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, mode=2, max_append=w.D)
     st = harness.run_step_protocol(pair, tokens, lps, [1, 2], steps=25, warm=0, start_lens=start, check_every=5)
     assert st["steps"] == 25
+
+
+# ---- an index that keeps tables for the shortest n-grams only ------------------------------------
+@pytest.mark.parametrize("index_max_n", [1, 2])
+@pytest.mark.parametrize("match_capacity", [0, 3000])
+def test_short_index_dense_tiny_vocab_every_step(index_max_n, match_capacity):
+    # queries longer than the longest indexed n-gram look up their last index_max_n tokens and verify (or scan for)
+    # all k; both through the single-launch build and (match_capacity below P*N*L) the probe / scan / dag kernels
+    G, N, L, V, D, k_max = 2, 6, 64, 4, 4, 4
+    tokens, lps = synth.small_random(G * N, L, V, 9700 + index_max_n)
+    for k in range(1, k_max + 1):
+        pair = Pair(G, N, L, V, k_max, D, alpha=0.5, B=3, Ke=2, index_max_n=index_max_n, match_capacity=match_capacity)
+        start = 3 + (np.arange(G * N) * 5) % 11
+        st = run_protocol(pair, tokens, lps, k, steps=25, warm=0, start_lens=start, commit_in_accept=True)
+        assert st["steps"] > 5
+
+
+@pytest.mark.parametrize("wid,index_max_n", [(2, 2), (2, 1), (5, 2)])
+def test_short_index_on_benchmark_workloads(wid, index_max_n):
+    w = synth.WORKLOADS[wid]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D, index_max_n=index_max_n)
+    if wid == 2:
+        start = 600 + (np.arange(w.P) * 37) % 300
+        st = harness.run_step_protocol(pair, tokens, lps, [4, 1, 3, 2], steps=100, warm=0, start_lens=start, check_every=5)
+        assert st["steps"] == 100
+        assert (pair.g.query_modes() > 0).any()
+    else:
+        start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+        pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+        for k in (3, 8):
+            pair.build_and_compare(k, check_dag=False, paths=list(range(0, w.P, 8)))
+        pair.trim(np.full(w.P, 4000, np.int32))                 # the rebuilt index has the same few tables
+        pair.build_and_compare(4, check_dag=False, paths=list(range(0, w.P, 8)))
+
+
+# ---- back-off of the suffix length on prompts that take the probe / scan / dag kernels ------------
+def test_backoff_by_rounds_dense_tiny_vocab():
+    G, N, L, V, D, k_max = 2, 6, 64, 4, 4, 4
+    tokens, lps = synth.small_random(G * N, L, V, 9800)
+    pair = Pair(G, N, L, V, k_max, D, alpha=0.5, match_capacity=3000)
+    start = (2 + (np.arange(G * N) * 5) % 11).astype(np.int32)
+    pair.append(tokens[:, :16], lps[:, :16], start, expect_status=0)
+    seen = set()
+    for step in range(20):
+        lens = pair.o.lengths()
+        _, _, used = pair.backoff_and_compare(k_max if step % 3 else 2)
+        seen |= set(used.tolist())
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
+        pair.accept_and_compare(sampled, sampled_lp)
+        pair.build_and_compare(1 + step % k_max, check_dag=False)      # an ordinary build in between finds a clean state
+    assert len(seen) >= 3
+    pair.check_history()
+
+
+def test_backoff_by_rounds_config5():
+    w = synth.WORKLOADS[5]
+    tokens, lps = synth.make_streams(w)
+    pair = Pair(w.G, w.N, w.L, w.V, w.k_max, w.D, max_append=w.D)
+    start = (w.L - 40 - (np.arange(w.P) * 29) % 3000).astype(np.int32)
+    pair.append(tokens[:, :int(start.max())], lps[:, :int(start.max())], start, expect_status=0)
+    pair.g.build_drafts_backoff(w.k_max)
+    assert pair.g.status() == 0
+    used_g = pair.g.used_k.cpu().numpy()
+    gt, gl = pair.g.draft_tok.cpu().numpy(), pair.g.draft_len.cpu().numpy()
+    off, gpos = pair.g.matches()
+    off, gpos = off.numpy(), gpos.numpy()
+    for i in range(0, w.P, 8):                                          # oracle: fixed-k builds composed per path
+        used = 0
+        for k in range(w.k_max, 0, -1):
+            pair.o.build_path(k, i)
+            if len(pair.o.matches(i)) > 0:
+                used = k
+                break
+        assert used_g[i] == used, (i, used_g[i], used)
+        d, _, _ = pair.o.draft(i)
+        assert gl[i] == len(d) and np.array_equal(gt[i, :len(d)], d), i
+        assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), pair.o.matches(i)), i
+    assert len(set(used_g.tolist())) >= 3

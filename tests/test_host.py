@@ -31,12 +31,13 @@ def test_workspace_bytes_and_config_validation(lib):
     # path store (tokens + probabilities) plus k_max tables of 2*N*L 32-byte buckets
     assert n >= 2 * 16 * 1024 * 4 + 4 * 2 * 16 * 1024 * 32
     assert n % 256 == 0
+    assert binding.sdms_workspace_bytes(binding.make_config(1, 16, 1024, 128256, 4, 8, index_max_n=2)) < n - 2 * 2 * 16 * 1024 * 32 + 4096
     bigger = binding.make_config(1, 16, 1024, 128256, 4, 8, B=8, Ke=4)
     assert binding.sdms_workspace_bytes(bigger) > n
     bad = [dict(G=0), dict(N=0), dict(N=2000), dict(L=1), dict(V=0), dict(k_max=0), dict(k_max=17), dict(D=0),
            dict(D=33), dict(max_append=0), dict(max_append=10), dict(B=33), dict(B=4, Ke=0), dict(search_mode=3), dict(search_mode=2, pool_mode=1),
            dict(alpha=1.5), dict(alpha=-0.1), dict(match_capacity=-1), dict(epsilon=2), dict(epsilon=-1), dict(pool_mode=3), dict(pool_mode=-1),
-           dict(max_matches_per_path=-1), dict(max_beams=9), dict(max_beams=-1), dict(max_beams=2, pool_mode=1)]
+           dict(max_matches_per_path=-1), dict(max_beams=9), dict(max_beams=-1), dict(max_beams=2, pool_mode=1), dict(index_max_n=4), dict(index_max_n=-1)]
     base = dict(G=1, N=4, L=64, V=100, k_max=3, D=4)
     for change in bad:
         kw = dict(base, **change)

@@ -507,10 +507,11 @@ def gather_at_scale(device, G=64, N=256, L=8192, V=16384, D=16):
            "store_bytes": 8 * P * n, "workspace_bytes": s.workspace_bytes,
            "matches": int(m.sum()), "mean_matches_per_query": float(m.mean()), "max_matches_per_query": int(m.max())}
     nbytes = int(8 * n_m.sum() + 4 * len(gpos) + P * (12 * D + 4))
-    for name in ("dag", "dag_heavy"):
+    for name in ("dag", "dag_wide"):
         if name in prof and prof[name][1]:
             ms, launches = prof[name]
             out[name + "_us_per_launch"] = 1e3 * ms / launches
+    out["queries_by_mode"] = {str(k): int(v) for k, v in zip(*np.unique(s.query_modes(), return_counts=True))}
     us = sum(out[k] for k in out if k.endswith("_us_per_launch"))
     out.update(algorithmic_bytes=nbytes, us_per_build_gather_side=us, gbs=nbytes / (us * 1e-6) / 1e9)
     del s
@@ -767,9 +768,16 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the build-only figures of the other workloads")
     ap.add_argument("--steady", type=int, default=0,
                     help="only print the build-only figures of this workload at 97 %% full histories (for profiling)")
+    ap.add_argument("--gather-scale", type=int, default=0,
+                    help="only run the gather / DAG kernels on this many prompts of 256 paths x 8192 tokens (for profiling)")
     ap.add_argument("--scan-scale", type=int, default=0,
                     help="only run the tile-scan kernel on this many prompts of 256 paths x 8192 tokens (for profiling)")
     args = ap.parse_args()
+    if args.gather_scale:
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps({"gather_at_scale": gather_at_scale("cuda:0", G=args.gather_scale)}), flush=True)
+        return
     if args.scan_scale:
         import torch
         torch.cuda.set_device(0)

@@ -85,9 +85,10 @@ typedef struct {
                                        successors of best(d+1,.), summed from the path's end; the
                                        walk follows the largest best(), ties to the smaller token.
                                        DAG pool only.  Paths with more matches than shared memory
-                                       takes are searched over node tables in the workspace's table
-                                       area (wide_table_bytes); only if that is switched off or full
-                                       do they get the mode-0 draft and raise SDMS_STATUS_SEARCH_FALLBACK */
+                                       takes are searched by one more launch after the build, over
+                                       node tables in the workspace's table area (wide_table_bytes);
+                                       only if that is switched off or full do they keep the mode-0
+                                       draft and raise SDMS_STATUS_SEARCH_FALLBACK               */
   float    alpha;                /* Eq. 5 mixing weight; the paper's experiments use 1        */
   int64_t  match_capacity;       /* match-list entries in the workspace, 0 = default          */
   int32_t  epsilon;              /* Eq. 4 edit-distance tolerance of the suffix match: 0 (exact)
@@ -213,7 +214,8 @@ int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draf
  * When a prompt's paths fit one thread-block cluster (paths_per_group <= 16, the
  * single-launch build applies and the device can hold the clusters of all prompts
  * at once) the step is ONE kernel launch: the paths of a prompt commit, meet at a cluster
- * barrier, and build.  Otherwise the call issues the separate launches.
+ * barrier, and build (search_mode 2 adds the launch that searches the paths with many
+ * matches).  Otherwise the call issues the separate launches.
  * sdms_step_is_single_launch reports which (1 / 0).
  */
 int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d_sampled_logprobs,

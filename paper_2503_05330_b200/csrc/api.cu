@@ -13,7 +13,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
   size_t tok, pq, len, rec, status, index, q_fp, q_mode, q_reserved, q_off, q_cursor, match_cursor, g_nscan, g_trim, matches;
-  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_key, w_item, b_ent, b_ctl;
+  size_t w_ctl, w_desc, w_pred, w_edge, w_tab, w_key, w_item, b_ent, b_ctl, bp_todo;
   bool wide_on;
   uint64_t w_slots;
   size_t x_draft_tok, x_draft_len, x_node_tok, x_node_S, x_node_cnt, x_node_count, x_edge_dst, x_edge_S, x_edge_cnt, x_out_degree;
@@ -94,7 +94,8 @@ Layout make_layout(const sdms_config* c) {
   }
   l.w_slots = (l.wide_on || (stride > 0 && wide > 0)) ? (uint64_t)wide / slot_bytes : 0;
   l.w_ctl = take((size_t)kWideCtlWords * 8);
-  l.b_ctl = take(8);
+  l.b_ctl = take(16);
+  l.bp_todo = take(P * 4);
   l.w_desc = take(l.wide_on ? (size_t)kMaxWide * 16 : 0);
   l.w_pred = take(l.wide_on ? (size_t)kMaxWide * SDMS_MAX_DRAFT * sizeof(WidePred) : 0);
   l.w_edge = take(l.wide_on ? (size_t)kMaxWide * SDMS_MAX_DRAFT * 8 : 0);
@@ -162,11 +163,15 @@ int drain_pending(sdms_ctx* ctx, size_t count) {
   return SDMS_OK;
 }
 
-// Best-path builds may reserve node tables in the workspace's table area (paths with more matches than
-// shared memory takes): the cursor they reserve with starts every build at zero.  Other contexts: nothing.
-int reset_table_cursor(sdms_ctx* ctx, cudaStream_t stream) {
+// A best-path build marks the paths with more matches than its shared-memory search takes; this launch
+// searches them over node tables in the workspace's table area and replaces their (greedy) drafts.
+// Other contexts: nothing.
+int finish_best_paths(sdms_ctx* ctx, int32_t* draft_tok, int32_t* draft_len, float* draft_score, float* draft_edge_w,
+                      cudaStream_t stream) {
   if (ctx->cfg.search_mode != 2 || ctx->dev.beam_stride == 0) return SDMS_OK;
-  return cudaMemsetAsync(ctx->dev.b_ctl, 0, 8, stream) == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
+  ++ctx->launches;
+  return launch_best_path_fix(ctx->dev, draft_tok, draft_len, draft_score, draft_edge_w, stream) == cudaSuccess
+             ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
 template <class F>
@@ -262,7 +267,7 @@ int sdms_create(const sdms_config* cfg, void* d_workspace, size_t bytes, sdms_ct
   d.w_tab = (WideSlot*)(w + lay.w_tab); d.w_key = (uint32_t*)(w + lay.w_key); d.w_item = (int32_t*)(w + lay.w_item);
   d.w_grid = lay.wide_on ? wide_kernel_grid() : 0;   // 0 (also without cooperative launch on this device): one thread block per query
   d.w_slots = lay.w_slots;
-  d.b_ent = (BeamEnt*)(w + lay.b_ent); d.b_ctl = (unsigned long long*)(w + lay.b_ctl); d.beam_stride = lay.w_slots ? (cfg->max_beams > 0 ? cfg->max_beams : (cfg->search_mode == 2 ? 1 : 0)) : 0;
+  d.b_ent = (BeamEnt*)(w + lay.b_ent); d.b_ctl = (unsigned long long*)(w + lay.b_ctl); d.bp_todo = (int32_t*)(w + lay.bp_todo); d.beam_stride = lay.w_slots ? (cfg->max_beams > 0 ? cfg->max_beams : (cfg->search_mode == 2 ? 1 : 0)) : 0;
   ctx->step_fits = step_kernel_fits(d);
   d.build_cluster = build_cluster_size(d);
   *out = ctx;
@@ -301,12 +306,12 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
   if (k < 1 || k > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   if (ctx->dev.fused) {
     const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
       return launch_build_fused(ctx->dev, k, k, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, nullptr, st); });
-    if (rc == SDMS_OK) ctx->built = true;
-    return rc;
+    if (rc != SDMS_OK) return rc;
+    ctx->built = true;
+    return finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
   }
   int rc;
   if (ctx->dev.eps > 0) {                            // matches with tolerance: sized by counting, four launches
@@ -323,8 +328,9 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   if (rc == SDMS_OK && ctx->dev.w_grid > 0)
     rc = timed(ctx, SDMS_KERNEL_DAG_WIDE, st, [&] {
       return launch_dag_wide(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
-  if (rc == SDMS_OK) ctx->built = true;
-  return rc;
+  if (rc != SDMS_OK) return rc;
+  ctx->built = true;
+  return finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
 }
 
 int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok, int32_t* d_draft_len,
@@ -332,7 +338,6 @@ int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok,
   if (!ctx || !d_draft_tok || !d_draft_len) return SDMS_ERR_INVALID_ARG;
   if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   if (!ctx->dev.fused) {
     // large prompts: one probe / scan / dag (/ wide) round per suffix length, longest first; a path that has found
     // matches keeps them and its draft, the others try again with a shorter suffix
@@ -348,14 +353,17 @@ int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok,
         rc = timed(ctx, SDMS_KERNEL_DAG_WIDE, st, [&] {
           return launch_dag_wide(ctx->dev, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st); });
       if (rc != SDMS_OK) return rc;
+      rc = finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
+      if (rc != SDMS_OK) return rc;
     }
     ctx->built = true;
     return SDMS_OK;
   }
   const int rc = timed(ctx, SDMS_KERNEL_BUILD_FUSED, st, [&] {
     return launch_build_fused(ctx->dev, k_hi, 1, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, d_used_k, st); });
-  if (rc == SDMS_OK) ctx->built = true;
-  return rc;
+  if (rc != SDMS_OK) return rc;
+  ctx->built = true;
+  return finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
 }
 
 int sdms_accept(sdms_ctx* ctx, const int32_t* d_draft_tok, const int32_t* d_draft_len, const int32_t* d_sampled,
@@ -392,12 +400,12 @@ int sdms_step(sdms_ctx* ctx, int32_t k, const int32_t* d_sampled, const float* d
   }
   cudaStream_t st = (cudaStream_t)stream;
   ctx->built = false;
-  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
     return launch_step(ctx->dev, k, k, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
                        d_draft_score, d_draft_edge_w, nullptr, st); });
-  if (rc == SDMS_OK) ctx->built = true;
-  return rc;
+  if (rc != SDMS_OK) return rc;
+  ctx->built = true;
+  return finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
 }
 
 int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, const float* d_sampled_logprobs,
@@ -415,12 +423,12 @@ int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, con
   }
   cudaStream_t st = (cudaStream_t)stream;
   ctx->built = false;
-  if (reset_table_cursor(ctx, st) != SDMS_OK) return SDMS_ERR_CUDA;
   const int rc = timed(ctx, SDMS_KERNEL_STEP, st, [&] {
     return launch_step(ctx->dev, k_hi, 1, d_sampled, d_sampled_logprobs, d_accept_len, d_draft_tok, d_draft_len,
                        d_draft_score, d_draft_edge_w, d_used_k, st); });
-  if (rc == SDMS_OK) ctx->built = true;
-  return rc;
+  if (rc != SDMS_OK) return rc;
+  ctx->built = true;
+  return finish_best_paths(ctx, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st);
 }
 
 int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes) {

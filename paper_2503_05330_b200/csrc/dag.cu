@@ -31,7 +31,6 @@
 #include "sdms_internal.h"
 #include "append_dev.cuh"
 #include "wide_dev.cuh"
-#include "beam_dev.cuh"
 
 namespace sdms {
 
@@ -1204,26 +1203,14 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
       dag_best_path(s, sm, i, M, cap, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
       return;
     }
-    // too many matches for tables in shared memory: the same search over node tables in the workspace's table area
-    if (blockDim.x == kWideThreads && s.beam_stride > 0 && M <= kWideMaxMatches) {
-      __shared__ long long sh_first;
-      __shared__ float sh_value;
-      const int lcap = beam_lcap(M);
-      if (threadIdx.x == 0) {
-        const unsigned long long need = (unsigned long long)s.D << lcap;
-        const unsigned long long at = atomicAdd(s.b_ctl, need);
-        sh_first = at + need <= s.w_slots ? (long long)at : -1;
-      }
-      __syncthreads();
-      if (sh_first >= 0) {
-        beams_of_query(s, i, M, mlist, (unsigned)sh_first, lcap, 1, draft_tok + (size_t)i * s.D, draft_len + i, &sh_value, true,
-                       draft_score ? draft_score + (size_t)i * s.D : nullptr,
-                       draft_edge_w ? draft_edge_w + (size_t)i * s.D : nullptr);
-        return;
-      }
+    // too many matches for tables in shared memory: the path gets the greedy draft for now and is marked; the
+    // launch that follows a best-path build (beams.cu) searches the marked paths over node tables in the
+    // workspace's table area and replaces their drafts.  Without a table area the greedy draft stays, and says so.
+    if (s.beam_stride > 0) {
+      if (threadIdx.x == 0) s.bp_todo[i] = 1;
+    } else if (threadIdx.x == 0) {
+      atomicOr(s.status, SDMS_STATUS_SEARCH_FALLBACK);
     }
-    // no room there either: this path gets the greedy walk, and says so
-    if (threadIdx.x == 0) atomicOr(s.status, SDMS_STATUS_SEARCH_FALLBACK);
   }
   if (!EXPORT && s.pool == 2) list_pool(s, i, M, mlist, plen, poff, draft_tok, draft_len, draft_score, draft_edge_w);
   else if (M <= 32) dag_small<EXPORT>(s, sm, i, M, mlist, plen, poff, root, draft_tok, draft_len, draft_score, draft_edge_w);

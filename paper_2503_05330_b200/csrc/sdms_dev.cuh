@@ -80,8 +80,9 @@ struct Dev {
   int32_t* w_item;                     // [w_slots] per (layer, match): slot of the item's token in the layer's table
   unsigned long long w_slots;
   BeamEnt* b_ent;                      // [w_slots][beam_stride] continuations kept per node (sdms_get_beams)
-  unsigned long long* b_ctl;           // [1] slots handed out by the beam kernel
-  int32_t beam_stride;                 // the context's max_beams
+  unsigned long long* b_ctl;           // [2] slots handed out by the beam kernel / by the best-path launch after a build
+  int32_t beam_stride;                 // continuations kept per node: the context's max_beams, 1 for search mode 2 alone
+  int32_t* bp_todo;                    // [P] search mode 2: the path's best path is still to be searched over global tables
   int32_t w_grid;                      // CTAs of the wide pass (all resident at once)
   // DAG export of the last build
   int32_t* x_node_tok; int64_t* x_node_S; int32_t* x_node_cnt; int32_t* x_node_count;

@@ -47,6 +47,8 @@ cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len
                             float* draft_edge_w, cudaStream_t stream);
 cudaError_t launch_beams(const Dev& s, int B, int32_t* beam_tok, int32_t* beam_len, float* beam_value,
                          cudaStream_t stream);
+cudaError_t launch_best_path_fix(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
+                                 float* draft_edge_w, cudaStream_t stream);
 cudaError_t dag_kernel_setup();
 cudaError_t scan_kernel_setup();
 

@@ -1220,7 +1220,7 @@ __device__ __forceinline__ void dag_phase(const Dev& s, const Smem& sm, int i, i
 }
 
 template <bool EXPORT>
-__global__ void __launch_bounds__(kDagThreads, 1) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
+__global__ void __launch_bounds__(kDagThreads, EXPORT ? 1 : 2) dag_kernel(Dev s, int32_t* __restrict__ draft_tok,
                                                           int32_t* __restrict__ draft_len,
                                                           float* __restrict__ draft_score,
                                                           float* __restrict__ draft_edge_w, int round, int k,

@@ -328,6 +328,7 @@ class Runner:
             results = s.results.numpy()
             seen = 0
             stream = torch.cuda.current_stream()
+            stream_ptr = stream.cuda_stream
         S = plan["steps"]
         for timed in timed_step_plan(K, S):
             self.start_run(first_drafts=True)
@@ -343,7 +344,10 @@ class Runner:
                         t0 = time.perf_counter()
                         a.record()
                     np.copyto(step_in, h_in[step])  # host to host: the model's answer lands in the mapped buffer
-                    self.step(step, s.sampled_in, s.sampled_lp_in)
+                    if self.backoff:
+                        self.step(step, s.sampled_in, s.sampled_lp_in)
+                    else:
+                        s.step_own_buffers(k_next, stream_ptr)
                     if on:
                         b.record()
                     stream.synchronize()            # the caller reads the result before its next step

@@ -132,6 +132,9 @@ def _dp(t):
 
 
 def _sp(stream):
+    """cudaStream_t of a torch stream (None: the current one) or of a raw handle given as int."""
+    if isinstance(stream, int):
+        return C.c_void_p(stream)
     if stream is None:
         stream = torch.cuda.current_stream()
     return C.c_void_p(stream.cuda_stream)
@@ -295,6 +298,7 @@ class Sdms:
         self.step_in = torch.empty(2 * P * (D_ + 1), **io)
         self.sampled_in = self.step_in[:P * (D_ + 1)].view(P, D_ + 1)
         self.sampled_lp_in = self.step_in[P * (D_ + 1):].view(torch.float32).view(P, D_ + 1)
+        self._own = None
 
     def close(self):
         if getattr(self, "ctx", None):
@@ -336,6 +340,14 @@ class Sdms:
         sdms_step(self.ctx, k, sampled, sampled_logprobs, self.accept_len, self.draft_tok, self.draft_len,
                   self.draft_score, self.draft_edge_w, stream)
         return self.accept_len, self.draft_tok, self.draft_len
+
+    def step_own_buffers(self, k, stream=None):
+        """`step` on the context's own input buffers (`sampled_in`, `sampled_lp_in`), with the pointers marshalled
+        once: for decode loops that count microseconds on the host."""
+        if self._own is None:
+            self._own = tuple(_dp(t) for t in (self.sampled_in, self.sampled_lp_in, self.accept_len, self.draft_tok,
+                                               self.draft_len, self.draft_score, self.draft_edge_w))
+        _check(lib().sdms_step(self.ctx, k, *self._own, _sp(stream)), "sdms_step")
 
     def step_backoff(self, k_hi, sampled, sampled_logprobs, stream=None):
         sdms_step_backoff(self.ctx, k_hi, sampled, sampled_logprobs, self.accept_len, self.draft_tok, self.draft_len,

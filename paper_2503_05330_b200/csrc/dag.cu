@@ -1358,7 +1358,9 @@ __device__ void shared_scan(const Dev& s, int g, int k, int nq, const int32_t (*
   }
 }
 
-template <bool EXPORT>
+// SHARE: the code of the cluster-shared scan is compiled in (kernels for prompts below kShareMinTokens leave it
+// out: after a cold start the step fetches every instruction it may run past)
+template <bool EXPORT, bool SHARE>
 __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                             float* draft_score, float* draft_edge_w, int32_t* used_k,
                             const int32_t* own_rec = nullptr, int csize = 0) {
@@ -1377,7 +1379,7 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
 
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
   // the cluster shares its scans (same decision in every CTA of the launch)
-  const bool share = csize > 1 && k_lo == k_hi && s.eps == 0 && (s.L & 3) == 0 && slice >= kShareMinTokens;
+  const bool share = SHARE && csize > 1 && k_lo == k_hi && s.eps == 0 && (s.L & 3) == 0 && slice >= kShareMinTokens;
   // With k_lo < k_hi the suffix length backs off: the longest k in [k_lo, k_hi] that has a match wins.
   int k = k_hi;
   for (;; --k) {
@@ -1581,7 +1583,7 @@ __device__ void build_phase(const Dev& s, const Smem& sm, int k_hi, int k_lo, in
                     draft_len, draft_score, draft_edge_w);
 }
 
-template <bool EXPORT>
+template <bool EXPORT, bool SHARE>
 __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, int k_hi, int k_lo, int32_t* draft_tok,
                                                                   int32_t* draft_len, float* draft_score,
                                                                   float* draft_edge_w, int32_t* used_k, int csize) {
@@ -1589,7 +1591,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
   grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
-  build_phase<EXPORT>(s, sm, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, nullptr, csize);
+  build_phase<EXPORT, SHARE>(s, sm, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, nullptr, csize);
 }
 
 // One launch per decode step.  The CTAs of a prompt form a thread-block cluster.  Each CTA first
@@ -1598,6 +1600,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) build_fused_kernel(Dev s, in
 // path of the prompt is up to date and each CTA builds its path's next draft.  draft_tok / draft_len
 // hold the previous drafts on entry and the new ones on exit.
 // k_lo < k: the suffix length backs off from k to k_lo (used_k, if given, receives each path's choice).
+template <bool SHARE>
 __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, int k_lo, const int32_t* sampled,
                                                            const float* sampled_lp, int32_t* accept_len,
                                                            int32_t* draft_tok, int32_t* draft_len,
@@ -1611,7 +1614,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) step_kernel(Dev s, int k, in
   accept_commit_phase(s, blockIdx.x, draft_tok, draft_len, sampled, sampled_lp, accept_len, sh_own_rec, k);
   // every thread of every CTA of the cluster gets here exactly once (no early exit above)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  build_phase<false>(s, sm, k, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, sh_own_rec, s.N);
+  build_phase<false, SHARE>(s, sm, k, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, sh_own_rec, s.N);
 }
 
 }  // namespace
@@ -1623,11 +1626,17 @@ cudaError_t dag_kernel_setup() {
     e = cudaFuncSetAttribute(dag_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)dag_smem_bytes<true>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(build_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(build_fused_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)dag_smem_bytes<false>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(build_fused_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dag_smem_bytes<false>());
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(step_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
@@ -1651,7 +1660,7 @@ bool step_kernel_fits(const Dev& s) {
   step_launch_config(s, 0, &cfg, attr);
   cfg.numAttrs = 1;                                   // occupancy only looks at the cluster shape
   int clusters = 0;
-  if (cudaOccupancyMaxActiveClusters(&clusters, step_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (cudaOccupancyMaxActiveClusters(&clusters, step_kernel<true>, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
   // every prompt's cluster resident at once: large clusters leave SMs of a GPC idle, and a launch whose
   // clusters queue up for the device is slower than the separate accept and build launches
   return (long long)clusters * s.N >= s.P;
@@ -1662,8 +1671,9 @@ cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, c
                         float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
   cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
   step_launch_config(s, stream, &cfg, attr);
-  return cudaLaunchKernelEx(&cfg, step_kernel, s, k, k_lo, sampled, sampled_lp, accept_len, draft_tok, draft_len,
-                            draft_score, draft_edge_w, used_k);
+  const bool share = (s.L & 3) == 0 && (long long)s.N * s.L >= kShareMinTokens;       // the prompt is worth sharing its scan
+  return cudaLaunchKernelEx(&cfg, share ? step_kernel<true> : step_kernel<false>, s, k, k_lo, sampled, sampled_lp, accept_len,
+                            draft_tok, draft_len, draft_score, draft_edge_w, used_k);
 }
 
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
@@ -1691,7 +1701,7 @@ int build_cluster_size(const Dev& s) {
     attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, build_fused_kernel<false>, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
+    if (cudaOccupancyMaxActiveClusters(&clusters, build_fused_kernel<false, true>, &cfg) != cudaSuccess) { cudaGetLastError(); continue; }
     if ((long long)clusters * c >= s.P) return c;
   }
   return 1;
@@ -1700,7 +1710,7 @@ int build_cluster_size(const Dev& s) {
 cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_tok, int32_t* draft_len,
                                float* draft_score, float* draft_edge_w, int32_t* used_k, cudaStream_t stream) {
   if (s.build_cluster <= 1 || k_lo != k_hi)
-    return launch_overlapped(build_fused_kernel<false>, dim3(s.P), dim3(kFusedThreads), dag_smem_bytes<false>(), stream,
+    return launch_overlapped(build_fused_kernel<false, false>, dim3(s.P), dim3(kFusedThreads), dag_smem_bytes<false>(), stream,
                              s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w, used_k, 0);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.P); cfg.blockDim = dim3(kFusedThreads);
@@ -1711,7 +1721,7 @@ cudaError_t launch_build_fused(const Dev& s, int k_hi, int k_lo, int32_t* draft_
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, build_fused_kernel<false>, s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w,
+  return cudaLaunchKernelEx(&cfg, build_fused_kernel<false, true>, s, k_hi, k_lo, draft_tok, draft_len, draft_score, draft_edge_w,
                             used_k, (int)s.build_cluster);
 }
 

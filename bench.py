@@ -29,8 +29,8 @@ UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel from its last ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); only quoted while the kernel sources are the ones profiled
-NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76544,
-               "sources_sha256": "e12a72d89f9b3dc814c0a39a784b393dfa7702be8b3587dc9255d39edc42cd0d"}
+NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 75968,
+               "sources_sha256": "bbab5f23f0fc00ce74c0caacda7f00fb8806953bbb54dda165b640f12f48617b"}
 
 
 def kernel_sources_sha():

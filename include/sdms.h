@@ -303,6 +303,12 @@ int sdms_debug_read_history(sdms_ctx* ctx, int32_t* d_tok, int32_t* d_pq, int32_
  * 0 = no query or no index entry, 1 = from the index bucket, 2 = by scanning. */
 int sdms_debug_read_query_modes(sdms_ctx* ctx, int32_t* d_modes, void* stream);
 
+/* Every wait inside a kernel (grid barrier of the wide pass, copy barriers of the streaming scan) is bounded:
+ * when it runs out, the kernel raises SDMS_STATUS_TIMEOUT and returns, and the context stays usable.  This call
+ * shows what that looks like without anything going wrong: one thread waits, with the same bounded wait, about
+ * half a millisecond for a count that nobody raises, sets the status bit and returns. */
+int sdms_debug_wait_timeout(sdms_ctx* ctx, void* stream);
+
 /* Waits for `stream`, returns the status bits in *host_flags and clears them. */
 int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream);
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff", "sdms_get_beams",
+    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff", "sdms_get_beams", "sdms_debug_wait_timeout",
 )
 
 
@@ -84,6 +84,7 @@ def lib():
         l.sdms_debug_read_history.argtypes = [vp] * 5
         l.sdms_debug_read_query_modes.argtypes = [vp, vp, vp]
         l.sdms_get_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        l.sdms_debug_wait_timeout.argtypes = [vp, vp]
         l.sdms_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         l.sdms_profile_enable.argtypes = [vp, i32]
         l.sdms_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_uint64)]
@@ -233,6 +234,10 @@ def sdms_get_status(ctx, stream=None) -> int:
     f = C.c_uint32(0)
     _check(lib().sdms_get_status(ctx, C.byref(f), _sp(stream)), "sdms_get_status")
     return f.value
+
+
+def sdms_debug_wait_timeout(ctx, stream=None):
+    _check(lib().sdms_debug_wait_timeout(ctx, _sp(stream)), "sdms_debug_wait_timeout")
 
 
 def sdms_launch_count(ctx) -> int:

@@ -506,6 +506,12 @@ int sdms_debug_read_query_modes(sdms_ctx* ctx, int32_t* d_modes, void* stream) {
                          (cudaStream_t)stream) == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
 }
 
+int sdms_debug_wait_timeout(sdms_ctx* ctx, void* stream) {
+  if (!ctx) return SDMS_ERR_INVALID_ARG;
+  ++ctx->launches;
+  return launch_wait_timeout(ctx->dev, 1000000LL, (cudaStream_t)stream) == cudaSuccess ? SDMS_OK : SDMS_ERR_CUDA;
+}
+
 int sdms_get_status(sdms_ctx* ctx, uint32_t* host_flags, void* stream) {
   if (!ctx || !host_flags) return SDMS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;

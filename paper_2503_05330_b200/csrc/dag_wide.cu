@@ -36,7 +36,7 @@ namespace sdms {
 
 namespace {
 
-constexpr long long kBarrierCycles = 2000000000LL;   // about a second: a barrier that takes that long has failed
+constexpr long long kBarrierCycles = 200000000LL;    // about a tenth of a second (the pass takes 0.1-0.3 ms): a barrier that takes that long has failed
 constexpr u64 kSumMask = (1ull << kWideSumShift) - 1;
 
 __device__ __forceinline__ u64 ld_u64(const u64* p) { return __ldcg(p); }
@@ -45,6 +45,15 @@ __device__ __forceinline__ uint32_t ld_u32(const uint32_t* p) { return __ldcg(p)
 // All CTAs of the grid arrive; returns false (in every thread of the CTA) if the others did not show
 // up in time.  Arrivals are spread over kWideBarrierWays counters in lines of their own (hundreds of
 // atomics on one address take microseconds); one thread per counter waits for it.
+__device__ __forceinline__ bool wait_for_count(const u64* ctr, u64 target, long long cycles) {
+  const long long t0 = clock64();
+  while (ld_u64(ctr) < target) {
+    if (clock64() - t0 > cycles) return false;
+    __nanosleep(32);
+  }
+  return true;
+}
+
 __device__ bool grid_barrier(const Dev& s, unsigned phase) {
   __syncthreads();
   int ok = 1;
@@ -53,14 +62,15 @@ __device__ bool grid_barrier(const Dev& s, unsigned phase) {
     u64* ctr = s.w_ctl + kWideBarrierAt + t * kWideBarrierStride;
     if (t == (int)(blockIdx.x & (kWideBarrierWays - 1))) { __threadfence(); atomicAdd(ctr, 1ull); }
     const u64 target = (u64)((gridDim.x + kWideBarrierWays - 1 - t) / kWideBarrierWays) * phase;
-    const long long t0 = clock64();
-    while (ld_u64(ctr) < target) {
-      if (clock64() - t0 > kBarrierCycles) { ok = 0; break; }
-      __nanosleep(32);
-    }
+    ok = wait_for_count(ctr, target, kBarrierCycles);
     __threadfence();
   }
   return __syncthreads_and(ok) != 0;
+}
+
+// sdms_debug_wait_timeout: the bounded wait of the grid barrier on a count that nobody raises.
+__global__ void wait_timeout_kernel(Dev s, long long cycles) {
+  if (threadIdx.x == 0 && !wait_for_count(s.b_ctl + 1, ~0ull, cycles)) atomicOr(s.status, SDMS_STATUS_TIMEOUT);
 }
 
 __device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
@@ -247,6 +257,11 @@ int wide_kernel_grid() {
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dag_wide_kernel, kWideThreads, 0) != cudaSuccess) { cudaGetLastError(); return 0; }
   return sms * (per_sm < 1 ? per_sm : 1);
+}
+
+cudaError_t launch_wait_timeout(const Dev& s, long long cycles, cudaStream_t stream) {
+  wait_timeout_kernel<<<1, 32, 0, stream>>>(s, cycles);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,

@@ -194,7 +194,7 @@ constexpr int kStreamStages = 4;
 constexpr int kStreamTile = 2 * kScanTile;           // tokens per stage: a thread takes eight of them
 constexpr int kStreamThreads = kScanThreads + 32;   // eight scanning warps and one warp that issues the copies
 constexpr int kStreamSmemMax = 96 * 1024;             // dynamic shared memory the streaming form may ask for
-constexpr long long kWaitCycles = 4000000000LL;      // about two seconds: a wait that long has failed
+constexpr long long kWaitCycles = 400000000LL;       // about a fifth of a second (the kernel takes 20-140 us): a wait that long has failed
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -416,7 +416,7 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
     if (STREAM) {
       if (!__all_sync(FULL_MASK, mbar_wait(&sh_full[stage], phase))) {  // cannot happen; the warp leaves in an orderly way
         atomicOr(s.status, SDMS_STATUS_TIMEOUT);
-        for (int it = 0; it < 100000; ++it) __nanosleep(1000);         // copies still in flight land in live shared memory
+        for (int it = 0; it < 10000; ++it) __nanosleep(1000);         // copies still in flight land in live shared memory
         break;
       }
       const int4* const st4 = reinterpret_cast<const int4*>(sh_stage + stage * TILE);

@@ -43,6 +43,7 @@ cudaError_t launch_step(const Dev& s, int k, int k_lo, const int32_t* sampled, c
 cudaError_t launch_compact_matches(const Dev& s, int32_t* offsets, int32_t* gpos, size_t cap, cudaStream_t stream);
 // queries with many matches, aggregated by all SMs (dag_wide.cu)
 int wide_kernel_grid();
+cudaError_t launch_wait_timeout(const Dev& s, long long cycles, cudaStream_t stream);
 cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                             float* draft_edge_w, cudaStream_t stream);
 cudaError_t launch_beams(const Dev& s, int B, int32_t* beam_tok, int32_t* beam_len, float* beam_value,

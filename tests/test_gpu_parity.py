@@ -1014,3 +1014,16 @@ def test_backoff_by_rounds_config5():
         assert gl[i] == len(d) and np.array_equal(gt[i, :len(d)], d), i
         assert np.array_equal(np.sort(gpos[off[i]:off[i + 1]]), pair.o.matches(i)), i
     assert len(set(used_g.tolist())) >= 3
+
+
+def test_a_wait_that_runs_out_sets_the_status_bit_and_leaves_the_context_usable():
+    # the bounded wait of the kernels, on a count that nobody raises (about half a millisecond)
+    from paper_2503_05330_b200 import binding
+    G, N, L, V, D = 1, 4, 48, 3, 4
+    tokens, lps = synth.small_random(G * N, L, V, 77)
+    pair = Pair(G, N, L, V, 2, D)
+    pair.append(tokens[:, :30], lps[:, :30], np.full(N, 30, np.int32), expect_status=0)
+    binding.sdms_debug_wait_timeout(pair.g.ctx)
+    assert pair.g.status() == binding.STATUS_TIMEOUT
+    assert pair.g.status() == 0                      # read and cleared
+    pair.build_and_compare(1, check_dag=False)       # nothing else has changed

@@ -420,7 +420,14 @@ def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=
         modes = s.query_modes()
         glen = lens.reshape(wl.G, wl.N).sum(1).repeat(wl.N)
         fused = wl.N * wl.L <= 131072
-        scan_bytes = int(4 * (glen - lens)[modes == 2].sum()) if fused else (4 * int(lens.sum()) if (modes == 2).any() else 0)
+        csize = binding.sdms_build_cluster_size(s.ctx)
+        if fused and csize > 1:          # a cluster of csize paths reads its prompt once for all its scan queries
+            scanning = (modes == 2).reshape(-1, csize).any(1)
+            scan_bytes = int(4 * glen.reshape(-1, csize)[:, 0][scanning].sum())
+        elif fused:                      # every scanning query reads the other paths of its prompt
+            scan_bytes = int(4 * (glen - lens)[modes == 2].sum())
+        else:                            # one shared pass over the store
+            scan_bytes = 4 * int(lens.sum()) if (modes == 2).any() else 0
         nbytes = scan_bytes + int((modes > 0).sum()) * (32 + 4 * k) + int(m.sum()) * (4 + 8 * wl.D) + wl.P * (12 * wl.D + 4)
         shared_scan = 4 * int(lens.reshape(wl.G, wl.N)[(modes == 2).reshape(wl.G, wl.N).any(1)].sum())   # scan model: once per prompt
         out[str(k)] = {"us": us, "p10_us": float(np.percentile(t_us, 10)), "p90_us": float(np.percentile(t_us, 90)),
@@ -444,7 +451,7 @@ def steady_state(wl, device, iters=20, peak=None, max_matches=0, ks=None, beams=
     assert s.status() == 0
     return {"groups": wl.G, "paths_per_group": wl.N, "capacity": wl.L, "max_draft_len": wl.D, "fill": 0.97,
             "max_matches_per_path": max_matches, "index_max_n": index_max_n or wl.k_max,
-            "launches_per_build": 1 if fused else 4, "workspace_bytes": s.workspace_bytes, "build_by_k": out}
+            "launches_per_build": 1 if fused else 4, "build_cluster_size": binding.sdms_build_cluster_size(s.ctx), "workspace_bytes": s.workspace_bytes, "build_by_k": out}
 
 
 def scan_at_scale(device, G=64, N=256, L=8192, V=151936):

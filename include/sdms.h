@@ -226,6 +226,9 @@ int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, con
                       int32_t* d_accept_len, int32_t* d_draft_tok, int32_t* d_draft_len, float* d_draft_score,
                       float* d_draft_edge_w, int32_t* d_used_k, void* stream);
 int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes);
+/* Thread blocks (= consecutive paths of one prompt) that share the scan of their prompt in the single-launch
+ * build: 1 = every query scans for itself (also on contexts that do not take that build). */
+int sdms_build_cluster_size(sdms_ctx* ctx, int32_t* paths);
 
 /*
  * Sliding window for runs longer than the capacity (the paper's runs end long

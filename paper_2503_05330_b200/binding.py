@@ -30,7 +30,7 @@ EXPORTS = (
     "sdms_build_drafts", "sdms_build_drafts_backoff", "sdms_accept", "sdms_get_matches", "sdms_get_dag",
     "sdms_debug_read_history", "sdms_debug_read_query_modes", "sdms_get_status", "sdms_launch_count", "sdms_profile_enable",
     "sdms_profile_read", "sdms_strerror", "sdms_kernel_name", "sdms_match_noalloc", "sdms_step",
-    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff", "sdms_get_beams", "sdms_debug_wait_timeout",
+    "sdms_step_is_single_launch", "sdms_trim", "sdms_host_pointer", "sdms_step_backoff", "sdms_get_beams", "sdms_debug_wait_timeout", "sdms_build_cluster_size",
 )
 
 
@@ -78,6 +78,7 @@ def lib():
         l.sdms_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         l.sdms_step_backoff.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         l.sdms_step_is_single_launch.argtypes = [vp, C.POINTER(C.c_int32)]
+        l.sdms_build_cluster_size.argtypes = [vp, C.POINTER(C.c_int32)]
         l.sdms_get_matches.argtypes = [vp, vp, vp, C.c_size_t, vp]
         l.sdms_get_dag.argtypes = [vp] * 10
         l.sdms_get_beams.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -206,6 +207,12 @@ def sdms_step_is_single_launch(ctx) -> bool:
     yes = C.c_int32(0)
     _check(lib().sdms_step_is_single_launch(ctx, C.byref(yes)), "sdms_step_is_single_launch")
     return bool(yes.value)
+
+
+def sdms_build_cluster_size(ctx) -> int:
+    n = C.c_int32(0)
+    _check(lib().sdms_build_cluster_size(ctx, C.byref(n)), "sdms_build_cluster_size")
+    return n.value
 
 
 def sdms_get_matches(ctx, offsets, gpos, stream=None):

@@ -437,6 +437,12 @@ int sdms_step_is_single_launch(sdms_ctx* ctx, int32_t* yes) {
   return SDMS_OK;
 }
 
+int sdms_build_cluster_size(sdms_ctx* ctx, int32_t* paths) {
+  if (!ctx || !paths) return SDMS_ERR_INVALID_ARG;
+  *paths = ctx->dev.build_cluster > 1 ? ctx->dev.build_cluster : 1;
+  return SDMS_OK;
+}
+
 int sdms_host_pointer(const void* host_ptr, void** device_ptr) {
   if (!host_ptr || !device_ptr) return SDMS_ERR_INVALID_ARG;
   cudaPointerAttributes a{};

@@ -4,8 +4,9 @@
 // One CTA aggregates a query of a few dozen matches in its own shared memory (dag.cu).  A query with
 // hundreds or tens of thousands of matches keeps one SM busy for as long while the others idle, so
 // dag_kernel hands such queries over (wide_register) and this pass works through all of them at
-// once: every (match, layer) pair is one item, 128 matches are one unit of work, and the units of all
-// queries are dealt out to a grid that covers the device.  Each query owns, for every layer, a node
+// once: every (match, layer) pair is one item, 128 matches are one unit of work (split by layers into
+// two or four units when that still leaves CTAs without one), and the units of all queries are dealt
+// out to a grid that covers the device.  Each query owns, for every layer, a node
 // table in global memory (open addressing, one 32-byte slot per node and the keys apart, eight to a
 // sector; all of it zero when the pass begins and again when it ends).  Sums are integers and every choice has a tie rule, so the atomics'
 // order cannot show in a result.
@@ -80,6 +81,7 @@ __device__ __forceinline__ double weight_of(const Dev& s, u64 sum) {
 __global__ void __launch_bounds__(kWideThreads, 1)
 dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ draft_len,
                 float* __restrict__ draft_score, float* __restrict__ draft_edge_w) {
+  grid_wait();                                       // scheduled while dag_kernel drains; its list is complete from here on
   const u64 registered = ld_u64(&s.w_ctl[0]);
   if (registered == 0) return;                       // the same for every CTA: nobody waits for anybody
   const int nq = (int)(registered < (u64)kMaxWide ? registered : (u64)kMaxWide);
@@ -120,7 +122,14 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     if (tid == kWideThreads - 1) sh_cbase[nq] = before + c[0] + c[1];
     __syncthreads();
   }
-  const int units = sh_cbase[nq];
+  const int chunks = sh_cbase[nq];
+  // With fewer chunks than CTAs a chunk is split by layers as well: a thread's rounds (its layers d_first + 4 r) go to
+  // `split` units that run on different SMs.
+  const int rounds_all = (D + kLayerWays - 1) / kLayerWays;
+  int split = 1;
+  while (split * 2 <= rounds_all && chunks * split * 2 <= (int)gridDim.x) split *= 2;   // never two units for a CTA because of it: each unit walks the draft again
+  const int rounds_per = (rounds_all + split - 1) / split;
+  const int units = chunks * split;
 
   // unit c belongs to the last query whose first unit is not after c
   auto query_of = [&](int c) {
@@ -130,28 +139,30 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
   };
 
   // ---- pass A: node sums -------------------------------------------------------------------------
-  for (int c = blockIdx.x; c < units; c += gridDim.x) {
+  for (int u = blockIdx.x; u < units; u += gridDim.x) {
+    const int c = u / split, r_lo = (u - c * split) * rounds_per;
     const int q = query_of(c);
     const int4 de = sh_desc[q];
     const int i = de.x, M = de.y, lcap = de.z;
     const unsigned base = (unsigned)de.w;
-    const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
-    (void)nm;
-    wide_insert_unit(s, s.matches + s.q_off[i], base, lcap, M, m0);
+    const int m0 = (c - sh_cbase[q]) * kWideChunk;
+    wide_insert_unit(s, s.matches + s.q_off[i], base, lcap, M, m0, r_lo, r_lo + rounds_per);
   }
   if (!grid_barrier(s, 1)) { if (tid == 0) atomicOr(s.status, SDMS_STATUS_TIMEOUT); return; }
 
   // ---- passes B and C: the best successor of every node ------------------------------------------
   for (int pass = 0; pass < 2; ++pass) {
-    for (int c = blockIdx.x; c < units; c += gridDim.x) {
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+      const int c = u / split, r_lo = (u - c * split) * rounds_per;
       const int q = query_of(c);
       const int4 de = sh_desc[q];
       const int M = de.y, lcap = de.z;
       const unsigned base = (unsigned)de.w;
       const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
       const int* const item = s.w_item + base + m0 + ml;
+      const int d_end = min(D, d_first + (r_lo + rounds_per - 1) * kLayerWays);
 #pragma unroll 1
-      for (int d = d_first; d <= D; d += kLayerWays) {
+      for (int d = d_first + r_lo * kLayerWays; d <= d_end; d += kLayerWays) {
         int sv = -1, su = -1;
         if (ml < nm) {
           sv = item[(size_t)(d - 1) * M];
@@ -184,14 +195,15 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
   }
 
   // ---- pass D: walk, then the sums of the edges taken ---------------------------------------------
-  for (int c = blockIdx.x; c < units; c += gridDim.x) {
+  for (int u = blockIdx.x; u < units; u += gridDim.x) {
+    const int c = u / split, r_lo = (u - c * split) * rounds_per;
     const int q = query_of(c);
     const int4 de = sh_desc[q];
     const int i = de.x, M = de.y, lcap = de.z;
     const unsigned base = (unsigned)de.w;
     const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
     if (tid == 0) {
-      const bool writer = m0 == 0;                    // the query's first unit writes the draft out
+      const bool writer = m0 == 0 && r_lo == 0;       // the query's first unit writes the draft out
       const WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT;
       u64 next = ld_u64(&pr[0].succ);
       int emitted = 0;
@@ -215,8 +227,9 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     const int emitted = sh_emitted;
     const int* const item = s.w_item + base + m0 + ml;
     const int gpos = ml < nm ? s.matches[(size_t)s.q_off[i] + m0 + ml] : 0;
+    const int d_end = min(emitted, d_first + (r_lo + rounds_per - 1) * kLayerWays);
 #pragma unroll 1
-    for (int d = d_first; d <= emitted; d += kLayerWays) {
+    for (int d = d_first + r_lo * kLayerWays; d <= d_end; d += kLayerWays) {
       bool on = false;
       if (ml < nm) on = item[(size_t)(d - 1) * M] == sh_dslot[d - 1] && (d == 1 || item[(size_t)(d - 2) * M] == sh_dslot[d - 2]);
       const unsigned group = __ballot_sync(FULL, on);
@@ -268,10 +281,24 @@ cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len
                             float* draft_edge_w, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.w_grid); cfg.blockDim = dim3(kWideThreads); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeCooperative;
   attr[0].val.cooperative = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  // Scheduled early as well (its CTAs take their SMs while the kernel before drains: that kernel's CTAs have all
+  // started by then and wait for nobody) where the runtime takes both attributes together, else cooperative only.
+  static bool early = true;
+  if (early) {
+    cfg.numAttrs = 2;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, dag_wide_kernel, s, draft_tok, draft_len, draft_score, draft_edge_w);
+    if (e == cudaSuccess) return e;
+    if (e != cudaErrorInvalidValue && e != cudaErrorNotSupported) return e;
+    cudaGetLastError();
+    early = false;
+  }
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, dag_wide_kernel, s, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 

@@ -77,7 +77,10 @@ __device__ __forceinline__ u64 group_sum(unsigned group, unsigned shared, unsign
 // CTA.  The lanes of a warp hold 32 matches at the same layer; lanes whose followers are the same token
 // form a group and the group's leader claims the node's slot and sends one add for all of them.
 // Every item's slot (-1: the candidate has ended) is noted in w_item[base + (d - 1) * M + m].
-__device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* list, unsigned base, int lcap, int M, int m0) {
+// A thread's layers are d_first + 4 r; with r_lo / r_hi the call takes only the rounds r_lo <= r < r_hi of them (a unit
+// split by layers: more, shorter units when there are fewer units than CTAs).
+__device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* list, unsigned base, int lcap, int M, int m0,
+                                                 int r_lo = 0, int r_hi = SDMS_MAX_DRAFT) {
   const int tid = threadIdx.x, lane = tid & 31;
   const int D = s.D;
   const int ml = tid & (kWideChunk - 1), d_first = tid / kWideChunk + 1;   // d_first is the same in all lanes of a warp
@@ -90,14 +93,16 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
       const int j = path_of(s, gpos);
       n_m = min(D, __ldg(s.len + j) - 1 - (gpos - j * s.L));
     }
-  for (int d_base = d_first; d_base <= D; d_base += kMaxRounds * kLayerWays) {     // the same trip count for the whole warp
+  for (int r0 = r_lo; r0 < r_hi && d_first + r0 * kLayerWays <= D; r0 += kMaxRounds) {     // the same trip count for the whole warp
+    const int d_base = d_first + r0 * kLayerWays;
+    const int d_end = min(D, d_first + (r_hi - 1) * kLayerWays);    // the last layer of this thread that belongs to the unit
     int v[kMaxRounds];
     unsigned p[kMaxRounds];
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {            // every follower this thread needs is asked for before the first is used
       const int d = d_base + r * kLayerWays;
       v[r] = -1; p[r] = 0u;
-      if (d <= n_m) { v[r] = __ldg(s.tok + gpos + d); p[r] = (unsigned)__ldg(s.pq + gpos + d); }
+      if (d <= n_m && d <= d_end) { v[r] = __ldg(s.tok + gpos + d); p[r] = (unsigned)__ldg(s.pq + gpos + d); }
     }
     // the key sector and the slot every follower hashes to are asked for now: when the rounds below get to
     // them (one after the other, the lanes of a warp in step) they are on their way from memory
@@ -119,25 +124,29 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
     for (int r = 0; r < kMaxRounds; ++r) {
       const int d = d_base + r * kLayerWays;
       leader[r] = 0; sv[r] = -1; add[r] = 0ull;
-      if (d > D) continue;                              // the same for the whole warp
+      if (d > d_end) continue;                          // the same for the whole warp
       const unsigned group = __match_any_sync(FULL, v[r]);          // lanes whose items are the same node
       leader[r] = __ffs(group) - 1;
       const unsigned shared = __ballot_sync(FULL, v[r] >= 0 && (group & (group - 1)) != 0u);
       add[r] = ((u64)__popc(group) << kWideSumShift) | group_sum(group, shared, p[r]);
     }
-    // linear probing, eight keys (one sector) per round trip: the longest probe run of a half-full table
-    // of a thousand nodes is some forty slots
+    // Open addressing by sectors of eight keys (one round trip each).  A token's home sector is given by its hash; it
+    // may sit in any of the sector's eight slots, and only a sector without a free slot sends it on to the next one.
+    // Within a sector every claimer of a token tries the free slots in the same order (from the hash's low bits on,
+    // wrapping), so two claimers of one token end up at one slot: the slots before it in that order were taken by
+    // other tokens when the first of them passed, and slots are never given back during a pass.
     unsigned h[kMaxRounds];
     unsigned todo = 0;                                  // layers whose slot this thread still has to find
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
       const int d = d_base + r * kLayerWays;
       h[r] = ((unsigned)v[r] * 2654435761u) >> (32 - lcap);
-      if (d <= D && v[r] >= 0 && lane == leader[r]) todo |= 1u << r;
+      if (d <= d_end && v[r] >= 0 && lane == leader[r]) todo |= 1u << r;
     }
     uint4 ka[kMaxRounds], kb[kMaxRounds];                // the sector of keys each sequence is looking at
     unsigned fresh = 0;                                 // layers whose sector is in ka / kb
-    for (unsigned step = 0; step <= 2u * mask + 16u && todo; ++step) {   // every step moves each sequence on by at least one slot
+    unsigned taken = 0;                                 // eight bits per layer: slots of that sector a failed claim has shown to be somebody else's
+    for (unsigned step = 0; step <= 2u * mask + 16u && todo; ++step) {   // every step finds the slot, rules one out or leaves a full sector
 #pragma unroll
       for (int r = 0; r < kMaxRounds; ++r) {
         if (!(todo >> r & 1u) || (fresh >> r & 1u)) continue;
@@ -146,7 +155,7 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
         kb[r] = __ldcg(reinterpret_cast<const uint4*>(keys + 4));
       }
       fresh |= todo;
-      int at[kMaxRounds];                               // first slot of the sector, from h on, that is free or holds the token
+      int at[kMaxRounds];                               // the slot that holds the token, else the first free one in the token's order
       uint32_t seen[kMaxRounds];
 #pragma unroll
       for (int r = 0; r < kMaxRounds; ++r) {
@@ -154,36 +163,52 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
         if (!(todo >> r & 1u)) continue;
         const uint32_t want = (uint32_t)v[r] + 1u;
         const uint32_t kk[8] = {ka[r].x, ka[r].y, ka[r].z, ka[r].w, kb[r].x, kb[r].y, kb[r].z, kb[r].w};
+        unsigned hit = 0u, open = 0u;
 #pragma unroll
-        for (int x = 7; x >= 0; --x)
-          if ((unsigned)x >= (h[r] & 7u) && (kk[x] == 0u || kk[x] == want)) { at[r] = x; seen[r] = kk[x]; }
+        for (int x = 0; x < 8; ++x) { hit |= (unsigned)(kk[x] == want) << x; open |= (unsigned)(kk[x] == 0u) << x; }
+        open &= ~(taken >> (8 * r));
+        const unsigned start = h[r] & 7u;
+        if (hit) { at[r] = __ffs(hit) - 1; seen[r] = want; }
+        else if (open) { at[r] = (int)((start + __ffs(((open | (open << 8)) >> start) & 0xffu) - 1) & 7u); }
       }
+      unsigned claims = 0;
 #pragma unroll
-      for (int r = 0; r < kMaxRounds; ++r) {             // the claims of all layers go out together
+      for (int r = 0; r < kMaxRounds; ++r) {             // the claims of all layers go out together ...
         if (!(todo >> r & 1u) || at[r] < 0 || seen[r] != 0u) continue;
         uint32_t* keys = s.w_key + base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u);
         seen[r] = atomicCAS(&keys[at[r]], 0u, (uint32_t)v[r] + 1u);
-        if (seen[r] == 0u) {
-          seen[r] = (uint32_t)v[r] + 1u;
-          s.w_tab[base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u) + at[r]].tok1 = seen[r];
-        }
+        claims |= 1u << r;
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {             // ... and with them a new look at their sectors: should a claim fail (the
+        if (!(claims >> r & 1u)) continue;               // sector was read before its other claimers arrived), the next one knows better
+        const uint32_t* keys = s.w_key + base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u);
+        ka[r] = __ldcg(reinterpret_cast<const uint4*>(keys));
+        kb[r] = __ldcg(reinterpret_cast<const uint4*>(keys + 4));
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {
+        if (!(claims >> r & 1u) || seen[r] != 0u) continue;
+        seen[r] = (uint32_t)v[r] + 1u;
+        s.w_tab[base + ((size_t)(d_base + r * kLayerWays - 1) << lcap) + (h[r] & ~7u) + at[r]].tok1 = seen[r];
       }
 #pragma unroll
       for (int r = 0; r < kMaxRounds; ++r) {
         if (!(todo >> r & 1u)) continue;
-        if (at[r] < 0) { h[r] = ((h[r] & ~7u) + 8u) & mask; fresh &= ~(1u << r); continue; }   // nothing in this sector: on to the next
+        if (at[r] < 0) {                                  // no room in this sector: on to the next, same order within it
+          h[r] = (((h[r] & ~7u) + 8u) & mask) | (h[r] & 7u);
+          fresh &= ~(1u << r); taken &= ~(0xffu << (8 * r));
+          continue;
+        }
         if (seen[r] == (uint32_t)v[r] + 1u) { sv[r] = (int)((h[r] & ~7u) + at[r]); todo &= ~(1u << r); continue; }
-        // somebody else's token got there first: go on behind it, in the same sector as long as it lasts (a key that
-        // was free when the sector was read may be taken by now: the claim will tell)
-        h[r] = (h[r] & ~7u) + at[r] + 1u;
-        if ((h[r] & 7u) == 0u) { h[r] &= mask; fresh &= ~(1u << r); }
+        taken |= 1u << (8 * r + at[r]);                   // somebody else's token got there first: the next free slot of the (stale) sector
       }
     }
     if (todo) atomicOr(s.status, SDMS_STATUS_INDEX_FULL);             // more nodes than slots: cannot happen
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
       const int d = d_base + r * kLayerWays;
-      if (d > D) continue;
+      if (d > d_end) continue;
       if (sv[r] >= 0) atomicAdd(&s.w_tab[base + ((size_t)(d - 1) << lcap) + sv[r]].sum, add[r]);
       const int mine = __shfl_sync(FULL, sv[r], leader[r]);
       if (ml < nm) item[(size_t)(d - 1) * M] = v[r] >= 0 ? mine : -1;

@@ -30,6 +30,7 @@
 //   pass E  edge weights out; the slots that were used are zeroed again.
 // Between the passes all CTAs meet at a grid barrier (bounded wait; the launch is cooperative, so all
 // CTAs are resident).
+#include <cstddef>
 #include "sdms_internal.h"
 #include "wide_dev.cuh"
 
@@ -39,6 +40,9 @@ namespace {
 
 constexpr long long kBarrierCycles = 200000000LL;    // about a tenth of a second (the pass takes 0.1-0.3 ms): a barrier that takes that long has failed
 constexpr u64 kSumMask = (1ull << kWideSumShift) - 1;
+constexpr int kRivalsFrom = 4096;                    // matches of a query from which offers to one node are reduced in the warp first
+static_assert(offsetof(WideSlot, succ) == offsetof(WideSlot, succ_w) + 8 && offsetof(WidePred, succ) == offsetof(WidePred, succ_w) + 8,
+              "the best successor sits right behind its weight");
 
 __device__ __forceinline__ u64 ld_u64(const u64* p) { return __ldcg(p); }
 __device__ __forceinline__ uint32_t ld_u32(const uint32_t* p) { return __ldcg(p); }
@@ -161,33 +165,70 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
       const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
       const int* const item = s.w_item + base + m0 + ml;
       const int d_end = min(D, d_first + (r_lo + rounds_per - 1) * kLayerWays);
+      // a thread's layers four at a time: the loads of all four are on their way before the first is used
 #pragma unroll 1
-      for (int d = d_first + r_lo * kLayerWays; d <= d_end; d += kLayerWays) {
-        int sv = -1, su = -1;
-        if (ml < nm) {
-          sv = item[(size_t)(d - 1) * M];
-          if (d > 1 && s.mode != 1) su = item[(size_t)(d - 2) * M];
+      for (int d0 = d_first + r_lo * kLayerWays; d0 <= d_end; d0 += kMaxRounds * kLayerWays) {
+        int sv[kMaxRounds], su[kMaxRounds];
+#pragma unroll
+        for (int r = 0; r < kMaxRounds; ++r) {
+          const int d = d0 + r * kLayerWays;
+          sv[r] = -1; su[r] = -1;
+          if (d <= d_end && ml < nm) {
+            sv[r] = item[(size_t)(d - 1) * M];
+            if (d > 1 && s.mode != 1) su[r] = item[(size_t)(d - 2) * M];
+          }
         }
-        const bool on = sv >= 0 && (d == 1 || s.mode == 1 || su >= 0);
-        // items on the same edge (same node, under the layer-wise rule) bring the same offer: one lane speaks for them
-        const u64 edge = on ? ((u64)(unsigned)su << 32) | (u64)(unsigned)sv : ~(u64)lane;
-        const unsigned group = __match_any_sync(FULL, edge);
-        if (!on || lane != __ffs(group) - 1) continue;
-        const WideSlot* mine = s.w_tab + base + ((size_t)(d - 1) << lcap) + sv;
-        const u64 wbits = (u64)__double_as_longlong(weight_of(s, ld_u64(&mine->sum)));
-        u64* best_w; u64* best;
-        if (d == 1 || s.mode == 1) {
-          WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT + (d - 1);
-          best_w = &pr->succ_w; best = &pr->succ;
-        } else {
-          WideSlot* before = s.w_tab + base + ((size_t)(d - 2) << lcap) + su;
-          best_w = &before->succ_w; best = &before->succ;
+        unsigned lead = 0;                             // layers in which this lane speaks for its edge
+        u64 sum[kMaxRounds];
+        u64* best_w[kMaxRounds];
+#pragma unroll
+        for (int r = 0; r < kMaxRounds; ++r) {
+          const int d = d0 + r * kLayerWays;
+          sum[r] = 0ull; best_w[r] = nullptr;
+          if (d > d_end) continue;                     // the same for the whole warp
+          const bool on = sv[r] >= 0 && (d == 1 || s.mode == 1 || su[r] >= 0);
+          // items on the same edge (same node, under the layer-wise rule) bring the same offer: one lane speaks for them
+          const u64 edge = on ? ((u64)(unsigned)su[r] << 32) | (u64)(unsigned)sv[r] : ~(u64)lane;
+          const unsigned group = __match_any_sync(FULL, edge);
+          if (!on || lane != __ffs(group) - 1) continue;
+          lead |= 1u << r;
+          sum[r] = ld_u64(&s.w_tab[base + ((size_t)(d - 1) << lcap) + sv[r]].sum);
+          best_w[r] = d == 1 || s.mode == 1 ? &s.w_pred[(size_t)q * SDMS_MAX_DRAFT + (d - 1)].succ_w
+                                            : &s.w_tab[base + ((size_t)(d - 2) << lcap) + su[r]].succ_w;
         }
         if (pass == 0) {
-          atomicMax(best_w, wbits);
-        } else if (ld_u64(best_w) == wbits) {
-          const uint32_t tok = ld_u32(&mine->tok1) - 1u;
-          atomicMax(best, ((u64)(~tok) << 32) | (u64)(unsigned)sv);
+#pragma unroll
+          for (int r = 0; r < kMaxRounds; ++r) {
+            if (d0 + r * kLayerWays > d_end) continue;   // the same for the whole warp
+            // Of the lanes that offer to the same node only the one with the largest weight needs to: a popular
+            // n-gram's root or first nodes would otherwise take thousands of atomics on one address.
+            const bool on = lead >> r & 1u;
+            const u64 w = on ? (u64)__double_as_longlong(weight_of(s, sum[r])) : 0ull;
+            if (M < kRivalsFrom) { if (on) atomicMax(best_w[r], w); continue; }   // few offers per node: not worth the shuffles
+            const unsigned rivals = __match_any_sync(FULL, on ? (u64)(uintptr_t)best_w[r] : (u64)lane);
+            u64 top = w;
+            for (unsigned rem = __ballot_sync(FULL, on && (rivals & (rivals - 1)) != 0u); rem; rem &= rem - 1) {
+              const int src = __ffs(rem) - 1;
+              const u64 other = __shfl_sync(FULL, w, src);
+              if ((rivals >> src & 1u) && other > top) top = other;
+            }
+            if (on && w == top) atomicMax(best_w[r], w);
+          }
+        } else {
+          u64 cur[kMaxRounds];
+          uint32_t tok1[kMaxRounds];
+#pragma unroll
+          for (int r = 0; r < kMaxRounds; ++r) {
+            cur[r] = 0ull; tok1[r] = 0u;
+            if (!(lead >> r & 1u)) continue;
+            cur[r] = ld_u64(best_w[r]);
+            tok1[r] = ld_u32(&s.w_tab[base + ((size_t)(d0 + r * kLayerWays - 1) << lcap) + sv[r]].tok1);
+          }
+#pragma unroll
+          for (int r = 0; r < kMaxRounds; ++r) {
+            if (!(lead >> r & 1u) || cur[r] != (u64)__double_as_longlong(weight_of(s, sum[r]))) continue;
+            atomicMax(best_w[r] + 1, ((u64)(~(tok1[r] - 1u)) << 32) | (u64)(unsigned)sv[r]);   // succ sits behind succ_w
+          }
         }
       }
     }

@@ -5,9 +5,9 @@
 namespace sdms {
 
 // log2 of the slots of one layer's node table: a power of two above 5/2 of the matches.  A layer in which
-// every candidate is a node of its own fills at most 40 % of it: with linear probing the LONGEST probe
-// run of the table decides how long a pass takes (the whole grid waits for the unluckiest lane), and
-// that run grows quickly with the fill.
+// every candidate is a node of its own fills at most 40 % of it: the whole grid waits for the unluckiest
+// lane of a pass, that is for the fullest eight-key sector of all tables (every claimer that meets
+// somebody else's token there pays another round trip), and how full that sector is grows quickly with the fill.
 __device__ __forceinline__ int wide_lcap(int M) {
   int l = 6;
   while ((1ll << l) < (5ll * M) / 2 + 1) ++l;

@@ -243,6 +243,25 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     const int i = de.x, M = de.y, lcap = de.z;
     const unsigned base = (unsigned)de.w;
     const int m0 = (c - sh_cbase[q]) * kWideChunk, nm = min(kWideChunk, M - m0);
+    // what the edge sums below need of this thread's first four layers is asked for now: it arrives while
+    // thread 0 walks (a dependent load per layer)
+    const int* const item = s.w_item + base + m0 + ml;
+    const int gpos = ml < nm ? s.matches[(size_t)s.q_off[i] + m0 + ml] : 0;
+    const int d_lo = d_first + r_lo * kLayerWays, d_hi = min(D, d_first + (r_lo + rounds_per - 1) * kLayerWays);
+    int it1[kMaxRounds], it0[kMaxRounds];
+    unsigned pv[kMaxRounds];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+      const int d = d_lo + r * kLayerWays;
+      it1[r] = -1; it0[r] = -1; pv[r] = 0u;
+      if (ml < nm && d <= d_hi) {
+        it1[r] = item[(size_t)(d - 1) * M];
+        if (d > 1) it0[r] = item[(size_t)(d - 2) * M];
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r)
+      if (it1[r] >= 0) pv[r] = (unsigned)__ldg(s.pq + gpos + d_lo + r * kLayerWays);    // the item exists, so its follower does
     if (tid == 0) {
       const bool writer = m0 == 0 && r_lo == 0;       // the query's first unit writes the draft out
       const WidePred* pr = s.w_pred + (size_t)q * SDMS_MAX_DRAFT;
@@ -266,18 +285,32 @@ dag_wide_kernel(Dev s, int32_t* __restrict__ draft_tok, int32_t* __restrict__ dr
     }
     __syncthreads();
     const int emitted = sh_emitted;
-    const int* const item = s.w_item + base + m0 + ml;
-    const int gpos = ml < nm ? s.matches[(size_t)s.q_off[i] + m0 + ml] : 0;
-    const int d_end = min(emitted, d_first + (r_lo + rounds_per - 1) * kLayerWays);
+    const int d_end = min(emitted, d_hi);
 #pragma unroll 1
-    for (int d = d_first + r_lo * kLayerWays; d <= d_end; d += kLayerWays) {
-      bool on = false;
-      if (ml < nm) on = item[(size_t)(d - 1) * M] == sh_dslot[d - 1] && (d == 1 || item[(size_t)(d - 2) * M] == sh_dslot[d - 2]);
-      const unsigned group = __ballot_sync(FULL, on);
-      if (group == 0u) continue;
-      const u64 sum = group_sum(group, group, on ? (unsigned)__ldg(s.pq + gpos + d) : 0u);
-      if (lane == __ffs(group) - 1)
-        atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
+    for (int d0 = d_lo; d0 <= d_end; d0 += kMaxRounds * kLayerWays) {
+      if (d0 != d_lo) {                                 // more than four layers per thread (D > 16, unit not split): the next four
+#pragma unroll
+        for (int r = 0; r < kMaxRounds; ++r) {
+          const int d = d0 + r * kLayerWays;
+          it1[r] = -1; it0[r] = -1; pv[r] = 0u;
+          if (ml < nm && d <= d_end) {
+            it1[r] = item[(size_t)(d - 1) * M];
+            it0[r] = item[(size_t)(d - 2) * M];
+            if (it1[r] >= 0) pv[r] = (unsigned)__ldg(s.pq + gpos + d);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRounds; ++r) {
+        const int d = d0 + r * kLayerWays;
+        if (d > d_end) continue;                        // the same for the whole warp
+        const bool on = it1[r] >= 0 && it1[r] == sh_dslot[d - 1] && (d == 1 || it0[r] == sh_dslot[d - 2]);
+        const unsigned group = __ballot_sync(FULL, on);
+        if (group == 0u) continue;
+        const u64 sum = group_sum(group, group, on ? pv[r] : 0u);
+        if (lane == __ffs(group) - 1)
+          atomicAdd(&s.w_edge[(size_t)q * SDMS_MAX_DRAFT + d - 1], ((u64)__popc(group) << kWideSumShift) | sum);
+      }
     }
     __syncthreads();
   }

@@ -840,6 +840,29 @@ def test_wide_pass_with_many_distinct_followers_and_ragged_ends():
     assert prof["dag_wide"][1] == 1
 
 
+@pytest.mark.parametrize("N,L,V,D,match_capacity", [(4, 400, 3, 32, 5000), (4, 400, 3, 10, 5000), (5, 300, 2, 3, 7000),
+                                                     (24, 900, 50, 32, 400000)])
+def test_wide_pass_units_split_by_layers_and_drafts_longer_than_a_batch(N, L, V, D, match_capacity):
+    # few heavy queries: their chunks of 128 matches are split by layers into 2, 4 or 8 units (D = 32: eight rounds of
+    # layers per thread; D = 10: three, so the last unit is short; D = 3: one, no split); many heavy queries: no split,
+    # several units per CTA, and with D = 32 a thread's layers take two batches of four
+    G = 1
+    tokens, lps = synth.small_random(G * N, L, V, 4260 + D)
+    pair = Pair(G, N, L, V, 2, D, match_capacity=match_capacity, alpha=0.5)
+    n = L - 4 * (D + 1) - 4
+    lens = (n - (np.arange(G * N) * 29) % (L // 3)).astype(np.int32)
+    pair.append(tokens[:, :n], lps[:, :n], lens, expect_status=0)
+    from paper_2503_05330_b200 import binding
+    binding.sdms_profile_enable(pair.g.ctx, True)
+    for k in (1, 2, 1):
+        pair.build_and_compare(k, check_dag=False)
+        lens = pair.o.lengths()
+        sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
+        pair.accept_and_compare(sampled, sampled_lp)
+    assert binding.sdms_profile_read(pair.g.ctx)["dag_wide"][1] >= 3
+    pair.check_history()
+
+
 # ---- several drafts per path: the B best paths of the pool ----------------------------------------
 def test_beams_hand_worked_pool_on_device():
     paths = [[5, 9], [9, 1, 3, 7], [9, 2, 4, 7], [9, 2, 5, 7]]

@@ -187,7 +187,10 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
  * enough for the single-launch build (N*L <= 131072 tokens and G*N*N*L <=
  * match_capacity); on larger ones one round of launches per suffix length, longest
  * first (a path that has found matches keeps them; sdms_debug_read_query_modes then
- * reports 3 for it), there not together with epsilon = 1 (SDMS_ERR_BAD_STATE).
+ * reports 3 for it).  With epsilon = 1 a path that gets down to k = 1 matches every
+ * position of its prompt (one substitution away from any token): on such a large
+ * prompt that is more than a match list holds, the path gets no draft and
+ * SDMS_STATUS_MATCH_OVERFLOW is raised.
  */
 int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok, int32_t* d_draft_len,
                               float* d_draft_score, float* d_draft_edge_w, int32_t* d_used_k, void* stream);

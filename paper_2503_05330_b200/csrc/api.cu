@@ -315,7 +315,7 @@ int sdms_build_drafts(sdms_ctx* ctx, int32_t k, int32_t* d_draft_tok, int32_t* d
   }
   int rc;
   if (ctx->dev.eps > 0) {                            // matches with tolerance: sized by counting, four launches
-    rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_fuzzy_match(ctx->dev, k, st); });
+    rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_fuzzy_match(ctx->dev, k, 0, st); });
     ctx->launches += 3;
   } else {
     rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, 0, st); });
@@ -341,11 +341,16 @@ int sdms_build_drafts_backoff(sdms_ctx* ctx, int32_t k_hi, int32_t* d_draft_tok,
   if (!ctx->dev.fused) {
     // large prompts: one probe / scan / dag (/ wide) round per suffix length, longest first; a path that has found
     // matches keeps them and its draft, the others try again with a shorter suffix
-    if (ctx->dev.eps > 0) return SDMS_ERR_BAD_STATE;
     for (int k = k_hi; k >= 1; --k) {
       const int round = kRoundBackoff | (k < k_hi ? kRoundNotFirst : 0) | (k == 1 ? kRoundLast : 0);
-      int rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, k < k_hi, st); });
-      if (rc == SDMS_OK) rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+      int rc;
+      if (ctx->dev.eps > 0) {
+        rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_fuzzy_match(ctx->dev, k, k < k_hi, st); });
+        ctx->launches += 3;
+      } else {
+        rc = timed(ctx, SDMS_KERNEL_PROBE, st, [&] { return launch_probe(ctx->dev, k, k < k_hi, st); });
+        if (rc == SDMS_OK) rc = timed(ctx, SDMS_KERNEL_SCAN, st, [&] { return launch_scan(ctx->dev, k, st); });
+      }
       if (rc == SDMS_OK)
         rc = timed(ctx, SDMS_KERNEL_DAG, st, [&] {
           return launch_dag(ctx->dev, false, d_draft_tok, d_draft_len, d_draft_score, d_draft_edge_w, st, round, k, d_used_k); });
@@ -414,7 +419,6 @@ int sdms_step_backoff(sdms_ctx* ctx, int32_t k_hi, const int32_t* d_sampled, con
   if (!ctx || !d_sampled || !d_sampled_logprobs || !d_accept_len || !d_draft_tok || !d_draft_len)
     return SDMS_ERR_INVALID_ARG;
   if (k_hi < 1 || k_hi > ctx->cfg.k_max) return SDMS_ERR_INVALID_ARG;
-  if (!ctx->dev.fused && ctx->dev.eps > 0) return SDMS_ERR_BAD_STATE;
   if (!ctx->step_fits) {
     const int rc = sdms_accept(ctx, d_draft_tok, d_draft_len, d_sampled, d_sampled_logprobs, d_accept_len, stream);
     if (rc != SDMS_OK) return rc;

@@ -33,12 +33,13 @@ constexpr int kFzQueries = 128;                    // queries whose tokens are s
 
 __device__ __forceinline__ uint32_t fz_bit(int32_t tok) { return ((uint32_t)tok * 2654435761u) >> 16; }
 
-__global__ void __launch_bounds__(256) fuzzy_prepare_kernel(Dev s, int k) {
+__global__ void __launch_bounds__(256) fuzzy_prepare_kernel(Dev s, int k, int skip_done) {
   grid_wait();
   grid_release();
   if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_grid) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= s.P) return;
+  if (skip_done && s.q_mode[i] == Q_DONE) return;                // back-off: this path has its matches from a longer suffix
   const int len = s.len[i];
   s.q_fp[i] = 0u;
   s.q_mode[i] = len >= k && len < s.L ? Q_SCAN : Q_NONE;
@@ -160,10 +161,10 @@ __global__ void __launch_bounds__(kFzThreads) fuzzy_scan_kernel(Dev s, int k, in
 }  // namespace
 
 // probe + scan of a build with tolerance 1 on a context that does not take the single-launch build
-cudaError_t launch_fuzzy_match(const Dev& s, int k, cudaStream_t stream) {
+cudaError_t launch_fuzzy_match(const Dev& s, int k, int skip_done, cudaStream_t stream) {
   const int tiles = (s.L + kFzTile - 1) / kFzTile;
   const unsigned blocks = (unsigned)((s.P + 255) / 256);
-  cudaError_t e = launch_overlapped(fuzzy_prepare_kernel, dim3(blocks), dim3(256), 0, stream, s, k);
+  cudaError_t e = launch_overlapped(fuzzy_prepare_kernel, dim3(blocks), dim3(256), 0, stream, s, k, skip_done);
   if (e == cudaSuccess)
     e = launch_overlapped(fuzzy_scan_kernel<false>, dim3((unsigned)(s.P * tiles)), dim3(kFzThreads), 0, stream, s, k, tiles);
   if (e == cudaSuccess) e = launch_overlapped(fuzzy_alloc_kernel, dim3(blocks), dim3(256), 0, stream, s);

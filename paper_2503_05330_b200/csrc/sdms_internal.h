@@ -27,7 +27,7 @@ cudaError_t launch_accept(const Dev& s, const int32_t* draft_tok, const int32_t*
 cudaError_t launch_probe(const Dev& s, int k, int skip_done, cudaStream_t stream);
 cudaError_t launch_scan(const Dev& s, int k, cudaStream_t stream);
 // tolerance 1 on large prompts: mark the queries, count, hand out slices, fill (four launches)
-cudaError_t launch_fuzzy_match(const Dev& s, int k, cudaStream_t stream);
+cudaError_t launch_fuzzy_match(const Dev& s, int k, int skip_done, cudaStream_t stream);
 // round: 0 for an ordinary build; kRound* flags, k and used_k for one round of a back-off build on a large prompt
 cudaError_t launch_dag(const Dev& s, bool with_export, int32_t* draft_tok, int32_t* draft_len, float* draft_score,
                        float* draft_edge_w, cudaStream_t stream, int round = 0, int k = 0, int32_t* used_k = nullptr);

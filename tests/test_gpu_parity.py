@@ -995,10 +995,12 @@ def test_short_index_on_benchmark_workloads(wid, index_max_n):
 
 
 # ---- back-off of the suffix length on prompts that take the probe / scan / dag kernels ------------
-def test_backoff_by_rounds_dense_tiny_vocab():
-    G, N, L, V, D, k_max = 2, 6, 64, 4, 4, 4
+@pytest.mark.parametrize("eps,L,match_capacity", [(0, 64, 3000), (1, 128, 9000)])
+def test_backoff_by_rounds_dense_tiny_vocab(eps, L, match_capacity):
+    # (with tolerance 1 a path that gets down to k = 1 matches every position: the list must hold N * L per path)
+    G, N, V, D, k_max = 2, 6, 4, 4, 4
     tokens, lps = synth.small_random(G * N, L, V, 9800)
-    pair = Pair(G, N, L, V, k_max, D, alpha=0.5, match_capacity=3000)
+    pair = Pair(G, N, L, V, k_max, D, alpha=0.5, match_capacity=match_capacity, eps=eps)
     start = (2 + (np.arange(G * N) * 5) % 11).astype(np.int32)
     pair.append(tokens[:, :16], lps[:, :16], start, expect_status=0)
     seen = set()
@@ -1009,8 +1011,23 @@ def test_backoff_by_rounds_dense_tiny_vocab():
         sampled, sampled_lp = synth.sampled_window(tokens, lps, lens, D + 1)
         pair.accept_and_compare(sampled, sampled_lp)
         pair.build_and_compare(1 + step % k_max, check_dag=False)      # an ordinary build in between finds a clean state
-    assert len(seen) >= 3
+    assert len(seen) >= (3 if eps == 0 else 2)
     pair.check_history()
+
+
+def test_backoff_by_rounds_with_tolerance_on_a_prompt_too_large_for_one_launch():
+    # 40 paths x 4096 tokens (more than 128 Ki tokens): count / hand out / fill / dag (/ wide) once per suffix length
+    G, N, L, V, D, k_max = 1, 40, 4096, 60, 6, 4
+    tokens, lps = synth.small_random(G * N, L, V, 9810)
+    pair = Pair(G, N, L, V, k_max, D, eps=1)
+    lens = (4000 - (np.arange(G * N) * 61) % 1500).astype(np.int32)
+    pair.append(tokens[:, :4000], lps[:, :4000], lens, expect_status=0)
+    _, _, used = pair.backoff_and_compare(k_max)
+    assert len(set(used.tolist())) >= 2 and used.min() >= 2
+    sampled, sampled_lp = synth.sampled_window(tokens, lps, pair.o.lengths(), D + 1)
+    pair.accept_and_compare(sampled, sampled_lp)
+    pair.backoff_and_compare(3)
+    pair.build_and_compare(2, check_dag=False)                          # an ordinary build afterwards finds a clean state
 
 
 def test_backoff_by_rounds_config5():

@@ -1225,29 +1225,35 @@ __global__ void __launch_bounds__(kDagThreads, EXPORT ? 1 : 2) dag_kernel(Dev s,
                                                           float* __restrict__ draft_score,
                                                           float* __restrict__ draft_edge_w, int round, int k,
                                                           int32_t* __restrict__ used_k) {
-  grid_wait();
-  grid_release();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Smem sm = carve<EXPORT>(smem_raw);
   __shared__ int32_t sh_len[SDMS_MAX_PATHS_PER_GROUP];
   const int i = blockIdx.x;
+  // the path lengths are older than the kernels this one follows (probe, scan: their CTAs let it start only after
+  // their own wait): fetched while those drain
+  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + (i / s.N) * s.N + n);
+  const int32_t root = ldm(s.rec + (size_t)i * kRecWords + 1);
+  grid_wait();
+  grid_release();
+  // what probe and scan left for this path, in one round trip
+  const int32_t q_mode = s.q_mode[i];
+  const int q_found = min(s.q_cursor[i], s.q_reserved[i]), q_off = s.q_off[i];
   if (i == 0) {                                       // probe and scan are done with these: the next build finds them at zero
     for (int x = threadIdx.x; x < s.G; x += blockDim.x) s.g_nscan[x] = 0;
     // (the slices of a back-off build's earlier rounds stay where they are until its last round)
     if (threadIdx.x == 0 && (!(round & kRoundBackoff) || (round & kRoundLast))) *s.match_cursor = 0ull;
   }
-  if ((round & kRoundNotFirst) && s.q_mode[i] == Q_DONE) return;     // drafted in an earlier round, from a longer suffix
+  if ((round & kRoundNotFirst) && q_mode == Q_DONE) return;     // drafted in an earlier round, from a longer suffix
   write_defaults<EXPORT>(s, i, draft_tok, draft_score, draft_edge_w);
-  const int M = s.q_mode[i] == Q_NONE ? 0 : min(s.q_cursor[i], s.q_reserved[i]);
+  const int M = q_mode == Q_NONE ? 0 : q_found;
   if (M == 0) {
     if (threadIdx.x == 0) { draft_len[i] = 0; if (used_k) used_k[i] = 0; }
     return;
   }
   if ((round & kRoundBackoff) && threadIdx.x == 0) { s.q_mode[i] = Q_DONE; if (used_k) used_k[i] = k; }
   const int g = i / s.N;
-  for (int n = threadIdx.x; n < s.N; n += blockDim.x) sh_len[n] = ldm(s.len + g * s.N + n);
   __syncthreads();
-  int32_t* const mlist = s.matches + s.q_off[i];
+  int32_t* const mlist = s.matches + q_off;
   int Mk = M;
   if (s.R > 0) {                                    // (a second pass over the same build finds nothing left to cut)
     Mk = cap_matches(s, g, M, mlist, sm.st_tok);
@@ -1256,8 +1262,7 @@ __global__ void __launch_bounds__(kDagThreads, EXPORT ? 1 : 2) dag_kernel(Dev s,
   }
   // more matches than a warp holds: all SMs share the work (the pass that follows this kernel)
   if (!EXPORT && s.pool == 0 && s.mode != 2 && Mk > 32 && wide_register(s, i, Mk)) return;
-  dag_phase<EXPORT>(s, sm, i, Mk, mlist, sh_len, g * s.N, ldm(s.rec + (size_t)i * kRecWords + 1),
-                    draft_tok, draft_len, draft_score, draft_edge_w);
+  dag_phase<EXPORT>(s, sm, i, Mk, mlist, sh_len, g * s.N, root, draft_tok, draft_len, draft_score, draft_edge_w);
 }
 
 // Whole draft construction of one query path in one CTA, for prompts whose

@@ -245,11 +245,7 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 template <bool STREAM>
 __global__ void __launch_bounds__(STREAM ? kStreamThreads : kScanThreads, STREAM ? 4 : 6)
 scan_kernel(Dev s, int k, int ctas, int set_slots) {
-  grid_wait();
-  grid_release();
-  if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_grid) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
   const int g = blockIdx.x / ctas, first = blockIdx.x - g * ctas;
-  if (s.g_nscan[g] == 0) return;
   constexpr int TILE = STREAM ? kStreamTile : kScanTile;
   const int ntiles = (s.L + TILE - 1) / TILE, total = s.N * ntiles;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -277,6 +273,20 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
     for (int st = 0; st < kStreamStages; ++st) { mbar_init(&sh_full[st], 1); mbar_init(&sh_empty[st], kScanThreads); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // the last token of the first path this thread will look at below (path records are older than the probe too)
+  const int i_pre = g * s.N + (int)threadIdx.x;
+  int32_t last_pre = 0;
+  if ((int)threadIdx.x < s.N) last_pre = s.rec[(size_t)i_pre * kRecWords + 1];
+  // Up to here nothing was read that the probe writes (path lengths, records and tokens are older than the probe: its
+  // CTAs let this kernel start only after their own wait), so the set-up above overlaps the probe's tail.
+  grid_wait();
+  grid_release();
+  if (blockIdx.x == 0 && threadIdx.x < kWideCtlWords && s.w_grid) s.w_ctl[threadIdx.x] = 0ull;   // the wide pass of this build starts with an empty list
+  // what the probe left for that path, asked for together with the prompt's count of scan queries: one round trip
+  int32_t mode_pre = Q_NONE;
+  uint32_t fp_pre = 0u;
+  if ((int)threadIdx.x < s.N) { mode_pre = s.q_mode[i_pre]; fp_pre = s.q_fp[i_pre]; }
+  if (s.g_nscan[g] == 0) return;
   __syncthreads();
   // (path, tile) of the CTA's current tile and of the one after it; they advance by `ctas` tiles without a division
   const int step_j = ctas / ntiles, step_t = ctas - step_j * ntiles;
@@ -312,14 +322,15 @@ scan_kernel(Dev s, int k, int ctas, int set_slots) {
   // the prompt's scan queries
   for (int n = threadIdx.x; n < s.N; n += blockDim.x) {
     const int i = g * s.N + n;
-    if (s.q_mode[i] == Q_SCAN) {
+    const bool have = n == (int)threadIdx.x;                         // the thread's first path: already here
+    if ((have ? mode_pre : s.q_mode[i]) == Q_SCAN) {
       const int sl = atomicAdd(&sh_nq, 1);
-      const uint32_t fp = s.q_fp[i];
+      const uint32_t fp = have ? fp_pre : s.q_fp[i];
       sh_qid[sl] = i;
       sh_qfp[sl] = fp;
       uint32_t hs = (fp >> 1) & (set_slots - 1);
       while (atomicCAS(&sh_set[hs], -1, sl) != -1) hs = (hs + 1) & (set_slots - 1);
-      const int32_t last = s.rec[(size_t)i * kRecWords + 1];
+      const int32_t last = have ? last_pre : s.rec[(size_t)i * kRecWords + 1];
       sh_qlast[sl] = last;
       const uint32_t lb = last_bit(last), lb2 = last_bit2(last);      // two bits per query token: few false alarms
       atomicOr(&sh_last[lb >> 5], 1u << (lb & 31));

@@ -79,8 +79,6 @@ __device__ __forceinline__ bool one_edit_end(const int32_t* row, int e, const in
 
 template <bool FILL>
 __global__ void __launch_bounds__(kFzThreads) fuzzy_scan_kernel(Dev s, int k, int tiles) {
-  grid_wait();
-  grid_release();
   __shared__ int32_t sh_tok[kFzHalo + kFzTile];            // sh_tok[kFzHalo + x] = token at t0 + x
   __shared__ uint32_t sh_bits[kFzBits / 32];
   __shared__ int32_t sh_q[kFzQueries][SDMS_MAX_K];
@@ -99,6 +97,10 @@ __global__ void __launch_bounds__(kFzThreads) fuzzy_scan_kernel(Dev s, int k, in
   }
   for (int x = tid; x < kFzBits / 32; x += blockDim.x) sh_bits[x] = 0u;
   if (tid == 0) sh_ncand = 0;
+  // tokens and path lengths are older than the kernels this one follows (their CTAs let it start only after their own
+  // wait): the tile was staged while those drained; the queries' state is read from here on
+  grid_wait();
+  grid_release();
   __syncthreads();
   // the tokens that can sit at the end of a match: the last two of every query of the prompt
   if (k >= 2)

@@ -368,8 +368,7 @@ cudaError_t launch_dag_wide(const Dev& s, int32_t* draft_tok, int32_t* draft_len
     cfg.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, dag_wide_kernel, s, draft_tok, draft_len, draft_score, draft_edge_w);
     if (e == cudaSuccess) return e;
-    if (e != cudaErrorInvalidValue && e != cudaErrorNotSupported) return e;
-    cudaGetLastError();
+    cudaGetLastError();                               // whatever the reason: once more without the second attribute
     early = false;
   }
   cfg.numAttrs = 1;

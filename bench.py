@@ -29,8 +29,8 @@ UNIT = "paths*steps/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel from its last ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); only quoted while the kernel sources are the ones profiled
-NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 75968,
-               "sources_sha256": "bbab5f23f0fc00ce74c0caacda7f00fb8806953bbb54dda165b640f12f48617b"}
+NCU_TRAFFIC = {"kernel": "step", "bytes_per_launch": 76032,
+               "sources_sha256": "82c4fa773fa1eba361a55396feeb945f28cf039ae1940f656ce90e8d14e5ec53"}
 
 
 def kernel_sources_sha():

@@ -58,6 +58,7 @@ constexpr int kWideThreads = 512;
 constexpr int kWideChunk = 128;                      // matches per unit of work: thread t owns match t % 128 ...
 constexpr int kLayerWays = kWideThreads / kWideChunk;  // ... and the layers d = t / 128 + 1, + 5, + 9, ...
 constexpr int kMaxRounds = 4;                          // layers of a thread that are in flight together (16 layers of the query)
+static_assert(kMaxRounds * 8 <= 32, "eight slot bits per layer in flight fit one word");
 
 // Sum of p over the lanes of this lane's group (`group` from __match_any_sync).  The same loop in every
 // lane, over the lanes that share their group with somebody (`shared`: whole groups only); a lane that is
@@ -163,13 +164,13 @@ __device__ __forceinline__ void wide_insert_unit(const Dev& s, const int32_t* li
         if (!(todo >> r & 1u)) continue;
         const uint32_t want = (uint32_t)v[r] + 1u;
         const uint32_t kk[8] = {ka[r].x, ka[r].y, ka[r].z, ka[r].w, kb[r].x, kb[r].y, kb[r].z, kb[r].w};
-        unsigned hit = 0u, open = 0u;
+        unsigned hit = 0u, vacant = 0u;
 #pragma unroll
-        for (int x = 0; x < 8; ++x) { hit |= (unsigned)(kk[x] == want) << x; open |= (unsigned)(kk[x] == 0u) << x; }
-        open &= ~(taken >> (8 * r));
+        for (int x = 0; x < 8; ++x) { hit |= (unsigned)(kk[x] == want) << x; vacant |= (unsigned)(kk[x] == 0u) << x; }
+        vacant &= ~(taken >> (8 * r));
         const unsigned start = h[r] & 7u;
         if (hit) { at[r] = __ffs(hit) - 1; seen[r] = want; }
-        else if (open) { at[r] = (int)((start + __ffs(((open | (open << 8)) >> start) & 0xffu) - 1) & 7u); }
+        else if (vacant) { at[r] = (int)((start + __ffs(((vacant | (vacant << 8)) >> start) & 0xffu) - 1) & 7u); }
       }
       unsigned claims = 0;
 #pragma unroll
